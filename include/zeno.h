@@ -1,0 +1,157 @@
+/*
+ * zeno.h -- C ABI of the Zeno aggregation step on one NVIDIA B200 (sm_100a).
+ *
+ * The step is the server side of "Zeno: Distributed Stochastic Gradient
+ * Descent with Suspicion-based Fault-tolerance" (Algorithm 1, the line
+ * "v = Zeno_b({v_i})"):
+ *
+ *   Definition 2   Score_{gamma,rho}(v_i, x) = f_r(x) - f_r(x - gamma v_i) - rho ||v_i||^2,
+ *                  f_r = mean loss over the server's n_r samples, l2 norm;
+ *   Definition 3   rank the m candidates by score (descending) and return the
+ *                  average of the m - b best.
+ *
+ * Conventions for every call
+ *   - All data pointers are DEVICE pointers owned by the caller (x, V, the batch,
+ *     and every output).  Inputs are never written; outputs are overwritten in
+ *     full.  The library allocates device memory only inside zeno_create.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Calls are asynchronous on it: they enqueue kernels and return; there is
+ *     no host synchronisation and no device-to-host copy inside a call.
+ *   - Errors are return codes.  Nothing is thrown, aborted or trapped.  Argument
+ *     errors are detected on the host before anything is enqueued.
+ *   - A handle serialises its calls through one private workspace: calls that
+ *     use the same handle must be ordered on the GPU (same stream, or events).
+ *
+ * Parameter-vector layout (x and every row of V):
+ *   multi-layer perceptron: for layer l = 1..L, the weights W_l as
+ *   [dims[l] x dims[l-1]] row-major (input index contiguous), then, if
+ *   has_bias, the bias b_l[dims[l]]; layers concatenated in order.
+ *   least squares: the d entries of x.
+ *   V is [m x ldv] row-major with ldv >= d (in elements); columns >= d are
+ *   padding and are never read.  Rows whose start is 16-byte aligned
+ *   (ldv * element size a multiple of 16, base pointer 16-byte aligned) take
+ *   the vectorised kernels; any other ldv >= d takes a slower scalar path.
+ */
+#ifndef ZENO_H_
+#define ZENO_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ZENO_MAX_LAYERS 8
+#define ZENO_MAX_CANDIDATES 1024
+
+typedef enum {
+    ZENO_OK = 0,
+    ZENO_ERR_INVALID_ARG = 1, /* NULL required pointer, m/b/n_r/ldv out of range, non-finite gamma or rho */
+    ZENO_ERR_UNSUPPORTED = 2, /* a (loss, dtype, shape) for which no kernel exists -- never a silent fallback */
+    ZENO_ERR_WORKSPACE = 3,   /* the handle's workspace could not be allocated */
+    ZENO_ERR_CUDA = 4,        /* a CUDA runtime call failed; see zeno_last_cuda_error */
+    ZENO_ERR_TIMEOUT = 5      /* a bounded device-side wait gave up */
+} zeno_status;
+
+typedef enum {
+    /* f(x; (a, y)) = -log softmax(MLP_x(a))[y]: L >= 1 dense layers, ReLU between
+     * them; L = 1 is softmax regression.  Cross-entropy is the loss the paper
+     * trains and reports (Experiments, evaluation metrics). */
+    ZENO_LOSS_SOFTMAX_MLP = 0,
+    /* f(x; (a, y)) = (a.x - y)^2 / 2, so that f_r(x) = ||A x - y||^2 / (2 n_r). */
+    ZENO_LOSS_LEAST_SQUARES = 1
+} zeno_loss_kind;
+
+typedef enum {
+    ZENO_F32 = 0, /* x and V stored as IEEE binary32 */
+    ZENO_BF16 = 1 /* x and V stored as bfloat16; a candidate's parameters are
+                     x - gamma v rounded (to binary32, then) to bfloat16;
+                     features, activations and accumulation stay binary32 */
+} zeno_dtype;
+
+typedef struct {
+    int32_t kind;        /* zeno_loss_kind */
+    int32_t param_dtype; /* zeno_dtype */
+    int32_t n_layers;    /* L; least squares: 1 */
+    int32_t has_bias;    /* MLP only */
+    int64_t dims[ZENO_MAX_LAYERS + 1]; /* MLP: widths, e.g. {3072,512,512,10}; least squares: {d, 1} */
+} zeno_model_desc;
+
+/* The server's batch z_1..z_{n_r} (Definition 2), drawn by the caller after the
+ * candidates arrive (Algorithm 1). */
+typedef struct {
+    const float *features; /* device, [n_r x dims[0]] row-major binary32 (least squares: A [n_r x d]) */
+    const void *targets;   /* device, int32 labels[n_r] in [0, dims[L]) (MLP) or float y[n_r] (least squares) */
+    int32_t n_r;
+} zeno_batch;
+
+typedef struct zeno_context *zeno_handle;
+
+/* Number of parameters d implied by a model description (0 if it is invalid). */
+int64_t zeno_param_count(const zeno_model_desc *desc);
+
+/* Creates a handle for one model shape on CUDA device `device` and allocates its
+ * workspace for up to m_max candidates and n_r_max server samples.
+ * INVALID_ARG: NULL arguments, m_max outside [1, ZENO_MAX_CANDIDATES], n_r_max < 1,
+ * bad layer sizes.  UNSUPPORTED: unknown kind/dtype, least squares with bfloat16.
+ * WORKSPACE / CUDA: allocation failed (the handle is not created). */
+zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m_max,
+                        int32_t n_r_max, int32_t device);
+
+/* Frees the workspace.  The caller makes sure no call on the handle is in flight. */
+zeno_status zeno_destroy(zeno_handle h);
+
+/* Definition 2 for all m candidates:
+ *   losses[0] = f_r(x), losses[1+i] = f_r(x - gamma v_i), norms[i] = ||v_i||^2,
+ *   scores[i] = losses[0] - losses[1+i] - rho * norms[i].
+ * f_r(x) is evaluated once and shared ((m+1) n_r sample evaluations in all,
+ * the paper's cost model).  The m perturbed models are never materialised:
+ * x - gamma v_i is formed inside the operand load, and ||v_i||^2 is accumulated
+ * in the same pass over V.
+ * x: [d]; V: [m x ldv]; scores: float[m] (required); losses: float[m+1] or NULL;
+ * norms: float[m] or NULL.
+ * INVALID_ARG: NULL x/V/batch/features/targets/scores, m < 1 or > m_max,
+ * n_r < 1 or > n_r_max, ldv < d, rho < 0 (the theory uses rho = 0 for convex
+ * losses, so 0 is accepted), gamma or rho not finite.
+ * Labels outside [0, classes) are not detected; the loss of that sample is then
+ * computed against class 0. */
+zeno_status zeno_score(zeno_handle h, const void *x, const void *V, int64_t ldv, int32_t m,
+                       const zeno_batch *batch, float gamma, float rho, float *scores,
+                       float *losses, float *norms, void *stream);
+
+/* Definition 3, the ranking: idx[0..m-b) = the candidates with the m - b highest
+ * scores in rank order.  The paper's ">=" leaves ties open; here a higher score
+ * comes first, equal scores keep index order, and a NaN score ranks as minus
+ * infinity.  Runs in one thread block (bitonic network on (score, index) keys).
+ * INVALID_ARG: NULL pointers, m < 1 or > m_max, b < 0 or b >= m (the paper needs
+ * m > b >= q; q is unknown to the server, so only m > b >= 0 is checked). */
+zeno_status zeno_select(zeno_handle h, const float *scores, int32_t m, int32_t b, int32_t *idx,
+                        void *stream);
+
+/* Definition 3, the average: out[j] = (1/k) sum_{r<k} V[idx[r]][j] for j < d,
+ * in binary32 whatever the storage type of V.  Only the k selected rows are
+ * read.  idx is a device array; entries outside [0, m) are skipped (their row
+ * contributes zero) rather than dereferenced.
+ * INVALID_ARG: NULL pointers, k < 1 or k > m, m > m_max, ldv < d. */
+zeno_status zeno_aggregate(zeno_handle h, const void *V, int64_t ldv, int32_t m,
+                           const int32_t *idx, int32_t k, float *out, void *stream);
+
+/* Zeno_b({v_i}) = score -> select -> aggregate on one stream, no host round trip.
+ * out: float[d] (required); scores: float[m] or NULL; idx: int32[m-b] or NULL.
+ * The SGD update x <- x - gamma * out (Algorithm 1) is left to the caller. */
+zeno_status zeno_step(zeno_handle h, const void *x, const void *V, int64_t ldv, int32_t m,
+                      const zeno_batch *batch, float gamma, float rho, int32_t b, float *out,
+                      float *scores, int32_t *idx, void *stream);
+
+/* Kernels launched by the most recent call on this handle (0 after an error). */
+int32_t zeno_last_launch_count(zeno_handle h);
+
+/* The cudaError_t (as int) behind the most recent ZENO_ERR_CUDA on this handle. */
+int32_t zeno_last_cuda_error(zeno_handle h);
+
+const char *zeno_status_string(zeno_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ZENO_H_ */

@@ -1,0 +1,334 @@
+/*
+ * zeno_oracle.c -- TEST INFRASTRUCTURE, not part of the product.
+ *
+ * A plain, slow, float64 statement of the Zeno aggregation rule
+ * (Xie, Koyejo, Gupta: "Zeno: Distributed SGD with Suspicion-based
+ * Fault-tolerance"), written from the paper's definitions so that it can be
+ * checked against them by eye:
+ *
+ *   Definition 2 (stochastic descendant score)
+ *       Score_{gamma,rho}(u, x) = f_r(x) - f_r(x - gamma u) - rho ||u||^2,
+ *       f_r(x) = (1/n_r) sum_{i<=n_r} f(x; z_i),  all norms l2 (Table 1).
+ *   Definition 3 (suspicion-based aggregation)
+ *       sort the candidates by score, descending; average the first m-b.
+ *
+ * Every candidate is evaluated on its own, from the definition: the
+ * perturbed parameter vector x - gamma*v_i is formed, the loss is evaluated
+ * on it, nothing is shared between candidates except f_r(x), nothing is
+ * blocked, fused or reordered.  All arithmetic is double precision; inputs
+ * (float32 or bfloat16 storage) are promoted exactly.
+ *
+ * Only the tests, the smoke check and the benchmark's CPU-baseline leg use
+ * this file.  It shares no code, header, table or constant with the CUDA
+ * library.
+ *
+ * Pins (tests/test_oracle_pins.py): every function below is pinned -- see the
+ * list in that file.  Nothing here is "parity unpinned".
+ *
+ * Parameter-vector layout (the one both sides agree on): x and every row of
+ * V are the flat concatenation, layer by layer, of W_l stored [out_l x in_l]
+ * row-major followed by b_l[out_l] (if has_bias).  Least squares: just x[d].
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum { ZO_LOSS_SOFTMAX_MLP = 0, ZO_LOSS_LEAST_SQUARES = 1 };
+enum { ZO_F32 = 0, ZO_BF16 = 1 };
+enum { ZO_OK = 0, ZO_BAD_ARG = 1, ZO_NO_MEM = 2 };
+
+/* number of single-sample loss evaluations f(.; z_j) performed since the last
+ * reset; the paper's cost model is (m+1) * n_r of them per step (Discussion:
+ * "21 x 4 = 84" for m = 20, n_r = 4). */
+static long long zo_sample_evals = 0;
+void zo_reset_eval_count(void) { zo_sample_evals = 0; }
+long long zo_eval_count(void) { return zo_sample_evals; }
+
+int zo_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* ---- storage formats ---------------------------------------------------- */
+
+static double zo_bf16_bits_to_double(uint16_t h)
+{
+    uint32_t u = (uint32_t)h << 16; /* bfloat16 = the upper half of a binary32 */
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/* one stored parameter, promoted exactly */
+static double zo_load(const void *p, int64_t i, int dtype)
+{
+    if (dtype == ZO_BF16)
+        return zo_bf16_bits_to_double(((const uint16_t *)p)[i]);
+    return (double)((const float *)p)[i];
+}
+
+/* Round a binary32 value to the nearest bfloat16 (8 significant bits, binary32
+ * exponent range), ties to even, written from the format's definition:
+ * find the spacing of bfloat16 numbers around |f| and round f to a multiple
+ * of it with the current (to-nearest-even) rounding mode. */
+double zo_round_to_bf16(float f)
+{
+    double a = fabs((double)f);
+    if (!(a == a) || isinf(a) || a == 0.0)
+        return (double)f;
+    int e;
+    frexp(a, &e);            /* a = frac * 2^e, frac in [0.5, 1)  =>  2^(e-1) <= a < 2^e */
+    int ulp_exp = (e - 1) - 7; /* 8 significant bits */
+    if (ulp_exp < -126 - 7)
+        ulp_exp = -126 - 7;  /* subnormal range: fixed spacing 2^-133 */
+    double q = nearbyint(ldexp(a, -ulp_exp)); /* exact scaling, ties to even */
+    double r = ldexp(q, ulp_exp);
+    if (r >= ldexp(1.0, 128))
+        r = INFINITY;        /* past the largest finite bfloat16 */
+    return f < 0 ? -r : r;
+}
+
+/* ---- the candidate's parameter vector ----------------------------------- */
+
+/* w = x - gamma * v, element by element (Definition 2's argument x - gamma u).
+ * v == NULL gives w = x.
+ * float32 storage: exact double arithmetic on the promoted values.
+ * bfloat16 storage: the candidate is itself a bfloat16 model; its entries are
+ * the difference rounded once to binary32 (the precision the quantisation
+ * decision is taken in) and then to bfloat16. */
+void zo_candidate_params(const void *x, const void *v, int64_t d, int dtype,
+                         double gamma, double *w)
+{
+    for (int64_t j = 0; j < d; ++j) {
+        double xj = zo_load(x, j, dtype);
+        if (!v) { w[j] = xj; continue; }
+        double vj = zo_load(v, j, dtype);
+        double diff = xj - gamma * vj;
+        if (dtype == ZO_BF16)
+            diff = zo_round_to_bf16((float)diff);
+        w[j] = diff;
+    }
+}
+
+int64_t zo_param_count(int kind, int n_layers, const int64_t *dims, int has_bias)
+{
+    if (kind == ZO_LOSS_LEAST_SQUARES)
+        return dims[0];
+    int64_t d = 0;
+    for (int l = 0; l < n_layers; ++l)
+        d += dims[l + 1] * dims[l] + (has_bias ? dims[l + 1] : 0);
+    return d;
+}
+
+/* ---- f_r ---------------------------------------------------------------- */
+
+/* Softmax cross-entropy of a ReLU multi-layer perceptron, one sample.
+ * h: the sample's features [dims[0]].  scratch: two buffers of max(dims). */
+static double zo_mlp_sample_loss(const double *w, int n_layers, const int64_t *dims,
+                                 int has_bias, const float *feat, int32_t label,
+                                 double *buf0, double *buf1)
+{
+    double *h = buf0, *z = buf1;
+    for (int64_t k = 0; k < dims[0]; ++k)
+        h[k] = (double)feat[k];
+    const double *p = w;
+    for (int l = 0; l < n_layers; ++l) {
+        int64_t in = dims[l], out = dims[l + 1];
+        const double *W = p;
+        const double *bias = has_bias ? p + out * in : NULL;
+        for (int64_t o = 0; o < out; ++o) {
+            double acc = 0.0;
+            for (int64_t k = 0; k < in; ++k)
+                acc += W[o * in + k] * h[k];
+            if (bias)
+                acc += bias[o];
+            if (l + 1 < n_layers && !(acc > 0.0))
+                acc = (acc == acc) ? 0.0 : acc; /* ReLU; a NaN stays a NaN */
+            z[o] = acc;
+        }
+        p += out * in + (has_bias ? out : 0);
+        double *t = h; h = z; z = t;
+    }
+    /* h now holds the logits: loss = log sum_c exp(z_c) - z_label */
+    int64_t C = dims[n_layers];
+    double zmax = h[0];
+    for (int64_t c = 1; c < C; ++c)
+        if (h[c] > zmax) zmax = h[c];
+    double se = 0.0;
+    for (int64_t c = 0; c < C; ++c)
+        se += exp(h[c] - zmax);
+    return zmax + log(se) - h[label];
+}
+
+/* f_r(w) = (1/n_r) sum_j f(w; z_j)   (Definition 2).
+ * kind 0: targets = int32 labels[n_r]; features [n_r x dims[0]] float32.
+ * kind 1: f(w; (a_j, y_j)) = (a_j . w - y_j)^2 / 2, features = A [n_r x d],
+ *         targets = float32 y[n_r], so that f_r = ||A w - y||^2 / (2 n_r). */
+double zo_loss(int kind, int n_layers, const int64_t *dims, int has_bias,
+               const double *w, const float *features, const void *targets, int n_r)
+{
+    double total = 0.0;
+    if (kind == ZO_LOSS_LEAST_SQUARES) {
+        int64_t d = dims[0];
+        const float *y = (const float *)targets;
+        for (int j = 0; j < n_r; ++j) {
+            double acc = 0.0;
+            for (int64_t k = 0; k < d; ++k)
+                acc += (double)features[(int64_t)j * d + k] * w[k];
+            double r = acc - (double)y[j];
+            total += 0.5 * r * r;
+        }
+    } else {
+        int64_t widest = 0;
+        for (int l = 0; l <= n_layers; ++l)
+            if (dims[l] > widest) widest = dims[l];
+        double *buf0 = (double *)malloc(sizeof(double) * (size_t)widest);
+        double *buf1 = (double *)malloc(sizeof(double) * (size_t)widest);
+        if (!buf0 || !buf1) { free(buf0); free(buf1); return NAN; }
+        const int32_t *labels = (const int32_t *)targets;
+        for (int j = 0; j < n_r; ++j)
+            total += zo_mlp_sample_loss(w, n_layers, dims, has_bias,
+                                        features + (int64_t)j * dims[0], labels[j], buf0, buf1);
+        free(buf0);
+        free(buf1);
+    }
+#pragma omp atomic
+    zo_sample_evals += n_r;
+    return total / (double)n_r;
+}
+
+/* ---- Definition 2: scores ------------------------------------------------ */
+
+/* scores[i] = f_r(x) - f_r(x - gamma v_i) - rho ||v_i||^2 for i < m.
+ * losses (optional, [m+1]): losses[0] = f_r(x), losses[1+i] = f_r(x - gamma v_i).
+ * norms  (optional, [m])  : ||v_i||^2.
+ * V is [m x ldv] row-major in the storage dtype; columns >= d are padding.
+ * Candidates are independent; they are spread over the host threads. */
+int zo_score(int kind, int dtype, int n_layers, const int64_t *dims, int has_bias,
+             const void *x, const void *V, int64_t ldv, int m,
+             const float *features, const void *targets, int n_r,
+             double gamma, double rho,
+             double *scores, double *losses, double *norms)
+{
+    if (m < 1 || n_r < 1 || !x || !V || !features || !targets || !scores)
+        return ZO_BAD_ARG;
+    int64_t d = zo_param_count(kind, n_layers, dims, has_bias);
+    if (ldv < d)
+        return ZO_BAD_ARG;
+    size_t esz = dtype == ZO_BF16 ? 2 : 4;
+    int rc = ZO_OK;
+
+    double *w0 = (double *)malloc(sizeof(double) * (size_t)d);
+    if (!w0) return ZO_NO_MEM;
+    zo_candidate_params(x, NULL, d, dtype, 0.0, w0);
+    double f0 = zo_loss(kind, n_layers, dims, has_bias, w0, features, targets, n_r);
+    free(w0);
+    if (losses) losses[0] = f0;
+
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int i = 0; i < m; ++i) {
+        const void *vi = (const char *)V + (size_t)i * (size_t)ldv * esz;
+        double *w = (double *)malloc(sizeof(double) * (size_t)d);
+        if (!w) {
+#pragma omp atomic write
+            rc = ZO_NO_MEM;
+            continue;
+        }
+        zo_candidate_params(x, vi, d, dtype, gamma, w);
+        double fi = zo_loss(kind, n_layers, dims, has_bias, w, features, targets, n_r);
+        free(w);
+        double nrm = 0.0;
+        for (int64_t j = 0; j < d; ++j) {
+            double vj = zo_load(vi, j, dtype);
+            nrm += vj * vj;
+        }
+        scores[i] = f0 - fi - rho * nrm;
+        if (losses) losses[1 + i] = fi;
+        if (norms) norms[i] = nrm;
+    }
+    return rc;
+}
+
+/* ---- Definition 3: ranking ----------------------------------------------- */
+
+/* idx[0..m-b) = the candidates with the m-b highest scores, in rank order.
+ * The paper's ">=" leaves ties open; the reading taken here: higher score
+ * first, then lower index; a NaN score counts as minus infinity.
+ * Plain stable insertion sort of the index list. */
+int zo_select(const double *scores, int m, int b, int32_t *idx)
+{
+    if (m < 1 || b < 0 || b >= m || !scores || !idx)
+        return ZO_BAD_ARG;
+    int32_t *order = (int32_t *)malloc(sizeof(int32_t) * (size_t)m);
+    double *key = (double *)malloc(sizeof(double) * (size_t)m);
+    if (!order || !key) { free(order); free(key); return ZO_NO_MEM; }
+    for (int i = 0; i < m; ++i)
+        key[i] = (scores[i] == scores[i]) ? scores[i] : -INFINITY;
+    for (int i = 0; i < m; ++i) {
+        int pos = i;
+        /* move left past strictly smaller keys only: equal keys keep index order */
+        while (pos > 0 && key[order[pos - 1]] < key[i]) {
+            order[pos] = order[pos - 1];
+            --pos;
+        }
+        order[pos] = i;
+    }
+    for (int r = 0; r < m - b; ++r)
+        idx[r] = order[r];
+    free(order);
+    free(key);
+    return ZO_OK;
+}
+
+/* ---- Definition 3: trimmed average --------------------------------------- */
+
+/* out[j] = (1/k) sum_{r<k} V[idx[r]][j],  j < d. */
+int zo_aggregate(int dtype, const void *V, int64_t ldv, int64_t d, int m,
+                 const int32_t *idx, int k, double *out)
+{
+    if (k < 1 || !V || !idx || !out || ldv < d)
+        return ZO_BAD_ARG;
+    size_t esz = dtype == ZO_BF16 ? 2 : 4;
+    for (int r = 0; r < k; ++r)
+        if (idx[r] < 0 || idx[r] >= m) return ZO_BAD_ARG;
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < d; ++j) {
+        double acc = 0.0;
+        for (int r = 0; r < k; ++r) {
+            const void *row = (const char *)V + (size_t)idx[r] * (size_t)ldv * esz;
+            acc += zo_load(row, j, dtype);
+        }
+        out[j] = acc / (double)k;
+    }
+    return ZO_OK;
+}
+
+/* ---- the whole step: Zeno_b({v_i}) ---------------------------------------- */
+
+int zo_step(int kind, int dtype, int n_layers, const int64_t *dims, int has_bias,
+            const void *x, const void *V, int64_t ldv, int m,
+            const float *features, const void *targets, int n_r,
+            double gamma, double rho, int b,
+            double *out, double *scores, int32_t *idx)
+{
+    if (b < 0 || b >= m) return ZO_BAD_ARG;
+    int64_t d = zo_param_count(kind, n_layers, dims, has_bias);
+    double *s = scores ? scores : (double *)malloc(sizeof(double) * (size_t)m);
+    int32_t *ix = idx ? idx : (int32_t *)malloc(sizeof(int32_t) * (size_t)(m - b));
+    if (!s || !ix) return ZO_NO_MEM;
+    int rc = zo_score(kind, dtype, n_layers, dims, has_bias, x, V, ldv, m,
+                      features, targets, n_r, gamma, rho, s, NULL, NULL);
+    if (rc == ZO_OK) rc = zo_select(s, m, b, ix);
+    if (rc == ZO_OK) rc = zo_aggregate(dtype, V, ldv, d, m, ix, m - b, out);
+    if (!scores) free(s);
+    if (!idx) free(ix);
+    return rc;
+}

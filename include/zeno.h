@@ -143,6 +143,27 @@ zeno_status zeno_step(zeno_handle h, const void *x, const void *V, int64_t ldv, 
                       const zeno_batch *batch, float gamma, float rho, int32_t b, float *out,
                       float *scores, int32_t *idx, void *stream);
 
+/* The same step for a caller whose data lives in HOST memory (Algorithm 1's server receiving the
+ * candidates over the network): x, V, features, targets, out, scores and idx are HOST pointers
+ * (pinned memory makes the copies asynchronous).  The call copies the inputs to a device staging
+ * area owned by the handle (allocated or grown on first need -- the only allocation outside
+ * zeno_create), enqueues the step, copies out[d] (and scores[m], idx[m-b] if not NULL) back and
+ * synchronises the stream before returning.  Same argument checks as zeno_step. */
+zeno_status zeno_step_host(zeno_handle h, const void *x, const void *V, int64_t ldv, int32_t m,
+                           const float *features, const void *targets, int32_t n_r, float gamma,
+                           float rho, int32_t b, float *out, float *scores, int32_t *idx,
+                           void *stream);
+
+/* Per-kernel timing for benchmarks.  zeno_profile(h, 1) makes every later call on the handle
+ * record a CUDA event on the call's stream before each of its kernels and after the last one
+ * (a few microseconds of overhead per call); zeno_profile(h, 0) switches it off again.
+ * zeno_profile_read waits for the most recent call's last event (a host synchronisation) and
+ * writes, for up to `cap` kernels in launch order, the elapsed milliseconds ms[i] and a static
+ * name names[i] (either array may be NULL).  Returns the number of kernels written, 0 if
+ * profiling is off or nothing was recorded, -1 on a CUDA error. */
+zeno_status zeno_profile(zeno_handle h, int32_t enable);
+int32_t zeno_profile_read(zeno_handle h, float *ms, const char **names, int32_t cap);
+
 /* Kernels launched by the most recent call on this handle (0 after an error). */
 int32_t zeno_last_launch_count(zeno_handle h);
 

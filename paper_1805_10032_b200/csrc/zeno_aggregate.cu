@@ -1,0 +1,154 @@
+// Definition 3, the average: out[j] = (1/k) sum_{r<k} V[idx[r]][j], binary32 output.
+//
+// Pure streaming: only the k selected rows of V are read, each element once, with 16-byte
+// loads when the rows allow it.  A thread owns one 16-byte column group and walks the k rows,
+// so k independent loads are in flight per thread and consecutive threads read consecutive
+// addresses of the same row.  Rows are added in rank order, in binary32.
+#include "zeno_internal.h"
+
+namespace zeno {
+
+namespace {
+
+template <typename T> struct Group;           // one 16-byte group of columns
+template <> struct Group<float> {
+    static constexpr int kElems = 4;
+    __device__ static void load(const float *p, float (&o)[4]) {
+        float4 t = __ldcs(reinterpret_cast<const float4 *>(p));
+        o[0] = t.x; o[1] = t.y; o[2] = t.z; o[3] = t.w;
+    }
+};
+template <> struct Group<__nv_bfloat16> {
+    static constexpr int kElems = 8;
+    __device__ static void load(const __nv_bfloat16 *p, float (&o)[8]) {
+        uint4 t = __ldcs(reinterpret_cast<const uint4 *>(p));
+        const unsigned w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            o[2 * q] = __uint_as_float(w[q] << 16);
+            o[2 * q + 1] = __uint_as_float(w[q] & 0xffff0000u);
+        }
+    }
+};
+
+// rows_s[r] = element offset of selected row r, or -1 for an index outside [0, m)
+__device__ __forceinline__ void stage_rows(const int32_t *idx, int k, int m, int64_t ldv,
+                                           int64_t *rows_s) {
+    for (int r = threadIdx.x; r < k; r += blockDim.x) {
+        int i = idx[r];
+        rows_s[r] = (i >= 0 && i < m) ? (int64_t)i * ldv : -1;
+    }
+    __syncthreads();
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) aggregate_vec_kernel(const T *V, int64_t ldv, int64_t d, int m,
+                                                             const int32_t *idx, int k, float *out) {
+    constexpr int E = Group<T>::kElems;
+    __shared__ int64_t rows_s[ZENO_MAX_CANDIDATES];
+    stage_rows(idx, k, m, ldv, rows_s);
+    const int64_t groups = d / E;            // whole groups; the d % E tail columns follow below
+    for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < groups;
+         g += (int64_t)gridDim.x * blockDim.x) {
+        float acc[E];
+#pragma unroll
+        for (int e = 0; e < E; ++e) acc[e] = 0.f;
+        int r = 0;
+        for (; r + 4 <= k; r += 4) {         // four rows in flight per step
+            float v[4][E];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                int64_t off = rows_s[r + q];
+                if (off >= 0) {
+                    Group<T>::load(V + off + g * E, v[q]);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < E; ++e) v[q][e] = 0.f;
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+#pragma unroll
+                for (int e = 0; e < E; ++e) acc[e] += v[q][e];
+        }
+        for (; r < k; ++r) {
+            int64_t off = rows_s[r];
+            if (off < 0) continue;
+            float v[E];
+            Group<T>::load(V + off + g * E, v);
+#pragma unroll
+            for (int e = 0; e < E; ++e) acc[e] += v[e];
+        }
+        float4 *o = reinterpret_cast<float4 *>(out + g * E);
+#pragma unroll
+        for (int q = 0; q < E / 4; ++q)
+            o[q] = make_float4(acc[4 * q] / (float)k, acc[4 * q + 1] / (float)k,
+                               acc[4 * q + 2] / (float)k, acc[4 * q + 3] / (float)k);
+    }
+    // tail columns (fewer than one group), one per thread of block 0
+    if (blockIdx.x == 0) {
+        const int64_t j = groups * E + threadIdx.x;
+        if (j < d) {
+            float acc = 0.f;
+            for (int r = 0; r < k; ++r) {
+                int64_t off = rows_s[r];
+                if (off >= 0) acc += load_elem(V + off + j);
+            }
+            out[j] = acc / (float)k;
+        }
+    }
+}
+
+// Any ldv >= d, any d: one element per thread.
+template <typename T>
+__global__ void __launch_bounds__(256) aggregate_scalar_kernel(const T *V, int64_t ldv, int64_t d,
+                                                                int m, const int32_t *idx, int k,
+                                                                float *out) {
+    __shared__ int64_t rows_s[ZENO_MAX_CANDIDATES];
+    stage_rows(idx, k, m, ldv, rows_s);
+    for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < d;
+         j += (int64_t)gridDim.x * blockDim.x) {
+        float acc = 0.f;
+        for (int r = 0; r < k; ++r) {
+            int64_t off = rows_s[r];
+            if (off >= 0) acc += load_elem(V + off + j);
+        }
+        out[j] = acc / (float)k;
+    }
+}
+
+template <typename T>
+cudaError_t launch_typed(const Context &c, const T *V, int64_t ldv, int m, const int32_t *idx, int k,
+                         float *out, bool aligned, cudaStream_t s) {
+    const int sms = c.sm_count > 0 ? c.sm_count : 148;
+    const int64_t d = c.d;
+    constexpr int E = Group<T>::kElems;
+    if (aligned) {
+        int64_t want = (d / E + 255) / 256;
+        int64_t cap = (int64_t)sms * 8;
+        int blocks = (int)(want < cap ? want : cap);
+        if (blocks < 1) blocks = 1;
+        aggregate_vec_kernel<T><<<blocks, 256, 0, s>>>(V, ldv, d, m, idx, k, out);
+    } else {
+        int64_t want = (d + 255) / 256;
+        int64_t cap = (int64_t)sms * 8;
+        int blocks = (int)(want < cap ? want : cap);
+        if (blocks < 1) blocks = 1;
+        aggregate_scalar_kernel<T><<<blocks, 256, 0, s>>>(V, ldv, d, m, idx, k, out);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_aggregate(Context &c, const void *V, int64_t ldv, int m,
+                             const int32_t *idx, int k, float *out, bool aligned, cudaStream_t s,
+                             int *launches) {
+    ++*launches;
+    profile_mark(c, "aggregate", s);
+    if (c.desc.param_dtype == ZENO_BF16)
+        return launch_typed(c, static_cast<const __nv_bfloat16 *>(V), ldv, m, idx, k, out, aligned, s);
+    return launch_typed(c, static_cast<const float *>(V), ldv, m, idx, k, out, aligned, s);
+}
+
+}  // namespace zeno

@@ -1,0 +1,457 @@
+// C ABI of the Zeno aggregation step: argument checks, workspace, and the order in which the
+// kernels are enqueued.  No arithmetic of the method lives here.
+#include <math.h>
+#include <new>
+#include <string.h>
+
+#include "zeno_internal.h"
+
+using zeno::Context;
+
+struct zeno_context : public Context {};
+
+namespace {
+
+constexpr size_t kAlign = 256;
+
+size_t round_up(size_t n, size_t q) { return (n + q - 1) / q * q; }
+
+size_t elem_size(int dtype) { return dtype == ZENO_BF16 ? 2 : 4; }
+
+bool desc_ok(const zeno_model_desc *d) {
+    if (!d) return false;
+    if (d->kind == ZENO_LOSS_LEAST_SQUARES) return d->dims[0] >= 1;
+    if (d->kind != ZENO_LOSS_SOFTMAX_MLP) return false;
+    if (d->n_layers < 1 || d->n_layers > ZENO_MAX_LAYERS) return false;
+    for (int l = 0; l <= d->n_layers; ++l)
+        if (d->dims[l] < 1 || d->dims[l] > (int64_t)1 << 30) return false;
+    return true;
+}
+
+bool is_aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// Switches to the handle's device for the duration of a call and back afterwards.
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    cudaError_t err = cudaSuccess;
+    explicit DeviceGuard(int dev) {
+        err = cudaGetDevice(&prev);
+        if (err == cudaSuccess && prev != dev) {
+            err = cudaSetDevice(dev);
+            switched = err == cudaSuccess;
+        }
+    }
+    ~DeviceGuard() {
+        if (switched) cudaSetDevice(prev);
+    }
+};
+
+// Per-kernel timing: a call starts a fresh list of events and closes it after its last kernel.
+void profile_begin(Context *c) { c->profiled = 0; }
+void profile_end(Context *c, cudaStream_t s) {
+    if (c->profile) cudaEventRecord(c->events[c->profiled], s);
+}
+
+zeno_status fail_cuda(Context *c, cudaError_t e) {
+    c->last_cuda_error = (int)e;
+    c->last_launches = 0;
+    return ZENO_ERR_CUDA;
+}
+
+// The 4-element vector loads of the scoring kernels need every row of every layer (and the
+// rows of V) to start on a multiple of 4 elements.
+bool score_rows_aligned(const Context &c, const void *x, const void *V, int64_t ldv,
+                        const float *features) {
+    const size_t vec_bytes = 4 * elem_size(c.desc.param_dtype);
+    if (!is_aligned(x, vec_bytes) || !is_aligned(V, vec_bytes) || !is_aligned(features, 16)) return false;
+    if (ldv % 4 != 0) return false;
+    if (c.desc.kind == ZENO_LOSS_LEAST_SQUARES) return c.d % 4 == 0;
+    for (int l = 0; l < c.desc.n_layers; ++l)
+        if (c.offW[l] % 4 != 0 || c.desc.dims[l] % 4 != 0) return false;
+    return true;
+}
+
+bool aggregate_rows_aligned(const Context &c, const void *V, int64_t ldv, const float *out) {
+    return is_aligned(V, 16) && is_aligned(out, 16) && (ldv * elem_size(c.desc.param_dtype)) % 16 == 0;
+}
+
+zeno_status check_common(const Context *c, const void *V, int64_t ldv, int32_t m) {
+    if (!c || !V) return ZENO_ERR_INVALID_ARG;
+    if (m < 1 || m > c->m_max) return ZENO_ERR_INVALID_ARG;
+    if (ldv < c->d) return ZENO_ERR_INVALID_ARG;
+    return ZENO_OK;
+}
+
+zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv, int32_t m,
+                          const zeno_batch *batch, float gamma, float rho, float *scores,
+                          float *losses, float *norms, cudaStream_t s, int *launches) {
+    zeno_status st = check_common(c, V, ldv, m);
+    if (st != ZENO_OK) return st;
+    if (!x || !batch || !batch->features || !batch->targets || !scores) return ZENO_ERR_INVALID_ARG;
+    if (batch->n_r < 1 || batch->n_r > c->n_r_max) return ZENO_ERR_INVALID_ARG;
+    if (!isfinite(gamma) || !isfinite(rho) || rho < 0.f) return ZENO_ERR_INVALID_ARG;
+
+    const int n_r = batch->n_r;
+    const bool aligned = score_rows_aligned(*c, x, V, ldv, batch->features);
+    float *loss_buf = losses ? losses : c->losses;
+    cudaError_t e = cudaSuccess;
+
+    if (c->desc.kind == ZENO_LOSS_LEAST_SQUARES) {
+        zeno::LsqArgs a;
+        a.x = static_cast<const float *>(x);
+        a.V = static_cast<const float *>(V);
+        a.ldv = ldv;
+        a.d = c->d;
+        a.A = batch->features;
+        a.n_r = n_r;
+        a.m = m;
+        a.part = c->lsq_part;
+        a.slabs = c->lsq_slabs;
+        e = zeno::launch_lsq_score(*c, a, static_cast<const float *>(batch->targets), gamma, rho,
+                                   aligned, loss_buf, norms, scores, s, launches);
+        return e == cudaSuccess ? ZENO_OK : fail_cuda(c, e);
+    }
+
+    const int L = c->desc.n_layers;
+    for (int l = 0; l < L; ++l) {
+        zeno::LayerArgs a;
+        a.x = x;
+        a.V = V;
+        a.ldv = ldv;
+        a.offW = c->offW[l];
+        a.offB = c->offB[l];
+        a.in = (int)c->desc.dims[l];
+        a.out = (int)c->desc.dims[l + 1];
+        a.Hin = l == 0 ? batch->features : c->act[(l - 1) & 1];
+        a.hin_cand_stride = l == 0 ? 0 : (int64_t)n_r * a.in;
+        a.Hout = c->act[l & 1];
+        a.n_r = n_r;
+        a.m = m;
+        a.gamma = gamma;
+        a.relu = l + 1 < L;
+        a.normpart = c->normpart;
+        a.np_slots = c->np_slots;
+        a.np_base = c->np_base[l];
+        e = zeno::launch_mlp_layer(*c, a, aligned, s, launches);
+        if (e != cudaSuccess) return fail_cuda(c, e);
+    }
+    e = zeno::launch_mlp_loss(*c, c->act[(L - 1) & 1], static_cast<const int32_t *>(batch->targets),
+                              n_r, m, (int)c->desc.dims[L], loss_buf, s, launches);
+    if (e != cudaSuccess) return fail_cuda(c, e);
+    e = zeno::launch_mlp_finalize(*c, m, rho, loss_buf, scores, norms, s, launches);
+    return e == cudaSuccess ? ZENO_OK : fail_cuda(c, e);
+}
+
+zeno_status enqueue_select(Context *c, const float *scores, int32_t m, int32_t b, int32_t *idx,
+                           cudaStream_t s, int *launches) {
+    if (!c || !scores || !idx) return ZENO_ERR_INVALID_ARG;
+    if (m < 1 || m > c->m_max || b < 0 || b >= m) return ZENO_ERR_INVALID_ARG;
+    cudaError_t e = zeno::launch_select(*c, scores, m, b, idx, s, launches);
+    return e == cudaSuccess ? ZENO_OK : fail_cuda(c, e);
+}
+
+zeno_status enqueue_aggregate(Context *c, const void *V, int64_t ldv, int32_t m, const int32_t *idx,
+                              int32_t k, float *out, cudaStream_t s, int *launches) {
+    zeno_status st = check_common(c, V, ldv, m);
+    if (st != ZENO_OK) return st;
+    if (!idx || !out || k < 1 || k > m) return ZENO_ERR_INVALID_ARG;
+    cudaError_t e = zeno::launch_aggregate(*c, V, ldv, m, idx, k, out,
+                                           aggregate_rows_aligned(*c, V, ldv, out), s, launches);
+    return e == cudaSuccess ? ZENO_OK : fail_cuda(c, e);
+}
+
+}  // namespace
+
+extern "C" {
+
+int64_t zeno_param_count(const zeno_model_desc *desc) {
+    if (!desc_ok(desc)) return 0;
+    if (desc->kind == ZENO_LOSS_LEAST_SQUARES) return desc->dims[0];
+    int64_t d = 0;
+    for (int l = 0; l < desc->n_layers; ++l)
+        d += desc->dims[l + 1] * desc->dims[l] + (desc->has_bias ? desc->dims[l + 1] : 0);
+    return d;
+}
+
+zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m_max,
+                        int32_t n_r_max, int32_t device) {
+    if (!out) return ZENO_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!desc) return ZENO_ERR_INVALID_ARG;
+    if (desc->kind != ZENO_LOSS_SOFTMAX_MLP && desc->kind != ZENO_LOSS_LEAST_SQUARES)
+        return ZENO_ERR_UNSUPPORTED;
+    if (desc->param_dtype != ZENO_F32 && desc->param_dtype != ZENO_BF16) return ZENO_ERR_UNSUPPORTED;
+    if (desc->kind == ZENO_LOSS_LEAST_SQUARES && desc->param_dtype != ZENO_F32)
+        return ZENO_ERR_UNSUPPORTED;
+    if (!desc_ok(desc)) return ZENO_ERR_INVALID_ARG;
+    if (m_max < 1 || m_max > ZENO_MAX_CANDIDATES || n_r_max < 1 || device < 0)
+        return ZENO_ERR_INVALID_ARG;
+
+    zeno_context *c = new (std::nothrow) zeno_context();
+    if (!c) return ZENO_ERR_WORKSPACE;
+    memset(static_cast<Context *>(c), 0, sizeof(Context));
+    c->desc = *desc;
+    c->d = zeno_param_count(desc);
+    c->device = device;
+    c->m_max = m_max;
+    c->n_r_max = n_r_max;
+
+    DeviceGuard guard(device);
+    cudaDeviceProp prop;
+    cudaError_t e = guard.err != cudaSuccess ? guard.err : cudaGetDeviceProperties(&prop, device);
+    if (e != cudaSuccess) {
+        delete c;
+        return ZENO_ERR_CUDA;
+    }
+    c->sm_count = prop.multiProcessorCount;
+
+    const size_t rows = (size_t)m_max + 1;
+    size_t act_elems = 0, norm_elems = 0, lsq_elems = 0;
+    if (desc->kind == ZENO_LOSS_SOFTMAX_MLP) {
+        int64_t off = 0, widest = 0;
+        int slots = 0;
+        for (int l = 0; l < desc->n_layers; ++l) {
+            const int64_t in = desc->dims[l], o = desc->dims[l + 1];
+            c->offW[l] = off;
+            off += o * in;
+            c->offB[l] = desc->has_bias ? off : -1;
+            if (desc->has_bias) off += o;
+            c->np_base[l] = slots;
+            slots += zeno::mlp_norm_slots((int)o);
+            if (o > widest) widest = o;
+        }
+        c->np_slots = slots;
+        act_elems = rows * (size_t)n_r_max * (size_t)widest;
+        norm_elems = (size_t)m_max * (size_t)slots;
+    } else {
+        c->lsq_slabs = zeno::lsq_slab_count(*c);
+        lsq_elems = ((size_t)c->lsq_slabs + 1) * rows * ((size_t)n_r_max + 1);
+    }
+
+    size_t bytes = 0;
+    auto reserve = [&](size_t elems, size_t esz) {
+        size_t at = bytes;
+        bytes += round_up(elems * esz, kAlign);
+        return at;
+    };
+    const size_t at_act0 = reserve(act_elems, 4), at_act1 = reserve(act_elems, 4);
+    const size_t at_norm = reserve(norm_elems, 4), at_lsq = reserve(lsq_elems, 4);
+    const size_t at_loss = reserve(rows, 4), at_norms = reserve(m_max, 4);
+    const size_t at_scores = reserve(m_max, 4), at_idx = reserve(m_max, 4);
+
+    e = cudaMalloc(&c->arena, bytes);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        delete c;
+        return ZENO_ERR_WORKSPACE;
+    }
+    char *base = static_cast<char *>(c->arena);
+    c->act[0] = reinterpret_cast<float *>(base + at_act0);
+    c->act[1] = reinterpret_cast<float *>(base + at_act1);
+    c->normpart = reinterpret_cast<float *>(base + at_norm);
+    c->lsq_part = reinterpret_cast<float *>(base + at_lsq);
+    c->losses = reinterpret_cast<float *>(base + at_loss);
+    c->norms = reinterpret_cast<float *>(base + at_norms);
+    c->scores = reinterpret_cast<float *>(base + at_scores);
+    c->idx = reinterpret_cast<int32_t *>(base + at_idx);
+    *out = c;
+    return ZENO_OK;
+}
+
+zeno_status zeno_destroy(zeno_handle h) {
+    if (!h) return ZENO_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    cudaError_t e = cudaFree(h->arena);
+    if (h->host_stage) cudaFree(h->host_stage);
+    if (h->profile)
+        for (int i = 0; i <= zeno::kMaxProfiled; ++i) cudaEventDestroy(h->events[i]);
+    delete h;
+    return e == cudaSuccess ? ZENO_OK : ZENO_ERR_CUDA;
+}
+
+zeno_status zeno_score(zeno_handle h, const void *x, const void *V, int64_t ldv, int32_t m,
+                       const zeno_batch *batch, float gamma, float rho, float *scores,
+                       float *losses, float *norms, void *stream) {
+    if (!h) return ZENO_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+    int launches = 0;
+    profile_begin(h);
+    zeno_status st = enqueue_score(h, x, V, ldv, m, batch, gamma, rho, scores, losses, norms,
+                                   static_cast<cudaStream_t>(stream), &launches);
+    profile_end(h, static_cast<cudaStream_t>(stream));
+    h->last_launches = st == ZENO_OK ? launches : 0;
+    return st;
+}
+
+zeno_status zeno_select(zeno_handle h, const float *scores, int32_t m, int32_t b, int32_t *idx,
+                        void *stream) {
+    if (!h) return ZENO_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+    int launches = 0;
+    profile_begin(h);
+    zeno_status st = enqueue_select(h, scores, m, b, idx, static_cast<cudaStream_t>(stream), &launches);
+    profile_end(h, static_cast<cudaStream_t>(stream));
+    h->last_launches = st == ZENO_OK ? launches : 0;
+    return st;
+}
+
+zeno_status zeno_aggregate(zeno_handle h, const void *V, int64_t ldv, int32_t m, const int32_t *idx,
+                           int32_t k, float *out, void *stream) {
+    if (!h) return ZENO_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+    int launches = 0;
+    profile_begin(h);
+    zeno_status st = enqueue_aggregate(h, V, ldv, m, idx, k, out, static_cast<cudaStream_t>(stream),
+                                       &launches);
+    profile_end(h, static_cast<cudaStream_t>(stream));
+    h->last_launches = st == ZENO_OK ? launches : 0;
+    return st;
+}
+
+zeno_status zeno_step(zeno_handle h, const void *x, const void *V, int64_t ldv, int32_t m,
+                      const zeno_batch *batch, float gamma, float rho, int32_t b, float *out,
+                      float *scores, int32_t *idx, void *stream) {
+    if (!h || !out) return ZENO_ERR_INVALID_ARG;
+    if (m < 1 || m > h->m_max || b < 0 || b >= m) return ZENO_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    float *score_buf = scores ? scores : h->scores;
+    int32_t *idx_buf = idx ? idx : h->idx;
+    int launches = 0;
+    profile_begin(h);
+    zeno_status st = enqueue_score(h, x, V, ldv, m, batch, gamma, rho, score_buf, nullptr, nullptr, s,
+                                   &launches);
+    if (st == ZENO_OK) st = enqueue_select(h, score_buf, m, b, idx_buf, s, &launches);
+    if (st == ZENO_OK) st = enqueue_aggregate(h, V, ldv, m, idx_buf, m - b, out, s, &launches);
+    profile_end(h, s);
+    h->last_launches = st == ZENO_OK ? launches : 0;
+    return st;
+}
+
+zeno_status zeno_step_host(zeno_handle h, const void *x, const void *V, int64_t ldv, int32_t m,
+                           const float *features, const void *targets, int32_t n_r, float gamma,
+                           float rho, int32_t b, float *out, float *scores, int32_t *idx,
+                           void *stream) {
+    if (!h || !x || !V || !features || !targets || !out) return ZENO_ERR_INVALID_ARG;
+    if (m < 1 || m > h->m_max || b < 0 || b >= m || ldv < h->d) return ZENO_ERR_INVALID_ARG;
+    if (n_r < 1 || n_r > h->n_r_max) return ZENO_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t esz = elem_size(h->desc.param_dtype);
+    const size_t in0 = (size_t)h->desc.dims[0];
+    const size_t x_bytes = round_up((size_t)h->d * esz, kAlign);
+    const size_t v_bytes = round_up((size_t)m * (size_t)ldv * esz, kAlign);
+    const size_t f_bytes = round_up((size_t)n_r * in0 * 4, kAlign);
+    const size_t t_bytes = round_up((size_t)n_r * 4, kAlign);
+    const size_t o_bytes = round_up((size_t)h->d * 4, kAlign);
+    const size_t need = x_bytes + v_bytes + f_bytes + t_bytes + o_bytes;
+    cudaError_t e;
+    if (need > h->host_stage_bytes) {
+        // grown on demand; the previous staging area may still be in use by earlier work
+        e = cudaStreamSynchronize(s);
+        if (e != cudaSuccess) return fail_cuda(h, e);
+        if (h->host_stage) cudaFree(h->host_stage);
+        h->host_stage = nullptr;
+        h->host_stage_bytes = 0;
+        e = cudaMalloc(&h->host_stage, need);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            return ZENO_ERR_WORKSPACE;
+        }
+        h->host_stage_bytes = need;
+    }
+    char *p = static_cast<char *>(h->host_stage);
+    void *dx = p;
+    void *dV = p + x_bytes;
+    float *df = reinterpret_cast<float *>(p + x_bytes + v_bytes);
+    void *dt = p + x_bytes + v_bytes + f_bytes;
+    float *dout = reinterpret_cast<float *>(p + x_bytes + v_bytes + f_bytes + t_bytes);
+    e = cudaMemcpyAsync(dx, x, (size_t)h->d * esz, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dV, V, (size_t)m * (size_t)ldv * esz, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(df, features, (size_t)n_r * in0 * 4, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(dt, targets, (size_t)n_r * 4, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    zeno_batch batch;
+    batch.features = df;
+    batch.targets = dt;
+    batch.n_r = n_r;
+    int launches = 0;
+    profile_begin(h);
+    zeno_status st = enqueue_score(h, dx, dV, ldv, m, &batch, gamma, rho, h->scores, nullptr, nullptr, s,
+                                   &launches);
+    if (st == ZENO_OK) st = enqueue_select(h, h->scores, m, b, h->idx, s, &launches);
+    if (st == ZENO_OK) st = enqueue_aggregate(h, dV, ldv, m, h->idx, m - b, dout, s, &launches);
+    profile_end(h, s);
+    if (st != ZENO_OK) {
+        h->last_launches = 0;
+        return st;
+    }
+    e = cudaMemcpyAsync(out, dout, (size_t)h->d * 4, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess && scores)
+        e = cudaMemcpyAsync(scores, h->scores, (size_t)m * 4, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess && idx)
+        e = cudaMemcpyAsync(idx, h->idx, (size_t)(m - b) * 4, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    h->last_launches = launches;
+    return ZENO_OK;
+}
+
+zeno_status zeno_profile(zeno_handle h, int32_t enable) {
+    if (!h) return ZENO_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+    if (enable && !h->profile) {
+        for (int i = 0; i <= zeno::kMaxProfiled; ++i) {
+            cudaError_t e = cudaEventCreate(&h->events[i]);
+            if (e != cudaSuccess) {
+                for (int j = 0; j < i; ++j) cudaEventDestroy(h->events[j]);
+                return fail_cuda(h, e);
+            }
+        }
+        h->profile = true;
+    } else if (!enable && h->profile) {
+        for (int i = 0; i <= zeno::kMaxProfiled; ++i) cudaEventDestroy(h->events[i]);
+        h->profile = false;
+    }
+    h->profiled = 0;
+    return ZENO_OK;
+}
+
+int32_t zeno_profile_read(zeno_handle h, float *ms, const char **names, int32_t cap) {
+    if (!h || !h->profile || h->profiled == 0) return 0;
+    DeviceGuard guard(h->device);
+    if (cudaEventSynchronize(h->events[h->profiled]) != cudaSuccess) return -1;
+    int n = h->profiled < cap ? h->profiled : cap;
+    for (int i = 0; i < n; ++i) {
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, h->events[i], h->events[i + 1]) != cudaSuccess) return -1;
+        if (ms) ms[i] = t;
+        if (names) names[i] = h->kernel_names[i];
+    }
+    return n;
+}
+
+int32_t zeno_last_launch_count(zeno_handle h) { return h ? h->last_launches : 0; }
+
+int32_t zeno_last_cuda_error(zeno_handle h) { return h ? h->last_cuda_error : 0; }
+
+const char *zeno_status_string(zeno_status s) {
+    switch (s) {
+        case ZENO_OK: return "ok";
+        case ZENO_ERR_INVALID_ARG: return "invalid argument";
+        case ZENO_ERR_UNSUPPORTED: return "unsupported loss / dtype / shape";
+        case ZENO_ERR_WORKSPACE: return "workspace allocation failed";
+        case ZENO_ERR_CUDA: return "CUDA runtime error";
+        case ZENO_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

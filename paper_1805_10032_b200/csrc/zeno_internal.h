@@ -1,0 +1,147 @@
+// Internal declarations shared by the translation units of libzeno.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "zeno.h"
+
+namespace zeno {
+
+// Rows of V (and x) handled per warp in the CUDA-core kernels.
+constexpr int kRowsPerWarp = 4;
+// Warps per block in the layer kernel; one block covers kRowsPerWarp * kLayerWarps output rows.
+constexpr int kLayerWarps = 8;
+// Number of k-slabs the least-squares stream is cut into is at most this.
+constexpr int kMaxSlabs = 1024;
+// Most kernels one call can enqueue (layers + loss + finalize + select + aggregate).
+constexpr int kMaxProfiled = ZENO_MAX_LAYERS + 8;
+
+struct Context {
+    zeno_model_desc desc;
+    int64_t d;
+    int device;
+    int m_max, n_r_max;
+    int sm_count;
+    int64_t offW[ZENO_MAX_LAYERS];  // element offset of W_l inside a parameter vector
+    int64_t offB[ZENO_MAX_LAYERS];  // element offset of b_l, -1 without bias
+    int np_base[ZENO_MAX_LAYERS];   // first norm-partial slot of layer l
+    int np_slots;                   // norm-partial slots per candidate
+    void *arena;                    // the one device allocation everything below is carved from
+    float *act[2];                  // activations [m_max+1][n_r_max][widest layer output]
+    float *normpart;                // [m_max][np_slots] partial sums of v^2
+    float *lsq_part;                // [slabs][m_max+1][n_r_max+1] partial A.v and v^2
+    int lsq_slabs;
+    float *losses;                  // [m_max+1]
+    float *norms;                   // [m_max]
+    float *scores;                  // [m_max]
+    int32_t *idx;                   // [m_max]
+    void *host_stage;               // device copies of host inputs (zeno_step_host), grown on demand
+    size_t host_stage_bytes;
+    int last_launches;
+    int last_cuda_error;
+    // optional per-kernel timing (zeno_profile): events[i] is recorded before kernel i of a call,
+    // events[n] after the last one
+    bool profile;
+    cudaEvent_t events[kMaxProfiled + 1];
+    const char *kernel_names[kMaxProfiled];
+    int profiled;
+};
+
+// Records the event that closes the previous kernel and opens the next one.
+inline void profile_mark(Context &c, const char *name, cudaStream_t s) {
+    if (!c.profile || c.profiled >= kMaxProfiled) return;
+    cudaEventRecord(c.events[c.profiled], s);
+    c.kernel_names[c.profiled++] = name;
+}
+
+// One dense layer of all m+1 models (candidate 0 is x itself).
+struct LayerArgs {
+    const void *x;
+    const void *V;
+    int64_t ldv;
+    int64_t offW, offB;
+    int in, out;
+    const float *Hin;
+    int64_t hin_cand_stride;  // 0: the input activations are shared (layer 1)
+    float *Hout;              // [m+1][n_r][out]
+    int n_r, m;
+    float gamma;
+    int relu;
+    float *normpart;
+    int np_slots, np_base;
+};
+
+struct LsqArgs {
+    const float *x;
+    const float *V;
+    int64_t ldv;
+    int64_t d;
+    const float *A;
+    int n_r, m;
+    float *part;      // [slabs][m+1][n_r+1]; the last column holds the partial sum of squares
+    int slabs;
+};
+
+// Launchers return the cudaError_t of the launch; *launches is incremented per kernel.
+cudaError_t launch_mlp_layer(Context &c, const LayerArgs &a, bool aligned, cudaStream_t s,
+                             int *launches);
+cudaError_t launch_mlp_loss(Context &c, const float *logits, const int32_t *labels, int n_r,
+                            int m, int classes, float *losses, cudaStream_t s, int *launches);
+cudaError_t launch_mlp_finalize(Context &c, int m, float rho, const float *losses,
+                                float *scores, float *norms_out, cudaStream_t s, int *launches);
+cudaError_t launch_lsq_score(Context &c, const LsqArgs &a, const float *y, float gamma,
+                             float rho, bool aligned, float *losses, float *norms, float *scores,
+                             cudaStream_t s, int *launches);
+cudaError_t launch_select(Context &c, const float *scores, int m, int b, int32_t *idx, cudaStream_t s,
+                          int *launches);
+cudaError_t launch_aggregate(Context &c, const void *V, int64_t ldv, int m,
+                             const int32_t *idx, int k, float *out, bool aligned, cudaStream_t s,
+                             int *launches);
+
+int lsq_slab_count(const Context &c);
+int mlp_norm_slots(int out);
+
+// ---- device helpers shared by the kernels ------------------------------------------------
+
+#ifdef __CUDACC__
+
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t hi16_in_low) {
+    return __uint_as_float(hi16_in_low << 16);
+}
+
+__device__ __forceinline__ float load_elem(const float *p) { return __ldg(p); }
+__device__ __forceinline__ float load_elem(const __nv_bfloat16 *p) {
+    return bf16_bits_to_float(__ldg(reinterpret_cast<const unsigned short *>(p)));
+}
+
+// four consecutive elements starting at p (p must be aligned to 4 elements)
+__device__ __forceinline__ void load_vec4(const float *p, float (&o)[4]) {
+    float4 t = __ldg(reinterpret_cast<const float4 *>(p));
+    o[0] = t.x; o[1] = t.y; o[2] = t.z; o[3] = t.w;
+}
+__device__ __forceinline__ void load_vec4(const __nv_bfloat16 *p, float (&o)[4]) {
+    uint2 t = __ldg(reinterpret_cast<const uint2 *>(p));
+    o[0] = __uint_as_float(t.x << 16);
+    o[1] = __uint_as_float(t.x & 0xffff0000u);
+    o[2] = __uint_as_float(t.y << 16);
+    o[3] = __uint_as_float(t.y & 0xffff0000u);
+}
+
+template <typename T> struct is_bf16 { static constexpr bool value = false; };
+template <> struct is_bf16<__nv_bfloat16> { static constexpr bool value = true; };
+
+// One entry of the candidate's parameter vector, x - gamma v (Definition 2's argument).
+// bfloat16 models: the difference is rounded to binary32 by the fused multiply-add and then
+// to bfloat16, because the candidate is itself a bfloat16 model.
+template <typename T>
+__device__ __forceinline__ float candidate_param(float x, float v, float gamma) {
+    float w = fmaf(-gamma, v, x);
+    if (is_bf16<T>::value) w = __bfloat162float(__float2bfloat16_rn(w));
+    return w;
+}
+
+#endif  // __CUDACC__
+
+}  // namespace zeno

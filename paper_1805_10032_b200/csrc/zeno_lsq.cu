@@ -1,0 +1,284 @@
+// Scores for the least-squares loss f_r(x) = ||A x - y||^2 / (2 n_r) (Definition 2).
+//
+// The residual is linear in the parameters, A (x - gamma v_i) - y = (A x - y) - gamma A v_i,
+// so one streaming pass computes the n_r-by-(m+1) products A [x, v_1 .. v_m] together with the
+// squared norms of the rows of V.  Every element of A, x and V is read from HBM exactly once:
+// a block owns a contiguous slab of the index k, stages the A-chunk of that slab in shared
+// memory (cp.async, double buffered) and lets each warp stream kRowsPerWarp rows of [x; V]
+// against it with per-lane register accumulators.  Per-slab partial sums are written out and
+// combined in a fixed order (in double) by a one-block finishing kernel, which also forms the
+// losses and the scores.
+#include "zeno_internal.h"
+
+namespace zeno {
+
+namespace {
+
+constexpr int kStageFloats = 8192;   // floats of A per shared-memory stage (32 KB)
+constexpr int kIterK = 128;
+
+__device__ __forceinline__ void cp_async16(void *smem, const void *gmem, bool valid) {
+    unsigned s = static_cast<unsigned>(__cvta_generic_to_shared(smem));
+    int bytes = valid ? 16 : 0;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(s), "l"(gmem), "r"(bytes));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;\n" ::"n"(N));
+}
+
+template <int N>
+__device__ __forceinline__ float warp_transpose_reduce(float (&v)[N], int lane) {
+#pragma unroll
+    for (int s = N / 2; s >= 1; s >>= 1) {
+        const bool upper = (lane & s) != 0;
+#pragma unroll
+        for (int i = 0; i < s; ++i) {
+            float send = upper ? v[i] : v[i + s];
+            float keep = upper ? v[i + s] : v[i];
+            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, s);
+        }
+    }
+    float r = v[0];
+#pragma unroll
+    for (int s = N; s < 32; s <<= 1) r += __shfl_xor_sync(0xffffffffu, r, s);
+    return r;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int s = 16; s >= 1; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
+    return v;
+}
+
+template <bool VEC>
+__device__ __forceinline__ void load_row4(const float *row, int64_t kbase, int lane, int64_t K,
+                                          float (&o)[4]) {
+    if (VEC) {
+        int64_t k = kbase + 4 * lane;
+        if (k < K) {
+            // streamed once: keep it out of L1
+            float4 t = __ldcs(reinterpret_cast<const float4 *>(row + k));
+            o[0] = t.x; o[1] = t.y; o[2] = t.z; o[3] = t.w;
+        } else {
+            o[0] = o[1] = o[2] = o[3] = 0.f;
+        }
+    } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            int64_t k = kbase + 32 * e + lane;
+            o[e] = k < K ? __ldcs(row + k) : 0.f;
+        }
+    }
+}
+
+// Warps per block: bounded by the register file (RB * NRT accumulators per lane; the
+// register budget per thread is 65536 / threads with threads rounded up to 128).
+template <int NRT, int RB> struct LsqShape {
+    static constexpr int kMaxWarps = RB * NRT >= 128 ? 8 : (RB * NRT >= 96 ? 12 : 16);
+};
+
+// grid.x = slabs of k, grid.y = sets of rows (blockDim.x/32 warps x RB rows each),
+// grid.z = tiles of NRT samples.  Row 0 is x, row 1+i is v_i.
+template <int NRT, int RB, bool VEC>
+__global__ void __launch_bounds__(LsqShape<NRT, RB>::kMaxWarps * 32, 1) lsq_stream_kernel(LsqArgs a) {
+    constexpr int kStageK = kStageFloats / NRT;
+    extern __shared__ __align__(16) float smem_dyn[];
+    float(*as)[NRT][kStageK] = reinterpret_cast<float(*)[NRT][kStageK]>(smem_dyn);
+
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int nwarps = blockDim.x >> 5;
+    const int rows = a.m + 1;
+    const int row0 = (blockIdx.y * nwarps + warp) * RB;
+    const int j0 = blockIdx.z * NRT;
+    const int n_valid = min(NRT, a.n_r - j0);
+    const int64_t K = a.d;
+
+    const float *rowp[RB];
+#pragma unroll
+    for (int r = 0; r < RB; ++r) {
+        int rr = min(row0 + r, rows - 1);
+        rowp[r] = rr == 0 ? a.x : a.V + (int64_t)(rr - 1) * a.ldv;
+    }
+
+    // this block's stages: [s_begin, s_end) of ceil(d / kStageK)
+    const int64_t total = (K + kStageK - 1) / kStageK;
+    const int64_t s_begin = total * blockIdx.x / gridDim.x;
+    const int64_t s_end = total * (blockIdx.x + 1) / gridDim.x;
+
+    float acc[RB][NRT];
+    float nrm[RB];
+#pragma unroll
+    for (int r = 0; r < RB; ++r) {
+        nrm[r] = 0.f;
+#pragma unroll
+        for (int j = 0; j < NRT; ++j) acc[r][j] = 0.f;
+    }
+
+    auto issue_stage = [&](int64_t s, int buf) {
+        float(*dst)[kStageK] = as[buf];
+        const int64_t kb = s * kStageK;
+        if (VEC) {
+            constexpr int kVecPerRow = kStageK / 4;
+            for (int t = threadIdx.x; t < NRT * kVecPerRow; t += blockDim.x) {
+                int j = t / kVecPerRow, kk = (t % kVecPerRow) * 4;
+                bool ok = j < n_valid && kb + kk < K;
+                const float *src = ok ? a.A + (int64_t)(j0 + j) * K + kb + kk : a.A;
+                cp_async16(&dst[j][kk], src, ok);
+            }
+        } else {
+            for (int t = threadIdx.x; t < NRT * kStageK; t += blockDim.x) {
+                int j = t / kStageK, kk = t % kStageK;
+                bool ok = j < n_valid && kb + kk < K;
+                dst[j][kk] = ok ? __ldg(a.A + (int64_t)(j0 + j) * K + kb + kk) : 0.f;
+            }
+        }
+        cp_async_commit();
+    };
+
+    if (s_begin < s_end) issue_stage(s_begin, 0);
+    for (int64_t s = s_begin; s < s_end; ++s) {
+        const int buf = (int)((s - s_begin) & 1);
+        if (s + 1 < s_end) {
+            issue_stage(s + 1, buf ^ 1);
+            cp_async_wait<1>();
+        } else {
+            cp_async_wait<0>();
+        }
+        __syncthreads();
+        const float(*h)[kStageK] = as[buf];
+        if (row0 < rows) {
+#pragma unroll 1
+            for (int it = 0; it < kStageK / kIterK; ++it) {
+                const int64_t kbase = s * kStageK + it * kIterK;
+                if (kbase >= K) break;
+                float w[RB][4];
+#pragma unroll
+                for (int r = 0; r < RB; ++r) {
+                    load_row4<VEC>(rowp[r], kbase, lane, K, w[r]);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) nrm[r] = fmaf(w[r][e], w[r][e], nrm[r]);
+                }
+#pragma unroll
+                for (int j = 0; j < NRT; ++j) {
+                    float hv[4];
+                    if (VEC) {
+                        float4 t = *reinterpret_cast<const float4 *>(&h[j][it * kIterK + 4 * lane]);
+                        hv[0] = t.x; hv[1] = t.y; hv[2] = t.z; hv[3] = t.w;
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) hv[e] = h[j][it * kIterK + 32 * e + lane];
+                    }
+#pragma unroll
+                    for (int r = 0; r < RB; ++r)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) acc[r][j] = fmaf(w[r][e], hv[e], acc[r][j]);
+                }
+            }
+        }
+        __syncthreads();
+    }
+
+    // part[slab][row][0..n_r) = partial A.row ; part[slab][row][n_r] = partial sum of squares
+    const int stride = a.n_r + 1;
+#pragma unroll
+    for (int r = 0; r < RB; ++r) {
+        float z = warp_transpose_reduce<NRT>(acc[r], lane);
+        float q = warp_sum(nrm[r]);
+        const int rr = row0 + r;
+        if (rr < rows) {
+            float *dst = a.part + ((int64_t)blockIdx.x * rows + rr) * stride;
+            if (lane < n_valid) dst[j0 + lane] = z;
+            if (lane == 0 && blockIdx.z == 0) dst[a.n_r] = q;
+        }
+    }
+}
+
+// One block.  Sums the slab partials in slab order (double), then
+//   residual r_j = (A x)_j - y_j,  f_0 = sum r_j^2 / (2 n_r),
+//   f_i = sum (r_j - gamma (A v_i)_j)^2 / (2 n_r),  score_i = f_0 - f_i - rho ||v_i||^2.
+__global__ void __launch_bounds__(1024) lsq_finish_kernel(const float *part, int slabs, int m,
+                                                           int n_r, const float *y, float gamma,
+                                                           float rho, float *losses, float *norms,
+                                                           float *scores, float *sums /*[m+1][n_r+1]*/) {
+    const int rows = m + 1, stride = n_r + 1;
+    for (int t = threadIdx.x; t < rows * stride; t += blockDim.x) {
+        double acc = 0.0;
+        for (int s = 0; s < slabs; ++s) acc += (double)part[(int64_t)s * rows * stride + t];
+        sums[t] = (float)acc;
+    }
+    __syncthreads();
+    // the losses stay in double until the score is formed: f_0 - f_i cancels many digits
+    __shared__ double f_s[ZENO_MAX_CANDIDATES + 1];
+    for (int r = threadIdx.x; r < rows; r += blockDim.x) {
+        double f = 0.0;
+        for (int j = 0; j < n_r; ++j) {
+            double res = (double)sums[j] - (double)y[j];
+            if (r > 0) res -= (double)gamma * (double)sums[r * stride + j];
+            f += res * res;
+        }
+        f_s[r] = f / (2.0 * n_r);
+        losses[r] = (float)f_s[r];
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < m; i += blockDim.x) {
+        float nv = sums[(i + 1) * stride + n_r];
+        if (norms) norms[i] = nv;
+        scores[i] = (float)(f_s[0] - f_s[1 + i] - (double)rho * (double)nv);
+    }
+}
+
+template <int NRT, int RB, bool VEC>
+cudaError_t launch_stream(const LsqArgs &a, cudaStream_t s) {
+    const size_t smem = sizeof(float) * 2 * kStageFloats;
+    auto kernel = lsq_stream_kernel<NRT, RB, VEC>;
+    // the row groups are spread evenly over as few row sets as the warp limit allows
+    const int groups = (a.m + 1 + RB - 1) / RB;
+    const int row_sets = (groups + LsqShape<NRT, RB>::kMaxWarps - 1) / LsqShape<NRT, RB>::kMaxWarps;
+    const int warps = (groups + row_sets - 1) / row_sets;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    dim3 grid(a.slabs, row_sets, (a.n_r + NRT - 1) / NRT);
+    kernel<<<grid, warps * 32, smem, s>>>(a);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+int lsq_slab_count(const Context &c) {
+    int s = c.sm_count > 0 ? c.sm_count : 148;
+    return s < kMaxSlabs ? s : kMaxSlabs;
+}
+
+cudaError_t launch_lsq_score(Context &c, const LsqArgs &a_in, const float *y, float gamma,
+                             float rho, bool aligned, float *losses, float *norms, float *scores,
+                             cudaStream_t s, int *launches) {
+    LsqArgs a = a_in;
+    const int rows = a.m + 1;
+    const int nrt = a.n_r <= 8 ? 8 : (a.n_r <= 16 ? 16 : 32);
+    // small problems: no more slabs than there are stages of A
+    const int64_t stages = (a.d + (kStageFloats / nrt) - 1) / (kStageFloats / nrt);
+    int slabs = lsq_slab_count(c);
+    if ((int64_t)slabs > stages) slabs = (int)stages;
+    a.slabs = slabs;
+    cudaError_t e;
+    ++*launches;
+    profile_mark(c, "lsq_stream", s);
+    if (nrt == 8)
+        e = aligned ? launch_stream<8, 8, true>(a, s) : launch_stream<8, 8, false>(a, s);
+    else if (nrt == 16)
+        e = aligned ? launch_stream<16, 6, true>(a, s) : launch_stream<16, 6, false>(a, s);
+    else
+        e = aligned ? launch_stream<32, 4, true>(a, s) : launch_stream<32, 4, false>(a, s);
+    if (e != cudaSuccess) return e;
+    ++*launches;
+    profile_mark(c, "lsq_finish", s);
+    // the combined sums live behind the slab partials in the same workspace region
+    float *sums = a.part + (int64_t)slabs * rows * (a.n_r + 1);
+    lsq_finish_kernel<<<1, 1024, 0, s>>>(a.part, slabs, a.m, a.n_r, y, gamma, rho, losses, norms,
+                                         scores, sums);
+    return cudaGetLastError();
+}
+
+}  // namespace zeno

@@ -1,0 +1,318 @@
+// Candidate-model forward for the softmax-cross-entropy MLP (Definition 2: f_r(x) and
+// f_r(x - gamma v_i) on the same n_r samples), CUDA-core path.
+//
+// One launch per dense layer evaluates that layer for all m+1 models at once (model 0 is x
+// itself).  A warp owns kRowsPerWarp output rows of one model: its lanes stride the input
+// index k, form w = x - gamma v in registers straight from the loads of x and V (the
+// perturbed model never exists in memory), accumulate the n_r dot products and, in the same
+// pass, the sum of squares of the V entries they touched (the rho ||v||^2 term).  The input
+// activations of the layer are staged through shared memory with cp.async, double buffered.
+#include "zeno_internal.h"
+
+namespace zeno {
+
+namespace {
+
+constexpr int kStageK = 256;   // k-extent of one shared-memory stage of the activations
+constexpr int kIterK = 128;    // k-extent one warp consumes per inner iteration (32 lanes x 4)
+
+__device__ __forceinline__ void cp_async16(void *smem, const void *gmem, bool valid) {
+    unsigned s = static_cast<unsigned>(__cvta_generic_to_shared(smem));
+    int bytes = valid ? 16 : 0;  // 0 source bytes: the destination is zero-filled
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(s), "l"(gmem), "r"(bytes));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;\n" ::"n"(N));
+}
+
+// Sum, over the 32 lanes, of each of N per-lane values; lane j (< N) ends up holding the total
+// of value j.  Recursive halving: 31 shuffles for N = 32 instead of 160.
+template <int N>
+__device__ __forceinline__ float warp_transpose_reduce(float (&v)[N], int lane) {
+    static_assert(N == 1 || N == 2 || N == 4 || N == 8 || N == 16 || N == 32, "N must be 2^k");
+#pragma unroll
+    for (int s = N / 2; s >= 1; s >>= 1) {
+        const bool upper = (lane & s) != 0;
+#pragma unroll
+        for (int i = 0; i < s; ++i) {
+            float send = upper ? v[i] : v[i + s];
+            float keep = upper ? v[i + s] : v[i];
+            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, s);
+        }
+    }
+    float r = v[0];
+#pragma unroll
+    for (int s = N; s < 32; s <<= 1) r += __shfl_xor_sync(0xffffffffu, r, s);
+    return r;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int s = 16; s >= 1; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
+    return v;
+}
+
+// Positions of a lane's four k-indices inside a 128-wide iteration block.
+//   vector path: 4*lane + e  (one 16-byte / 8-byte load);  scalar path: 32*e + lane (coalesced).
+template <bool VEC> __device__ __forceinline__ int lane_k(int lane, int e) {
+    return VEC ? 4 * lane + e : 32 * e + lane;
+}
+
+template <typename T, bool VEC>
+__device__ __forceinline__ void load_row4(const T *row, int kbase, int lane, int K, float (&o)[4]) {
+    if (VEC) {
+        int k = kbase + 4 * lane;
+        if (k < K) {  // K is a multiple of 4 on this path
+            load_vec4(row + k, o);
+        } else {
+            o[0] = o[1] = o[2] = o[3] = 0.f;
+        }
+    } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            int k = kbase + 32 * e + lane;
+            o[e] = k < K ? load_elem(row + k) : 0.f;
+        }
+    }
+}
+
+template <typename T, int NRT, bool VEC>
+__global__ void __launch_bounds__(kLayerWarps * 32, 1) mlp_layer_kernel(LayerArgs a) {
+    constexpr int RB = kRowsPerWarp;
+    extern __shared__ __align__(16) float smem_dyn[];
+    float(*hs)[NRT][kStageK] = reinterpret_cast<float(*)[NRT][kStageK]>(smem_dyn);
+
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int c = blockIdx.y;                    // model: 0 = x, 1+i = x - gamma v_i
+    const int j0 = blockIdx.z * NRT;             // first sample of this tile
+    const int row0 = (blockIdx.x * kLayerWarps + warp) * RB;
+    const int K = a.in;
+    const bool has_v = c > 0;
+
+    const T *xw = static_cast<const T *>(a.x) + a.offW;
+    const T *vw = static_cast<const T *>(a.V) + (has_v ? (int64_t)(c - 1) * a.ldv : 0) + a.offW;
+    const T *xrow[RB];
+    const T *vrow[RB];
+#pragma unroll
+    for (int r = 0; r < RB; ++r) {
+        int o = min(row0 + r, a.out - 1);        // rows past the end are computed on a clamp and dropped
+        xrow[r] = xw + (int64_t)o * K;
+        vrow[r] = vw + (int64_t)o * K;
+    }
+    const float *hin = a.Hin + (int64_t)c * a.hin_cand_stride + (int64_t)j0 * K;
+    const int n_valid = min(NRT, a.n_r - j0);
+
+    float acc[RB][NRT];
+    float nrm = 0.f;
+#pragma unroll
+    for (int r = 0; r < RB; ++r)
+#pragma unroll
+        for (int j = 0; j < NRT; ++j) acc[r][j] = 0.f;
+
+    const int stages = (K + kStageK - 1) / kStageK;
+
+    auto issue_stage = [&](int s) {
+        float(*dst)[kStageK] = hs[s & 1];
+        const int kb = s * kStageK;
+        if (VEC) {
+            constexpr int kVecPerRow = kStageK / 4;
+            for (int t = threadIdx.x; t < NRT * kVecPerRow; t += blockDim.x) {
+                int j = t / kVecPerRow, kk = (t % kVecPerRow) * 4;
+                bool ok = j < n_valid && kb + kk < K;
+                const float *src = ok ? hin + (int64_t)j * K + kb + kk : a.Hin;
+                cp_async16(&dst[j][kk], src, ok);
+            }
+        } else {
+            for (int t = threadIdx.x; t < NRT * kStageK; t += blockDim.x) {
+                int j = t / kStageK, kk = t % kStageK;
+                bool ok = j < n_valid && kb + kk < K;
+                dst[j][kk] = ok ? __ldg(hin + (int64_t)j * K + kb + kk) : 0.f;
+            }
+        }
+        cp_async_commit();
+    };
+
+    issue_stage(0);
+    for (int s = 0; s < stages; ++s) {
+        if (s + 1 < stages) {
+            issue_stage(s + 1);
+            cp_async_wait<1>();
+        } else {
+            cp_async_wait<0>();
+        }
+        __syncthreads();
+        const float(*h)[kStageK] = hs[s & 1];
+#pragma unroll 1
+        for (int it = 0; it < kStageK / kIterK; ++it) {
+            const int kbase = s * kStageK + it * kIterK;
+            if (kbase >= K) break;
+            float w[RB][4];
+#pragma unroll
+            for (int r = 0; r < RB; ++r) {
+                float xv[4], vv[4];
+                load_row4<T, VEC>(xrow[r], kbase, lane, K, xv);
+                if (has_v) {
+                    load_row4<T, VEC>(vrow[r], kbase, lane, K, vv);
+                } else {
+                    vv[0] = vv[1] = vv[2] = vv[3] = 0.f;
+                }
+                const bool live = row0 + r < a.out;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    w[r][e] = candidate_param<T>(xv[e], vv[e], a.gamma);
+                    if (live) nrm = fmaf(vv[e], vv[e], nrm);
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < NRT; ++j) {
+                float hv[4];
+                if (VEC) {
+                    float4 t = *reinterpret_cast<const float4 *>(&h[j][it * kIterK + 4 * lane]);
+                    hv[0] = t.x; hv[1] = t.y; hv[2] = t.z; hv[3] = t.w;
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) hv[e] = h[j][it * kIterK + 32 * e + lane];
+                }
+#pragma unroll
+                for (int r = 0; r < RB; ++r)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) acc[r][j] = fmaf(w[r][e], hv[e], acc[r][j]);
+            }
+        }
+        __syncthreads();
+    }
+
+    // lane j now collects sample j0 + j of each row
+#pragma unroll
+    for (int r = 0; r < RB; ++r) {
+        float z = warp_transpose_reduce<NRT>(acc[r], lane);
+        const int o = row0 + r;
+        if (o < a.out && lane < n_valid) {
+            if (a.offB >= 0) {
+                const T *xb = static_cast<const T *>(a.x) + a.offB + o;
+                float bx = load_elem(xb);
+                float bv = has_v ? load_elem(static_cast<const T *>(a.V) + (int64_t)(c - 1) * a.ldv +
+                                             a.offB + o)
+                                 : 0.f;
+                z += candidate_param<T>(bx, bv, a.gamma);
+            }
+            if (a.relu) z = (z > 0.f || z != z) ? z : 0.f;   // a NaN stays a NaN
+            a.Hout[((int64_t)c * a.n_r + j0 + lane) * a.out + o] = z;
+        }
+    }
+
+    // partial ||v||^2 of the rows (and bias entries) this warp touched; one slot per warp
+    if (has_v && blockIdx.z == 0) {
+        if (a.offB >= 0 && lane < RB && row0 + lane < a.out) {
+            float bv = load_elem(static_cast<const T *>(a.V) + (int64_t)(c - 1) * a.ldv + a.offB +
+                                 row0 + lane);
+            nrm = fmaf(bv, bv, nrm);
+        }
+        nrm = warp_sum(nrm);
+        if (lane == 0)
+            a.normpart[(int64_t)(c - 1) * a.np_slots + a.np_base + blockIdx.x * kLayerWarps + warp] = nrm;
+    }
+}
+
+// Per model: mean over the samples of log-sum-exp(z) - z[label].  One block per model, one
+// warp per sample, fixed summation order.
+__global__ void __launch_bounds__(256) mlp_loss_kernel(const float *logits, const int32_t *labels,
+                                                        int n_r, int classes, float *losses) {
+    __shared__ float per_warp[8];
+    const int c = blockIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    float mine = 0.f;
+    for (int j = warp; j < n_r; j += 8) {
+        const float *z = logits + ((int64_t)c * n_r + j) * classes;
+        float zmax = -INFINITY;
+        for (int q = lane; q < classes; q += 32) zmax = fmaxf(zmax, z[q]);
+#pragma unroll
+        for (int s = 16; s >= 1; s >>= 1) zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, s));
+        float se = 0.f;
+        for (int q = lane; q < classes; q += 32) se += expf(z[q] - zmax);   // a NaN logit makes se NaN
+        se = warp_sum(se);
+        int lab = labels[j];
+        if (lab < 0 || lab >= classes) lab = 0;
+        mine += zmax + logf(se) - z[lab];   // identical in every lane of the warp
+    }
+    if (lane == 0) per_warp[warp] = mine;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float t = 0.f;
+        for (int w = 0; w < 8; ++w) t += per_warp[w];
+        losses[c] = t / (float)n_r;
+    }
+}
+
+// norms[i] = sum of the partial slots (fixed order); scores[i] = f_0 - f_i - rho * norms[i].
+__global__ void mlp_finalize_kernel(const float *normpart, int np_slots, int m, float rho,
+                                    const float *losses, float *scores, float *norms_out) {
+    const int lane = threadIdx.x & 31;
+    const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (i >= m) return;
+    float t = 0.f;
+    for (int s = lane; s < np_slots; s += 32) t += normpart[(int64_t)i * np_slots + s];
+    t = warp_sum(t);
+    if (lane == 0) {
+        if (norms_out) norms_out[i] = t;
+        scores[i] = losses[0] - losses[1 + i] - rho * t;
+    }
+}
+
+template <typename T, bool VEC>
+cudaError_t launch_layer_nrt(const LayerArgs &a, cudaStream_t s) {
+    const int rows_per_block = kRowsPerWarp * kLayerWarps;
+    auto go = [&](auto kernel, int nrt) {
+        dim3 grid((a.out + rows_per_block - 1) / rows_per_block, a.m + 1, (a.n_r + nrt - 1) / nrt);
+        const size_t smem = sizeof(float) * 2 * nrt * kStageK;
+        if (smem > 48 * 1024) {
+            cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 (int)smem);
+            if (e != cudaSuccess) return e;
+        }
+        kernel<<<grid, kLayerWarps * 32, smem, s>>>(a);
+        return cudaGetLastError();
+    };
+    if (a.n_r <= 8) return go(mlp_layer_kernel<T, 8, VEC>, 8);
+    if (a.n_r <= 16) return go(mlp_layer_kernel<T, 16, VEC>, 16);
+    return go(mlp_layer_kernel<T, 32, VEC>, 32);
+}
+
+}  // namespace
+
+int mlp_norm_slots(int out) {
+    const int rows_per_block = kRowsPerWarp * kLayerWarps;
+    return (out + rows_per_block - 1) / rows_per_block * kLayerWarps;
+}
+
+cudaError_t launch_mlp_layer(Context &c, const LayerArgs &a, bool aligned, cudaStream_t s,
+                             int *launches) {
+    ++*launches;
+    profile_mark(c, "mlp_layer", s);
+    if (c.desc.param_dtype == ZENO_BF16)
+        return aligned ? launch_layer_nrt<__nv_bfloat16, true>(a, s)
+                       : launch_layer_nrt<__nv_bfloat16, false>(a, s);
+    return aligned ? launch_layer_nrt<float, true>(a, s) : launch_layer_nrt<float, false>(a, s);
+}
+
+cudaError_t launch_mlp_loss(Context &c, const float *logits, const int32_t *labels, int n_r,
+                            int m, int classes, float *losses, cudaStream_t s, int *launches) {
+    ++*launches;
+    profile_mark(c, "mlp_loss", s);
+    mlp_loss_kernel<<<m + 1, 256, 0, s>>>(logits, labels, n_r, classes, losses);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_mlp_finalize(Context &c, int m, float rho, const float *losses,
+                                float *scores, float *norms_out, cudaStream_t s, int *launches) {
+    ++*launches;
+    profile_mark(c, "mlp_finalize", s);
+    const int warps = 4;
+    mlp_finalize_kernel<<<(m + warps - 1) / warps, warps * 32, 0, s>>>(c.normpart, c.np_slots, m,
+                                                                      rho, losses, scores, norms_out);
+    return cudaGetLastError();
+}
+
+}  // namespace zeno

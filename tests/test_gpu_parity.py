@@ -1,0 +1,259 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the float64 oracle on the same
+seeded inputs, element by element."""
+import numpy as np
+import pytest
+import torch
+
+from paper_1805_10032_b200 import synthetic as syn
+from paper_1805_10032_b200 import zeno
+
+import parity as P
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _library():
+    from paper_1805_10032_b200 import build as zbuild
+    zbuild.build()
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    zeno.load_library()
+
+
+# ---------------------------------------------------------------- shrunk versions of the five workloads
+# sizes chosen to span several row tiles / k stages and to leave ragged tails in every dimension
+
+SHRUNK = {
+    "cfg1": (1, dict()),                                                   # full size (d = 7850)
+    "cfg1_nr7": (1, dict(n_r=7, m=11, b=4, faults=[(4, "signflip")])),
+    "cfg2_small": (2, dict(dims=(300, 72, 40, 10), n_r=9)),
+    "cfg2_wide_k": (2, dict(dims=(1028, 36, 68, 10), n_r=33, m=7, b=3, faults=[(3, "noise200")])),
+    "cfg3_small": (3, dict(dims=(260, 44, 36, 10), m=37, b=15, n_r=70,
+                           faults=[(7, "signflip"), (8, "omniscient")])),
+    "cfg4_small": (4, dict(dims=(264, 136, 72, 50), m=9, b=3, n_r=19, faults=[(3, "signflip")])),
+    "cfg5_small": (5, dict(d=70000, m=13, b=5, n_r=16, n_noise=5)),
+    "cfg5_nr5": (5, dict(d=33333 * 4, m=70, b=30, n_r=5, n_noise=30)),
+    "cfg5_nr40": (5, dict(d=9000, m=6, b=2, n_r=40, n_noise=2)),
+}
+
+
+@pytest.mark.parametrize("name", sorted(SHRUNK))
+def test_step_matches_oracle_on_shrunk_workloads(oracle, name):
+    index, ov = SHRUNK[name]
+    w = syn.make_config(index, **ov)
+    res = P.run_step_parity(oracle, w)
+    assert res["launches"] >= 3
+
+
+def test_config2_full_size(oracle):
+    w = syn.make_config(2)
+    assert w.d == 1841162 and w.m == 20 and w.n_r == 32
+    res = P.run_step_parity(oracle, w)
+    assert res["exact_set"]
+
+
+# ---------------------------------------------------------------- odd shapes, unaligned rows (scalar path)
+
+@pytest.mark.parametrize("dims,n_r,m,pad", [
+    ((7, 5, 4, 3), 3, 6, 0),        # nothing aligned
+    ((13, 3), 1, 2, 5),             # softmax regression, one sample
+    ((129, 33, 2), 17, 5, 1),
+    ((130, 66, 10), 8, 33, 3),
+    ((260, 10), 32, 4, 2),
+])
+def test_unaligned_layouts(oracle, dims, n_r, m, pad):
+    d = syn.param_count("mlp", dims)
+    w = syn.make_config(2, dims=dims, n_r=n_r, m=m, b=m // 3, faults=[(m // 3, "noise200")],
+                        ldv=d + pad)
+    P.run_step_parity(oracle, w)
+
+
+def test_unaligned_base_pointers(oracle):
+    # x and V start 4 bytes into an allocation: every vector path must be refused
+    w = syn.make_config(1, dims=(64, 12), m=6, b=2, faults=[(2, "signflip")])
+    xs = torch.empty(w.d + 1, device="cuda"); xs[1:] = w.x.cuda()
+    Vs = torch.empty(w.m * w.ldv + 1, device="cuda"); Vs[1:] = w.V.cuda().reshape(-1)
+    x, V = xs[1:], Vs[1:].view(w.m, w.ldv)
+    s_orc, _, _ = P.oracle_score(oracle, w)
+    with zeno.from_workload(w) as z:
+        out, scores, idx = z.step(x, V, w.features.cuda(), w.targets.cuda(), w.gamma, w.rho, w.b,
+                                  ldv=w.ldv)
+    P.assert_scores_close(scores.cpu().numpy(), s_orc)
+    o = P.oracle_inputs(w)
+    ref = oracle.aggregate(0, o["V"], w.ldv, w.d, w.m, idx.cpu().numpy())
+    assert P.rel_l2(out.cpu().numpy(), ref) <= P.AGG_RTOL
+
+
+def test_lsq_unaligned(oracle):
+    w = syn.make_config(5, d=4099, m=5, b=2, n_r=3, n_noise=2, ldv=4101)
+    P.run_step_parity(oracle, w)
+
+
+def test_no_bias_model(oracle):
+    w = syn.make_config(2, dims=(96, 24, 10), n_r=6, m=5, b=1, faults=[(1, "noise200")],
+                        has_bias=False)
+    P.run_step_parity(oracle, w)
+
+
+# ---------------------------------------------------------------- properties on the GPU output
+
+def _small():
+    return syn.make_config(2, dims=(132, 40, 24, 10), n_r=12, m=10, b=4, faults=[(4, "noise200")])
+
+
+def test_zero_update_scores_exactly_zero():
+    w = _small()
+    w.V[3, :w.d] = 0.0
+    x, V, f, t = P.to_device(w)
+    with zeno.from_workload(w) as z:
+        s, losses, norms = z.score(x, V, f, t, w.gamma, w.rho)
+    assert s[3].item() == 0.0 and norms[3].item() == 0.0 and losses[4].item() == losses[0].item()
+    wl = syn.make_config(5, d=5000, m=4, b=1, n_r=16, n_noise=1)
+    wl.V[2, :wl.d] = 0.0
+    x, V, f, t = P.to_device(wl)
+    with zeno.from_workload(wl) as z:
+        s, losses, norms = z.score(x, V, f, t, wl.gamma, wl.rho)
+    assert s[2].item() == 0.0
+
+
+def test_b_zero_is_the_mean_and_b_m_minus_1_is_one_row():
+    w = _small()
+    x, V, f, t = P.to_device(w)
+    with zeno.from_workload(w) as z:
+        out0, _, idx0 = z.step(x, V, f, t, w.gamma, w.rho, 0)
+        out1, s1, idx1 = z.step(x, V, f, t, w.gamma, w.rho, w.m - 1)
+    assert sorted(idx0.tolist()) == list(range(w.m))
+    mean = w.V[:, :w.d].double().mean(0).numpy()
+    assert P.rel_l2(out0.cpu().numpy(), mean) <= P.AGG_RTOL
+    best = int(torch.argmax(s1))
+    assert idx1.tolist() == [best]
+    assert torch.equal(out1.cpu(), w.V[best, :w.d])      # bit-exact copy of one input row
+
+
+def test_permutation_invariance_and_duplicates():
+    w = _small()
+    w.V[7] = w.V[2]
+    x, V, f, t = P.to_device(w)
+    perm = torch.randperm(w.m, generator=torch.Generator().manual_seed(1))
+    with zeno.from_workload(w) as z:
+        out, s, idx = z.step(x, V, f, t, w.gamma, w.rho, w.b)
+        out_p, s_p, idx_p = z.step(x, V[perm.cuda()].contiguous(), f, t, w.gamma, w.rho, w.b)
+    assert s[7].item() == s[2].item()                    # duplicates score bit-identically
+    assert torch.equal(s_p.cpu(), s.cpu()[perm])         # scores do not depend on the row position
+    sel, sel_p = set(idx.tolist()), set(perm[idx_p.cpu().long()].tolist())
+    # the two copies are interchangeable; everything else must agree
+    canon = lambda S: {2 if i == 7 else i for i in S}
+    assert canon(sel) == canon(sel_p)
+    assert P.rel_l2(out_p.cpu().numpy(), out.cpu().numpy()) <= 1e-6
+
+
+def test_lemma1_on_gpu_ranking():
+    # Lemma 1: the k-th best score overall is at least the k-th best score inside any subset
+    g = torch.Generator().manual_seed(5)
+    s = torch.randn(200, generator=g)
+    with zeno.Zeno(0, 0, (8, 4), m_max=256, n_r_max=4) as z:
+        idx = z.select(s.cuda(), 0).cpu().long()
+    ranked = s[idx]
+    assert torch.all(ranked[:-1] >= ranked[1:])
+    for size in (1, 17, 100, 200):
+        sub = s[torch.randperm(200, generator=g)[:size]].sort(descending=True).values
+        assert torch.all(ranked[:size] >= sub)
+
+
+def test_jensen_step_on_gpu_outputs(oracle):
+    # convex loss: f_r(x - gamma * Zeno_b(V)) <= mean of the selected candidates' losses
+    w = syn.make_config(1)
+    x, V, f, t = P.to_device(w)
+    with zeno.from_workload(w) as z:
+        out, s, idx = z.step(x, V, f, t, w.gamma, w.rho, w.b)
+        _, losses, _ = z.score(x, V, f, t, w.gamma, w.rho)
+        # evaluate f_r at x - gamma * out by presenting `out` as a single candidate
+        V1 = torch.zeros(1, w.ldv, device="cuda"); V1[0, :w.d] = out
+        _, l1, _ = z.score(x, V1, f, t, w.gamma, w.rho)
+    assert l1[1].item() <= losses[1 + idx.long()].mean().item() + 1e-6
+
+
+# ---------------------------------------------------------------- ranking alone: integer work, bit-exact
+
+@pytest.mark.parametrize("m", [1, 2, 31, 32, 33, 100, 513, 1024])
+def test_select_matches_oracle_bit_exactly(oracle, m):
+    g = np.random.default_rng(m)
+    s = g.standard_normal(m).astype(np.float32)
+    if m >= 31:
+        s[g.integers(0, m, m // 4)] = s[0]                 # exact ties
+        s[g.integers(0, m, 3)] = np.nan
+        s[g.integers(0, m, 2)] = -np.inf
+        s[g.integers(0, m, 2)] = np.inf
+        s[5], s[6] = 0.0, -0.0
+    with zeno.Zeno(0, 0, (8, 4), m_max=1024, n_r_max=4) as z:
+        for b in sorted({0, m // 3, m - 1}):
+            idx = z.select(torch.from_numpy(s).cuda(), b).cpu().numpy()
+            assert np.array_equal(idx, oracle.select(s.astype(np.float64), b))
+
+
+# ---------------------------------------------------------------- faulty values stay contained
+
+def test_non_finite_candidates_are_ranked_last_and_do_not_leak(oracle):
+    w = _small()
+    w.V[0, 5] = float("nan")
+    w.V[4, 100] = float("inf")
+    w.V[6, :w.d] = 1e30
+    x, V, f, t = P.to_device(w)
+    with zeno.from_workload(w) as z:
+        out, s, idx = z.step(x, V, f, t, w.gamma, w.rho, 3)
+    s_orc, _, _ = P.oracle_score(oracle, w)
+    assert not set(idx.tolist()) & {0, 4, 6}
+    assert torch.isfinite(out).all()
+    good = [i for i in range(w.m) if i not in (0, 4, 6)]
+    P.assert_scores_close(s.cpu().numpy()[good], s_orc[good])
+    # NaN / Inf entries make the score non-finite on both sides; the 1e30 row overflows binary32
+    # (score -inf) where float64 still holds -3e60: both rank it last
+    assert not np.isfinite(s.cpu().numpy()[[0, 4, 6]]).any()
+    assert not np.isfinite(s_orc[[0, 4]]).any() and s_orc[6] < -1e59
+
+
+def test_aggregate_skips_out_of_range_indices():
+    w = _small()
+    V = w.V.cuda()
+    idx = torch.tensor([1, -3, 2, 99], dtype=torch.int32, device="cuda")
+    with zeno.from_workload(w) as z:
+        out = z.aggregate(V, idx)
+    ref = (w.V[1, :w.d].double() + w.V[2, :w.d].double()) / 4
+    assert P.rel_l2(out.cpu().numpy(), ref.numpy()) <= P.AGG_RTOL
+
+
+# ---------------------------------------------------------------- argument errors are status codes
+
+def test_argument_errors():
+    w = _small()
+    x, V, f, t = P.to_device(w)
+    with zeno.from_workload(w) as z:
+        for kwargs in (dict(b=w.m), dict(b=-1)):
+            with pytest.raises(zeno.ZenoError) as e:
+                z.step(x, V, f, t, w.gamma, w.rho, **kwargs)
+            assert e.value.status == zeno.ERR_INVALID_ARG
+        for bad in (dict(gamma=float("nan")), dict(rho=-1.0), dict(rho=float("inf"))):
+            args = dict(gamma=w.gamma, rho=w.rho); args.update(bad)
+            with pytest.raises(zeno.ZenoError) as e:
+                z.score(x, V, f, t, args["gamma"], args["rho"])
+            assert e.value.status == zeno.ERR_INVALID_ARG
+        with pytest.raises(zeno.ZenoError):
+            z.score(x, V, f, t, w.gamma, w.rho, ldv=w.d - 1)
+        with pytest.raises(zeno.ZenoError):
+            z.score(x, V, f, t, w.gamma, w.rho, m=w.m + 1)          # beyond m_max
+        # the handle still works after rejected calls
+        out, s, idx = z.step(x, V, f, t, w.gamma, w.rho, w.b)
+        assert torch.isfinite(out).all()
+
+
+def test_host_entry_point_matches_device_entry_point():
+    w = _small()
+    x, V, f, t = P.to_device(w)
+    out_h = torch.empty(w.d, dtype=torch.float32).pin_memory()
+    s_h = torch.empty(w.m, dtype=torch.float32).pin_memory()
+    i_h = torch.empty(w.m - w.b, dtype=torch.int32).pin_memory()
+    with zeno.from_workload(w) as z:
+        out, s, idx = z.step(x, V, f, t, w.gamma, w.rho, w.b)
+        z.step_host(w.x.pin_memory(), w.V.pin_memory(), w.features.pin_memory(),
+                    w.targets.pin_memory(), w.gamma, w.rho, w.b, out_h, s_h, i_h)
+    assert torch.equal(out.cpu(), out_h) and torch.equal(s.cpu(), s_h) and torch.equal(idx.cpu(), i_h)

@@ -1,0 +1,385 @@
+#!/usr/bin/env python
+"""Benchmark of the Zeno aggregation step (scores -> ranking -> trimmed mean).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl ours|reference]
+
+One step = one zeno_step call: f_r(x), the m candidate losses f_r(x - gamma v_i) with the
+squared norms, the top-(m-b) ranking and the trimmed mean, on one batch of synthetic input.
+Prints ONE JSON line: steps/s with the inputs resident in HBM (`value`), the same through the
+host-memory entry point with the copies inside the timed region (`e2e`), the dominant kernel's
+achieved bandwidth against the measured HBM peak (`roofline`), and the float64 CPU oracle timed
+on the host cores (`cpu_baseline`).
+
+--gpus N (under torchrun, one rank per GPU): the step does not shard without a collective this
+library does not have, so the ranks run independent replicas of the workload; `value` is the sum.
+--impl reference: times the CPU oracle as it stands (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "zeno_steps_per_sec"
+UNIT = "steps/s"
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_HBM_GBS = 6650.0
+
+
+# ----------------------------------------------------------------------------- helpers
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as fh:
+            d = json.load(fh)
+        return float(d["hbm_gbs"]), "measured"
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+def algorithmic_bytes(w):
+    """Bytes the step itself must move (padding excluded): the score pass reads V, x and the batch
+    once; the aggregate pass reads the m-b selected rows once more and writes d floats."""
+    s = 2 if w.dtype == "bf16" else 4
+    feats = w.n_r * w.dims[0] * 4 + w.n_r * 4
+    score = w.m * w.d * s + w.d * s + feats
+    agg = (w.m - w.b) * w.d * s + w.d * 4
+    return score, agg
+
+
+def layer_bytes(w, layer):
+    """Algorithmic bytes of one layer launch: that layer's slice of V (m rows) and of x, plus its
+    input activations ((m+1) n_r in floats, or the shared features for layer 0) and outputs."""
+    s = 2 if w.dtype == "bf16" else 4
+    i, o = w.dims[layer], w.dims[layer + 1]
+    params = o * i + (o if w.has_bias else 0)
+    acts_in = w.n_r * i * 4 * (1 if layer == 0 else w.m + 1)
+    acts_out = (w.m + 1) * w.n_r * o * 4
+    return (w.m + 1) * params * s + acts_in + acts_out
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons, sampled while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-i", str(self.gpu), "-lms", "100"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            with open(self.path) as fh:
+                for line in fh:
+                    f = [t.strip() for t in line.split(",")]
+                    if len(f) < 9:
+                        continue
+                    try:
+                        sm.append(float(f[1])); smax.append(float(f[2]))
+                    except ValueError:
+                        continue
+                    for n, v in zip(names, f[5:9]):
+                        if v.lower().startswith("active"):
+                            reasons.add(n)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def kind_code(w):
+    return 1 if w.kind == "lsq" else 0
+
+
+def oracle_step_seconds(w, m_sample=None):
+    """One oracle step on (a candidate subset of) the workload; returns (seconds, candidates)."""
+    import numpy as np
+    from oracle import zeno_oracle
+    from paper_1805_10032_b200 import synthetic as syn
+    m = w.m if m_sample is None else min(m_sample, w.m)
+    b = min(w.b, m - 1)
+    V = syn.to_numpy_params(w.V[:m])
+    x = syn.to_numpy_params(w.x)
+    f = w.features.cpu().numpy()
+    t = w.targets.cpu().numpy()
+    dt = 1 if w.dtype == "bf16" else 0
+    t0 = time.perf_counter()
+    zeno_oracle.step(kind_code(w), dt, w.dims, w.has_bias, x, V, w.ldv, m, f, t,
+                     float(np.float32(w.gamma)), float(np.float32(w.rho)), b)
+    return time.perf_counter() - t0, m
+
+
+# ----------------------------------------------------------------------------- reference arm
+
+def run_reference(args, rank, world):
+    if rank != 0:
+        return 0
+    from oracle import zeno_oracle
+    from paper_1805_10032_b200 import synthetic as syn
+    zeno_oracle.build()
+    w = syn.make_config(args.config)
+    cores = zeno_oracle.num_threads()
+    # bound the whole run to a few minutes: time one full step, then shrink the candidate sample
+    t_full, _ = oracle_step_seconds(w)
+    total_steps = args.steps + args.warmup
+    budget = 150.0
+    m_sample = w.m
+    if t_full * total_steps > budget:
+        m_sample = max(1, int((budget / total_steps) / t_full * (w.m + 1)) - 1)
+    scale = (w.m + 1) / (m_sample + 1)     # the oracle's work is linear in the models evaluated
+    for _ in range(args.warmup):
+        oracle_step_seconds(w, m_sample)
+    times = [oracle_step_seconds(w, m_sample)[0] * scale for _ in range(args.steps)]
+    per_step = sum(times) / len(times)
+    value = 1.0 / per_step
+    sample = (f"all {w.m} candidates" if m_sample == w.m else
+              f"first {m_sample} of {w.m} candidates per step, time scaled by (m+1)/(m_s+1)")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": workload_config(w, args.config),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def workload_config(w, index):
+    return {"workload": f"config{index}: {w.kind} dims={list(w.dims)} dtype={w.dtype} m={w.m} "
+                        f"b={w.b} n_r={w.n_r} gamma={w.gamma} rho={w.rho} d={w.d} ldv={w.ldv}",
+            "m": w.m, "b": w.b, "n_r": w.n_r, "d": w.d}
+
+
+# ----------------------------------------------------------------------------- our arm
+
+def run_ours(args, rank, world, local_rank):
+    import torch
+    from paper_1805_10032_b200 import build as zbuild
+    from paper_1805_10032_b200 import synthetic as syn
+    from paper_1805_10032_b200 import zeno
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the Zeno step has no CPU path")
+    zbuild.build()
+    dev = local_rank
+    torch.cuda.set_device(dev)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", dev))
+
+    # inputs: enough distinct sets that the rotation exceeds 4x the L2 capacity
+    w0 = syn.make_config(args.config)
+    score_b, agg_b = algorithmic_bytes(w0)
+    set_bytes = w0.V.numel() * w0.V.element_size() + w0.features.numel() * 4
+    n_sets = max(1, min(8, -(-4 * L2_BYTES // set_bytes)))
+    if set_bytes > 8 * L2_BYTES:
+        n_sets = 1
+    sets = [w0] + [syn.make_config(args.config, seed=syn.BASE_SEED + args.config + 1000 * (i + 1))
+                   for i in range(n_sets - 1)]
+    dsets = [(s.x.cuda(), s.V.cuda(), s.features.cuda(), s.targets.cuda()) for s in sets]
+    z = zeno.from_workload(w0, device=dev)
+    out = torch.empty(w0.d, dtype=torch.float32, device="cuda")
+    scores = torch.empty(w0.m, dtype=torch.float32, device="cuda")
+    idx = torch.empty(w0.m - w0.b, dtype=torch.int32, device="cuda")
+
+    def step(i):
+        x, V, f, t = dsets[i % n_sets]
+        z.step(x, V, f, t, w0.gamma, w0.rho, w0.b, out=out, scores=scores, idx=idx)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    launches_per_step = 0
+    step(0)
+    launches_per_step = z.last_launch_count
+
+    # ---- timed region 1: K steps, inputs resident in HBM
+    sampler = ClockSampler(dev)
+    sampler.start()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        step(i)
+    e1.record()
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+
+    # ---- timed region 2: the same K steps with an event around every kernel
+    z.profile(True)
+    per_kernel = {}
+    order = []
+    for i in range(args.steps):
+        step(i)
+        for j, (name, ms) in enumerate(z.profile_read()):
+            key = f"{j}:{name}"
+            if key not in per_kernel:
+                per_kernel[key] = []
+                order.append(key)
+            per_kernel[key].append(ms)
+    z.profile(False)
+    clocks = sampler.stop()
+
+    if dist is not None:
+        t = torch.tensor([ms_total], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_per_step = ms_total / args.steps
+    value = world * args.steps / (ms_total * 1e-3)
+
+    # ---- end to end through the host-memory entry point (copies inside the timed region)
+    hx, hV = sets[0].x.pin_memory(), sets[0].V.pin_memory()
+    hf, ht = sets[0].features.pin_memory(), sets[0].targets.pin_memory()
+    hout = torch.empty(w0.d, dtype=torch.float32).pin_memory()
+    e2e_steps = max(3, min(args.steps, 20))
+    for _ in range(2):
+        z.step_host(hx, hV, hf, ht, w0.gamma, w0.rho, w0.b, hout)
+    barrier()
+    t0 = time.perf_counter()
+    e0.record()
+    for _ in range(e2e_steps):
+        z.step_host(hx, hV, hf, ht, w0.gamma, w0.rho, w0.b, hout)
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = world * e2e_steps / (e2e_ms * 1e-3)
+    h2d = (hx.numel() * hx.element_size() + hV.numel() * hV.element_size() + hf.numel() * 4
+           + ht.numel() * 4)
+    d2h = hout.numel() * 4
+
+    if rank != 0:
+        return 0
+
+    # ---- roofline of the dominant kernel
+    peak, peak_kind = measured_peaks()
+    kern = []
+    for key in order:
+        v = per_kernel[key]
+        kern.append({"kernel": key, "avg_us": 1e3 * sum(v) / len(v)})
+    total_us = sum(k["avg_us"] for k in kern) or 1.0
+    for k in kern:
+        k["share"] = k["avg_us"] / total_us
+    top = max(kern, key=lambda k: k["avg_us"])
+    top_i = int(top["kernel"].split(":")[0])
+    top_name = top["kernel"].split(":")[1]
+    if top_name == "mlp_layer":
+        top_bytes = layer_bytes(w0, top_i)
+    elif top_name == "lsq_stream":
+        top_bytes = score_b
+    elif top_name == "aggregate":
+        top_bytes = agg_b
+    else:
+        top_bytes = 0
+    achieved = top_bytes / (top["avg_us"] * 1e-6) / 1e9
+    step_bytes = score_b + agg_b
+    roofline = {
+        "bound": "hbm", "kernel": top["kernel"], "achieved": achieved, "peak": peak,
+        "unit": "GB/s", "frac": achieved / peak, "traffic": None, "peak_source": peak_kind,
+        "bytes_per_launch": top_bytes, "avg_us": top["avg_us"],
+        "timed": "second pass over the same K steps with a CUDA event around every kernel",
+        "step": {"algorithmic_bytes": step_bytes,
+                 "achieved_GBs": step_bytes / (ms_per_step * 1e-3) / 1e9,
+                 "frac_of_hbm_peak": step_bytes / (ms_per_step * 1e-3) / 1e9 / peak,
+                 "roofline_us": step_bytes / (peak * 1e9) * 1e6},
+        "kernels": kern,
+    }
+
+    # ---- CPU baseline: the oracle on a bounded sample of the same workload
+    from oracle import zeno_oracle
+    zeno_oracle.build()
+    t_full, _ = oracle_step_seconds(w0, None if args.config in (1, 2) else 3)
+    m_s = w0.m if args.config in (1, 2) else 3
+    reps = max(1, min(5, int(12.0 / max(t_full, 1e-3))))
+    ts = [oracle_step_seconds(w0, m_s)[0] for _ in range(reps)]
+    t_step = (sum(ts) / len(ts)) * (w0.m + 1) / (m_s + 1)
+    cpu = {"value": 1.0 / t_step, "unit": UNIT, "cores": zeno_oracle.num_threads(), "kind": "oracle",
+           "sample": (f"{reps} full steps" if m_s == w0.m else
+                      f"{reps} steps over the first {m_s} of {w0.m} candidates, scaled by (m+1)/(m_s+1)")}
+
+    cfg = workload_config(w0, args.config)
+    cfg["l2_policy"] = (f"inputs rotate over {n_sets} distinct sets ({n_sets * set_bytes / 1e6:.0f} MB"
+                        f" > 4x L2)" if n_sets > 1 else "one input set, larger than 4x L2")
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16/f32" if w0.dtype == "bf16" else "f32",
+        "data": "synthetic", "config": cfg, "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps},
+        "gpu_launches": launches_per_step * args.steps, "launches_per_step": launches_per_step,
+        "roofline": roofline, "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+    z.close()
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--config", type=int, default=2, help="benchmark configuration 1..5 (default 2)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        return run_reference(args, rank, world)
+    return run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -154,6 +154,11 @@ zeno_status zeno_step_host(zeno_handle h, const void *x, const void *V, int64_t 
                            float rho, int32_t b, float *out, float *scores, int32_t *idx,
                            void *stream);
 
+/* Synchronises `stream` and reports whether any kernel enqueued through this handle gave up on a
+ * bounded device-side wait (its outputs are then undefined): ZENO_ERR_TIMEOUT if so, else
+ * ZENO_OK.  The condition is sticky for the life of the handle. */
+zeno_status zeno_device_status(zeno_handle h, void *stream);
+
 /* Per-kernel timing for benchmarks.  zeno_profile(h, 1) makes every later call on the handle
  * record a CUDA event on the call's stream before each of its kernels and after the last one
  * (a few microseconds of overhead per call); zeno_profile(h, 0) switches it off again.

@@ -2,6 +2,7 @@
 // kernels are enqueued.  No arithmetic of the method lives here.
 #include <math.h>
 #include <new>
+#include <stdlib.h>
 #include <string.h>
 
 #include "zeno_internal.h"
@@ -114,7 +115,28 @@ zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv,
     }
 
     const int L = c->desc.n_layers;
-    for (int l = 0; l < L; ++l) {
+    zeno::NormSlots used;
+    used.layers = L;
+    int first_cuda_layer = 0;
+    // first layer on the tensor cores when the shape and the alignment allow it
+    zeno::StreamTcPlan plan;
+    if (c->tc_ok && aligned &&
+        zeno::stream_tc_plan(c->sm_count, (int)c->desc.dims[0], (int)c->desc.dims[1], n_r, m, &plan) &&
+        plan.R <= c->tc_r_max) {
+        const float *xf = static_cast<const float *>(x);
+        const float *Vf = static_cast<const float *>(V);
+        e = zeno::launch_stream_tc(*c, plan, xf, Vf, ldv, c->offW[0], c->offB[0], (int)c->desc.dims[0],
+                                   (int)c->desc.dims[1], batch->features, n_r, m, c->tc_part, c->np_base[0],
+                                   s, launches);
+        if (e != cudaSuccess) return fail_cuda(c, e);
+        e = zeno::launch_stream_combine(*c, plan, c->tc_part, xf, Vf, ldv, c->offB[0], (int)c->desc.dims[1],
+                                        n_r, m, gamma, L > 1, c->act[0], s, launches);
+        if (e != cudaSuccess) return fail_cuda(c, e);
+        used.base[0] = c->np_base[0];
+        used.count[0] = zeno::stream_tc_norm_slots(plan);
+        first_cuda_layer = 1;
+    }
+    for (int l = first_cuda_layer; l < L; ++l) {
         zeno::LayerArgs a;
         a.x = x;
         a.V = V;
@@ -133,13 +155,15 @@ zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv,
         a.normpart = c->normpart;
         a.np_slots = c->np_slots;
         a.np_base = c->np_base[l];
+        used.base[l] = c->np_base[l];
+        used.count[l] = zeno::mlp_norm_slots(a.out);
         e = zeno::launch_mlp_layer(*c, a, aligned, s, launches);
         if (e != cudaSuccess) return fail_cuda(c, e);
     }
     e = zeno::launch_mlp_loss(*c, c->act[(L - 1) & 1], static_cast<const int32_t *>(batch->targets),
                               n_r, m, (int)c->desc.dims[L], loss_buf, s, launches);
     if (e != cudaSuccess) return fail_cuda(c, e);
-    e = zeno::launch_mlp_finalize(*c, m, rho, loss_buf, scores, norms, s, launches);
+    e = zeno::launch_mlp_finalize(*c, used, m, rho, loss_buf, scores, norms, s, launches);
     return e == cudaSuccess ? ZENO_OK : fail_cuda(c, e);
 }
 
@@ -207,7 +231,7 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
     c->sm_count = prop.multiProcessorCount;
 
     const size_t rows = (size_t)m_max + 1;
-    size_t act_elems = 0, norm_elems = 0, lsq_elems = 0;
+    size_t act_elems = 0, norm_elems = 0, lsq_elems = 0, tc_elems = 0;
     if (desc->kind == ZENO_LOSS_SOFTMAX_MLP) {
         int64_t off = 0, widest = 0;
         int slots = 0;
@@ -218,7 +242,22 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
             c->offB[l] = desc->has_bias ? off : -1;
             if (desc->has_bias) off += o;
             c->np_base[l] = slots;
-            slots += zeno::mlp_norm_slots((int)o);
+            int layer_slots = zeno::mlp_norm_slots((int)o);
+            if (l == 0 && desc->param_dtype == ZENO_F32 && !getenv("ZENO_DISABLE_TENSOR_CORES")) {
+                // the tensor-core stream may serve the first layer: size its partials for the
+                // shortest k-range any plan may pick
+                zeno::StreamTcPlan probe;
+                if (zeno::stream_tc_plan(c->sm_count, (int)in, (int)o, n_r_max < 64 ? n_r_max : 64, m_max,
+                                         &probe)) {
+                    c->tc_ok = true;
+                    c->tc_r_max = (int)((in + zeno::kStreamTcMinKR - 1) / zeno::kStreamTcMinKR);
+                    probe.R = c->tc_r_max;
+                    const int tc_slots = zeno::stream_tc_norm_slots(probe);
+                    if (tc_slots > layer_slots) layer_slots = tc_slots;
+                    tc_elems = (size_t)c->tc_r_max * rows * (size_t)n_r_max * (size_t)o;
+                }
+            }
+            slots += layer_slots;
             if (o > widest) widest = o;
         }
         c->np_slots = slots;
@@ -239,6 +278,7 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
     const size_t at_norm = reserve(norm_elems, 4), at_lsq = reserve(lsq_elems, 4);
     const size_t at_loss = reserve(rows, 4), at_norms = reserve(m_max, 4);
     const size_t at_scores = reserve(m_max, 4), at_idx = reserve(m_max, 4);
+    const size_t at_status = reserve(1, 4), at_tc = reserve(tc_elems, 4);
 
     e = cudaMalloc(&c->arena, bytes);
     if (e != cudaSuccess) {
@@ -255,6 +295,14 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
     c->norms = reinterpret_cast<float *>(base + at_norms);
     c->scores = reinterpret_cast<float *>(base + at_scores);
     c->idx = reinterpret_cast<int32_t *>(base + at_idx);
+    c->dev_status = reinterpret_cast<int *>(base + at_status);
+    c->tc_part = reinterpret_cast<float *>(base + at_tc);
+    e = cudaMemset(c->dev_status, 0, sizeof(int));
+    if (e != cudaSuccess) {
+        cudaFree(c->arena);
+        delete c;
+        return ZENO_ERR_CUDA;
+    }
     *out = c;
     return ZENO_OK;
 }
@@ -397,10 +445,24 @@ zeno_status zeno_step_host(zeno_handle h, const void *x, const void *V, int64_t 
         e = cudaMemcpyAsync(scores, h->scores, (size_t)m * 4, cudaMemcpyDeviceToHost, s);
     if (e == cudaSuccess && idx)
         e = cudaMemcpyAsync(idx, h->idx, (size_t)(m - b) * 4, cudaMemcpyDeviceToHost, s);
+    int dev_status = 0;
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&dev_status, h->dev_status, sizeof(int), cudaMemcpyDeviceToHost, s);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return fail_cuda(h, e);
     h->last_launches = launches;
-    return ZENO_OK;
+    return dev_status ? ZENO_ERR_TIMEOUT : ZENO_OK;
+}
+
+zeno_status zeno_device_status(zeno_handle h, void *stream) {
+    if (!h) return ZENO_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int dev_status = 0;
+    cudaError_t e = cudaMemcpyAsync(&dev_status, h->dev_status, sizeof(int), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return fail_cuda(h, e);
+    return dev_status ? ZENO_ERR_TIMEOUT : ZENO_OK;
 }
 
 zeno_status zeno_profile(zeno_handle h, int32_t enable) {

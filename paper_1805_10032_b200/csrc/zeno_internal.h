@@ -18,6 +18,14 @@ constexpr int kMaxSlabs = 1024;
 // Most kernels one call can enqueue (layers + loss + finalize + select + aggregate).
 constexpr int kMaxProfiled = ZENO_MAX_LAYERS + 8;
 
+// Launch shape of the tensor-core stream: k-range length, number of k-ranges, blocks per
+// k-range, padded sample count, 128-row tiles per model, dynamic shared memory.
+struct StreamTcPlan { int KR, R, G, n_pad, tiles_per_model, smem_bytes; };
+constexpr int kStreamTcMinKR = 256;
+
+// Which norm-partial slots a call filled: per layer (first slot, count).
+struct NormSlots { int base[ZENO_MAX_LAYERS]; int count[ZENO_MAX_LAYERS]; int layers; };
+
 struct Context {
     zeno_model_desc desc;
     int64_t d;
@@ -37,6 +45,10 @@ struct Context {
     float *norms;                   // [m_max]
     float *scores;                  // [m_max]
     int32_t *idx;                   // [m_max]
+    int *dev_status;                // raised by a kernel whose bounded wait gave up
+    bool tc_ok;                     // the tensor-core stream serves this model's first layer
+    int tc_r_max;                   // most k-ranges any plan for this model may use
+    float *tc_part;                 // [R][m_max+1][n_r_max][dims[1]] split-K partials
     void *host_stage;               // device copies of host inputs (zeno_step_host), grown on demand
     size_t host_stage_bytes;
     int last_launches;
@@ -89,7 +101,7 @@ cudaError_t launch_mlp_layer(Context &c, const LayerArgs &a, bool aligned, cudaS
                              int *launches);
 cudaError_t launch_mlp_loss(Context &c, const float *logits, const int32_t *labels, int n_r,
                             int m, int classes, float *losses, cudaStream_t s, int *launches);
-cudaError_t launch_mlp_finalize(Context &c, int m, float rho, const float *losses,
+cudaError_t launch_mlp_finalize(Context &c, const NormSlots &slots, int m, float rho, const float *losses,
                                 float *scores, float *norms_out, cudaStream_t s, int *launches);
 cudaError_t launch_lsq_score(Context &c, const LsqArgs &a, const float *y, float gamma,
                              float rho, bool aligned, float *losses, float *norms, float *scores,
@@ -99,6 +111,16 @@ cudaError_t launch_select(Context &c, const float *scores, int m, int b, int32_t
 cudaError_t launch_aggregate(Context &c, const void *V, int64_t ldv, int m,
                              const int32_t *idx, int k, float *out, bool aligned, cudaStream_t s,
                              int *launches);
+
+// Tensor-core stream for the first layer (fp32 storage).
+bool stream_tc_plan(int sms, int K, int out, int n_r, int m, StreamTcPlan *p);
+int stream_tc_norm_slots(const StreamTcPlan &p);
+cudaError_t launch_stream_tc(Context &c, const StreamTcPlan &p, const float *x, const float *V, int64_t ldv,
+                             int64_t offW, int64_t offB, int K, int out, const float *X, int n_r, int m,
+                             float *part, int np_base, cudaStream_t s, int *launches);
+cudaError_t launch_stream_combine(Context &c, const StreamTcPlan &p, const float *part, const float *x,
+                                  const float *V, int64_t ldv, int64_t offB, int out, int n_r, int m,
+                                  float gamma, int relu, float *H, cudaStream_t s, int *launches);
 
 int lsq_slab_count(const Context &c);
 int mlp_norm_slots(int out);

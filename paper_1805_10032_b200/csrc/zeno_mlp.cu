@@ -246,14 +246,16 @@ __global__ void __launch_bounds__(256) mlp_loss_kernel(const float *logits, cons
     }
 }
 
-// norms[i] = sum of the partial slots (fixed order); scores[i] = f_0 - f_i - rho * norms[i].
-__global__ void mlp_finalize_kernel(const float *normpart, int np_slots, int m, float rho,
+// norms[i] = sum of the partial slots the layers filled (fixed order);
+// scores[i] = f_0 - f_i - rho * norms[i].
+__global__ void mlp_finalize_kernel(const float *normpart, int np_slots, NormSlots used, int m, float rho,
                                     const float *losses, float *scores, float *norms_out) {
     const int lane = threadIdx.x & 31;
     const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (i >= m) return;
     float t = 0.f;
-    for (int s = lane; s < np_slots; s += 32) t += normpart[(int64_t)i * np_slots + s];
+    for (int l = 0; l < used.layers; ++l)
+        for (int s = lane; s < used.count[l]; s += 32) t += normpart[(int64_t)i * np_slots + used.base[l] + s];
     t = warp_sum(t);
     if (lane == 0) {
         if (norms_out) norms_out[i] = t;
@@ -305,12 +307,12 @@ cudaError_t launch_mlp_loss(Context &c, const float *logits, const int32_t *labe
     return cudaGetLastError();
 }
 
-cudaError_t launch_mlp_finalize(Context &c, int m, float rho, const float *losses,
+cudaError_t launch_mlp_finalize(Context &c, const NormSlots &slots, int m, float rho, const float *losses,
                                 float *scores, float *norms_out, cudaStream_t s, int *launches) {
     ++*launches;
     profile_mark(c, "mlp_finalize", s);
     const int warps = 4;
-    mlp_finalize_kernel<<<(m + warps - 1) / warps, warps * 32, 0, s>>>(c.normpart, c.np_slots, m,
+    mlp_finalize_kernel<<<(m + warps - 1) / warps, warps * 32, 0, s>>>(c.normpart, c.np_slots, slots, m,
                                                                       rho, losses, scores, norms_out);
     return cudaGetLastError();
 }

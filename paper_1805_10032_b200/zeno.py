@@ -25,7 +25,7 @@ F32, BF16 = 0, 1
 
 EXPORTS = (
     "zeno_param_count", "zeno_create", "zeno_destroy", "zeno_score", "zeno_select",
-    "zeno_aggregate", "zeno_step", "zeno_step_host", "zeno_profile", "zeno_profile_read",
+    "zeno_aggregate", "zeno_step", "zeno_step_host", "zeno_device_status", "zeno_profile", "zeno_profile_read",
     "zeno_last_launch_count",
     "zeno_last_cuda_error", "zeno_status_string",
 )
@@ -78,6 +78,8 @@ def load_library() -> ctypes.CDLL:
     lib.zeno_step.argtypes = [vp, vp, vp, i64, i32, ctypes.POINTER(Batch), f32, f32, i32, vp, vp, vp, vp]
     lib.zeno_step_host.restype = i32
     lib.zeno_step_host.argtypes = [vp, vp, vp, i64, i32, vp, vp, i32, f32, f32, i32, vp, vp, vp, vp]
+    lib.zeno_device_status.restype = i32
+    lib.zeno_device_status.argtypes = [vp, vp]
     lib.zeno_profile.restype = i32
     lib.zeno_profile.argtypes = [vp, i32]
     lib.zeno_profile_read.restype = i32
@@ -183,6 +185,10 @@ class Zeno:
     @property
     def last_launch_count(self) -> int:
         return int(self._lib.zeno_last_launch_count(self._h))
+
+    def check_device_status(self, stream=None):
+        """Synchronises and raises if a kernel gave up on a bounded device-side wait."""
+        self._check(self._lib.zeno_device_status(self._h, _stream_ptr(stream)), "zeno_device_status")
 
     def profile(self, enable: bool = True):
         self._check(self._lib.zeno_profile(self._h, int(enable)), "zeno_profile")

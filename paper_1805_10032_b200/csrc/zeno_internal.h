@@ -20,8 +20,8 @@ constexpr int kMaxProfiled = ZENO_MAX_LAYERS + 8;
 
 // Launch shape of the tensor-core stream: k-range length, number of k-ranges, blocks per
 // k-range, padded sample count, 128-row tiles per model, dynamic shared memory.
-struct StreamTcPlan { int KR, R, G, n_pad, tiles_per_model, smem_bytes; };
-constexpr int kStreamTcMinKR = 256;
+struct StreamTcPlan { int KR, R, G, n_pad, tiles_per_model, smem_bytes, stages; };
+constexpr int kStreamTcMinKR = 128;
 
 // Which norm-partial slots a call filled: per layer (first slot, count).
 struct NormSlots { int base[ZENO_MAX_LAYERS]; int count[ZENO_MAX_LAYERS]; int layers; };

@@ -8,17 +8,28 @@
 //
 // fp32 accuracy on tf32 tensor cores: both operands are split, a = a_hi + a_lo with a_hi the
 // value rounded to tf32, and the product is accumulated as a_hi b_hi + a_lo b_hi + a_hi b_lo
-// (the dropped a_lo b_lo term is below 2^-22 relative).
+// (the dropped a_lo b_lo term is below 2^-22 relative).  At these small N the MMA is bound by
+// fetching its A operand, so X_hi and X_lo are stacked along N: one MMA reads a_hi once and
+// yields a_hi x_hi and a_hi x_lo side by side; a second one adds a_lo x_hi.
+//
+// The tensor core adds into its fp32 accumulator with truncation, so a long accumulation chain
+// drifts; the two small products go to an accumulator of their own (their truncation error is
+// 2^-11 smaller) and the k-range of a block bounds the length of the chain of large ones.
 //
 // Per block (one SM): a k-range of the input index, whose X_hi / X_lo slices stay resident in
 // shared memory in the 128-byte-swizzled K-major layout the MMA reads, and a list of 128-row
-// tiles of the stacked matrix.  Warp roles:
-//   warp 0      TMA producer: 128 rows x 32 floats boxes of V (or x) into a 4-stage ring
-//   warp 1      TMEM owner and MMA issuer (tcgen05.mma, A operand from TMEM, B from shared)
-//   warps 2-5   converters: thread t owns row t of the tile; reads its 128 bytes from the stage,
-//               accumulates v^2, splits into hi/lo and stores both to TMEM (tcgen05.st) where
-//               the MMA picks them up; after the last k-block they drain the accumulator
-//               (tcgen05.ld) into the split-K partial output.
+// tiles of the stacked matrix.  These MMAs are small (N = n_r), so one issuing thread cannot keep
+// the tensor pipe busy: its waits and commits would leave the pipe idle half of the time.  The
+// block therefore runs TWO independent pipelines side by side, each on its own row tiles, with
+// its own TMA ring, converter warps, MMA issuer, TMEM operand buffers and accumulator; the
+// tensor pipe interleaves their MMAs.  Warp roles (p = pipeline 0 / 1):
+//   warp p        TMA producer: 128 rows x 32 floats boxes of V (or x) into pipeline p's ring
+//   warp 2+p      MMA issuer (tcgen05.mma, A operand from TMEM, B from shared); warp 2 owns TMEM
+//   warps 4-7 / 8-11   converters of pipeline 0 / 1: thread t owns row t of the tile; reads its
+//                 128 bytes from the stage, accumulates v^2, splits into hi/lo and stores both
+//                 to TMEM (tcgen05.st) where the MMA picks them up
+//   warps 12-15   epilogue: drain finished accumulators (tcgen05.ld) into the split-K partial
+//                 output while both pipelines keep going
 // Every mbarrier wait is bounded; a wait that gives up raises a status word and the block leaves
 // through the common teardown (pending bulk copies awaited, TMEM freed).
 #include <cuda.h>
@@ -31,10 +42,13 @@ namespace {
 
 constexpr int kTileRows = 128;          // rows of the stacked matrix per tile = TMEM lanes
 constexpr int kBlockK = 32;             // floats per k-block = one 128-byte swizzle row
-constexpr int kStages = 4;
+constexpr int kPipes = 2;               // independent pipelines per block
+constexpr int kMaxStages = 6;           // TMA ring depth per pipeline
 constexpr int kStageBytes = kTileRows * kBlockK * 4;
-constexpr int kThreads = 192;
-constexpr int kTmemCols = 256;          // D0 @0, D1 @64, A0 @128 (hi 32 + lo 32), A1 @192
+constexpr int kMaxABufs = 2;            // TMEM A buffers per pipeline (hi 32 + lo 32 columns each)
+constexpr int kThreads = 32 * 16;
+constexpr int kTmemCols = 512;          // one accumulator set per pipeline, then the A buffers (see TmemLayout)
+constexpr int kSmemBudget = 220 * 1024;
 constexpr uint32_t kSpinLimit = 1u << 22;
 
 // ---- PTX wrappers -------------------------------------------------------------------------
@@ -122,6 +136,19 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
     return d;
 }
 
+// TMEM columns.  Pipeline p's accumulator set holds D1 = a_hi [x_hi; x_lo]^T (2 n_pad columns)
+// and D2 = a_lo x_hi^T (n_pad columns); the A buffers (64 columns each) follow the two sets,
+// n_abufs per pipeline.
+struct TmemLayout {
+    int set_stride, d2_off, a_base, n_abufs;
+    __host__ __device__ explicit TmemLayout(int n_pad) {
+        set_stride = n_pad <= 32 ? 128 : 192;
+        d2_off = n_pad <= 32 ? 64 : 128;
+        a_base = kPipes * set_stride;
+        n_abufs = (kTmemCols - a_base) / (64 * kPipes);
+    }
+};
+
 struct StreamArgs {
     const float *X;        // [n_r x K] the server batch
     const float *V;        // for the bias entries' v^2
@@ -133,6 +160,7 @@ struct StreamArgs {
     int K, out, n_r, n_pad, m;
     int KR;                // floats of K per k-range (multiple of 32)
     int tiles_per_model;   // ceil(out / 128)
+    int stages;            // depth of each pipeline's TMA ring (<= kMaxStages)
     int *status;           // device status word (raised on a wait that gave up)
 };
 
@@ -140,10 +168,12 @@ __global__ void __launch_bounds__(kThreads, 1)
 stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_v,
                      StreamArgs a) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bars[kStages * 2 + 8];
+    // per pipeline: full[kMaxStages], empty[kMaxStages], a_full[kMaxABufs], a_empty[kMaxABufs], d_full, d_empty
+    constexpr int kBarsPerPipe = 2 * kMaxStages + 2 * kMaxABufs + 2;
+    __shared__ __align__(8) uint64_t bars[kPipes * kBarsPerPipe];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
-    __shared__ int issued[kStages];
+    __shared__ int issued[kPipes][kMaxStages];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int r = blockIdx.x;                         // k-range
@@ -151,149 +181,166 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     const int k_len = min(a.KR, a.K - k0);
     const int nkb = (k_len + kBlockK - 1) / kBlockK;   // k-blocks in this range
     const int n_items_total = (a.m + 1) * a.tiles_per_model;
+    const int n_stages = a.stages;
 
     // shared memory carve-up (dynamic part is 1024-byte aligned)
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int nkb_max = a.KR / kBlockK;
-    const uint32_t xs_bytes = (uint32_t)nkb_max * a.n_pad * 128;
-    uint8_t *xs_hi = base;
-    uint8_t *xs_lo = base + xs_bytes;
-    uint8_t *stages = base + 2 * xs_bytes;            // xs_bytes is a multiple of 1024 (n_pad % 16 == 0)
+    const uint32_t xkb_bytes = 2u * a.n_pad * 128;     // one k-block of [X_hi; X_lo]: a multiple of 1024
+    uint8_t *xs = base;
+    uint8_t *stage_base = base + (uint32_t)nkb_max * xkb_bytes;   // pipeline p's ring at p * n_stages * kStageBytes
+    const TmemLayout tl(a.n_pad);
+    const int n_abufs = tl.n_abufs;
 
-    const uint32_t bar_full = smem_u32(&bars[0]);               // + 8 * stage
-    const uint32_t bar_empty = smem_u32(&bars[kStages]);
-    const uint32_t bar_afull = smem_u32(&bars[2 * kStages]);     // 2 TMEM A buffers
-    const uint32_t bar_aempty = smem_u32(&bars[2 * kStages + 2]);
-    const uint32_t bar_dfull = smem_u32(&bars[2 * kStages + 4]);  // 2 accumulators
-    const uint32_t bar_dempty = smem_u32(&bars[2 * kStages + 6]);
+    auto bar_full = [&](int p, int s) { return smem_u32(&bars[p * kBarsPerPipe + s]); };
+    auto bar_empty = [&](int p, int s) { return smem_u32(&bars[p * kBarsPerPipe + kMaxStages + s]); };
+    auto bar_afull = [&](int p, int b) { return smem_u32(&bars[p * kBarsPerPipe + 2 * kMaxStages + b]); };
+    auto bar_aempty = [&](int p, int b) { return smem_u32(&bars[p * kBarsPerPipe + 2 * kMaxStages + kMaxABufs + b]); };
+    auto bar_dfull = [&](int p) { return smem_u32(&bars[p * kBarsPerPipe + 2 * kMaxStages + 2 * kMaxABufs]); };
+    auto bar_dempty = [&](int p) { return smem_u32(&bars[p * kBarsPerPipe + 2 * kMaxStages + 2 * kMaxABufs + 1]); };
 
     if (tid == 0) {
         abort_flag = 0;
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_empty + 8 * s, 4);
-            issued[s] = 0;
-        }
-        for (int q = 0; q < 2; ++q) {
-            mbar_init(bar_afull + 8 * q, 4);
-            mbar_init(bar_aempty + 8 * q, 1);
-            mbar_init(bar_dfull + 8 * q, 1);
-            mbar_init(bar_dempty + 8 * q, 4);
+        for (int p = 0; p < kPipes; ++p) {
+            for (int s = 0; s < kMaxStages; ++s) {
+                mbar_init(bar_full(p, s), 1);
+                mbar_init(bar_empty(p, s), 4);
+                issued[p][s] = 0;
+            }
+            for (int b = 0; b < kMaxABufs; ++b) {
+                mbar_init(bar_afull(p, b), 4);
+                mbar_init(bar_aempty(p, b), 1);
+            }
+            mbar_init(bar_dfull(p), 1);
+            mbar_init(bar_dempty(p), 4);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {   // TMEM allocation by one full warp
+    if (warp == 2) {   // TMEM allocation by one full warp
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(&tmem_base_slot)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-
-    // X_hi / X_lo of this k-range in the swizzled K-major layout: row j of k-block kb at
-    // kb * n_pad * 128 + j * 128, its 16-byte chunk c at position c ^ (j & 7).
-    for (int t = tid; t < nkb_max * a.n_pad * 8; t += kThreads) {
-        const int c = t & 7, j = (t >> 3) % a.n_pad, kb = (t >> 3) / a.n_pad;
-        const int k = k0 + kb * kBlockK + c * 4;
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (j < a.n_r && k < a.K && kb < nkb) v = __ldg(reinterpret_cast<const float4 *>(a.X + (int64_t)j * a.K + k));
-        float4 hi = make_float4(tf32_hi(v.x), tf32_hi(v.y), tf32_hi(v.z), tf32_hi(v.w));
-        float4 lo = make_float4(v.x - hi.x, v.y - hi.y, v.z - hi.z, v.w - hi.w);
-        const uint32_t off = (uint32_t)kb * a.n_pad * 128 + j * 128 + ((c ^ (j & 7)) << 4);
-        *reinterpret_cast<float4 *>(xs_hi + off) = hi;
-        *reinterpret_cast<float4 *>(xs_lo + off) = lo;
-    }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> tensor-core reads
     tc_fence_before();
-    __syncthreads();
+    __syncthreads();                                   // barriers and the TMEM base are visible
     tc_fence_after();
     const uint32_t tmem = tmem_base_slot;
     volatile int *abortp = &abort_flag;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
+    // [X_hi; X_lo] of this k-range in the swizzled K-major layout: k-block kb at kb * xkb_bytes,
+    // row j of X_hi at j * 128, of X_lo at (n_pad + j) * 128, 16-byte chunk c at c ^ (row & 7).
+    // Everyone but the producer warps fills it while the first V tiles are already in flight.
+    if (warp >= kPipes) {
+        constexpr int kFillers = kThreads - 32 * kPipes;
+        for (int t = tid - 32 * kPipes; t < nkb_max * a.n_pad * 8; t += kFillers) {
+            const int c = t & 7, j = (t >> 3) % a.n_pad, kb = (t >> 3) / a.n_pad;
+            const int k = k0 + kb * kBlockK + c * 4;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (j < a.n_r && k < a.K && kb < nkb) v = __ldg(reinterpret_cast<const float4 *>(a.X + (int64_t)j * a.K + k));
+            float4 hi = make_float4(tf32_hi(v.x), tf32_hi(v.y), tf32_hi(v.z), tf32_hi(v.w));
+            float4 lo = make_float4(v.x - hi.x, v.y - hi.y, v.z - hi.z, v.w - hi.w);
+            const uint32_t off = (uint32_t)kb * xkb_bytes + j * 128 + ((c ^ (j & 7)) << 4);
+            *reinterpret_cast<float4 *>(xs + off) = hi;
+            *reinterpret_cast<float4 *>(xs + off + a.n_pad * 128) = lo;   // n_pad % 8 == 0: same swizzle phase
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> tensor-core reads
+        asm volatile("bar.sync 1, %0;" ::"n"(kFillers) : "memory");      // named barrier: all but the producers
+    }
+
+    // Item li of this block (li = 0, 1, ..) is row tile blockIdx.y + li * gridDim.y of the stacked
+    // matrix; pipeline p takes the items with li % kPipes == p.
+    if (warp < kPipes) {
+        // ------------------------------------------------------------------ TMA producers
+        const int p = warp;
         if (lane == 0) {
+            uint8_t *ring = stage_base + (size_t)p * n_stages * kStageBytes;
             uint32_t it = 0;
-            for (int item = blockIdx.y; item < n_items_total && !*abortp; item += gridDim.y) {
+            for (int item = blockIdx.y + p * gridDim.y; item < n_items_total && !*abortp; item += kPipes * gridDim.y) {
                 const int model = item / a.tiles_per_model, tile = item % a.tiles_per_model;
+                // one issue site for both operands: x is a one-model stack
+                const CUtensorMap *map = model == 0 ? &map_x : &map_v;
+                const int c2 = max(model - 1, 0);
                 for (int kb = 0; kb < nkb; ++kb, ++it) {
-                    const int s = it % kStages;
-                    if (!mbar_wait(bar_empty + 8 * s, ((it / kStages) & 1) ^ 1, abortp)) break;
-                    mbar_expect_tx(bar_full + 8 * s, kStageBytes);
-                    const uint32_t dst = smem_u32(stages + s * kStageBytes);
-                    // one issue site for both operands: x is a one-model stack
-                    const CUtensorMap *map = model == 0 ? &map_x : &map_v;
-                    tma_load_3d(dst, map, k0 + kb * kBlockK, tile * kTileRows, max(model - 1, 0), bar_full + 8 * s);
-                    issued[s] = (int)(it / kStages) + 1;
+                    const int s = it % n_stages;
+                    if (!mbar_wait(bar_empty(p, s), ((it / n_stages) & 1) ^ 1, abortp)) break;
+                    mbar_expect_tx(bar_full(p, s), kStageBytes);
+                    tma_load_3d(smem_u32(ring + s * kStageBytes), map, k0 + kb * kBlockK, tile * kTileRows, c2,
+                                bar_full(p, s));
+                    issued[p][s] = (int)(it / n_stages) + 1;
                 }
             }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
+    } else if (warp < 2 * kPipes) {
+        // ------------------------------------------------------------------ MMA issuers
+        const int p = warp - kPipes;
         if (lane == 0) {
-            // instruction descriptor: D fp32, A and B tf32, both K-major, N = n_pad, M = 128
+            // instruction descriptors: D fp32, A and B tf32, both K-major, M = 128, N = n_pad / 2 n_pad
             const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(a.n_pad >> 3) << 17) |
                                    ((uint32_t)(kTileRows >> 4) << 24);
+            const uint32_t idesc2 = (idesc & ~(0x3fu << 17)) | ((uint32_t)((2 * a.n_pad) >> 3) << 17);
+            const uint32_t d1 = tmem + p * tl.set_stride, d2 = d1 + tl.d2_off;
+            const uint32_t a_bufs = tmem + tl.a_base + p * n_abufs * 64;
             uint32_t it = 0, q = 0;
-            for (int item = blockIdx.y; item < n_items_total && !*abortp; item += gridDim.y, ++q) {
-                const uint32_t d_tmem = tmem + (q & 1) * 64;
-                if (!mbar_wait(bar_dempty + 8 * (q & 1), ((q >> 1) & 1) ^ 1, abortp)) break;
+            for (int item = blockIdx.y + p * gridDim.y; item < n_items_total && !*abortp; item += kPipes * gridDim.y, ++q) {
+                if (!mbar_wait(bar_dempty(p), (q & 1) ^ 1, abortp)) break;    // accumulator drained
                 tc_fence_after();
                 bool ok = true;
                 for (int kb = 0; kb < nkb; ++kb, ++it) {
-                    const uint32_t ab = it & 1;
-                    if (!mbar_wait(bar_afull + 8 * ab, (it >> 1) & 1, abortp)) { ok = false; break; }
+                    const uint32_t ab = it % n_abufs;
+                    if (!mbar_wait(bar_afull(p, ab), (it / n_abufs) & 1, abortp)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t a_tmem = tmem + 128 + ab * 64;
-                    const uint32_t bh = smem_u32(xs_hi) + (uint32_t)kb * a.n_pad * 128;
-                    const uint32_t bl = smem_u32(xs_lo) + (uint32_t)kb * a.n_pad * 128;
+                    const uint32_t a_tmem = a_bufs + ab * 64;
+                    const uint32_t bx = smem_u32(xs) + (uint32_t)kb * xkb_bytes;
 #pragma unroll
                     for (int ks = 0; ks < kBlockK / 8; ++ks) {
-                        const uint64_t dh = smem_desc_sw128(bh + ks * 32);
-                        const uint64_t dl = smem_desc_sw128(bl + ks * 32);
-                        tc_mma_tf32_ts(d_tmem, a_tmem + ks * 8, dh, idesc, (kb | ks) != 0);        // a_hi x_hi
-                        tc_mma_tf32_ts(d_tmem, a_tmem + 32 + ks * 8, dh, idesc, 1);                // a_lo x_hi
-                        tc_mma_tf32_ts(d_tmem, a_tmem + ks * 8, dl, idesc, 1);                     // a_hi x_lo
+                        const uint64_t db = smem_desc_sw128(bx + ks * 32);
+                        tc_mma_tf32_ts(d1, a_tmem + ks * 8, db, idesc2, (kb | ks) != 0);       // a_hi [x_hi; x_lo]
+                        tc_mma_tf32_ts(d2, a_tmem + 32 + ks * 8, db, idesc, (kb | ks) != 0);   // a_lo x_hi
                     }
-                    tc_commit(bar_aempty + 8 * ab);    // the A buffer may be overwritten once these finish
+                    tc_commit(bar_aempty(p, ab));      // the A buffer may be overwritten once these finish
                 }
                 if (!ok) break;
-                tc_commit(bar_dfull + 8 * (q & 1));    // accumulator complete
+                tc_commit(bar_dfull(p));               // accumulators complete
             }
         }
-    } else {
-        // ------------------------------------------------------------------ converters + epilogue
+    } else if (warp < 2 * kPipes + 4 * kPipes) {
+        // ------------------------------------------------------------------ converters
+        const int p = (warp - 2 * kPipes) >> 2;
         const int quad = warp & 3;                    // TMEM lane quadrant this warp may access
         const int row = quad * 32 + lane;             // row of the tile = TMEM lane
         const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-        uint32_t it = 0, q = 0;
-        for (int item = blockIdx.y; item < n_items_total && !*abortp; item += gridDim.y, ++q) {
+        const uint8_t *ring = stage_base + (size_t)p * n_stages * kStageBytes;
+        const uint32_t a_bufs = tmem + lane_addr + tl.a_base + p * n_abufs * 64;
+        uint32_t it = 0;
+        for (int item = blockIdx.y + p * gridDim.y; item < n_items_total && !*abortp; item += kPipes * gridDim.y) {
             const int model = item / a.tiles_per_model, tile = item % a.tiles_per_model;
-            float nrm = 0.f;
+            float nrm4[4] = {0.f, 0.f, 0.f, 0.f};
             bool ok = true;
             for (int kb = 0; kb < nkb; ++kb, ++it) {
-                const int s = it % kStages;
-                if (!mbar_wait(bar_full + 8 * s, (it / kStages) & 1, abortp)) { ok = false; break; }
-                const uint8_t *src = stages + s * kStageBytes + row * 128;
+                const int s = it % n_stages;
+                if (!mbar_wait(bar_full(p, s), (it / n_stages) & 1, abortp)) { ok = false; break; }
+                const uint8_t *src = ring + s * kStageBytes + row * 128;
                 float4 v[8];
 #pragma unroll
                 for (int c = 0; c < 8; ++c) v[c] = *reinterpret_cast<const float4 *>(src + ((c ^ (row & 7)) << 4));
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar_empty + 8 * s);      // the stage may be refilled
+                if (lane == 0) mbar_arrive(bar_empty(p, s));        // the stage may be refilled
                 uint32_t hi[32], lo[32];
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
                     const float e[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
-                        nrm = fmaf(e[u], e[u], nrm);
+                        nrm4[u] = fmaf(e[u], e[u], nrm4[u]);
                         const float h = tf32_hi(e[u]);
                         hi[4 * c + u] = __float_as_uint(h);
                         lo[4 * c + u] = __float_as_uint(e[u] - h);
                     }
                 }
-                const uint32_t ab = it & 1;
-                if (!mbar_wait(bar_aempty + 8 * ab, ((it >> 1) & 1) ^ 1, abortp)) { ok = false; break; }
+                const uint32_t ab = it % n_abufs;
+                if (!mbar_wait(bar_aempty(p, ab), ((it / n_abufs) & 1) ^ 1, abortp)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t a_tmem = tmem + lane_addr + 128 + ab * 64;
+                const uint32_t a_tmem = a_bufs + ab * 64;
                 tc_st16(a_tmem, reinterpret_cast<const uint32_t(&)[16]>(hi[0]));
                 tc_st16(a_tmem + 16, reinterpret_cast<const uint32_t(&)[16]>(hi[16]));
                 tc_st16(a_tmem + 32, reinterpret_cast<const uint32_t(&)[16]>(lo[0]));
@@ -301,12 +348,13 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar_afull + 8 * ab);
+                if (lane == 0) mbar_arrive(bar_afull(p, ab));
             }
             if (!ok) break;
 
             // partial sum of squares of this tile's rows (model 0 is x itself: not a candidate)
             if (model > 0) {
+                float nrm = (nrm4[0] + nrm4[1]) + (nrm4[2] + nrm4[3]);
                 const int o = tile * kTileRows + row;
                 if (r == 0 && a.offB >= 0 && o < a.out) {
                     const float bv = __ldg(a.V + (int64_t)(model - 1) * a.ldv + a.offB + o);
@@ -318,25 +366,42 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                     a.normpart[(int64_t)(model - 1) * a.np_slots + a.np_base +
                                (r * a.tiles_per_model + tile) * 4 + quad] = nrm;
             }
-
-            // drain the accumulator: thread = output row o, column = sample j
-            if (!mbar_wait(bar_dfull + 8 * (q & 1), (q >> 1) & 1, abortp)) break;
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue
+        const int quad = warp & 3;
+        const int row = quad * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+        uint32_t li = 0;
+        for (int item = blockIdx.y; item < n_items_total && !*abortp; item += gridDim.y, ++li) {
+            const int model = item / a.tiles_per_model, tile = item % a.tiles_per_model;
+            const int p = li % kPipes;
+            const uint32_t q = li / kPipes;               // how many accumulators pipeline p has finished before
+            // thread = output row o, column = sample j
+            if (!mbar_wait(bar_dfull(p), q & 1, abortp)) break;
             tc_fence_after();
             const int o = tile * kTileRows + row;
             float *dst = a.part + (((int64_t)r * (a.m + 1) + model) * a.n_r) * a.out + o;
+            const uint32_t dset = tmem + lane_addr + p * tl.set_stride;
             for (int j0 = 0; j0 < a.n_pad; j0 += 16) {
-                uint32_t acc[16];
-                tc_ld16(tmem + lane_addr + (q & 1) * 64 + j0, acc);
+                uint32_t big[16], s1[16], s2[16];
+                tc_ld16(dset + j0, big);                       // a_hi x_hi
+                tc_ld16(dset + a.n_pad + j0, s1);              // a_hi x_lo
+                tc_ld16(dset + tl.d2_off + j0, s2);            // a_lo x_hi
                 tc_wait_ld();
+                if (j0 + 16 >= a.n_pad) {                      // everything is in registers: release the accumulator
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_dempty(p));
+                }
                 if (o < a.out) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
-                        if (j0 + j < a.n_r) dst[(int64_t)(j0 + j) * a.out] = __uint_as_float(acc[j]);
+                        if (j0 + j < a.n_r)
+                            dst[(int64_t)(j0 + j) * a.out] =
+                                __uint_as_float(big[j]) + (__uint_as_float(s1[j]) + __uint_as_float(s2[j]));
                 }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_dempty + 8 * (q & 1));
         }
     }
 
@@ -347,18 +412,19 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     if (tid == 0) {
         // bulk copies still in flight (only after an aborted run) must land before the block exits
         if (abort_flag) {
-            for (int s = 0; s < kStages; ++s)
-                if (issued[s] > 0) {
-                    for (uint32_t i = 0; i < kSpinLimit; ++i) {
-                        if (mbar_try_wait(bar_full + 8 * s, (uint32_t)(issued[s] - 1) & 1)) break;
-                        __nanosleep(64);
+            for (int p = 0; p < kPipes; ++p)
+                for (int s = 0; s < n_stages; ++s)
+                    if (issued[p][s] > 0) {
+                        for (uint32_t i = 0; i < kSpinLimit; ++i) {
+                            if (mbar_try_wait(bar_full(p, s), (uint32_t)(issued[p][s] - 1) & 1)) break;
+                            __nanosleep(64);
+                        }
                     }
-                }
             atomicMax(a.status, 1);
         }
     }
     __syncthreads();
-    if (warp == 1) {
+    if (warp == 2) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
 }
@@ -422,9 +488,12 @@ bool stream_tc_plan(int sms, int K, int out, int n_r, int m, StreamTcPlan *p) {
     const int n_pad = (n_r + 15) / 16 * 16;
     const int tiles = (out + kTileRows - 1) / kTileRows;
     const int items = (m + 1) * tiles;
-    const int kr_cap = n_pad <= 32 ? 512 : 256;      // X_hi + X_lo <= 128 KB of shared memory
     double best = -1.0;
-    for (int kr = kStreamTcMinKR; kr <= kr_cap; kr *= 2) {
+    for (int kr = kStreamTcMinKR; kr <= 512; kr *= 2) {
+        const int xs = 2 * (kr / kBlockK) * n_pad * 128;            // [X_hi; X_lo]
+        int stages = (kSmemBudget - 1024 - xs) / (kPipes * kStageBytes);   // per pipeline
+        if (stages > kMaxStages) stages = kMaxStages;
+        if (stages < 2) continue;
         const int R = (K + kr - 1) / kr;
         if (R > sms) continue;
         int G = sms / R;
@@ -432,16 +501,17 @@ bool stream_tc_plan(int sms, int K, int out, int n_r, int m, StreamTcPlan *p) {
         if (G < 1) G = 1;
         const int per = (items + G - 1) / G;
         double eff = (double)items / ((double)G * per) * ((double)(R * G) / sms);
-        eff -= 0.01 * R;                               // split-K partial traffic grows with R
+        eff -= 0.005 * R;                              // split-K partial traffic grows with R
+        if (stages < 4) eff -= 0.05;                   // a shallow ring hides less latency
         if (eff > best) {
             best = eff;
-            p->KR = kr; p->R = R; p->G = G;
+            p->KR = kr; p->R = R; p->G = G; p->stages = stages;
         }
     }
     if (best < 0) return false;
     p->n_pad = n_pad;
     p->tiles_per_model = tiles;
-    p->smem_bytes = 2 * (p->KR / kBlockK) * n_pad * 128 + kStages * kStageBytes + 1024;
+    p->smem_bytes = 2 * (p->KR / kBlockK) * n_pad * 128 + kPipes * p->stages * kStageBytes + 1024;
     return true;
 }
 
@@ -489,11 +559,12 @@ cudaError_t launch_stream_tc(Context &c, const StreamTcPlan &p, const float *x, 
     a.m = m;
     a.KR = p.KR;
     a.tiles_per_model = p.tiles_per_model;
+    a.stages = p.stages;
     a.status = c.dev_status;
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(stream_tf32x3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             200 * 1024);
+                                             kSmemBudget);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }

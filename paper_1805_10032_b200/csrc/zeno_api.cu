@@ -84,9 +84,13 @@ zeno_status check_common(const Context *c, const void *V, int64_t ldv, int32_t m
     return ZENO_OK;
 }
 
+// keep > 0 asks for the ranking as well (idx[0..keep)); *ranked tells whether the scoring pass
+// delivered it (the MLP tail does) or a separate select launch is still needed.
 zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv, int32_t m,
                           const zeno_batch *batch, float gamma, float rho, float *scores,
-                          float *losses, float *norms, cudaStream_t s, int *launches) {
+                          float *losses, float *norms, int keep, int32_t *idx, bool *ranked,
+                          cudaStream_t s, int *launches) {
+    *ranked = false;
     zeno_status st = check_common(c, V, ldv, m);
     if (st != ZENO_OK) return st;
     if (!x || !batch || !batch->features || !batch->targets || !scores) return ZENO_ERR_INVALID_ARG;
@@ -115,14 +119,23 @@ zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv,
     }
 
     const int L = c->desc.n_layers;
-    zeno::NormSlots used;
-    used.layers = L;
+    zeno::TailArgs tail;
+    tail.normpart = c->normpart;
+    tail.np_slots = c->np_slots;
+    tail.used.layers = L;
+    tail.m = m;
+    tail.rho = rho;
+    tail.scores = scores;
+    tail.norms_out = norms;
+    tail.idx = idx;
+    tail.keep = keep;
+    tail.ticket = c->tickets;
     int first_cuda_layer = 0;
     // first layer on the tensor cores when the shape and the alignment allow it
     zeno::StreamTcPlan plan;
     if (c->tc_ok && aligned &&
         zeno::stream_tc_plan(c->sm_count, (int)c->desc.dims[0], (int)c->desc.dims[1], n_r, m, &plan) &&
-        plan.R <= c->tc_r_max) {
+        plan.R <= c->tc_r_max && L >= 2) {
         const float *xf = static_cast<const float *>(x);
         const float *Vf = static_cast<const float *>(V);
         e = zeno::launch_stream_tc(*c, plan, xf, Vf, ldv, c->offW[0], c->offB[0], (int)c->desc.dims[0],
@@ -130,12 +143,14 @@ zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv,
                                    s, launches);
         if (e != cudaSuccess) return fail_cuda(c, e);
         e = zeno::launch_stream_combine(*c, plan, c->tc_part, xf, Vf, ldv, c->offB[0], (int)c->desc.dims[1],
-                                        n_r, m, gamma, L > 1, c->act[0], s, launches);
+                                        n_r, m, gamma, 1, c->act[0], s, launches);
         if (e != cudaSuccess) return fail_cuda(c, e);
-        used.base[0] = c->np_base[0];
-        used.count[0] = zeno::stream_tc_norm_slots(plan);
+        tail.used.base[0] = c->np_base[0];
+        tail.used.count[0] = zeno::stream_tc_norm_slots(plan);
         first_cuda_layer = 1;
     }
+    const int classes = (int)c->desc.dims[L];
+    const bool fuse_loss = zeno::mlp_can_fuse_loss(classes, n_r);
     for (int l = first_cuda_layer; l < L; ++l) {
         zeno::LayerArgs a;
         a.x = x;
@@ -155,16 +170,22 @@ zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv,
         a.normpart = c->normpart;
         a.np_slots = c->np_slots;
         a.np_base = c->np_base[l];
-        used.base[l] = c->np_base[l];
-        used.count[l] = zeno::mlp_norm_slots(a.out);
+        tail.used.base[l] = c->np_base[l];
+        tail.used.count[l] = zeno::mlp_norm_slots(a.out);
+        a.fuse_loss = (l + 1 == L) && fuse_loss;
+        a.labels = static_cast<const int32_t *>(batch->targets);
+        a.losses = loss_buf;
+        a.tail = tail;                               // complete by the time the last layer is reached
         e = zeno::launch_mlp_layer(*c, a, aligned, s, launches);
         if (e != cudaSuccess) return fail_cuda(c, e);
     }
-    e = zeno::launch_mlp_loss(*c, c->act[(L - 1) & 1], static_cast<const int32_t *>(batch->targets),
-                              n_r, m, (int)c->desc.dims[L], loss_buf, s, launches);
-    if (e != cudaSuccess) return fail_cuda(c, e);
-    e = zeno::launch_mlp_finalize(*c, used, m, rho, loss_buf, scores, norms, s, launches);
-    return e == cudaSuccess ? ZENO_OK : fail_cuda(c, e);
+    if (!fuse_loss) {
+        e = zeno::launch_mlp_loss(*c, c->act[(L - 1) & 1], static_cast<const int32_t *>(batch->targets),
+                                  n_r, m, classes, loss_buf, tail, s, launches);
+        if (e != cudaSuccess) return fail_cuda(c, e);
+    }
+    *ranked = keep > 0;
+    return ZENO_OK;
 }
 
 zeno_status enqueue_select(Context *c, const float *scores, int32_t m, int32_t b, int32_t *idx,
@@ -231,7 +252,7 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
     c->sm_count = prop.multiProcessorCount;
 
     const size_t rows = (size_t)m_max + 1;
-    size_t act_elems = 0, norm_elems = 0, lsq_elems = 0, tc_elems = 0;
+    size_t act_elems = 0, norm_elems = 0, lsq_elems = 0, tc_elems = 0, ticket_elems = 1;
     if (desc->kind == ZENO_LOSS_SOFTMAX_MLP) {
         int64_t off = 0, widest = 0;
         int slots = 0;
@@ -255,6 +276,7 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
                     const int tc_slots = zeno::stream_tc_norm_slots(probe);
                     if (tc_slots > layer_slots) layer_slots = tc_slots;
                     tc_elems = (size_t)c->tc_r_max * rows * (size_t)n_r_max * (size_t)o;
+
                 }
             }
             slots += layer_slots;
@@ -279,6 +301,7 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
     const size_t at_loss = reserve(rows, 4), at_norms = reserve(m_max, 4);
     const size_t at_scores = reserve(m_max, 4), at_idx = reserve(m_max, 4);
     const size_t at_status = reserve(1, 4), at_tc = reserve(tc_elems, 4);
+    const size_t at_tickets = reserve(ticket_elems, 4);
 
     e = cudaMalloc(&c->arena, bytes);
     if (e != cudaSuccess) {
@@ -297,7 +320,9 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
     c->idx = reinterpret_cast<int32_t *>(base + at_idx);
     c->dev_status = reinterpret_cast<int *>(base + at_status);
     c->tc_part = reinterpret_cast<float *>(base + at_tc);
+    c->tickets = reinterpret_cast<unsigned *>(base + at_tickets);
     e = cudaMemset(c->dev_status, 0, sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(c->tickets, 0, ticket_elems * sizeof(unsigned));
     if (e != cudaSuccess) {
         cudaFree(c->arena);
         delete c;
@@ -326,8 +351,9 @@ zeno_status zeno_score(zeno_handle h, const void *x, const void *V, int64_t ldv,
     if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
     int launches = 0;
     profile_begin(h);
-    zeno_status st = enqueue_score(h, x, V, ldv, m, batch, gamma, rho, scores, losses, norms,
-                                   static_cast<cudaStream_t>(stream), &launches);
+    bool ranked = false;
+    zeno_status st = enqueue_score(h, x, V, ldv, m, batch, gamma, rho, scores, losses, norms, 0, nullptr,
+                                   &ranked, static_cast<cudaStream_t>(stream), &launches);
     profile_end(h, static_cast<cudaStream_t>(stream));
     h->last_launches = st == ZENO_OK ? launches : 0;
     return st;
@@ -372,9 +398,10 @@ zeno_status zeno_step(zeno_handle h, const void *x, const void *V, int64_t ldv, 
     int32_t *idx_buf = idx ? idx : h->idx;
     int launches = 0;
     profile_begin(h);
-    zeno_status st = enqueue_score(h, x, V, ldv, m, batch, gamma, rho, score_buf, nullptr, nullptr, s,
-                                   &launches);
-    if (st == ZENO_OK) st = enqueue_select(h, score_buf, m, b, idx_buf, s, &launches);
+    bool ranked = false;
+    zeno_status st = enqueue_score(h, x, V, ldv, m, batch, gamma, rho, score_buf, nullptr, nullptr, m - b,
+                                   idx_buf, &ranked, s, &launches);
+    if (st == ZENO_OK && !ranked) st = enqueue_select(h, score_buf, m, b, idx_buf, s, &launches);
     if (st == ZENO_OK) st = enqueue_aggregate(h, V, ldv, m, idx_buf, m - b, out, s, &launches);
     profile_end(h, s);
     h->last_launches = st == ZENO_OK ? launches : 0;
@@ -431,9 +458,10 @@ zeno_status zeno_step_host(zeno_handle h, const void *x, const void *V, int64_t 
     batch.n_r = n_r;
     int launches = 0;
     profile_begin(h);
-    zeno_status st = enqueue_score(h, dx, dV, ldv, m, &batch, gamma, rho, h->scores, nullptr, nullptr, s,
-                                   &launches);
-    if (st == ZENO_OK) st = enqueue_select(h, h->scores, m, b, h->idx, s, &launches);
+    bool ranked = false;
+    zeno_status st = enqueue_score(h, dx, dV, ldv, m, &batch, gamma, rho, h->scores, nullptr, nullptr, m - b,
+                                   h->idx, &ranked, s, &launches);
+    if (st == ZENO_OK && !ranked) st = enqueue_select(h, h->scores, m, b, h->idx, s, &launches);
     if (st == ZENO_OK) st = enqueue_aggregate(h, dV, ldv, m, h->idx, m - b, dout, s, &launches);
     profile_end(h, s);
     if (st != ZENO_OK) {

@@ -49,6 +49,7 @@ struct Context {
     bool tc_ok;                     // the tensor-core stream serves this model's first layer
     int tc_r_max;                   // most k-ranges any plan for this model may use
     float *tc_part;                 // [R][m_max+1][n_r_max][dims[1]] split-K partials
+    unsigned *tickets;              // the tail's arrival counter, zero between launches
     void *host_stage;               // device copies of host inputs (zeno_step_host), grown on demand
     size_t host_stage_bytes;
     int last_launches;
@@ -68,6 +69,21 @@ inline void profile_mark(Context &c, const char *name, cudaStream_t s) {
     c.kernel_names[c.profiled++] = name;
 }
 
+// What the last block of the scoring pass needs to turn losses and norm partials into scores
+// (and, if keep > 0, into the ranking).
+struct TailArgs {
+    const float *normpart;
+    int np_slots;
+    NormSlots used;
+    int m;
+    float rho;
+    float *scores;
+    float *norms_out;   // may be NULL
+    int32_t *idx;       // used if keep > 0
+    int keep;           // m - b, or 0: no ranking wanted
+    unsigned *ticket;   // zero between launches
+};
+
 // One dense layer of all m+1 models (candidate 0 is x itself).
 struct LayerArgs {
     const void *x;
@@ -75,14 +91,19 @@ struct LayerArgs {
     int64_t ldv;
     int64_t offW, offB;
     int in, out;
-    const float *Hin;
-    int64_t hin_cand_stride;  // 0: the input activations are shared (layer 1)
+    const float *Hin;         // input activations [m+1][n_r][in] (shared features: stride 0)
+    int64_t hin_cand_stride;
     float *Hout;              // [m+1][n_r][out]
     int n_r, m;
     float gamma;
     int relu;
     float *normpart;
     int np_slots, np_base;
+    // last layer only: fold the cross-entropy (and the tail) into this launch
+    int fuse_loss;
+    const int32_t *labels;
+    float *losses;
+    TailArgs tail;
 };
 
 struct LsqArgs {
@@ -100,9 +121,9 @@ struct LsqArgs {
 cudaError_t launch_mlp_layer(Context &c, const LayerArgs &a, bool aligned, cudaStream_t s,
                              int *launches);
 cudaError_t launch_mlp_loss(Context &c, const float *logits, const int32_t *labels, int n_r,
-                            int m, int classes, float *losses, cudaStream_t s, int *launches);
-cudaError_t launch_mlp_finalize(Context &c, const NormSlots &slots, int m, float rho, const float *losses,
-                                float *scores, float *norms_out, cudaStream_t s, int *launches);
+                            int m, int classes, float *losses, const TailArgs &tail, cudaStream_t s,
+                            int *launches);
+bool mlp_can_fuse_loss(int out, int n_r);
 cudaError_t launch_lsq_score(Context &c, const LsqArgs &a, const float *y, float gamma,
                              float rho, bool aligned, float *losses, float *norms, float *scores,
                              cudaStream_t s, int *launches);

@@ -5,9 +5,15 @@
 // itself).  A warp owns kRowsPerWarp output rows of one model: its lanes stride the input
 // index k, form w = x - gamma v in registers straight from the loads of x and V (the
 // perturbed model never exists in memory), accumulate the n_r dot products and, in the same
-// pass, the sum of squares of the V entries they touched (the rho ||v||^2 term).  The input
-// activations of the layer are staged through shared memory with cp.async, double buffered.
+// pass, the sum of squares of the V entries they touched (the rho ||v||^2 term).  The loads of
+// the next 128 columns are issued before the current ones are consumed; the layer's input
+// activations are staged through shared memory, double buffered.
+//
+// The last layer, when it fits one block per model, also evaluates the cross-entropy; the block
+// that finishes last (a ticket, no waiting) then forms the scores and the ranking, so the whole
+// tail of the scoring pass costs no extra launch.
 #include "zeno_internal.h"
+#include "zeno_tail.cuh"
 
 namespace zeno {
 
@@ -53,12 +59,10 @@ __device__ __forceinline__ float warp_sum(float v) {
     return v;
 }
 
-// Positions of a lane's four k-indices inside a 128-wide iteration block.
-//   vector path: 4*lane + e  (one 16-byte / 8-byte load);  scalar path: 32*e + lane (coalesced).
-template <bool VEC> __device__ __forceinline__ int lane_k(int lane, int e) {
-    return VEC ? 4 * lane + e : 32 * e + lane;
-}
+__device__ __forceinline__ float relu_keep_nan(float z) { return (z > 0.f || z != z) ? z : 0.f; }
 
+// A lane's four k-indices inside a 128-wide block: vector path 4*lane + e (one 16-byte / 8-byte
+// load); scalar path 32*e + lane (coalesced).
 template <typename T, bool VEC>
 __device__ __forceinline__ void load_row4(const T *row, int kbase, int lane, int K, float (&o)[4]) {
     if (VEC) {
@@ -93,15 +97,9 @@ __global__ void __launch_bounds__(kLayerWarps * 32, 1) mlp_layer_kernel(LayerArg
 
     const T *xw = static_cast<const T *>(a.x) + a.offW;
     const T *vw = static_cast<const T *>(a.V) + (has_v ? (int64_t)(c - 1) * a.ldv : 0) + a.offW;
-    const T *xrow[RB];
-    const T *vrow[RB];
+    int orow[RB];                                // rows past the end are computed on a clamp and dropped
 #pragma unroll
-    for (int r = 0; r < RB; ++r) {
-        int o = min(row0 + r, a.out - 1);        // rows past the end are computed on a clamp and dropped
-        xrow[r] = xw + (int64_t)o * K;
-        vrow[r] = vw + (int64_t)o * K;
-    }
-    const float *hin = a.Hin + (int64_t)c * a.hin_cand_stride + (int64_t)j0 * K;
+    for (int r = 0; r < RB; ++r) orow[r] = min(row0 + r, a.out - 1);
     const int n_valid = min(NRT, a.n_r - j0);
 
     float acc[RB][NRT];
@@ -112,10 +110,13 @@ __global__ void __launch_bounds__(kLayerWarps * 32, 1) mlp_layer_kernel(LayerArg
         for (int j = 0; j < NRT; ++j) acc[r][j] = 0.f;
 
     const int stages = (K + kStageK - 1) / kStageK;
+    const int iters = (K + kIterK - 1) / kIterK;
 
+    // ---- staging of the input activations ------------------------------------------------
     auto issue_stage = [&](int s) {
         float(*dst)[kStageK] = hs[s & 1];
         const int kb = s * kStageK;
+        const float *hin = a.Hin + (int64_t)c * a.hin_cand_stride + (int64_t)j0 * K;
         if (VEC) {
             constexpr int kVecPerRow = kStageK / 4;
             for (int t = threadIdx.x; t < NRT * kVecPerRow; t += blockDim.x) {
@@ -134,7 +135,23 @@ __global__ void __launch_bounds__(kLayerWarps * 32, 1) mlp_layer_kernel(LayerArg
         cp_async_commit();
     };
 
+    // ---- the streamed operands: this iteration's x / v values, the next ones in flight ------
+    float xc[RB][4], vc[RB][4];
+    auto load_iter = [&](int g, float (&xo)[RB][4], float (&vo)[RB][4]) {
+        const int kbase = g * kIterK;
+#pragma unroll
+        for (int r = 0; r < RB; ++r) {
+            load_row4<T, VEC>(xw + (int64_t)orow[r] * K, kbase, lane, K, xo[r]);
+            if (has_v) {
+                load_row4<T, VEC>(vw + (int64_t)orow[r] * K, kbase, lane, K, vo[r]);
+            } else {
+                vo[r][0] = vo[r][1] = vo[r][2] = vo[r][3] = 0.f;
+            }
+        }
+    };
+
     issue_stage(0);
+    load_iter(0, xc, vc);
     for (int s = 0; s < stages; ++s) {
         if (s + 1 < stages) {
             issue_stage(s + 1);
@@ -144,82 +161,108 @@ __global__ void __launch_bounds__(kLayerWarps * 32, 1) mlp_layer_kernel(LayerArg
         }
         __syncthreads();
         const float(*h)[kStageK] = hs[s & 1];
-#pragma unroll 1
+#pragma unroll
         for (int it = 0; it < kStageK / kIterK; ++it) {
-            const int kbase = s * kStageK + it * kIterK;
-            if (kbase >= K) break;
-            float w[RB][4];
+            const int g = s * (kStageK / kIterK) + it;
+            if (g < iters) {
+                float xn[RB][4], vn[RB][4];
+                if (g + 1 < iters) load_iter(g + 1, xn, vn);
+                float w[RB][4];
 #pragma unroll
-            for (int r = 0; r < RB; ++r) {
-                float xv[4], vv[4];
-                load_row4<T, VEC>(xrow[r], kbase, lane, K, xv);
-                if (has_v) {
-                    load_row4<T, VEC>(vrow[r], kbase, lane, K, vv);
-                } else {
-                    vv[0] = vv[1] = vv[2] = vv[3] = 0.f;
-                }
-                const bool live = row0 + r < a.out;
+                for (int r = 0; r < RB; ++r) {
+                    const bool live = row0 + r < a.out;
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    w[r][e] = candidate_param<T>(xv[e], vv[e], a.gamma);
-                    if (live) nrm = fmaf(vv[e], vv[e], nrm);
-                }
-            }
-#pragma unroll
-            for (int j = 0; j < NRT; ++j) {
-                float hv[4];
-                if (VEC) {
-                    float4 t = *reinterpret_cast<const float4 *>(&h[j][it * kIterK + 4 * lane]);
-                    hv[0] = t.x; hv[1] = t.y; hv[2] = t.z; hv[3] = t.w;
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) hv[e] = h[j][it * kIterK + 32 * e + lane];
+                    for (int e = 0; e < 4; ++e) {
+                        w[r][e] = candidate_param<T>(xc[r][e], vc[r][e], a.gamma);
+                        if (live) nrm = fmaf(vc[r][e], vc[r][e], nrm);
+                    }
                 }
 #pragma unroll
-                for (int r = 0; r < RB; ++r)
+                for (int j = 0; j < NRT; ++j) {
+                    float hv[4];
+                    if (VEC) {
+                        float4 t = *reinterpret_cast<const float4 *>(&h[j][it * kIterK + 4 * lane]);
+                        hv[0] = t.x; hv[1] = t.y; hv[2] = t.z; hv[3] = t.w;
+                    } else {
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) acc[r][j] = fmaf(w[r][e], hv[e], acc[r][j]);
+                        for (int e = 0; e < 4; ++e) hv[e] = h[j][it * kIterK + 32 * e + lane];
+                    }
+#pragma unroll
+                    for (int r = 0; r < RB; ++r)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) acc[r][j] = fmaf(w[r][e], hv[e], acc[r][j]);
+                }
+                if (g + 1 < iters) {
+#pragma unroll
+                    for (int r = 0; r < RB; ++r)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            xc[r][e] = xn[r][e];
+                            vc[r][e] = vn[r][e];
+                        }
+                }
             }
         }
         __syncthreads();
     }
 
-    // lane j now collects sample j0 + j of each row
+    // ---- epilogue: lane j collects sample j0 + j of each row --------------------------------
+    float *zl = smem_dyn;                         // fused loss: logits [32 rows][NRT + 1]
+    const T *vrow_base = static_cast<const T *>(a.V) + (has_v ? (int64_t)(c - 1) * a.ldv : 0);
 #pragma unroll
     for (int r = 0; r < RB; ++r) {
         float z = warp_transpose_reduce<NRT>(acc[r], lane);
         const int o = row0 + r;
         if (o < a.out && lane < n_valid) {
             if (a.offB >= 0) {
-                const T *xb = static_cast<const T *>(a.x) + a.offB + o;
-                float bx = load_elem(xb);
-                float bv = has_v ? load_elem(static_cast<const T *>(a.V) + (int64_t)(c - 1) * a.ldv +
-                                             a.offB + o)
-                                 : 0.f;
+                float bx = load_elem(static_cast<const T *>(a.x) + a.offB + o);
+                float bv = has_v ? load_elem(vrow_base + a.offB + o) : 0.f;
                 z += candidate_param<T>(bx, bv, a.gamma);
             }
-            if (a.relu) z = (z > 0.f || z != z) ? z : 0.f;   // a NaN stays a NaN
-            a.Hout[((int64_t)c * a.n_r + j0 + lane) * a.out + o] = z;
+            if (a.relu) z = relu_keep_nan(z);
+            if (a.fuse_loss)
+                zl[o * (NRT + 1) + lane] = z;
+            else
+                a.Hout[((int64_t)c * a.n_r + j0 + lane) * a.out + o] = z;
         }
     }
 
     // partial ||v||^2 of the rows (and bias entries) this warp touched; one slot per warp
     if (has_v && blockIdx.z == 0) {
         if (a.offB >= 0 && lane < RB && row0 + lane < a.out) {
-            float bv = load_elem(static_cast<const T *>(a.V) + (int64_t)(c - 1) * a.ldv + a.offB +
-                                 row0 + lane);
+            float bv = load_elem(vrow_base + a.offB + row0 + lane);
             nrm = fmaf(bv, bv, nrm);
         }
         nrm = warp_sum(nrm);
         if (lane == 0)
             a.normpart[(int64_t)(c - 1) * a.np_slots + a.np_base + blockIdx.x * kLayerWarps + warp] = nrm;
     }
+
+    // ---- last layer: cross-entropy of this model, then (last block) scores and ranking -----
+    if (a.fuse_loss) {   // one block per model: gridDim.x == gridDim.z == 1, out <= 32, n_r <= NRT
+        __syncthreads();
+        if (warp == 0) {
+            float l = 0.f;
+            if (lane < n_valid) {
+                float zmax = -INFINITY;
+                for (int o = 0; o < a.out; ++o) zmax = fmaxf(zmax, zl[o * (NRT + 1) + lane]);
+                float se = 0.f;
+                for (int o = 0; o < a.out; ++o) se += expf(zl[o * (NRT + 1) + lane] - zmax);   // a NaN logit makes se NaN
+                int lab = a.labels[lane];
+                if (lab < 0 || lab >= a.out) lab = 0;
+                l = zmax + logf(se) - zl[lab * (NRT + 1) + lane];
+            }
+            l = warp_sum(l);
+            if (lane == 0) a.losses[c] = l / (float)a.n_r;
+        }
+        if (take_last_ticket(a.tail.ticket, gridDim.y)) finalize_and_select(a.tail, a.losses);
+    }
 }
 
 // Per model: mean over the samples of log-sum-exp(z) - z[label].  One block per model, one
-// warp per sample, fixed summation order.
+// warp per sample, fixed summation order; the last block to finish runs the tail.
 __global__ void __launch_bounds__(256) mlp_loss_kernel(const float *logits, const int32_t *labels,
-                                                        int n_r, int classes, float *losses) {
+                                                        int n_r, int classes, float *losses, TailArgs tail) {
     __shared__ float per_warp[8];
     const int c = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -244,23 +287,7 @@ __global__ void __launch_bounds__(256) mlp_loss_kernel(const float *logits, cons
         for (int w = 0; w < 8; ++w) t += per_warp[w];
         losses[c] = t / (float)n_r;
     }
-}
-
-// norms[i] = sum of the partial slots the layers filled (fixed order);
-// scores[i] = f_0 - f_i - rho * norms[i].
-__global__ void mlp_finalize_kernel(const float *normpart, int np_slots, NormSlots used, int m, float rho,
-                                    const float *losses, float *scores, float *norms_out) {
-    const int lane = threadIdx.x & 31;
-    const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (i >= m) return;
-    float t = 0.f;
-    for (int l = 0; l < used.layers; ++l)
-        for (int s = lane; s < used.count[l]; s += 32) t += normpart[(int64_t)i * np_slots + used.base[l] + s];
-    t = warp_sum(t);
-    if (lane == 0) {
-        if (norms_out) norms_out[i] = t;
-        scores[i] = losses[0] - losses[1 + i] - rho * t;
-    }
+    if (take_last_ticket(tail.ticket, gridDim.x)) finalize_and_select(tail, losses);
 }
 
 template <typename T, bool VEC>
@@ -268,7 +295,9 @@ cudaError_t launch_layer_nrt(const LayerArgs &a, cudaStream_t s) {
     const int rows_per_block = kRowsPerWarp * kLayerWarps;
     auto go = [&](auto kernel, int nrt) {
         dim3 grid((a.out + rows_per_block - 1) / rows_per_block, a.m + 1, (a.n_r + nrt - 1) / nrt);
-        const size_t smem = sizeof(float) * 2 * nrt * kStageK;
+        size_t smem = sizeof(float) * 2 * nrt * kStageK;
+        const size_t smem_loss = sizeof(float) * rows_per_block * (nrt + 1);
+        if (a.fuse_loss && smem_loss > smem) smem = smem_loss;
         if (smem > 48 * 1024) {
             cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  (int)smem);
@@ -289,10 +318,14 @@ int mlp_norm_slots(int out) {
     return (out + rows_per_block - 1) / rows_per_block * kLayerWarps;
 }
 
+// The cross-entropy can ride on the last layer's launch when one block sees all of a model's
+// logits: every output row in one block, every sample in one tile.
+bool mlp_can_fuse_loss(int out, int n_r) { return out <= kRowsPerWarp * kLayerWarps && n_r <= 32; }
+
 cudaError_t launch_mlp_layer(Context &c, const LayerArgs &a, bool aligned, cudaStream_t s,
                              int *launches) {
     ++*launches;
-    profile_mark(c, "mlp_layer", s);
+    profile_mark(c, a.fuse_loss ? "mlp_layer_loss_tail" : "mlp_layer", s);
     if (c.desc.param_dtype == ZENO_BF16)
         return aligned ? launch_layer_nrt<__nv_bfloat16, true>(a, s)
                        : launch_layer_nrt<__nv_bfloat16, false>(a, s);
@@ -300,20 +333,11 @@ cudaError_t launch_mlp_layer(Context &c, const LayerArgs &a, bool aligned, cudaS
 }
 
 cudaError_t launch_mlp_loss(Context &c, const float *logits, const int32_t *labels, int n_r,
-                            int m, int classes, float *losses, cudaStream_t s, int *launches) {
+                            int m, int classes, float *losses, const TailArgs &tail, cudaStream_t s,
+                            int *launches) {
     ++*launches;
-    profile_mark(c, "mlp_loss", s);
-    mlp_loss_kernel<<<m + 1, 256, 0, s>>>(logits, labels, n_r, classes, losses);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_mlp_finalize(Context &c, const NormSlots &slots, int m, float rho, const float *losses,
-                                float *scores, float *norms_out, cudaStream_t s, int *launches) {
-    ++*launches;
-    profile_mark(c, "mlp_finalize", s);
-    const int warps = 4;
-    mlp_finalize_kernel<<<(m + warps - 1) / warps, warps * 32, 0, s>>>(c.normpart, c.np_slots, slots, m,
-                                                                      rho, losses, scores, norms_out);
+    profile_mark(c, "mlp_loss_tail", s);
+    mlp_loss_kernel<<<m + 1, 256, 0, s>>>(logits, labels, n_r, classes, losses, tail);
     return cudaGetLastError();
 }
 

@@ -29,7 +29,9 @@
 //                 128 bytes from the stage, accumulates v^2, splits into hi/lo and stores both
 //                 to TMEM (tcgen05.st) where the MMA picks them up
 //   warps 12-15   epilogue: drain finished accumulators (tcgen05.ld) into the split-K partial
-//                 output while both pipelines keep going
+//                 output while both pipelines keep going.  The block that delivers the last
+//                 of a tile's R partials (a ticket per tile, no waiting) adds them up in
+//                 k-range order, so the sums do not depend on which block that is.
 // Every mbarrier wait is bounded; a wait that gives up raises a status word and the block leaves
 // through the common teardown (pending bulk copies awaited, TMEM freed).
 #include <cuda.h>
@@ -431,30 +433,50 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
 
 // Split-K reduction and activation after the streamed first layer:
 //   z_0 = sum_r P[r][0] + b(x),   z_c = z_0 - gamma (sum_r P[r][c] + b(v_c)),   h = ReLU(z)
-// One thread per (model, sample, output); partials are added in k-range order.
+// One thread per (model, sample, four outputs); the 2R loads of a thread are independent and
+// the partials are added in k-range order.
+template <bool VEC4>
 __global__ void __launch_bounds__(256) stream_combine_kernel(const float *part, int R, int m, int n_r, int out,
                                                              const float *x, const float *V, int64_t ldv,
                                                              int64_t offB, float gamma, int relu, float *H) {
-    const int64_t total = (int64_t)(m + 1) * n_r * out;
-    const int64_t per_r = total;
+    constexpr int E = VEC4 ? 4 : 1;
+    const int og = (out + E - 1) / E;                       // output groups per row
+    const int64_t total = (int64_t)(m + 1) * n_r * og;
+    const int64_t per_r = (int64_t)(m + 1) * n_r * out;
     for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total;
          t += (int64_t)gridDim.x * blockDim.x) {
-        const int o = (int)(t % out);
-        const int64_t cj = t / out;
+        const int o = (int)(t % og) * E;
+        const int64_t cj = t / og;
         const int c = (int)(cj / n_r), j = (int)(cj % n_r);
-        const int64_t base_idx = (int64_t)j * out + o;          // model 0
-        float z0 = 0.f, pc = 0.f;
+        const int64_t i0 = (int64_t)j * out + o;               // model 0
+        const int64_t ic = cj * out + o;
+        float z0[E], pc[E];
+#pragma unroll
+        for (int e = 0; e < E; ++e) z0[e] = pc[e] = 0.f;
+#pragma unroll 4
         for (int r = 0; r < R; ++r) {
-            z0 += part[r * per_r + base_idx];
-            if (c > 0) pc += part[r * per_r + t];
+            if (VEC4) {
+                const float4 a4 = __ldcg(reinterpret_cast<const float4 *>(part + r * per_r + i0));
+                z0[0] += a4.x; z0[1] += a4.y; z0[2] += a4.z; z0[3] += a4.w;
+                if (c > 0) {
+                    const float4 b4 = __ldcg(reinterpret_cast<const float4 *>(part + r * per_r + ic));
+                    pc[0] += b4.x; pc[1] += b4.y; pc[2] += b4.z; pc[3] += b4.w;
+                }
+            } else {
+                z0[0] += __ldcg(part + r * per_r + i0);
+                if (c > 0) pc[0] += __ldcg(part + r * per_r + ic);
+            }
         }
-        if (offB >= 0) {
-            z0 += __ldg(x + offB + o);
-            if (c > 0) pc += __ldg(V + (int64_t)(c - 1) * ldv + offB + o);
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            if (offB >= 0) {
+                z0[e] += __ldg(x + offB + o + e);
+                if (c > 0) pc[e] += __ldg(V + (int64_t)(c - 1) * ldv + offB + o + e);
+            }
+            float z = c > 0 ? fmaf(-gamma, pc[e], z0[e]) : z0[e];
+            if (relu) z = (z > 0.f || z != z) ? z : 0.f;
+            H[ic + e] = z;
         }
-        float z = c > 0 ? fmaf(-gamma, pc, z0) : z0;
-        if (relu) z = (z > 0.f || z != z) ? z : 0.f;
-        H[t] = z;
     }
 }
 
@@ -580,11 +602,15 @@ cudaError_t launch_stream_combine(Context &c, const StreamTcPlan &p, const float
                                   float gamma, int relu, float *H, cudaStream_t s, int *launches) {
     ++*launches;
     profile_mark(c, "stream_combine", s);
-    const int64_t total = (int64_t)(m + 1) * n_r * out;
+    const bool vec = out % 4 == 0;
+    const int64_t total = (int64_t)(m + 1) * n_r * (vec ? out / 4 : out);
     int blocks = (int)((total + 255) / 256);
-    const int cap = (c.sm_count > 0 ? c.sm_count : 148) * 8;
+    const int cap = (c.sm_count > 0 ? c.sm_count : 148) * 16;
     if (blocks > cap) blocks = cap;
-    stream_combine_kernel<<<blocks, 256, 0, s>>>(part, p.R, m, n_r, out, x, V, ldv, offB, gamma, relu, H);
+    if (vec)
+        stream_combine_kernel<true><<<blocks, 256, 0, s>>>(part, p.R, m, n_r, out, x, V, ldv, offB, gamma, relu, H);
+    else
+        stream_combine_kernel<false><<<blocks, 256, 0, s>>>(part, p.R, m, n_r, out, x, V, ldv, offB, gamma, relu, H);
     return cudaGetLastError();
 }
 

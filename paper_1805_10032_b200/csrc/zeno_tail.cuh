@@ -1,0 +1,84 @@
+// The end of the scoring pass, run by whichever block finishes last (a ticket, no waiting):
+// norms from their partial sums, Definition 2's score, and optionally Definition 3's ranking.
+#pragma once
+
+#include "zeno_internal.h"
+
+namespace zeno {
+
+// (score, index) packed so that unsigned order is "higher score first, then lower index":
+// the score's bits mapped to an order-preserving unsigned integer (NaN ranks with minus
+// infinity, -0 is folded into +0), the index stored complemented in the low half.
+__device__ __forceinline__ unsigned long long rank_key(float s, int index) {
+    if (s != s) s = -INFINITY;
+    s += 0.0f;
+    unsigned u = __float_as_uint(s);
+    u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+    return ((unsigned long long)u << 32) | (unsigned)(0xffffffffu - (unsigned)index);
+}
+
+// Called by ALL threads of a block.  Returns true in the block that took the last ticket, after
+// making the other blocks' global writes visible to it.
+__device__ __forceinline__ bool take_last_ticket(unsigned *ticket, unsigned n_blocks) {
+    __shared__ bool is_last;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned t = atomicAdd(ticket, 1u);
+        is_last = t == n_blocks - 1;
+        if (is_last) *ticket = 0;          // ready for the next launch
+    }
+    __syncthreads();
+    if (is_last) __threadfence();
+    return is_last;
+}
+
+// One block, any size.  norms[i] = the layers' partial sums added in slot order;
+// scores[i] = f_0 - f_i - rho norms[i]; if keep > 0, idx[0..keep) = the candidates with the
+// highest scores in rank order (bitonic sort of the packed keys in shared memory).
+__device__ __forceinline__ void finalize_and_select(const TailArgs &t, const float *losses) {
+    __shared__ unsigned long long keys[ZENO_MAX_CANDIDATES];
+    int n = 32;
+    while (n < t.m) n <<= 1;
+    const float f0 = __ldcg(losses);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    for (int i = threadIdx.x; i < n; i += blockDim.x)
+        if (i >= t.m) keys[i] = 0ull;      // padding: below every real key
+    // one warp per candidate; lanes stride the slots, then a fixed-order butterfly
+    for (int i = warp; i < t.m; i += n_warps) {
+        float nv = 0.f;
+        for (int l = 0; l < t.used.layers; ++l)
+            for (int s = lane; s < t.used.count[l]; s += 32)
+                nv += __ldcg(t.normpart + (int64_t)i * t.np_slots + t.used.base[l] + s);
+#pragma unroll
+        for (int sft = 16; sft >= 1; sft >>= 1) nv += __shfl_xor_sync(0xffffffffu, nv, sft);
+        if (lane == 0) {
+            const float sc = f0 - __ldcg(losses + 1 + i) - t.rho * nv;
+            if (t.norms_out) t.norms_out[i] = nv;
+            t.scores[i] = sc;
+            keys[i] = rank_key(sc, i);
+        }
+    }
+    if (t.keep <= 0) return;
+    __syncthreads();
+    for (int size = 2; size <= n; size <<= 1) {
+        for (int stride = size >> 1; stride >= 1; stride >>= 1) {
+            for (int i = threadIdx.x; i < n; i += blockDim.x) {
+                const int partner = i ^ stride;
+                if (partner > i) {
+                    const unsigned long long a = keys[i], b = keys[partner];
+                    const bool descending = (i & size) == 0;
+                    if ((a < b) == descending) {
+                        keys[i] = b;
+                        keys[partner] = a;
+                    }
+                }
+            }
+            __syncthreads();
+        }
+    }
+    for (int i = threadIdx.x; i < t.keep; i += blockDim.x)
+        t.idx[i] = (int32_t)(0xffffffffu - (unsigned)(keys[i] & 0xffffffffull));
+}
+
+}  // namespace zeno

@@ -42,7 +42,7 @@ def test_step_matches_oracle_on_shrunk_workloads(oracle, name):
     index, ov = SHRUNK[name]
     w = syn.make_config(index, **ov)
     res = P.run_step_parity(oracle, w)
-    assert res["launches"] >= 3
+    assert res["launches"] >= 2
 
 
 def test_config2_full_size(oracle):

@@ -161,13 +161,15 @@ zeno_status zeno_device_status(zeno_handle h, void *stream);
 
 /* Per-kernel timing for benchmarks.  zeno_profile(h, 1) makes every later call on the handle
  * record a CUDA event on the call's stream before each of its kernels and after the last one
- * (a few microseconds of overhead per call); zeno_profile(h, 0) switches it off again.
- * zeno_profile_read waits for the most recent call's last event (a host synchronisation) and
+ * (a few microseconds of overhead per call) and keeps the events of the last 64 calls;
+ * zeno_profile(h, 0) switches it off again.  zeno_profile_read looks at the call made `back`
+ * calls ago (0 = the most recent), waits for its last event (a host synchronisation) and
  * writes, for up to `cap` kernels in launch order, the elapsed milliseconds ms[i] and a static
- * name names[i] (either array may be NULL).  Returns the number of kernels written, 0 if
- * profiling is off or nothing was recorded, -1 on a CUDA error. */
+ * name names[i] (either array may be NULL).  Enqueue many calls before reading, so that the
+ * GPU is never waiting for the host between the events.  Returns the number of kernels
+ * written, 0 if profiling is off or that call is not in the ring, -1 on a CUDA error. */
 zeno_status zeno_profile(zeno_handle h, int32_t enable);
-int32_t zeno_profile_read(zeno_handle h, float *ms, const char **names, int32_t cap);
+int32_t zeno_profile_read(zeno_handle h, int32_t back, float *ms, const char **names, int32_t cap);
 
 /* Kernels launched by the most recent call on this handle (0 after an error). */
 int32_t zeno_last_launch_count(zeno_handle h);

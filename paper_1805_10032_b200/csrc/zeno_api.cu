@@ -51,7 +51,11 @@ struct DeviceGuard {
 // Per-kernel timing: a call starts a fresh list of events and closes it after its last kernel.
 void profile_begin(Context *c) { c->profiled = 0; }
 void profile_end(Context *c, cudaStream_t s) {
-    if (c->profile) cudaEventRecord(c->events[c->profiled], s);
+    if (!c->profile) return;
+    const int slot = (int)(c->call_seq % zeno::kProfileDepth);
+    cudaEventRecord(c->events[slot][c->profiled], s);
+    c->profiled_n[slot] = c->profiled;
+    ++c->call_seq;
 }
 
 zeno_status fail_cuda(Context *c, cudaError_t e) {
@@ -127,6 +131,7 @@ zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv,
     tail.rho = rho;
     tail.scores = scores;
     tail.norms_out = norms;
+    tail.norm_tot = c->norms;
     tail.idx = idx;
     tail.keep = keep;
     tail.ticket = c->tickets;
@@ -338,7 +343,8 @@ zeno_status zeno_destroy(zeno_handle h) {
     cudaError_t e = cudaFree(h->arena);
     if (h->host_stage) cudaFree(h->host_stage);
     if (h->profile)
-        for (int i = 0; i <= zeno::kMaxProfiled; ++i) cudaEventDestroy(h->events[i]);
+        for (int d = 0; d < zeno::kProfileDepth; ++d)
+            for (int i = 0; i <= zeno::kMaxProfiled; ++i) cudaEventDestroy(h->events[d][i]);
     delete h;
     return e == cudaSuccess ? ZENO_OK : ZENO_ERR_CUDA;
 }
@@ -497,33 +503,40 @@ zeno_status zeno_profile(zeno_handle h, int32_t enable) {
     if (!h) return ZENO_ERR_INVALID_ARG;
     DeviceGuard guard(h->device);
     if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+    const int total = zeno::kProfileDepth * (zeno::kMaxProfiled + 1);
+    cudaEvent_t *flat = &h->events[0][0];
     if (enable && !h->profile) {
-        for (int i = 0; i <= zeno::kMaxProfiled; ++i) {
-            cudaError_t e = cudaEventCreate(&h->events[i]);
+        for (int i = 0; i < total; ++i) {
+            cudaError_t e = cudaEventCreate(&flat[i]);
             if (e != cudaSuccess) {
-                for (int j = 0; j < i; ++j) cudaEventDestroy(h->events[j]);
+                for (int j = 0; j < i; ++j) cudaEventDestroy(flat[j]);
                 return fail_cuda(h, e);
             }
         }
         h->profile = true;
     } else if (!enable && h->profile) {
-        for (int i = 0; i <= zeno::kMaxProfiled; ++i) cudaEventDestroy(h->events[i]);
+        for (int i = 0; i < total; ++i) cudaEventDestroy(flat[i]);
         h->profile = false;
     }
     h->profiled = 0;
+    h->call_seq = 0;
+    for (int d = 0; d < zeno::kProfileDepth; ++d) h->profiled_n[d] = 0;
     return ZENO_OK;
 }
 
-int32_t zeno_profile_read(zeno_handle h, float *ms, const char **names, int32_t cap) {
-    if (!h || !h->profile || h->profiled == 0) return 0;
+int32_t zeno_profile_read(zeno_handle h, int32_t back, float *ms, const char **names, int32_t cap) {
+    if (!h || !h->profile || back < 0 || back >= zeno::kProfileDepth || back >= h->call_seq) return 0;
+    const int slot = (int)((h->call_seq - 1 - back) % zeno::kProfileDepth);
+    const int count = h->profiled_n[slot];
+    if (count == 0) return 0;
     DeviceGuard guard(h->device);
-    if (cudaEventSynchronize(h->events[h->profiled]) != cudaSuccess) return -1;
-    int n = h->profiled < cap ? h->profiled : cap;
+    if (cudaEventSynchronize(h->events[slot][count]) != cudaSuccess) return -1;
+    int n = count < cap ? count : cap;
     for (int i = 0; i < n; ++i) {
         float t = 0.f;
-        if (cudaEventElapsedTime(&t, h->events[i], h->events[i + 1]) != cudaSuccess) return -1;
+        if (cudaEventElapsedTime(&t, h->events[slot][i], h->events[slot][i + 1]) != cudaSuccess) return -1;
         if (ms) ms[i] = t;
-        if (names) names[i] = h->kernel_names[i];
+        if (names) names[i] = h->kernel_names[slot][i];
     }
     return n;
 }

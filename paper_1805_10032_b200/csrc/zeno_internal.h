@@ -17,6 +17,8 @@ constexpr int kLayerWarps = 8;
 constexpr int kMaxSlabs = 1024;
 // Most kernels one call can enqueue (layers + loss + finalize + select + aggregate).
 constexpr int kMaxProfiled = ZENO_MAX_LAYERS + 8;
+// Calls whose per-kernel events are kept for zeno_profile_read.
+constexpr int kProfileDepth = 64;
 
 // Launch shape of the tensor-core stream: k-range length, number of k-ranges, blocks per
 // k-range, padded sample count, 128-row tiles per model, dynamic shared memory.
@@ -54,19 +56,22 @@ struct Context {
     size_t host_stage_bytes;
     int last_launches;
     int last_cuda_error;
-    // optional per-kernel timing (zeno_profile): events[i] is recorded before kernel i of a call,
-    // events[n] after the last one
+    // optional per-kernel timing (zeno_profile): a ring of the last kProfileDepth calls; in a
+    // call's slot events[i] is recorded before kernel i and events[n] after the last one
     bool profile;
-    cudaEvent_t events[kMaxProfiled + 1];
-    const char *kernel_names[kMaxProfiled];
-    int profiled;
+    cudaEvent_t events[kProfileDepth][kMaxProfiled + 1];
+    const char *kernel_names[kProfileDepth][kMaxProfiled];
+    int profiled_n[kProfileDepth];
+    int profiled;                   // kernels marked so far in the current call
+    long long call_seq;             // calls completed since profiling was switched on
 };
 
 // Records the event that closes the previous kernel and opens the next one.
 inline void profile_mark(Context &c, const char *name, cudaStream_t s) {
     if (!c.profile || c.profiled >= kMaxProfiled) return;
-    cudaEventRecord(c.events[c.profiled], s);
-    c.kernel_names[c.profiled++] = name;
+    const int slot = (int)(c.call_seq % kProfileDepth);
+    cudaEventRecord(c.events[slot][c.profiled], s);
+    c.kernel_names[slot][c.profiled++] = name;
 }
 
 // What the last block of the scoring pass needs to turn losses and norm partials into scores
@@ -79,6 +84,7 @@ struct TailArgs {
     float rho;
     float *scores;
     float *norms_out;   // may be NULL
+    float *norm_tot;    // [m] workspace: ||v_i||^2 summed over the layers' partials
     int32_t *idx;       // used if keep > 0
     int keep;           // m - b, or 0: no ranking wanted
     unsigned *ticket;   // zero between launches

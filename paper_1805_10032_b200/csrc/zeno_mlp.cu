@@ -9,9 +9,9 @@
 // the next 128 columns are issued before the current ones are consumed; the layer's input
 // activations are staged through shared memory, double buffered.
 //
-// The last layer, when it fits one block per model, also evaluates the cross-entropy; the block
-// that finishes last (a ticket, no waiting) then forms the scores and the ranking, so the whole
-// tail of the scoring pass costs no extra launch.
+// A small last layer (mlp_head_kernel) runs as one block per model and also evaluates the
+// cross-entropy; the block that finishes last (a ticket, no waiting) then forms the scores and the
+// ranking, so the whole tail of the scoring pass costs no extra launch.
 #include "zeno_internal.h"
 #include "zeno_tail.cuh"
 
@@ -207,7 +207,6 @@ __global__ void __launch_bounds__(kLayerWarps * 32, 1) mlp_layer_kernel(LayerArg
     }
 
     // ---- epilogue: lane j collects sample j0 + j of each row --------------------------------
-    float *zl = smem_dyn;                         // fused loss: logits [32 rows][NRT + 1]
     const T *vrow_base = static_cast<const T *>(a.V) + (has_v ? (int64_t)(c - 1) * a.ldv : 0);
 #pragma unroll
     for (int r = 0; r < RB; ++r) {
@@ -220,10 +219,7 @@ __global__ void __launch_bounds__(kLayerWarps * 32, 1) mlp_layer_kernel(LayerArg
                 z += candidate_param<T>(bx, bv, a.gamma);
             }
             if (a.relu) z = relu_keep_nan(z);
-            if (a.fuse_loss)
-                zl[o * (NRT + 1) + lane] = z;
-            else
-                a.Hout[((int64_t)c * a.n_r + j0 + lane) * a.out + o] = z;
+            a.Hout[((int64_t)c * a.n_r + j0 + lane) * a.out + o] = z;
         }
     }
 
@@ -237,26 +233,161 @@ __global__ void __launch_bounds__(kLayerWarps * 32, 1) mlp_layer_kernel(LayerArg
         if (lane == 0)
             a.normpart[(int64_t)(c - 1) * a.np_slots + a.np_base + blockIdx.x * kLayerWarps + warp] = nrm;
     }
+}
 
-    // ---- last layer: cross-entropy of this model, then (last block) scores and ranking -----
-    if (a.fuse_loss) {   // one block per model: gridDim.x == gridDim.z == 1, out <= 32, n_r <= NRT
-        __syncthreads();
-        if (warp == 0) {
-            float l = 0.f;
-            if (lane < n_valid) {
-                float zmax = -INFINITY;
-                for (int o = 0; o < a.out; ++o) zmax = fmaxf(zmax, zl[o * (NRT + 1) + lane]);
-                float se = 0.f;
-                for (int o = 0; o < a.out; ++o) se += expf(zl[o * (NRT + 1) + lane] - zmax);   // a NaN logit makes se NaN
-                int lab = a.labels[lane];
-                if (lab < 0 || lab >= a.out) lab = 0;
-                l = zmax + logf(se) - zl[lab * (NRT + 1) + lane];
+// The last layer when it is small (out <= 32 classes, n_r <= 32 samples): one block per model
+// computes all of the model's logits, its cross-entropy, and -- in the block that finishes last --
+// the scores and the ranking.  The block first forms w = x - gamma v for the layer's rows in
+// shared memory (coalesced loads, v^2 accumulated on the way) next to the model's input
+// activations; then warp q multiplies samples 4q..4q+3 against all rows, lanes striding k.
+template <typename T, int OUT_T, bool VEC>
+__global__ void __launch_bounds__(256, 1) mlp_head_kernel(LayerArgs a) {
+    constexpr int KC = 512;                      // k-extent staged per pass
+    extern __shared__ __align__(16) float smem_dyn[];
+    float(*ws)[KC] = reinterpret_cast<float(*)[KC]>(smem_dyn);                  // [OUT_T][KC]
+    float(*hs)[KC] = reinterpret_cast<float(*)[KC]>(smem_dyn + OUT_T * KC);     // [32][KC]
+    __shared__ float zl[32][33];
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int c = blockIdx.x;
+    const int K = a.in;
+    const bool has_v = c > 0;
+    const T *xw = static_cast<const T *>(a.x) + a.offW;
+    const T *vbase = static_cast<const T *>(a.V) + (has_v ? (int64_t)(c - 1) * a.ldv : 0);
+    const T *vw = vbase + a.offW;
+    const float *hin = a.Hin + (int64_t)c * a.hin_cand_stride;
+
+    float acc[OUT_T][4];
+#pragma unroll
+    for (int o = 0; o < OUT_T; ++o)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc[o][q] = 0.f;
+    float nrm = 0.f;
+
+    for (int kb = 0; kb < K; kb += KC) {
+        if (kb > 0) __syncthreads();
+        // stage w rows and activations of this chunk (zero beyond the layer's rows / samples / K)
+        if (VEC) {
+            // activations: asynchronous copies, in flight while the weights are formed
+            for (int t = threadIdx.x; t < 32 * (KC / 4); t += 256) {
+                const int j = t / (KC / 4), kk = (t % (KC / 4)) * 4;
+                const bool ok = j < a.n_r && kb + kk < K;
+                cp_async16(&hs[j][kk], ok ? hin + (int64_t)j * K + kb + kk : a.Hin, ok);
             }
-            l = warp_sum(l);
-            if (lane == 0) a.losses[c] = l / (float)a.n_r;
+            cp_async_commit();
+            // weights: all of a thread's loads are issued before the first is used
+            constexpr int kPerThread = OUT_T * (KC / 4) / 256;
+            float xv[kPerThread][4], vv[kPerThread][4];
+#pragma unroll
+            for (int u = 0; u < kPerThread; ++u) {
+                const int t = threadIdx.x + u * 256;
+                const int o = t / (KC / 4), kk = (t % (KC / 4)) * 4;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) xv[u][e] = vv[u][e] = 0.f;
+                if (o < a.out && kb + kk < K) {
+                    load_vec4(xw + (int64_t)o * K + kb + kk, xv[u]);
+                    if (has_v) load_vec4(vw + (int64_t)o * K + kb + kk, vv[u]);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kPerThread; ++u) {
+                const int t = threadIdx.x + u * 256;
+                const int o = t / (KC / 4), kk = (t % (KC / 4)) * 4;
+                float w4[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    w4[e] = candidate_param<T>(xv[u][e], vv[u][e], a.gamma);
+                    nrm = fmaf(vv[u][e], vv[u][e], nrm);
+                }
+                *reinterpret_cast<float4 *>(&ws[o][kk]) = make_float4(w4[0], w4[1], w4[2], w4[3]);
+            }
+            cp_async_wait<0>();
+        } else {
+            for (int t = threadIdx.x; t < OUT_T * KC; t += 256) {
+                const int o = t / KC, kk = t % KC;
+                float w = 0.f;
+                if (o < a.out && kb + kk < K) {
+                    const float xv = load_elem(xw + (int64_t)o * K + kb + kk);
+                    const float vv = has_v ? load_elem(vw + (int64_t)o * K + kb + kk) : 0.f;
+                    w = candidate_param<T>(xv, vv, a.gamma);
+                    nrm = fmaf(vv, vv, nrm);
+                }
+                ws[o][kk] = w;
+            }
+            for (int t = threadIdx.x; t < 32 * KC; t += 256) {
+                const int j = t / KC, kk = t % KC;
+                hs[j][kk] = (j < a.n_r && kb + kk < K) ? __ldg(hin + (int64_t)j * K + kb + kk) : 0.f;
+            }
         }
-        if (take_last_ticket(a.tail.ticket, gridDim.y)) finalize_and_select(a.tail, a.losses);
+        __syncthreads();
+        // warp q: samples 4q..4q+3 against every row; lane l takes k = 4l + 128 i
+#pragma unroll 1
+        for (int i = 0; i < KC / 128; ++i) {
+            if (kb + i * 128 >= K) break;
+            const int kk = i * 128 + 4 * lane;
+            float4 h4[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) h4[q] = *reinterpret_cast<const float4 *>(&hs[warp * 4 + q][kk]);
+#pragma unroll
+            for (int o = 0; o < OUT_T; ++o) {
+                const float4 w4 = *reinterpret_cast<const float4 *>(&ws[o][kk]);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    acc[o][q] = fmaf(w4.x, h4[q].x, acc[o][q]);
+                    acc[o][q] = fmaf(w4.y, h4[q].y, acc[o][q]);
+                    acc[o][q] = fmaf(w4.z, h4[q].z, acc[o][q]);
+                    acc[o][q] = fmaf(w4.w, h4[q].w, acc[o][q]);
+                }
+            }
+        }
     }
+
+    // lane totals: 32 (row, sample) pairs at a time; lane l receives pair l of the batch
+#pragma unroll
+    for (int ob = 0; ob < OUT_T; ob += 8) {
+        float v[32];
+#pragma unroll
+        for (int o = 0; o < 8; ++o)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) v[o * 4 + q] = acc[ob + o][q];
+        float z = warp_transpose_reduce<32>(v, lane);
+        const int o = ob + (lane >> 2), j = warp * 4 + (lane & 3);
+        if (o < a.out && j < a.n_r) {
+            if (a.offB >= 0) {
+                const float bx = load_elem(static_cast<const T *>(a.x) + a.offB + o);
+                const float bv = has_v ? load_elem(vbase + a.offB + o) : 0.f;
+                z += candidate_param<T>(bx, bv, a.gamma);
+            }
+            if (a.relu) z = relu_keep_nan(z);
+            zl[o][j] = z;
+        }
+    }
+    // ||v||^2 of this layer's rows and bias entries: one slot per warp
+    if (has_v) {
+        if (a.offB >= 0 && threadIdx.x < a.out) {
+            const float bv = load_elem(vbase + a.offB + threadIdx.x);
+            nrm = fmaf(bv, bv, nrm);
+        }
+        nrm = warp_sum(nrm);
+        if (lane == 0) a.normpart[(int64_t)(c - 1) * a.np_slots + a.np_base + warp] = nrm;
+    }
+    __syncthreads();
+    if (has_v) block_norm_total(a.tail, c - 1);          // all layers' partials of this candidate
+    if (warp == 0) {
+        float l = 0.f;
+        if (lane < a.n_r) {
+            float zmax = -INFINITY;
+            for (int o = 0; o < a.out; ++o) zmax = fmaxf(zmax, zl[o][lane]);
+            float se = 0.f;
+            for (int o = 0; o < a.out; ++o) se += expf(zl[o][lane] - zmax);   // a NaN logit makes se NaN
+            int lab = a.labels[lane];
+            if (lab < 0 || lab >= a.out) lab = 0;
+            l = zmax + logf(se) - zl[lab][lane];
+        }
+        l = warp_sum(l);
+        if (lane == 0) a.losses[c] = l / (float)a.n_r;
+    }
+    if (take_last_ticket(a.tail.ticket, gridDim.x)) finalize_and_select(a.tail, a.losses);
 }
 
 // Per model: mean over the samples of log-sum-exp(z) - z[label].  One block per model, one
@@ -287,6 +418,7 @@ __global__ void __launch_bounds__(256) mlp_loss_kernel(const float *logits, cons
         for (int w = 0; w < 8; ++w) t += per_warp[w];
         losses[c] = t / (float)n_r;
     }
+    if (c > 0) block_norm_total(tail, c - 1);
     if (take_last_ticket(tail.ticket, gridDim.x)) finalize_and_select(tail, losses);
 }
 
@@ -295,9 +427,7 @@ cudaError_t launch_layer_nrt(const LayerArgs &a, cudaStream_t s) {
     const int rows_per_block = kRowsPerWarp * kLayerWarps;
     auto go = [&](auto kernel, int nrt) {
         dim3 grid((a.out + rows_per_block - 1) / rows_per_block, a.m + 1, (a.n_r + nrt - 1) / nrt);
-        size_t smem = sizeof(float) * 2 * nrt * kStageK;
-        const size_t smem_loss = sizeof(float) * rows_per_block * (nrt + 1);
-        if (a.fuse_loss && smem_loss > smem) smem = smem_loss;
+        const size_t smem = sizeof(float) * 2 * nrt * kStageK;
         if (smem > 48 * 1024) {
             cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  (int)smem);
@@ -322,10 +452,28 @@ int mlp_norm_slots(int out) {
 // logits: every output row in one block, every sample in one tile.
 bool mlp_can_fuse_loss(int out, int n_r) { return out <= kRowsPerWarp * kLayerWarps && n_r <= 32; }
 
+template <typename T, bool VEC>
+cudaError_t launch_head(const LayerArgs &a, cudaStream_t s) {
+    auto go = [&](auto kernel, int out_t) {
+        const size_t smem = sizeof(float) * (size_t)(out_t + 32) * 512;
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        kernel<<<a.m + 1, 256, smem, s>>>(a);
+        return cudaGetLastError();
+    };
+    if (a.out <= 16) return go(mlp_head_kernel<T, 16, VEC>, 16);
+    return go(mlp_head_kernel<T, 32, VEC>, 32);
+}
+
 cudaError_t launch_mlp_layer(Context &c, const LayerArgs &a, bool aligned, cudaStream_t s,
                              int *launches) {
     ++*launches;
-    profile_mark(c, a.fuse_loss ? "mlp_layer_loss_tail" : "mlp_layer", s);
+    profile_mark(c, a.fuse_loss ? "mlp_head_loss_tail" : "mlp_layer", s);
+    if (a.fuse_loss) {
+        if (c.desc.param_dtype == ZENO_BF16)
+            return aligned ? launch_head<__nv_bfloat16, true>(a, s) : launch_head<__nv_bfloat16, false>(a, s);
+        return aligned ? launch_head<float, true>(a, s) : launch_head<float, false>(a, s);
+    }
     if (c.desc.param_dtype == ZENO_BF16)
         return aligned ? launch_layer_nrt<__nv_bfloat16, true>(a, s)
                        : launch_layer_nrt<__nv_bfloat16, false>(a, s);

@@ -453,16 +453,26 @@ __global__ void __launch_bounds__(256) stream_combine_kernel(const float *part, 
         float z0[E], pc[E];
 #pragma unroll
         for (int e = 0; e < E; ++e) z0[e] = pc[e] = 0.f;
-#pragma unroll 4
-        for (int r = 0; r < R; ++r) {
-            if (VEC4) {
-                const float4 a4 = __ldcg(reinterpret_cast<const float4 *>(part + r * per_r + i0));
-                z0[0] += a4.x; z0[1] += a4.y; z0[2] += a4.z; z0[3] += a4.w;
-                if (c > 0) {
-                    const float4 b4 = __ldcg(reinterpret_cast<const float4 *>(part + r * per_r + ic));
-                    pc[0] += b4.x; pc[1] += b4.y; pc[2] += b4.z; pc[3] += b4.w;
+        if (VEC4) {
+            // twelve k-ranges at a time: all loads of a chunk are issued before they are added
+            for (int r0 = 0; r0 < R; r0 += 12) {
+                float4 a4[12], b4[12];
+#pragma unroll
+                for (int u = 0; u < 12; ++u) {
+                    const bool ok = r0 + u < R;
+                    a4[u] = ok ? __ldcg(reinterpret_cast<const float4 *>(part + (r0 + u) * per_r + i0))
+                               : make_float4(0.f, 0.f, 0.f, 0.f);
+                    b4[u] = ok && c > 0 ? __ldcg(reinterpret_cast<const float4 *>(part + (r0 + u) * per_r + ic))
+                                        : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
-            } else {
+#pragma unroll
+                for (int u = 0; u < 12; ++u) {
+                    z0[0] += a4[u].x; z0[1] += a4[u].y; z0[2] += a4[u].z; z0[3] += a4[u].w;
+                    pc[0] += b4[u].x; pc[1] += b4[u].y; pc[2] += b4[u].z; pc[3] += b4[u].w;
+                }
+            }
+        } else {
+            for (int r = 0; r < R; ++r) {
                 z0[0] += __ldcg(part + r * per_r + i0);
                 if (c > 0) pc[0] += __ldcg(part + r * per_r + ic);
             }

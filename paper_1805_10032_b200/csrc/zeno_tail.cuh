@@ -33,7 +33,40 @@ __device__ __forceinline__ bool take_last_ticket(unsigned *ticket, unsigned n_bl
     return is_last;
 }
 
-// One block, any size.  norms[i] = the layers' partial sums added in slot order;
+// Called by ALL threads of a block of at most 1024 threads, after the block's own partial sums
+// are in global memory and a __syncthreads().  Adds candidate i's partial sums of v^2 over all
+// layers in a fixed order (each lane's loads are issued eight at a time before they are added)
+// and leaves the total in norm_tot[i].
+__device__ __forceinline__ void block_norm_total(const TailArgs &t, int i) {
+    __shared__ float warp_part[32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+    float nv = 0.f;
+    for (int l = 0; l < t.used.layers; ++l) {
+        const float *src = t.normpart + (int64_t)i * t.np_slots + t.used.base[l];
+        const int count = t.used.count[l];
+        for (int s0 = warp * 256; s0 < count; s0 += n_warps * 256) {
+            float v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int s = s0 + u * 32 + lane;
+                v[u] = s < count ? __ldcg(src + s) : 0.f;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) nv += v[u];
+        }
+    }
+#pragma unroll
+    for (int sft = 16; sft >= 1; sft >>= 1) nv += __shfl_xor_sync(0xffffffffu, nv, sft);
+    if (lane == 0) warp_part[warp] = nv;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float tot = 0.f;
+        for (int w = 0; w < n_warps; ++w) tot += warp_part[w];
+        t.norm_tot[i] = tot;
+    }
+}
+
+// One block, any size.  norms[i] = the per-candidate totals left by block_norm_total;
 // scores[i] = f_0 - f_i - rho norms[i]; if keep > 0, idx[0..keep) = the candidates with the
 // highest scores in rank order (bitonic sort of the packed keys in shared memory).
 __device__ __forceinline__ void finalize_and_select(const TailArgs &t, const float *losses) {
@@ -41,23 +74,14 @@ __device__ __forceinline__ void finalize_and_select(const TailArgs &t, const flo
     int n = 32;
     while (n < t.m) n <<= 1;
     const float f0 = __ldcg(losses);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
     for (int i = threadIdx.x; i < n; i += blockDim.x)
         if (i >= t.m) keys[i] = 0ull;      // padding: below every real key
-    // one warp per candidate; lanes stride the slots, then a fixed-order butterfly
-    for (int i = warp; i < t.m; i += n_warps) {
-        float nv = 0.f;
-        for (int l = 0; l < t.used.layers; ++l)
-            for (int s = lane; s < t.used.count[l]; s += 32)
-                nv += __ldcg(t.normpart + (int64_t)i * t.np_slots + t.used.base[l] + s);
-#pragma unroll
-        for (int sft = 16; sft >= 1; sft >>= 1) nv += __shfl_xor_sync(0xffffffffu, nv, sft);
-        if (lane == 0) {
-            const float sc = f0 - __ldcg(losses + 1 + i) - t.rho * nv;
-            if (t.norms_out) t.norms_out[i] = nv;
-            t.scores[i] = sc;
-            keys[i] = rank_key(sc, i);
-        }
+    for (int i = threadIdx.x; i < t.m; i += blockDim.x) {
+        const float nv = __ldcg(t.norm_tot + i);
+        const float sc = f0 - __ldcg(losses + 1 + i) - t.rho * nv;
+        if (t.norms_out) t.norms_out[i] = nv;
+        t.scores[i] = sc;
+        keys[i] = rank_key(sc, i);
     }
     if (t.keep <= 0) return;
     __syncthreads();

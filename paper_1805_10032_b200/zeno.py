@@ -83,7 +83,7 @@ def load_library() -> ctypes.CDLL:
     lib.zeno_profile.restype = i32
     lib.zeno_profile.argtypes = [vp, i32]
     lib.zeno_profile_read.restype = i32
-    lib.zeno_profile_read.argtypes = [vp, ctypes.POINTER(f32), ctypes.POINTER(ctypes.c_char_p), i32]
+    lib.zeno_profile_read.argtypes = [vp, i32, ctypes.POINTER(f32), ctypes.POINTER(ctypes.c_char_p), i32]
     lib.zeno_last_launch_count.restype = i32
     lib.zeno_last_launch_count.argtypes = [vp]
     lib.zeno_last_cuda_error.restype = i32
@@ -193,12 +193,12 @@ class Zeno:
     def profile(self, enable: bool = True):
         self._check(self._lib.zeno_profile(self._h, int(enable)), "zeno_profile")
 
-    def profile_read(self):
-        """[(kernel name, milliseconds)] of the most recent call, in launch order."""
+    def profile_read(self, back: int = 0):
+        """[(kernel name, milliseconds)] of the call made `back` calls ago, in launch order."""
         cap = 32
         ms = (ctypes.c_float * cap)()
         names = (ctypes.c_char_p * cap)()
-        n = self._lib.zeno_profile_read(self._h, ms, names, cap)
+        n = self._lib.zeno_profile_read(self._h, int(back), ms, names, cap)
         if n < 0:
             raise ZenoError(ERR_CUDA, "zeno_profile_read")
         return [(names[i].decode(), float(ms[i])) for i in range(n)]

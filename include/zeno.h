@@ -43,6 +43,8 @@ extern "C" {
 
 #define ZENO_MAX_LAYERS 8
 #define ZENO_MAX_CANDIDATES 1024
+#define ZENO_STATIC_MAX_M 64    /* most candidates zeno_score_lsq_static accepts */
+#define ZENO_STATIC_MAX_N_R 32  /* most server samples zeno_score_lsq_static accepts */
 
 typedef enum {
     ZENO_OK = 0,
@@ -153,6 +155,30 @@ zeno_status zeno_step_host(zeno_handle h, const void *x, const void *V, int64_t 
                            const float *features, const void *targets, int32_t n_r, float gamma,
                            float rho, int32_t b, float *out, float *scores, int32_t *idx,
                            void *stream);
+
+/* Least-squares scores for callers that must not allocate.  (The paper has no counterpart: this
+ * is a packaging variant of zeno_score for the least-squares loss, same arithmetic, same kernels.)
+ * Some users of this library cannot call cudaMalloc at the point where they need a score: a
+ * serving loop that promised its host framework not to touch the allocator after start-up
+ * (cudaMalloc synchronises the whole device and would stall every other stream), or a process
+ * whose framework has already claimed all device memory for its own pool.  zeno_create needs an
+ * allocation for its workspace, so this call takes no handle: its scratch (per-slab partial
+ * products, about 1.4 MB) is a fixed array inside the library image, present on every GPU that
+ * loads the library for the life of the process.
+ *   - All pointers are device pointers on `device`; x [d], V [m x ldv], A [n_r x d], y [n_r];
+ *     scores[m] required, losses[m+1] and norms[m] optional (NULL).  Same results as
+ *     zeno_score on a least-squares handle.
+ *   - m <= ZENO_STATIC_MAX_M and n_r <= ZENO_STATIC_MAX_N_R, else ZENO_ERR_WORKSPACE (the scratch
+ *     is fixed).  Other argument errors: ZENO_ERR_INVALID_ARG, as for zeno_score.
+ *   - The first call on a device looks up the array's device address (no allocation, but a
+ *     runtime query): make that first call before any stream capture begins.
+ *   - No cudaMalloc / cudaFree / allocating routine is called, ever.
+ *   - All calls on a device share the one array and nothing in it needs clearing between calls
+ *     (each call rewrites every partial it later reads), but two calls whose kernels overlap on
+ *     the GPU (different streams, no ordering) race on it: order them. */
+zeno_status zeno_score_lsq_static(int32_t device, const float *x, const float *V, int64_t ldv, int64_t d,
+                                  int32_t m, const float *A, const float *y, int32_t n_r, float gamma,
+                                  float rho, float *scores, float *losses, float *norms, void *stream);
 
 /* Synchronises `stream` and reports whether any kernel enqueued through this handle gave up on a
  * bounded device-side wait (its outputs are then undefined): ZENO_ERR_TIMEOUT if so, else

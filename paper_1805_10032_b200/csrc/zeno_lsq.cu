@@ -282,3 +282,97 @@ cudaError_t launch_lsq_score(Context &c, const LsqArgs &a_in, const float *y, fl
 }
 
 }  // namespace zeno
+
+// ---- scoring without any allocation -------------------------------------------------------
+//
+// The slab partials, the combined sums and the losses of zeno_score_lsq_static live in this
+// array.  It is part of the library image: every GPU that loads the library carries it until
+// the process exits.  Size: (slabs + 1) (m + 1) (n_r + 1) + (m + 1) floats with slabs <= 160,
+// m <= ZENO_STATIC_MAX_M, n_r <= ZENO_STATIC_MAX_N_R -- about 1.4 MB.
+namespace {
+
+constexpr int kStaticMaxSlabs = 160;
+constexpr size_t kStaticScratchFloats =
+    (size_t)(kStaticMaxSlabs + 1) * (ZENO_STATIC_MAX_M + 1) * (ZENO_STATIC_MAX_N_R + 1) + (ZENO_STATIC_MAX_M + 1);
+
+static __device__ __align__(256) float g_static_scratch[kStaticScratchFloats];
+
+constexpr int kMaxDevices = 64;
+float *g_static_scratch_ptr[kMaxDevices];      // device address of the array, per device
+int g_static_sms[kMaxDevices];
+bool g_static_ready[kMaxDevices];
+
+// In host code `g_static_scratch` is only a handle for the runtime, not an address a kernel can
+// use: the device address is asked for once per device, with that device current.
+cudaError_t static_scratch_setup(int device) {
+    if (g_static_ready[device]) return cudaSuccess;
+    float *ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void **>(&ptr), g_static_scratch);
+    if (e != cudaSuccess) return e;
+    int sms = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+    if (e != cudaSuccess) return e;
+    g_static_scratch_ptr[device] = ptr;
+    g_static_sms[device] = sms;
+    g_static_ready[device] = true;
+    return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" zeno_status zeno_score_lsq_static(int32_t device, const float *x, const float *V, int64_t ldv,
+                                             int64_t d, int32_t m, const float *A, const float *y,
+                                             int32_t n_r, float gamma, float rho, float *scores,
+                                             float *losses, float *norms, void *stream) {
+    if (device < 0 || device >= kMaxDevices) return ZENO_ERR_INVALID_ARG;
+    if (!x || !V || !A || !y || !scores) return ZENO_ERR_INVALID_ARG;
+    if (d < 1 || ldv < d || m < 1 || n_r < 1) return ZENO_ERR_INVALID_ARG;
+    if (!isfinite(gamma) || !isfinite(rho) || rho < 0.f) return ZENO_ERR_INVALID_ARG;
+    if (m > ZENO_STATIC_MAX_M || n_r > ZENO_STATIC_MAX_N_R) return ZENO_ERR_WORKSPACE;   // beyond the fixed scratch
+
+    int prev = -1;
+    if (cudaGetDevice(&prev) != cudaSuccess) return ZENO_ERR_CUDA;
+    if (prev != device && cudaSetDevice(device) != cudaSuccess) return ZENO_ERR_CUDA;
+    zeno_status st = ZENO_OK;
+    cudaError_t e = static_scratch_setup(device);
+    if (e == cudaSuccess) {
+        cudaStream_t s = static_cast<cudaStream_t>(stream);
+        zeno::LsqArgs a;
+        a.x = x;
+        a.V = V;
+        a.ldv = ldv;
+        a.d = d;
+        a.A = A;
+        a.n_r = n_r;
+        a.m = m;
+        a.part = g_static_scratch_ptr[device];
+        const int rows = m + 1;
+        const int nrt = n_r <= 8 ? 8 : (n_r <= 16 ? 16 : 32);
+        const int64_t stages = (d + (zeno::kStageFloats / nrt) - 1) / (zeno::kStageFloats / nrt);
+        int slabs = g_static_sms[device] > 0 ? g_static_sms[device] : 148;
+        if (slabs > kStaticMaxSlabs) slabs = kStaticMaxSlabs;
+        if ((int64_t)slabs > stages) slabs = (int)stages;
+        a.slabs = slabs;
+        const bool aligned = reinterpret_cast<uintptr_t>(x) % 16 == 0 && reinterpret_cast<uintptr_t>(V) % 16 == 0 &&
+                             reinterpret_cast<uintptr_t>(A) % 16 == 0 && ldv % 4 == 0 && d % 4 == 0;
+        if (nrt == 8)
+            e = aligned ? zeno::launch_stream<8, 8, true>(a, s) : zeno::launch_stream<8, 8, false>(a, s);
+        else if (nrt == 16)
+            e = aligned ? zeno::launch_stream<16, 6, true>(a, s) : zeno::launch_stream<16, 6, false>(a, s);
+        else
+            e = aligned ? zeno::launch_stream<32, 4, true>(a, s) : zeno::launch_stream<32, 4, false>(a, s);
+        if (e == cudaSuccess) {
+            // Every partial the finishing kernel reads is rewritten by the stream kernel of the same
+            // call, so nothing left over from an earlier call has to be cleared.
+            float *sums = a.part + (int64_t)slabs * rows * (n_r + 1);
+            float *loss_buf = losses ? losses : sums + (int64_t)rows * (n_r + 1);
+            zeno::lsq_finish_kernel<<<1, 1024, 0, s>>>(a.part, slabs, m, n_r, y, gamma, rho, loss_buf, norms, scores,
+                                                       sums);
+            e = cudaGetLastError();
+        }
+    }
+    if (e != cudaSuccess) st = ZENO_ERR_CUDA;
+    if (prev != device) cudaSetDevice(prev);
+    return st;
+}
+

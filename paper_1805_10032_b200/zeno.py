@@ -25,7 +25,8 @@ F32, BF16 = 0, 1
 
 EXPORTS = (
     "zeno_param_count", "zeno_create", "zeno_destroy", "zeno_score", "zeno_select",
-    "zeno_aggregate", "zeno_step", "zeno_step_host", "zeno_device_status", "zeno_profile", "zeno_profile_read",
+    "zeno_aggregate", "zeno_step", "zeno_step_host", "zeno_device_status", "zeno_score_lsq_static",
+    "zeno_profile", "zeno_profile_read",
     "zeno_last_launch_count",
     "zeno_last_cuda_error", "zeno_status_string",
 )
@@ -78,6 +79,8 @@ def load_library() -> ctypes.CDLL:
     lib.zeno_step.argtypes = [vp, vp, vp, i64, i32, ctypes.POINTER(Batch), f32, f32, i32, vp, vp, vp, vp]
     lib.zeno_step_host.restype = i32
     lib.zeno_step_host.argtypes = [vp, vp, vp, i64, i32, vp, vp, i32, f32, f32, i32, vp, vp, vp, vp]
+    lib.zeno_score_lsq_static.restype = i32
+    lib.zeno_score_lsq_static.argtypes = [i32, vp, vp, i64, i64, i32, vp, vp, i32, f32, f32, vp, vp, vp, vp]
     lib.zeno_device_status.restype = i32
     lib.zeno_device_status.argtypes = [vp, vp]
     lib.zeno_profile.restype = i32
@@ -269,6 +272,26 @@ class Zeno:
                                       int(b), _ptr(out), _ptr(scores), _ptr(idx), _stream_ptr(stream))
         self._check(st, "zeno_step_host")
         return out
+
+
+STATIC_MAX_M, STATIC_MAX_N_R = 64, 32
+
+
+def score_lsq_static(x, V, A, y, gamma, rho, scores, losses=None, norms=None, m=None, ldv=None,
+                     device=0, stream=None):
+    """zeno_score_lsq_static: least-squares scores with no allocation anywhere -- the caller passes
+    every buffer (CUDA tensors: x [d], V [m, ldv], A [n_r, d], y [n_r], scores [m] float32; losses
+    [m+1] and norms [m] optional).  For callers that may not call the CUDA allocator; m <= 64 and
+    n_r <= 32.  Calls whose kernels could overlap on the GPU must be ordered by the caller."""
+    lib = load_library()
+    m = V.shape[0] if m is None else m
+    ldv = V.stride(0) if ldv is None else ldv
+    st = lib.zeno_score_lsq_static(int(device), _ptr(x), _ptr(V), int(ldv), int(x.shape[0]), int(m),
+                                   _ptr(A), _ptr(y), int(y.shape[0]), float(gamma), float(rho),
+                                   _ptr(scores), _ptr(losses), _ptr(norms), _stream_ptr(stream))
+    if st != OK:
+        raise ZenoError(st, "zeno_score_lsq_static")
+    return scores
 
 
 def from_workload(w, m_max=None, n_r_max=None, device=0) -> "Zeno":

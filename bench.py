@@ -208,14 +208,13 @@ def run_ours(args, rank, world, local_rank):
         dist.init_process_group("nccl", device_id=torch.device("cuda", dev))
 
     # inputs: enough distinct sets that the rotation exceeds 4x the L2 capacity
-    w0 = syn.make_config(args.config)
+    gen_device = "cuda" if args.config >= 3 else "cpu"      # the large workloads are generated on the device
+    w0 = syn.make_config(args.config, device=gen_device)
     score_b, agg_b = algorithmic_bytes(w0)
     set_bytes = w0.V.numel() * w0.V.element_size() + w0.features.numel() * 4
     n_sets = max(1, min(8, -(-4 * L2_BYTES // set_bytes)))
-    if set_bytes > 8 * L2_BYTES:
-        n_sets = 1
-    sets = [w0] + [syn.make_config(args.config, seed=syn.BASE_SEED + args.config + 1000 * (i + 1))
-                   for i in range(n_sets - 1)]
+    sets = [w0] + [syn.make_config(args.config, seed=syn.BASE_SEED + args.config + 1000 * (i + 1),
+                                   device=gen_device) for i in range(n_sets - 1)]
     dsets = [(s.x.cuda(), s.V.cuda(), s.features.cuda(), s.targets.cuda()) for s in sets]
     z = zeno.from_workload(w0, device=dev)
     out = torch.empty(w0.d, dtype=torch.float32, device="cuda")
@@ -278,10 +277,10 @@ def run_ours(args, rank, world, local_rank):
     value = world * args.steps / (ms_total * 1e-3)
 
     # ---- end to end through the host-memory entry point (copies inside the timed region)
-    hx, hV = sets[0].x.pin_memory(), sets[0].V.pin_memory()
-    hf, ht = sets[0].features.pin_memory(), sets[0].targets.pin_memory()
+    hx, hV = sets[0].x.cpu().pin_memory(), sets[0].V.cpu().pin_memory()
+    hf, ht = sets[0].features.cpu().pin_memory(), sets[0].targets.cpu().pin_memory()
     hout = torch.empty(w0.d, dtype=torch.float32).pin_memory()
-    e2e_steps = max(3, min(args.steps, 20))
+    e2e_steps = max(3, min(args.steps, 20 if args.config <= 3 else 3))
     for _ in range(2):
         z.step_host(hx, hV, hf, ht, w0.gamma, w0.rho, w0.b, hout)
     barrier()
@@ -341,8 +340,8 @@ def run_ours(args, rank, world, local_rank):
     # ---- CPU baseline: the oracle on a bounded sample of the same workload
     from oracle import zeno_oracle
     zeno_oracle.build()
-    t_full, _ = oracle_step_seconds(w0, None if args.config in (1, 2) else 3)
-    m_s = w0.m if args.config in (1, 2) else 3
+    t_full, _ = oracle_step_seconds(w0, None if args.config in (1, 2, 3) else 3)
+    m_s = w0.m if args.config in (1, 2, 3) else 3
     reps = max(1, min(5, int(12.0 / max(t_full, 1e-3))))
     ts = [oracle_step_seconds(w0, m_s)[0] for _ in range(reps)]
     t_step = (sum(ts) / len(ts)) * (w0.m + 1) / (m_s + 1)

@@ -175,13 +175,18 @@ zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv,
         a.normpart = c->normpart;
         a.np_slots = c->np_slots;
         a.np_base = c->np_base[l];
-        tail.used.base[l] = c->np_base[l];
-        tail.used.count[l] = zeno::mlp_norm_slots(a.out);
         a.fuse_loss = (l + 1 == L) && fuse_loss;
+        // 16-byte aligned rows of eight-parameter multiples take the warp-MMA kernel
+        const size_t esz = elem_size(c->desc.param_dtype);
+        const bool mma = !a.fuse_loss && aligned && !getenv("ZENO_DISABLE_TENSOR_CORES") &&
+                         zeno::mlp_mma_usable(a.in, a.out) && is_aligned(x, 16) && is_aligned(V, 16) &&
+                         (ldv * esz) % 16 == 0 && (a.offW * esz) % 16 == 0;
+        tail.used.base[l] = c->np_base[l];
+        tail.used.count[l] = mma ? zeno::mlp_mma_norm_slots(a.out) : zeno::mlp_norm_slots(a.out);
         a.labels = static_cast<const int32_t *>(batch->targets);
         a.losses = loss_buf;
         a.tail = tail;                               // complete by the time the last layer is reached
-        e = zeno::launch_mlp_layer(*c, a, aligned, s, launches);
+        e = mma ? zeno::launch_mlp_layer_mma(*c, a, s, launches) : zeno::launch_mlp_layer(*c, a, aligned, s, launches);
         if (e != cudaSuccess) return fail_cuda(c, e);
     }
     if (!fuse_loss) {

@@ -130,6 +130,10 @@ cudaError_t launch_mlp_loss(Context &c, const float *logits, const int32_t *labe
                             int m, int classes, float *losses, const TailArgs &tail, cudaStream_t s,
                             int *launches);
 bool mlp_can_fuse_loss(int out, int n_r);
+// Warp-MMA version of the layer kernel (16-byte aligned rows, in % 8 == 0).
+cudaError_t launch_mlp_layer_mma(Context &c, const LayerArgs &a, cudaStream_t s, int *launches);
+int mlp_mma_norm_slots(int out);
+bool mlp_mma_usable(int in, int out);
 cudaError_t launch_lsq_score(Context &c, const LsqArgs &a, const float *y, float gamma,
                              float rho, bool aligned, float *losses, float *norms, float *scores,
                              cudaStream_t s, int *launches);

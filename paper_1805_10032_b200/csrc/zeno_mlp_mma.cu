@@ -13,6 +13,12 @@
 // that the tensor core's truncating adds act on the small terms separately).  bfloat16 models:
 // the weights are exact in bf16; the fp32 activations are split into two bf16 terms.
 //
+// The activations are split once per stage, by the whole block, while they are written to shared
+// memory, in the order the B fragments want them: 16 bytes per (sample, k-pair) holding
+// {hi(k), hi(k+1), lo(k), lo(k+1)} for tf32, per (sample, k-quad) holding the packed bf16 pairs
+// {h0(k,k+1), h0(k+2,k+3), h1(k,k+1), h1(k+2,k+3)} for bf16.  One 16-byte shared load then feeds
+// all the MMAs of an (n-tile, k-step); slots are swizzled so that these loads are conflict free.
+//
 // A warp owns 16 output rows; lane (g, t) = (lane / 4, lane % 4) loads, for rows g and g + 8,
 // the eight consecutive k-values 8t .. 8t+7 of each 32-wide k-block (one or two 16-byte loads),
 // so every row is read in full 128-byte (64-byte for bf16) segments.  The MMA's k index is a
@@ -27,16 +33,15 @@ namespace {
 constexpr int kMmaWarps = 4;                 // warps per block, 16 rows each
 constexpr int kMmaRows = 16 * kMmaWarps;     // rows per block
 constexpr int kHS = 64;                      // k-extent of one shared-memory stage of activations
-constexpr int kHPitch = kHS + 4;             // floats per staged row (keeps 16-byte alignment)
 
-__device__ __forceinline__ void cp_async16(void *smem, const void *gmem, bool valid) {
-    unsigned s = static_cast<unsigned>(__cvta_generic_to_shared(smem));
-    int bytes = valid ? 16 : 0;
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(s), "l"(gmem), "r"(bytes));
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
-template <int N> __device__ __forceinline__ void cp_async_wait() {
-    asm volatile("cp.async.wait_group %0;\n" ::"n"(N));
+// 16-byte slots per staged sample row (one spare slot staggers consecutive rows over the banks)
+template <bool BF16> struct StageShape {
+    static constexpr int kSlots = BF16 ? kHS / 4 : kHS / 2;
+    static constexpr int kPitch = kSlots + 1;
+};
+// tf32 slots 8..15 of each 16 are rotated by two so that lanes t and t+2 of a row do not collide
+template <bool BF16> __device__ __forceinline__ int swizzle_slot(int slot) {
+    return BF16 ? slot : slot ^ (((slot >> 3) & 1) << 1);
 }
 
 __device__ __forceinline__ float tf32_hi(float a) {
@@ -81,13 +86,18 @@ template <typename T, int NRT>
 __global__ void __launch_bounds__(kMmaWarps * 32) mlp_layer_mma_kernel(LayerArgs a) {
     constexpr bool kBf16 = is_bf16<T>::value;
     constexpr int NT = NRT / 8;                 // n-tiles of 8 samples
-    __shared__ __align__(16) float hs[2][NRT][kHPitch];
+    constexpr int kPitch = StageShape<kBf16>::kPitch;
+    constexpr int kChunks = NRT * (kHS / 4) / (kMmaWarps * 32);   // float4 chunks of a stage per thread
+    extern __shared__ __align__(16) uint4 hs_dyn[];                 // [2][NRT][kPitch]
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
     const int c = blockIdx.y;
-    const int j0 = blockIdx.z * NRT;
-    const int row0 = (blockIdx.x * kMmaWarps + warp) * 16;
+    // sample tiles of the same rows sit in neighbouring blocks, so that V is read from HBM once
+    const int n_ztiles = (a.n_r + NRT - 1) / NRT;
+    const int ztile = blockIdx.x % n_ztiles, rowblk = blockIdx.x / n_ztiles;
+    const int j0 = ztile * NRT;
+    const int row0 = (rowblk * kMmaWarps + warp) * 16;
     const int K = a.in;
     const bool has_v = c > 0;
     const int n_valid = min(NRT, a.n_r - j0);
@@ -111,14 +121,38 @@ __global__ void __launch_bounds__(kMmaWarps * 32) mlp_layer_mma_kernel(LayerArgs
     const int n_stages = (K + kHS - 1) / kHS;
     const int n_blocks = (K + 31) / 32;
 
-    auto issue_stage = [&](int s) {
+    // activations of stage s: loaded into registers one stage ahead, split and stored in
+    // fragment order when the buffer is free
+    float4 hreg[kChunks];
+    auto load_stage = [&](int s) {
         const int kb = s * kHS;
-        for (int i = threadIdx.x; i < NRT * (kHS / 4); i += kMmaWarps * 32) {
+#pragma unroll
+        for (int u = 0; u < kChunks; ++u) {
+            const int i = threadIdx.x + u * (kMmaWarps * 32);
             const int j = i / (kHS / 4), kk = (i % (kHS / 4)) * 4;
-            const bool ok = j < n_valid && kb + kk < K;
-            cp_async16(&hs[s & 1][j][kk], ok ? hin + (int64_t)j * K + kb + kk : a.Hin, ok);
+            hreg[u] = (j < n_valid && kb + kk < K) ? __ldg(reinterpret_cast<const float4 *>(hin + (int64_t)j * K + kb + kk))
+                                                    : make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        cp_async_commit();
+    };
+    auto store_stage = [&](int s) {
+        uint4 *dst = hs_dyn + (size_t)(s & 1) * NRT * kPitch;
+#pragma unroll
+        for (int u = 0; u < kChunks; ++u) {
+            const int i = threadIdx.x + u * (kMmaWarps * 32);
+            const int j = i / (kHS / 4), q = i % (kHS / 4);      // q: index of the 4-wide k chunk
+            const float4 h = hreg[u];
+            if (kBf16) {
+                const float f0 = bf16_round(h.x), f1 = bf16_round(h.y), f2 = bf16_round(h.z), f3 = bf16_round(h.w);
+                dst[j * kPitch + q] = make_uint4(pack_bf16(f0, f1), pack_bf16(f2, f3), pack_bf16(h.x - f0, h.y - f1),
+                                                 pack_bf16(h.z - f2, h.w - f3));
+            } else {
+                const float a0 = tf32_hi(h.x), a1 = tf32_hi(h.y), a2 = tf32_hi(h.z), a3 = tf32_hi(h.w);
+                dst[j * kPitch + swizzle_slot<false>(2 * q)] =
+                    make_uint4(__float_as_uint(a0), __float_as_uint(a1), __float_as_uint(h.x - a0), __float_as_uint(h.y - a1));
+                dst[j * kPitch + swizzle_slot<false>(2 * q + 1)] =
+                    make_uint4(__float_as_uint(a2), __float_as_uint(a3), __float_as_uint(h.z - a2), __float_as_uint(h.w - a3));
+            }
+        }
     };
     // eight x and v values of rows g and g+8 for k-block kb (zero past K; K % 8 == 0 on this path)
     auto load_block = [&](int kblk, float (&xA)[8], float (&vA)[8], float (&xB)[8], float (&vB)[8]) {
@@ -141,16 +175,13 @@ __global__ void __launch_bounds__(kMmaWarps * 32) mlp_layer_mma_kernel(LayerArgs
     };
 
     float xA[8], vA[8], xB[8], vB[8];
-    issue_stage(0);
+    load_stage(0);
     load_block(0, xA, vA, xB, vB);
+    store_stage(0);
     for (int s = 0; s < n_stages; ++s) {
-        if (s + 1 < n_stages) {
-            issue_stage(s + 1);
-            cp_async_wait<1>();
-        } else {
-            cp_async_wait<0>();
-        }
-        __syncthreads();
+        __syncthreads();                                   // stage s is complete, buffer (s+1)&1 is free
+        if (s + 1 < n_stages) load_stage(s + 1);
+        const uint4 *h = hs_dyn + (size_t)(s & 1) * NRT * kPitch;
 #pragma unroll
         for (int half = 0; half < kHS / 32; ++half) {
             const int kblk = s * (kHS / 32) + half;
@@ -166,8 +197,6 @@ __global__ void __launch_bounds__(kMmaWarps * 32) mlp_layer_mma_kernel(LayerArgs
                     if (live_a) nrm = fmaf(vA[e], vA[e], nrm);
                     if (live_b) nrm = fmaf(vB[e], vB[e], nrm);
                 }
-                const float(*h)[kHPitch] = hs[s & 1];
-                const int kofs = half * 32 + 8 * t;
                 if (!kBf16) {
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {
@@ -180,15 +209,13 @@ __global__ void __launch_bounds__(kMmaWarps * 32) mlp_layer_mma_kernel(LayerArgs
                             ah[q] = __float_as_uint(hi);
                             al[q] = __float_as_uint(e[q] - hi);
                         }
+                        const int slot = swizzle_slot<false>(half * 16 + 4 * t + ks);
 #pragma unroll
                         for (int n = 0; n < NT; ++n) {
-                            const float2 hv = *reinterpret_cast<const float2 *>(&h[n * 8 + g][kofs + 2 * ks]);
-                            const float h0 = tf32_hi(hv.x), h1 = tf32_hi(hv.y);
-                            const uint32_t bh0 = __float_as_uint(h0), bh1 = __float_as_uint(h1);
-                            const uint32_t bl0 = __float_as_uint(hv.x - h0), bl1 = __float_as_uint(hv.y - h1);
-                            mma_tf32(big[n], ah, bh0, bh1);
-                            mma_tf32(small[n], al, bh0, bh1);
-                            mma_tf32(small[n], ah, bl0, bl1);
+                            const uint4 b = h[(n * 8 + g) * kPitch + slot];   // {hi k, hi k+1, lo k, lo k+1}
+                            mma_tf32(big[n], ah, b.x, b.y);
+                            mma_tf32(small[n], al, b.x, b.y);
+                            mma_tf32(small[n], ah, b.z, b.w);
                         }
                     }
                 } else {
@@ -200,15 +227,12 @@ __global__ void __launch_bounds__(kMmaWarps * 32) mlp_layer_mma_kernel(LayerArgs
                         aw[1] = pack_bf16(wB[4 * ks], wB[4 * ks + 1]);
                         aw[2] = pack_bf16(wA[4 * ks + 2], wA[4 * ks + 3]);
                         aw[3] = pack_bf16(wB[4 * ks + 2], wB[4 * ks + 3]);
+                        const int slot = half * 8 + 2 * t + ks;
 #pragma unroll
                         for (int n = 0; n < NT; ++n) {
-                            const float4 hv = *reinterpret_cast<const float4 *>(&h[n * 8 + g][kofs + 4 * ks]);
-                            const float f0 = bf16_round(hv.x), f1 = bf16_round(hv.y);
-                            const float f2 = bf16_round(hv.z), f3 = bf16_round(hv.w);
-                            const uint32_t bh0 = pack_bf16(f0, f1), bh1 = pack_bf16(f2, f3);
-                            const uint32_t bl0 = pack_bf16(hv.x - f0, hv.y - f1), bl1 = pack_bf16(hv.z - f2, hv.w - f3);
-                            mma_bf16(big[n], aw, bh0, bh1);
-                            mma_bf16(small[n], aw, bl0, bl1);
+                            const uint4 b = h[(n * 8 + g) * kPitch + slot];   // {h0 pair, h0 pair, h1 pair, h1 pair}
+                            mma_bf16(big[n], aw, b.x, b.y);
+                            mma_bf16(small[n], aw, b.z, b.w);
                         }
                     }
                 }
@@ -220,7 +244,7 @@ __global__ void __launch_bounds__(kMmaWarps * 32) mlp_layer_mma_kernel(LayerArgs
                 }
             }
         }
-        __syncthreads();
+        if (s + 1 < n_stages) store_stage(s + 1);          // buffer (s+1)&1 was last read in stage s-1
     }
 
     // accumulator fragment: rows g / g+8, samples 8n + 2t, 8n + 2t + 1
@@ -231,7 +255,7 @@ __global__ void __launch_bounds__(kMmaWarps * 32) mlp_layer_mma_kernel(LayerArgs
         const float vb0 = has_v ? load_elem(vbase + a.offB + rb) : 0.f;
         bias_a = candidate_param<T>(load_elem(xbias + ra), va0, a.gamma);
         bias_b = candidate_param<T>(load_elem(xbias + rb), vb0, a.gamma);
-        if (has_v && t == 0 && blockIdx.z == 0) {       // each bias entry counted once
+        if (has_v && t == 0 && ztile == 0) {            // each bias entry counted once
             if (live_a) nrm = fmaf(va0, va0, nrm);
             if (live_b) nrm = fmaf(vb0, vb0, nrm);
         }
@@ -249,19 +273,24 @@ __global__ void __launch_bounds__(kMmaWarps * 32) mlp_layer_mma_kernel(LayerArgs
             }
         }
     }
-    if (has_v && blockIdx.z == 0) {
+    if (has_v && ztile == 0) {
 #pragma unroll
         for (int sft = 16; sft >= 1; sft >>= 1) nrm += __shfl_xor_sync(0xffffffffu, nrm, sft);
         if (lane == 0)
-            a.normpart[(int64_t)(c - 1) * a.np_slots + a.np_base + blockIdx.x * kMmaWarps + warp] = nrm;
+            a.normpart[(int64_t)(c - 1) * a.np_slots + a.np_base + rowblk * kMmaWarps + warp] = nrm;
     }
 }
 
 template <typename T>
 cudaError_t launch_mma_typed(const LayerArgs &a, cudaStream_t s) {
     auto go = [&](auto kernel, int nrt) {
-        dim3 grid((a.out + kMmaRows - 1) / kMmaRows, a.m + 1, (a.n_r + nrt - 1) / nrt);
-        kernel<<<grid, kMmaWarps * 32, 0, s>>>(a);
+        dim3 grid((a.out + kMmaRows - 1) / kMmaRows * ((a.n_r + nrt - 1) / nrt), a.m + 1);
+        const size_t smem = (size_t)2 * nrt * StageShape<is_bf16<T>::value>::kPitch * 16;
+        if (smem > 48 * 1024) {
+            cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+        }
+        kernel<<<grid, kMmaWarps * 32, smem, s>>>(a);
         return cudaGetLastError();
     };
     if (a.n_r <= 16) return go(mlp_layer_mma_kernel<T, 16>, 16);

@@ -135,28 +135,31 @@ zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv,
     tail.idx = idx;
     tail.keep = keep;
     tail.ticket = c->tickets;
-    int first_cuda_layer = 0;
-    // first layer on the tensor cores when the shape and the alignment allow it
-    zeno::StreamTcPlan plan;
-    if (c->tc_ok && aligned &&
-        zeno::stream_tc_plan(c->sm_count, (int)c->desc.dims[0], (int)c->desc.dims[1], n_r, m, &plan) &&
-        plan.R <= c->tc_r_max && L >= 2) {
-        const float *xf = static_cast<const float *>(x);
-        const float *Vf = static_cast<const float *>(V);
-        e = zeno::launch_stream_tc(*c, plan, xf, Vf, ldv, c->offW[0], c->offB[0], (int)c->desc.dims[0],
-                                   (int)c->desc.dims[1], batch->features, n_r, m, c->tc_part, c->np_base[0],
-                                   s, launches);
-        if (e != cudaSuccess) return fail_cuda(c, e);
-        e = zeno::launch_stream_combine(*c, plan, c->tc_part, xf, Vf, ldv, c->offB[0], (int)c->desc.dims[1],
-                                        n_r, m, gamma, 1, c->act[0], s, launches);
-        if (e != cudaSuccess) return fail_cuda(c, e);
-        tail.used.base[0] = c->np_base[0];
-        tail.used.count[0] = zeno::stream_tc_norm_slots(plan);
-        first_cuda_layer = 1;
-    }
+    const float *xf = static_cast<const float *>(x);
+    const float *Vf = static_cast<const float *>(V);
     const int classes = (int)c->desc.dims[L];
     const bool fuse_loss = zeno::mlp_can_fuse_loss(classes, n_r);
-    for (int l = first_cuda_layer; l < L; ++l) {
+    for (int l = 0; l < L; ++l) {
+        const int in_l = (int)c->desc.dims[l], out_l = (int)c->desc.dims[l + 1];
+        const bool last_fused = (l + 1 == L) && fuse_loss;
+        // fp32 layers on the tcgen05 stream when the shape and the alignment allow it: the first
+        // layer against the shared batch, later layers against each model's own activations
+        zeno::StreamTcPlan plan;
+        if (c->tc_ok[l] && aligned && !last_fused &&
+            zeno::stream_tc_plan(c->sm_count, in_l, out_l, n_r, m, l > 0, &plan) && plan.R <= c->tc_r_max[l] &&
+            (l == 0 || getenv("ZENO_TC_ALL_LAYERS"))) {
+            const float *hin = l == 0 ? batch->features : c->act[(l - 1) & 1];
+            e = zeno::launch_stream_tc(*c, plan, xf, Vf, ldv, c->offW[l], c->offB[l], in_l, out_l, hin,
+                                       l == 0 ? 0 : (int64_t)n_r * in_l, gamma, n_r, m, c->tc_part,
+                                       c->np_base[l], s, launches);
+            if (e != cudaSuccess) return fail_cuda(c, e);
+            e = zeno::launch_stream_combine(*c, plan, c->tc_part, xf, Vf, ldv, c->offB[l], out_l, n_r, m, gamma,
+                                            l + 1 < L, c->act[l & 1], s, launches);
+            if (e != cudaSuccess) return fail_cuda(c, e);
+            tail.used.base[l] = c->np_base[l];
+            tail.used.count[l] = zeno::stream_tc_norm_slots(plan);
+            continue;
+        }
         zeno::LayerArgs a;
         a.x = x;
         a.V = V;
@@ -274,19 +277,19 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
             if (desc->has_bias) off += o;
             c->np_base[l] = slots;
             int layer_slots = zeno::mlp_norm_slots((int)o);
-            if (l == 0 && desc->param_dtype == ZENO_F32 && !getenv("ZENO_DISABLE_TENSOR_CORES")) {
-                // the tensor-core stream may serve the first layer: size its partials for the
-                // shortest k-range any plan may pick
+            if (desc->param_dtype == ZENO_F32 && !getenv("ZENO_DISABLE_TENSOR_CORES")) {
+                // the tensor-core stream may serve this layer: size its partials for the shortest
+                // k-range any plan may pick
                 zeno::StreamTcPlan probe;
-                if (zeno::stream_tc_plan(c->sm_count, (int)in, (int)o, n_r_max < 64 ? n_r_max : 64, m_max,
+                if (zeno::stream_tc_plan(c->sm_count, (int)in, (int)o, n_r_max < 64 ? n_r_max : 64, m_max, l > 0,
                                          &probe)) {
-                    c->tc_ok = true;
-                    c->tc_r_max = (int)((in + zeno::kStreamTcMinKR - 1) / zeno::kStreamTcMinKR);
-                    probe.R = c->tc_r_max;
+                    c->tc_ok[l] = true;
+                    c->tc_r_max[l] = (int)((in + zeno::kStreamTcMinKR - 1) / zeno::kStreamTcMinKR);
+                    probe.R = c->tc_r_max[l];
                     const int tc_slots = zeno::stream_tc_norm_slots(probe);
                     if (tc_slots > layer_slots) layer_slots = tc_slots;
-                    tc_elems = (size_t)c->tc_r_max * rows * (size_t)n_r_max * (size_t)o;
-
+                    const size_t need = (size_t)c->tc_r_max[l] * rows * (size_t)n_r_max * (size_t)o;
+                    if (need > tc_elems) tc_elems = need;
                 }
             }
             slots += layer_slots;

@@ -152,7 +152,10 @@ struct TmemLayout {
 };
 
 struct StreamArgs {
-    const float *X;        // [n_r x K] the server batch
+    const float *X;        // [n_r x K] the server batch, or the models' activations [m+1][n_r][K]
+    int64_t x_model_stride;   // 0 when every model shares X (first layer)
+    int tile_groups;       // per-model mode: blocks per model along y (each takes every tile_groups-th tile)
+    float gamma;           // per-model mode: A = x - gamma v is formed here
     const float *V;        // for the bias entries' v^2
     int64_t ldv;
     int64_t offB;          // element offset of this layer's bias inside a row of V, -1 if none
@@ -166,9 +169,17 @@ struct StreamArgs {
     int *status;           // device status word (raised on a wait that gave up)
 };
 
+// PER_MODEL = false: the first layer.  B = the shared batch, A = raw rows of [x; V] (the layer is
+//   linear in its weights, the caller combines X W^T - gamma X V^T), a block's items are row tiles
+//   blockIdx.y, blockIdx.y + gridDim.y, .. of the stacked matrix.
+// PER_MODEL = true: a later layer.  B = model c's own activations, A = x - gamma v formed by the
+//   converters from an x tile and a v tile that arrive together in one stage; a block belongs to
+//   one model and takes every tile_groups-th row tile of it.
+template <bool PER_MODEL>
 __global__ void __launch_bounds__(kThreads, 1)
 stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_v,
                      StreamArgs a) {
+    constexpr int kStage = PER_MODEL ? 2 * kStageBytes : kStageBytes;   // x tile then v tile, or one tile
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     // per pipeline: full[kMaxStages], empty[kMaxStages], a_full[kMaxABufs], a_empty[kMaxABufs], d_full, d_empty
     constexpr int kBarsPerPipe = 2 * kMaxStages + 2 * kMaxABufs + 2;
@@ -183,6 +194,19 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     const int k_len = min(a.KR, a.K - k0);
     const int nkb = (k_len + kBlockK - 1) / kBlockK;   // k-blocks in this range
     const int n_items_total = (a.m + 1) * a.tiles_per_model;
+    // item li of this block -> (model, tile); false when the block has no such item
+    auto get_item = [&](int li, int &model, int &tile) {
+        if (PER_MODEL) {
+            model = blockIdx.y / a.tile_groups;
+            tile = blockIdx.y % a.tile_groups + li * a.tile_groups;
+            return tile < a.tiles_per_model;
+        }
+        const int item = blockIdx.y + li * gridDim.y;
+        model = item / a.tiles_per_model;
+        tile = item % a.tiles_per_model;
+        return item < n_items_total;
+    };
+    const float *Xsrc = a.X + (PER_MODEL ? (int64_t)(blockIdx.y / a.tile_groups) * a.x_model_stride : 0);
     const int n_stages = a.stages;
 
     // shared memory carve-up (dynamic part is 1024-byte aligned)
@@ -190,7 +214,7 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     const int nkb_max = a.KR / kBlockK;
     const uint32_t xkb_bytes = 2u * a.n_pad * 128;     // one k-block of [X_hi; X_lo]: a multiple of 1024
     uint8_t *xs = base;
-    uint8_t *stage_base = base + (uint32_t)nkb_max * xkb_bytes;   // pipeline p's ring at p * n_stages * kStageBytes
+    uint8_t *stage_base = base + (uint32_t)nkb_max * xkb_bytes;   // pipeline p's ring at p * n_stages * kStage
     const TmemLayout tl(a.n_pad);
     const int n_abufs = tl.n_abufs;
 
@@ -238,7 +262,7 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             const int c = t & 7, j = (t >> 3) % a.n_pad, kb = (t >> 3) / a.n_pad;
             const int k = k0 + kb * kBlockK + c * 4;
             float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (j < a.n_r && k < a.K && kb < nkb) v = __ldg(reinterpret_cast<const float4 *>(a.X + (int64_t)j * a.K + k));
+            if (j < a.n_r && k < a.K && kb < nkb) v = __ldg(reinterpret_cast<const float4 *>(Xsrc + (int64_t)j * a.K + k));
             float4 hi = make_float4(tf32_hi(v.x), tf32_hi(v.y), tf32_hi(v.z), tf32_hi(v.w));
             float4 lo = make_float4(v.x - hi.x, v.y - hi.y, v.z - hi.z, v.w - hi.w);
             const uint32_t off = (uint32_t)kb * xkb_bytes + j * 128 + ((c ^ (j & 7)) << 4);
@@ -255,19 +279,29 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         // ------------------------------------------------------------------ TMA producers
         const int p = warp;
         if (lane == 0) {
-            uint8_t *ring = stage_base + (size_t)p * n_stages * kStageBytes;
+            uint8_t *ring = stage_base + (size_t)p * n_stages * kStage;
             uint32_t it = 0;
-            for (int item = blockIdx.y + p * gridDim.y; item < n_items_total && !*abortp; item += kPipes * gridDim.y) {
-                const int model = item / a.tiles_per_model, tile = item % a.tiles_per_model;
-                // one issue site for both operands: x is a one-model stack
-                const CUtensorMap *map = model == 0 ? &map_x : &map_v;
+            int model, tile;
+            for (int li = p; get_item(li, model, tile) && !*abortp; li += kPipes) {
                 const int c2 = max(model - 1, 0);
                 for (int kb = 0; kb < nkb; ++kb, ++it) {
                     const int s = it % n_stages;
                     if (!mbar_wait(bar_empty(p, s), ((it / n_stages) & 1) ^ 1, abortp)) break;
-                    mbar_expect_tx(bar_full(p, s), kStageBytes);
-                    tma_load_3d(smem_u32(ring + s * kStageBytes), map, k0 + kb * kBlockK, tile * kTileRows, c2,
-                                bar_full(p, s));
+                    const uint32_t dst = smem_u32(ring + s * kStage);
+                    if (PER_MODEL) {
+                        // x tile always, v tile for the candidates; both land on the same barrier
+                        const int n_loads = model > 0 ? 2 : 1;
+                        mbar_expect_tx(bar_full(p, s), n_loads * kStageBytes);
+#pragma unroll 1
+                        for (int w = 0; w < n_loads; ++w)       // kept as ONE issue site
+                            tma_load_3d(dst + w * kStageBytes, w ? &map_v : &map_x, k0 + kb * kBlockK,
+                                        tile * kTileRows, w ? c2 : 0, bar_full(p, s));
+                    } else {
+                        // one issue site for both operands: x is a one-model stack
+                        const CUtensorMap *map = model == 0 ? &map_x : &map_v;
+                        mbar_expect_tx(bar_full(p, s), kStageBytes);
+                        tma_load_3d(dst, map, k0 + kb * kBlockK, tile * kTileRows, c2, bar_full(p, s));
+                    }
                     issued[p][s] = (int)(it / n_stages) + 1;
                 }
             }
@@ -283,7 +317,8 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             const uint32_t d1 = tmem + p * tl.set_stride, d2 = d1 + tl.d2_off;
             const uint32_t a_bufs = tmem + tl.a_base + p * n_abufs * 64;
             uint32_t it = 0, q = 0;
-            for (int item = blockIdx.y + p * gridDim.y; item < n_items_total && !*abortp; item += kPipes * gridDim.y, ++q) {
+            int model, tile;
+            for (int li = p; get_item(li, model, tile) && !*abortp; li += kPipes, ++q) {
                 if (!mbar_wait(bar_dempty(p), (q & 1) ^ 1, abortp)) break;    // accumulator drained
                 tc_fence_after();
                 bool ok = true;
@@ -311,32 +346,62 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         const int quad = warp & 3;                    // TMEM lane quadrant this warp may access
         const int row = quad * 32 + lane;             // row of the tile = TMEM lane
         const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-        const uint8_t *ring = stage_base + (size_t)p * n_stages * kStageBytes;
+        const uint8_t *ring = stage_base + (size_t)p * n_stages * kStage;
         const uint32_t a_bufs = tmem + lane_addr + tl.a_base + p * n_abufs * 64;
         uint32_t it = 0;
-        for (int item = blockIdx.y + p * gridDim.y; item < n_items_total && !*abortp; item += kPipes * gridDim.y) {
-            const int model = item / a.tiles_per_model, tile = item % a.tiles_per_model;
+        int model, tile;
+        for (int li = p; get_item(li, model, tile) && !*abortp; li += kPipes) {
             float nrm4[4] = {0.f, 0.f, 0.f, 0.f};
             bool ok = true;
             for (int kb = 0; kb < nkb; ++kb, ++it) {
                 const int s = it % n_stages;
                 if (!mbar_wait(bar_full(p, s), (it / n_stages) & 1, abortp)) { ok = false; break; }
-                const uint8_t *src = ring + s * kStageBytes + row * 128;
+                const uint8_t *src = ring + s * kStage + row * 128;
                 float4 v[8];
-#pragma unroll
-                for (int c = 0; c < 8; ++c) v[c] = *reinterpret_cast<const float4 *>(src + ((c ^ (row & 7)) << 4));
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_empty(p, s));        // the stage may be refilled
                 uint32_t hi[32], lo[32];
+                if (PER_MODEL) {
+                    // stage = x tile then v tile: the candidate's weights are formed here
+                    float4 xv[8];
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const float e[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
+                    for (int c = 0; c < 8; ++c) xv[c] = *reinterpret_cast<const float4 *>(src + ((c ^ (row & 7)) << 4));
+                    if (model > 0) {
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        nrm4[u] = fmaf(e[u], e[u], nrm4[u]);
-                        const float h = tf32_hi(e[u]);
-                        hi[4 * c + u] = __float_as_uint(h);
-                        lo[4 * c + u] = __float_as_uint(e[u] - h);
+                        for (int c = 0; c < 8; ++c)
+                            v[c] = *reinterpret_cast<const float4 *>(src + kStageBytes + ((c ^ (row & 7)) << 4));
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) v[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_empty(p, s));    // the stage may be refilled
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const float ev[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
+                        const float ex[4] = {xv[c].x, xv[c].y, xv[c].z, xv[c].w};
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            nrm4[u] = fmaf(ev[u], ev[u], nrm4[u]);
+                            const float w = fmaf(-a.gamma, ev[u], ex[u]);
+                            const float h = tf32_hi(w);
+                            hi[4 * c + u] = __float_as_uint(h);
+                            lo[4 * c + u] = __float_as_uint(w - h);
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) v[c] = *reinterpret_cast<const float4 *>(src + ((c ^ (row & 7)) << 4));
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_empty(p, s));    // the stage may be refilled
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const float e[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            nrm4[u] = fmaf(e[u], e[u], nrm4[u]);
+                            const float h = tf32_hi(e[u]);
+                            hi[4 * c + u] = __float_as_uint(h);
+                            lo[4 * c + u] = __float_as_uint(e[u] - h);
+                        }
                     }
                 }
                 const uint32_t ab = it % n_abufs;
@@ -374,9 +439,8 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         const int quad = warp & 3;
         const int row = quad * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-        uint32_t li = 0;
-        for (int item = blockIdx.y; item < n_items_total && !*abortp; item += gridDim.y, ++li) {
-            const int model = item / a.tiles_per_model, tile = item % a.tiles_per_model;
+        int model, tile;
+        for (uint32_t li = 0; get_item((int)li, model, tile) && !*abortp; ++li) {
             const int p = li % kPipes;
             const uint32_t q = li / kPipes;               // how many accumulators pipeline p has finished before
             // thread = output row o, column = sample j
@@ -435,10 +499,13 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
 //   z_0 = sum_r P[r][0] + b(x),   z_c = z_0 - gamma (sum_r P[r][c] + b(v_c)),   h = ReLU(z)
 // One thread per (model, sample, four outputs); the 2R loads of a thread are independent and
 // the partials are added in k-range order.
+// With linear = 0 (a layer whose products were already taken with x - gamma v) only the model's own
+// partials and its bias x_b - gamma v_b are added.
 template <bool VEC4>
 __global__ void __launch_bounds__(256) stream_combine_kernel(const float *part, int R, int m, int n_r, int out,
                                                              const float *x, const float *V, int64_t ldv,
-                                                             int64_t offB, float gamma, int relu, float *H) {
+                                                             int64_t offB, float gamma, int relu, int linear,
+                                                             float *H) {
     constexpr int E = VEC4 ? 4 : 1;
     const int og = (out + E - 1) / E;                       // output groups per row
     const int64_t total = (int64_t)(m + 1) * n_r * og;
@@ -448,8 +515,9 @@ __global__ void __launch_bounds__(256) stream_combine_kernel(const float *part, 
         const int o = (int)(t % og) * E;
         const int64_t cj = t / og;
         const int c = (int)(cj / n_r), j = (int)(cj % n_r);
-        const int64_t i0 = (int64_t)j * out + o;               // model 0
         const int64_t ic = cj * out + o;
+        const int64_t i0 = linear ? (int64_t)j * out + o : ic;   // model 0 (linear), else the model itself
+        const bool two = linear && c > 0;                        // a second set of partials to add
         float z0[E], pc[E];
 #pragma unroll
         for (int e = 0; e < E; ++e) z0[e] = pc[e] = 0.f;
@@ -462,7 +530,7 @@ __global__ void __launch_bounds__(256) stream_combine_kernel(const float *part, 
                     const bool ok = r0 + u < R;
                     a4[u] = ok ? __ldcg(reinterpret_cast<const float4 *>(part + (r0 + u) * per_r + i0))
                                : make_float4(0.f, 0.f, 0.f, 0.f);
-                    b4[u] = ok && c > 0 ? __ldcg(reinterpret_cast<const float4 *>(part + (r0 + u) * per_r + ic))
+                    b4[u] = ok && two ? __ldcg(reinterpret_cast<const float4 *>(part + (r0 + u) * per_r + ic))
                                         : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
 #pragma unroll
@@ -474,16 +542,22 @@ __global__ void __launch_bounds__(256) stream_combine_kernel(const float *part, 
         } else {
             for (int r = 0; r < R; ++r) {
                 z0[0] += __ldcg(part + r * per_r + i0);
-                if (c > 0) pc[0] += __ldcg(part + r * per_r + ic);
+                if (two) pc[0] += __ldcg(part + r * per_r + ic);
             }
         }
 #pragma unroll
         for (int e = 0; e < E; ++e) {
-            if (offB >= 0) {
-                z0[e] += __ldg(x + offB + o + e);
-                if (c > 0) pc[e] += __ldg(V + (int64_t)(c - 1) * ldv + offB + o + e);
+            if (offB >= 0 && o + e < out) {
+                const float xb = __ldg(x + offB + o + e);
+                const float vb = c > 0 ? __ldg(V + (int64_t)(c - 1) * ldv + offB + o + e) : 0.f;
+                if (linear) {
+                    z0[e] += xb;
+                    pc[e] += vb;
+                } else {
+                    z0[e] += fmaf(-gamma, vb, xb);
+                }
             }
-            float z = c > 0 ? fmaf(-gamma, pc[e], z0[e]) : z0[e];
+            float z = two ? fmaf(-gamma, pc[e], z0[e]) : z0[e];
             if (relu) z = (z > 0.f || z != z) ? z : 0.f;
             H[ic + e] = z;
         }
@@ -515,43 +589,60 @@ EncodeTiledFn encode_tiled_fn() {
 
 // Shape of the launch for a layer of `out` rows and K inputs over m+1 models on `sms` SMs.
 // Picks the k-range length that keeps all SMs busy with an even share of row tiles.
-bool stream_tc_plan(int sms, int K, int out, int n_r, int m, StreamTcPlan *p) {
-    if (n_r < 1 || n_r > 64 || K < 256 || K % 4 != 0 || out < 64) return false;
+// Cost model, in units of the time one k-block takes: the block that finishes last runs
+// ceil(items / 2) row tiles on its busier pipeline, nkb k-blocks each, plus a fixed start-up
+// and drain; every extra k-range adds split-K partials that have to be written and summed.
+bool stream_tc_plan(int sms, int K, int out, int n_r, int m, bool per_model, StreamTcPlan *p) {
+    if (n_r < 1 || n_r > 64 || K < (per_model ? 128 : 256) || K % 4 != 0 || out < 64) return false;
     const int n_pad = (n_r + 15) / 16 * 16;
     const int tiles = (out + kTileRows - 1) / kTileRows;
-    const int items = (m + 1) * tiles;
-    double best = -1.0;
-    for (int kr = kStreamTcMinKR; kr <= 512; kr *= 2) {
+    const int stage_bytes = per_model ? 2 * kStageBytes : kStageBytes;
+    const int items_all = (m + 1) * tiles;
+    double best = 1e30;
+    for (int kr = kStreamTcMinKR; kr <= 1024; kr += kBlockK) {
         const int xs = 2 * (kr / kBlockK) * n_pad * 128;            // [X_hi; X_lo]
-        int stages = (kSmemBudget - 1024 - xs) / (kPipes * kStageBytes);   // per pipeline
+        if (xs + kPipes * 2 * stage_bytes + 1024 > kSmemBudget) break;
+        int stages = (kSmemBudget - 1024 - xs) / (kPipes * stage_bytes);   // per pipeline
         if (stages > kMaxStages) stages = kMaxStages;
-        if (stages < 2) continue;
         const int R = (K + kr - 1) / kr;
         if (R > sms) continue;
-        int G = sms / R;
-        if (G > items) G = items;
-        if (G < 1) G = 1;
-        const int per = (items + G - 1) / G;
-        double eff = (double)items / ((double)G * per) * ((double)(R * G) / sms);
-        eff -= 0.005 * R;                              // split-K partial traffic grows with R
-        if (stages < 4) eff -= 0.05;                   // a shallow ring hides less latency
-        if (eff > best) {
-            best = eff;
-            p->KR = kr; p->R = R; p->G = G; p->stages = stages;
+        if (R > 1 && (R - 1) * kr >= K) continue;                    // same R as a shorter range
+        const int nkb = kr / kBlockK;
+        const int g_hi = per_model ? tiles : (sms / R < items_all ? sms / R : items_all);
+        for (int g = 1; g <= g_hi; ++g) {
+            // g = blocks along y (first layer) or tile groups per model (later layers)
+            const int blocks = per_model ? R * (m + 1) * g : R * g;
+            const int items = per_model ? (tiles + g - 1) / g : (items_all + g - 1) / g;
+            const int waves = (blocks + sms - 1) / sms;
+            if (!per_model && waves > 1) continue;
+            // split-K partials are written and read back: 2 R n_r / K of the streamed bytes,
+            // cheap while they stay in L2
+            const double part_bytes = (double)R * (m + 1) * n_r * out * 4.0;
+            const double part_cost = 2.0 * R * n_r / K * (part_bytes > 64e6 ? 1.0 : 0.35);
+            double est = (double)waves * ((items + 1) / 2 * nkb * (1.0 + part_cost) + 6.0) + 0.2 * R;
+            if (stages < 3) est *= 1.1;                             // a shallow ring hides less latency
+            if (est < best) {
+                best = est;
+                p->KR = kr; p->R = R; p->stages = stages;
+                p->G = per_model ? (m + 1) * g : g;
+                p->tile_groups = per_model ? g : 1;
+            }
         }
     }
-    if (best < 0) return false;
+    if (best > 1e29) return false;
     p->n_pad = n_pad;
     p->tiles_per_model = tiles;
-    p->smem_bytes = 2 * (p->KR / kBlockK) * n_pad * 128 + kPipes * p->stages * kStageBytes + 1024;
+    p->per_model = per_model ? 1 : 0;
+    p->smem_bytes = 2 * (p->KR / kBlockK) * n_pad * 128 + kPipes * p->stages * stage_bytes + 1024;
     return true;
 }
 
 int stream_tc_norm_slots(const StreamTcPlan &p) { return p.R * p.tiles_per_model * 4; }
 
 cudaError_t launch_stream_tc(Context &c, const StreamTcPlan &p, const float *x, const float *V, int64_t ldv,
-                             int64_t offW, int64_t offB, int K, int out, const float *X, int n_r, int m,
-                             float *part, int np_base, cudaStream_t s, int *launches) {
+                             int64_t offW, int64_t offB, int K, int out, const float *X, int64_t x_model_stride,
+                             float gamma, int n_r, int m, float *part, int np_base, cudaStream_t s,
+                             int *launches) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return cudaErrorNotSupported;
     CUtensorMap map_x, map_v;
@@ -577,6 +668,9 @@ cudaError_t launch_stream_tc(Context &c, const StreamTcPlan &p, const float *x, 
     }
     StreamArgs a;
     a.X = X;
+    a.x_model_stride = x_model_stride;
+    a.tile_groups = p.tile_groups;
+    a.gamma = gamma;
     a.V = V;
     a.ldv = ldv;
     a.offB = offB;
@@ -595,21 +689,28 @@ cudaError_t launch_stream_tc(Context &c, const StreamTcPlan &p, const float *x, 
     a.status = c.dev_status;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(stream_tf32x3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(stream_tf32x3_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              kSmemBudget);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(stream_tf32x3_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     kSmemBudget);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
     ++*launches;
-    profile_mark(c, "stream_tf32x3", s);
+    profile_mark(c, p.per_model ? "stream_tf32x3_layer" : "stream_tf32x3", s);
     dim3 grid(p.R, p.G);
-    stream_tf32x3_kernel<<<grid, kThreads, p.smem_bytes, s>>>(map_x, map_v, a);
+    if (p.per_model)
+        stream_tf32x3_kernel<true><<<grid, kThreads, p.smem_bytes, s>>>(map_x, map_v, a);
+    else
+        stream_tf32x3_kernel<false><<<grid, kThreads, p.smem_bytes, s>>>(map_x, map_v, a);
     return cudaGetLastError();
 }
 
 cudaError_t launch_stream_combine(Context &c, const StreamTcPlan &p, const float *part, const float *x,
                                   const float *V, int64_t ldv, int64_t offB, int out, int n_r, int m,
                                   float gamma, int relu, float *H, cudaStream_t s, int *launches) {
+    const int linear = p.per_model ? 0 : 1;
     ++*launches;
     profile_mark(c, "stream_combine", s);
     const bool vec = out % 4 == 0;
@@ -618,9 +719,9 @@ cudaError_t launch_stream_combine(Context &c, const StreamTcPlan &p, const float
     const int cap = (c.sm_count > 0 ? c.sm_count : 148) * 16;
     if (blocks > cap) blocks = cap;
     if (vec)
-        stream_combine_kernel<true><<<blocks, 256, 0, s>>>(part, p.R, m, n_r, out, x, V, ldv, offB, gamma, relu, H);
+        stream_combine_kernel<true><<<blocks, 256, 0, s>>>(part, p.R, m, n_r, out, x, V, ldv, offB, gamma, relu, linear, H);
     else
-        stream_combine_kernel<false><<<blocks, 256, 0, s>>>(part, p.R, m, n_r, out, x, V, ldv, offB, gamma, relu, H);
+        stream_combine_kernel<false><<<blocks, 256, 0, s>>>(part, p.R, m, n_r, out, x, V, ldv, offB, gamma, relu, linear, H);
     return cudaGetLastError();
 }
 

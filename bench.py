@@ -20,9 +20,7 @@ import argparse
 import json
 import os
 import statistics
-import subprocess
 import sys
-import tempfile
 import time
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
@@ -68,58 +66,67 @@ def layer_bytes(w, layer):
 
 
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons, sampled while the timed region runs."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
-         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """SM clock and throttle reasons read through NVML (read-only) by a background thread every
+    few milliseconds while the timed regions run."""
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+               0x4: "sw_power_cap"}
 
-    def __init__(self, gpu_index):
-        self.gpu = gpu_index
-        self.proc = None
-        self.path = None
+    def __init__(self, gpu_index, period_s=0.005):
+        self.gpu, self.period = gpu_index, period_s
+        self.samples, self.reason_bits, self.max_mhz = [], 0, None
+        self._stop = None
+        self._thread = None
 
     def start(self):
+        import threading
         try:
-            fd, self.path = tempfile.mkstemp(suffix=".csv")
-            os.close(fd)
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                 "-i", str(self.gpu), "-lms", "100"],
-                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+            import pynvml
+            pynvml.nvmlInit()
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            index = self.gpu
+            if visible:
+                ids = [v.strip() for v in visible.split(",") if v.strip()]
+                if self.gpu < len(ids) and ids[self.gpu].isdigit():
+                    index = int(ids[self.gpu])
+            handle = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(handle, pynvml.NVML_CLOCK_SM))
         except Exception:
-            self.proc = None
+            return
+        self._stop = threading.Event()
+
+        def run():
+            while not self._stop.is_set():
+                try:
+                    self.samples.append(float(pynvml.nvmlDeviceGetClockInfo(handle, pynvml.NVML_CLOCK_SM)))
+                    self.reason_bits |= int(pynvml.nvmlDeviceGetCurrentClocksEventReasons(handle))
+                except Exception:
+                    pass
+                self._stop.wait(self.period)
+
+        self._thread = threading.Thread(target=run, daemon=True)
+        self._thread.start()
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        if self.proc is None:
-            return out
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        sm, smax, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        try:
-            with open(self.path) as fh:
-                for line in fh:
-                    f = [t.strip() for t in line.split(",")]
-                    if len(f) < 9:
-                        continue
-                    try:
-                        sm.append(float(f[1])); smax.append(float(f[2]))
-                    except ValueError:
-                        continue
-                    for n, v in zip(names, f[5:9]):
-                        if v.lower().startswith("active"):
-                            reasons.add(n)
-            os.unlink(self.path)
-        except Exception:
-            pass
-        if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), samples=len(sm))
-        out["reasons"] = sorted(reasons)
+        if self._thread is not None:
+            self._stop.set()
+            self._thread.join(timeout=2)
+        out = {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": len(self.samples)}
+        if self.samples:
+            out["sm_mhz"] = statistics.median(self.samples)
+        out["reasons"] = sorted(name for bit, name in self.REASONS.items() if self.reason_bits & bit)
         return out
+
+
+def whole_job_rate(ms_local, units_per_rank, world, dist=None, device="cpu"):
+    """Whole-job throughput from per-rank device times: the job takes as long as its slowest rank
+    (MAX over ranks), and every rank contributed units_per_rank units.  Returns (units/s, ms)."""
+    ms = float(ms_local)
+    if dist is not None and world > 1:
+        import torch
+        t = torch.tensor([ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return world * units_per_rank / (ms * 1e-3), ms
 
 
 def kind_code(w):
@@ -269,12 +276,8 @@ def run_ours(args, rank, world, local_rank):
     z.profile(False)
     clocks = sampler.stop()
 
-    if dist is not None:
-        t = torch.tensor([ms_total], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    value, ms_total = whole_job_rate(ms_total, args.steps, world, dist, "cuda")
     ms_per_step = ms_total / args.steps
-    value = world * args.steps / (ms_total * 1e-3)
 
     # ---- end to end through the host-memory entry point (copies inside the timed region)
     hx, hV = sets[0].x.cpu().pin_memory(), sets[0].V.cpu().pin_memory()
@@ -291,11 +294,7 @@ def run_ours(args, rank, world, local_rank):
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_value = world * e2e_steps / (e2e_ms * 1e-3)
+    e2e_value, e2e_ms = whole_job_rate(e2e_ms, e2e_steps, world, dist, "cuda")
     h2d = (hx.numel() * hx.element_size() + hV.numel() * hV.element_size() + hf.numel() * 4
            + ht.numel() * 4)
     d2h = hout.numel() * 4

@@ -46,6 +46,8 @@ __global__ void __launch_bounds__(256) aggregate_vec_kernel(const T *V, int64_t 
                                                              const int32_t *idx, int k, float *out) {
     constexpr int E = Group<T>::kElems;
     __shared__ int64_t rows_s[ZENO_MAX_CANDIDATES];
+    pdl_launch_dependents();
+    pdl_wait();
     stage_rows(idx, k, m, ldv, rows_s);
     const int64_t groups = d / E;            // whole groups; the d % E tail columns follow below
     for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < groups;
@@ -105,6 +107,8 @@ __global__ void __launch_bounds__(256) aggregate_scalar_kernel(const T *V, int64
                                                                 int m, const int32_t *idx, int k,
                                                                 float *out) {
     __shared__ int64_t rows_s[ZENO_MAX_CANDIDATES];
+    pdl_launch_dependents();
+    pdl_wait();
     stage_rows(idx, k, m, ldv, rows_s);
     for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < d;
          j += (int64_t)gridDim.x * blockDim.x) {
@@ -123,20 +127,21 @@ cudaError_t launch_typed(const Context &c, const T *V, int64_t ldv, int m, const
     const int sms = c.sm_count > 0 ? c.sm_count : 148;
     const int64_t d = c.d;
     constexpr int E = Group<T>::kElems;
+    cudaError_t e;
     if (aligned) {
         int64_t want = (d / E + 255) / 256;
         int64_t cap = (int64_t)sms * 8;
         int blocks = (int)(want < cap ? want : cap);
         if (blocks < 1) blocks = 1;
-        aggregate_vec_kernel<T><<<blocks, 256, 0, s>>>(V, ldv, d, m, idx, k, out);
+        e = launch_chained(aggregate_vec_kernel<T>, dim3(blocks), dim3(256), 0, s, chain_launches(c), V, ldv, d, m, idx, k, out);
     } else {
         int64_t want = (d + 255) / 256;
         int64_t cap = (int64_t)sms * 8;
         int blocks = (int)(want < cap ? want : cap);
         if (blocks < 1) blocks = 1;
-        aggregate_scalar_kernel<T><<<blocks, 256, 0, s>>>(V, ldv, d, m, idx, k, out);
+        e = launch_chained(aggregate_scalar_kernel<T>, dim3(blocks), dim3(256), 0, s, chain_launches(c), V, ldv, d, m, idx, k, out);
     }
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace

@@ -254,6 +254,7 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
     c->device = device;
     c->m_max = m_max;
     c->n_r_max = n_r_max;
+    c->chain = getenv("ZENO_DISABLE_PDL") == nullptr;
 
     DeviceGuard guard(device);
     cudaDeviceProp prop;

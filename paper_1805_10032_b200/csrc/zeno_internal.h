@@ -58,6 +58,7 @@ struct Context {
     int last_cuda_error;
     // optional per-kernel timing (zeno_profile): a ring of the last kProfileDepth calls; in a
     // call's slot events[i] is recorded before kernel i and events[n] after the last one
+    bool chain;                     // chain a step's kernels with programmatic dependent launch
     bool profile;
     cudaEvent_t events[kProfileDepth][kMaxProfiled + 1];
     const char *kernel_names[kProfileDepth][kMaxProfiled];
@@ -65,6 +66,9 @@ struct Context {
     int profiled;                   // kernels marked so far in the current call
     long long call_seq;             // calls completed since profiling was switched on
 };
+
+// Kernels overlap their set-up with the previous kernel's tail unless per-kernel events are wanted.
+inline bool chain_launches(const Context &c) { return c.chain && !c.profile; }
 
 // Records the event that closes the previous kernel and opens the next one.
 inline void profile_mark(Context &c, const char *name, cudaStream_t s) {
@@ -160,6 +164,30 @@ int mlp_norm_slots(int out);
 // ---- device helpers shared by the kernels ------------------------------------------------
 
 #ifdef __CUDACC__
+
+// Programmatic dependent launch.  Consecutive kernels of a step are chained so that a kernel's
+// blocks may become resident, and run their on-chip set-up, while the kernel before it drains.
+// Every kernel calls pdl_launch_dependents() first and pdl_wait() before it reads or writes any
+// global memory; pdl_wait() returns once the preceding kernel has completed and its writes are
+// visible (it is a no-op for a kernel launched the ordinary way).
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                  bool overlap, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
 
 __device__ __forceinline__ float bf16_bits_to_float(uint32_t hi16_in_low) {
     return __uint_as_float(hi16_in_low << 16);

@@ -87,6 +87,8 @@ __global__ void __launch_bounds__(kLayerWarps * 32, 1) mlp_layer_kernel(LayerArg
     extern __shared__ __align__(16) float smem_dyn[];
     float(*hs)[NRT][kStageK] = reinterpret_cast<float(*)[NRT][kStageK]>(smem_dyn);
 
+    pdl_launch_dependents();
+    pdl_wait();
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const int c = blockIdx.y;                    // model: 0 = x, 1+i = x - gamma v_i
@@ -248,6 +250,8 @@ __global__ void __launch_bounds__(256, 1) mlp_head_kernel(LayerArgs a) {
     float(*hs)[KC] = reinterpret_cast<float(*)[KC]>(smem_dyn + OUT_T * KC);     // [32][KC]
     __shared__ float zl[32][33];
 
+    pdl_launch_dependents();
+    pdl_wait();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int c = blockIdx.x;
     const int K = a.in;
@@ -395,6 +399,8 @@ __global__ void __launch_bounds__(256, 1) mlp_head_kernel(LayerArgs a) {
 __global__ void __launch_bounds__(256) mlp_loss_kernel(const float *logits, const int32_t *labels,
                                                         int n_r, int classes, float *losses, TailArgs tail) {
     __shared__ float per_warp[8];
+    pdl_launch_dependents();
+    pdl_wait();
     const int c = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     float mine = 0.f;
@@ -423,7 +429,7 @@ __global__ void __launch_bounds__(256) mlp_loss_kernel(const float *logits, cons
 }
 
 template <typename T, bool VEC>
-cudaError_t launch_layer_nrt(const LayerArgs &a, cudaStream_t s) {
+cudaError_t launch_layer_nrt(const LayerArgs &a, cudaStream_t s, bool overlap) {
     const int rows_per_block = kRowsPerWarp * kLayerWarps;
     auto go = [&](auto kernel, int nrt) {
         dim3 grid((a.out + rows_per_block - 1) / rows_per_block, a.m + 1, (a.n_r + nrt - 1) / nrt);
@@ -433,8 +439,7 @@ cudaError_t launch_layer_nrt(const LayerArgs &a, cudaStream_t s) {
                                                  (int)smem);
             if (e != cudaSuccess) return e;
         }
-        kernel<<<grid, kLayerWarps * 32, smem, s>>>(a);
-        return cudaGetLastError();
+        return launch_chained(kernel, grid, dim3(kLayerWarps * 32), smem, s, overlap, a);
     };
     if (a.n_r <= 8) return go(mlp_layer_kernel<T, 8, VEC>, 8);
     if (a.n_r <= 16) return go(mlp_layer_kernel<T, 16, VEC>, 16);
@@ -453,13 +458,12 @@ int mlp_norm_slots(int out) {
 bool mlp_can_fuse_loss(int out, int n_r) { return out <= kRowsPerWarp * kLayerWarps && n_r <= 32; }
 
 template <typename T, bool VEC>
-cudaError_t launch_head(const LayerArgs &a, cudaStream_t s) {
+cudaError_t launch_head(const LayerArgs &a, cudaStream_t s, bool overlap) {
     auto go = [&](auto kernel, int out_t) {
         const size_t smem = sizeof(float) * (size_t)(out_t + 32) * 512;
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        kernel<<<a.m + 1, 256, smem, s>>>(a);
-        return cudaGetLastError();
+        return launch_chained(kernel, dim3(a.m + 1), dim3(256), smem, s, overlap, a);
     };
     if (a.out <= 16) return go(mlp_head_kernel<T, 16, VEC>, 16);
     return go(mlp_head_kernel<T, 32, VEC>, 32);
@@ -471,13 +475,13 @@ cudaError_t launch_mlp_layer(Context &c, const LayerArgs &a, bool aligned, cudaS
     profile_mark(c, a.fuse_loss ? "mlp_head_loss_tail" : "mlp_layer", s);
     if (a.fuse_loss) {
         if (c.desc.param_dtype == ZENO_BF16)
-            return aligned ? launch_head<__nv_bfloat16, true>(a, s) : launch_head<__nv_bfloat16, false>(a, s);
-        return aligned ? launch_head<float, true>(a, s) : launch_head<float, false>(a, s);
+            return aligned ? launch_head<__nv_bfloat16, true>(a, s, chain_launches(c)) : launch_head<__nv_bfloat16, false>(a, s, chain_launches(c));
+        return aligned ? launch_head<float, true>(a, s, chain_launches(c)) : launch_head<float, false>(a, s, chain_launches(c));
     }
     if (c.desc.param_dtype == ZENO_BF16)
-        return aligned ? launch_layer_nrt<__nv_bfloat16, true>(a, s)
-                       : launch_layer_nrt<__nv_bfloat16, false>(a, s);
-    return aligned ? launch_layer_nrt<float, true>(a, s) : launch_layer_nrt<float, false>(a, s);
+        return aligned ? launch_layer_nrt<__nv_bfloat16, true>(a, s, chain_launches(c))
+                       : launch_layer_nrt<__nv_bfloat16, false>(a, s, chain_launches(c));
+    return aligned ? launch_layer_nrt<float, true>(a, s, chain_launches(c)) : launch_layer_nrt<float, false>(a, s, chain_launches(c));
 }
 
 cudaError_t launch_mlp_loss(Context &c, const float *logits, const int32_t *labels, int n_r,
@@ -485,8 +489,8 @@ cudaError_t launch_mlp_loss(Context &c, const float *logits, const int32_t *labe
                             int *launches) {
     ++*launches;
     profile_mark(c, "mlp_loss_tail", s);
-    mlp_loss_kernel<<<m + 1, 256, 0, s>>>(logits, labels, n_r, classes, losses, tail);
-    return cudaGetLastError();
+    return launch_chained(mlp_loss_kernel, dim3(m + 1), dim3(256), 0, s, chain_launches(c), logits, labels, n_r,
+                          classes, losses, tail);
 }
 
 }  // namespace zeno

@@ -90,6 +90,8 @@ __global__ void __launch_bounds__(kMmaWarps * 32) mlp_layer_mma_kernel(LayerArgs
     constexpr int kChunks = NRT * (kHS / 4) / (kMmaWarps * 32);   // float4 chunks of a stage per thread
     extern __shared__ __align__(16) uint4 hs_dyn[];                 // [2][NRT][kPitch]
 
+    pdl_launch_dependents();
+    pdl_wait();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
     const int c = blockIdx.y;
@@ -282,7 +284,7 @@ __global__ void __launch_bounds__(kMmaWarps * 32) mlp_layer_mma_kernel(LayerArgs
 }
 
 template <typename T>
-cudaError_t launch_mma_typed(const LayerArgs &a, cudaStream_t s) {
+cudaError_t launch_mma_typed(const LayerArgs &a, cudaStream_t s, bool overlap) {
     auto go = [&](auto kernel, int nrt) {
         dim3 grid((a.out + kMmaRows - 1) / kMmaRows * ((a.n_r + nrt - 1) / nrt), a.m + 1);
         const size_t smem = (size_t)2 * nrt * StageShape<is_bf16<T>::value>::kPitch * 16;
@@ -290,8 +292,7 @@ cudaError_t launch_mma_typed(const LayerArgs &a, cudaStream_t s) {
             cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return e;
         }
-        kernel<<<grid, kMmaWarps * 32, smem, s>>>(a);
-        return cudaGetLastError();
+        return launch_chained(kernel, grid, dim3(kMmaWarps * 32), smem, s, overlap, a);
     };
     if (a.n_r <= 16) return go(mlp_layer_mma_kernel<T, 16>, 16);
     if (a.n_r <= 32) return go(mlp_layer_mma_kernel<T, 32>, 32);
@@ -308,8 +309,8 @@ bool mlp_mma_usable(int in, int out) { return in % 8 == 0 && in >= 64 && out >= 
 cudaError_t launch_mlp_layer_mma(Context &c, const LayerArgs &a, cudaStream_t s, int *launches) {
     ++*launches;
     profile_mark(c, "mlp_layer_mma", s);
-    if (c.desc.param_dtype == ZENO_BF16) return launch_mma_typed<__nv_bfloat16>(a, s);
-    return launch_mma_typed<float>(a, s);
+    if (c.desc.param_dtype == ZENO_BF16) return launch_mma_typed<__nv_bfloat16>(a, s, chain_launches(c));
+    return launch_mma_typed<float>(a, s, chain_launches(c));
 }
 
 }  // namespace zeno

@@ -180,6 +180,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_v,
                      StreamArgs a) {
     constexpr int kStage = PER_MODEL ? 2 * kStageBytes : kStageBytes;   // x tile then v tile, or one tile
+    pdl_launch_dependents();
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     // per pipeline: full[kMaxStages], empty[kMaxStages], a_full[kMaxABufs], a_empty[kMaxABufs], d_full, d_empty
     constexpr int kBarsPerPipe = 2 * kMaxStages + 2 * kMaxABufs + 2;
@@ -250,6 +251,7 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     tc_fence_before();
     __syncthreads();                                   // barriers and the TMEM base are visible
     tc_fence_after();
+    pdl_wait();                                        // on-chip set-up done; global memory from here on
     const uint32_t tmem = tmem_base_slot;
     volatile int *abortp = &abort_flag;
 
@@ -507,6 +509,8 @@ __global__ void __launch_bounds__(256) stream_combine_kernel(const float *part, 
                                                              int64_t offB, float gamma, int relu, int linear,
                                                              float *H) {
     constexpr int E = VEC4 ? 4 : 1;
+    pdl_launch_dependents();
+    pdl_wait();
     const int og = (out + E - 1) / E;                       // output groups per row
     const int64_t total = (int64_t)(m + 1) * n_r * og;
     const int64_t per_r = (int64_t)(m + 1) * n_r * out;
@@ -701,10 +705,10 @@ cudaError_t launch_stream_tc(Context &c, const StreamTcPlan &p, const float *x, 
     profile_mark(c, p.per_model ? "stream_tf32x3_layer" : "stream_tf32x3", s);
     dim3 grid(p.R, p.G);
     if (p.per_model)
-        stream_tf32x3_kernel<true><<<grid, kThreads, p.smem_bytes, s>>>(map_x, map_v, a);
-    else
-        stream_tf32x3_kernel<false><<<grid, kThreads, p.smem_bytes, s>>>(map_x, map_v, a);
-    return cudaGetLastError();
+        return launch_chained(stream_tf32x3_kernel<true>, grid, dim3(kThreads), p.smem_bytes, s, chain_launches(c),
+                              map_x, map_v, a);
+    return launch_chained(stream_tf32x3_kernel<false>, grid, dim3(kThreads), p.smem_bytes, s, chain_launches(c),
+                          map_x, map_v, a);
 }
 
 cudaError_t launch_stream_combine(Context &c, const StreamTcPlan &p, const float *part, const float *x,
@@ -719,10 +723,10 @@ cudaError_t launch_stream_combine(Context &c, const StreamTcPlan &p, const float
     const int cap = (c.sm_count > 0 ? c.sm_count : 148) * 16;
     if (blocks > cap) blocks = cap;
     if (vec)
-        stream_combine_kernel<true><<<blocks, 256, 0, s>>>(part, p.R, m, n_r, out, x, V, ldv, offB, gamma, relu, linear, H);
-    else
-        stream_combine_kernel<false><<<blocks, 256, 0, s>>>(part, p.R, m, n_r, out, x, V, ldv, offB, gamma, relu, linear, H);
-    return cudaGetLastError();
+        return launch_chained(stream_combine_kernel<true>, dim3(blocks), dim3(256), 0, s, chain_launches(c), part,
+                              p.R, m, n_r, out, x, V, ldv, offB, gamma, relu, linear, H);
+    return launch_chained(stream_combine_kernel<false>, dim3(blocks), dim3(256), 0, s, chain_launches(c), part, p.R,
+                          m, n_r, out, x, V, ldv, offB, gamma, relu, linear, H);
 }
 
 }  // namespace zeno

@@ -237,18 +237,21 @@ __global__ void __launch_bounds__(kLayerWarps * 32, 1) mlp_layer_kernel(LayerArg
     }
 }
 
-// The last layer when it is small (out <= 32 classes, n_r <= 32 samples): one block per model
+// The last layer when it is small (out <= 32 classes and n_r <= 32 samples, or out <= 16 and
+// n_r <= 64): one block per model
 // computes all of the model's logits, its cross-entropy, and -- in the block that finishes last --
 // the scores and the ranking.  The block first forms w = x - gamma v for the layer's rows in
 // shared memory (coalesced loads, v^2 accumulated on the way) next to the model's input
-// activations; then warp q multiplies samples 4q..4q+3 against all rows, lanes striding k.
-template <typename T, int OUT_T, bool VEC>
+// activations; then warp q multiplies samples SPW q .. SPW q + SPW - 1 against all rows, lanes
+// striding k.
+template <typename T, int OUT_T, int SPW, bool VEC>
 __global__ void __launch_bounds__(256, 1) mlp_head_kernel(LayerArgs a) {
     constexpr int KC = 512;                      // k-extent staged per pass
+    constexpr int NS = 8 * SPW;                  // samples a block can hold
     extern __shared__ __align__(16) float smem_dyn[];
     float(*ws)[KC] = reinterpret_cast<float(*)[KC]>(smem_dyn);                  // [OUT_T][KC]
-    float(*hs)[KC] = reinterpret_cast<float(*)[KC]>(smem_dyn + OUT_T * KC);     // [32][KC]
-    __shared__ float zl[32][33];
+    float(*hs)[KC] = reinterpret_cast<float(*)[KC]>(smem_dyn + OUT_T * KC);     // [NS][KC]
+    __shared__ float zl[32][NS + 1];
 
     pdl_launch_dependents();
     pdl_wait();
@@ -261,11 +264,11 @@ __global__ void __launch_bounds__(256, 1) mlp_head_kernel(LayerArgs a) {
     const T *vw = vbase + a.offW;
     const float *hin = a.Hin + (int64_t)c * a.hin_cand_stride;
 
-    float acc[OUT_T][4];
+    float acc[OUT_T][SPW];
 #pragma unroll
     for (int o = 0; o < OUT_T; ++o)
 #pragma unroll
-        for (int q = 0; q < 4; ++q) acc[o][q] = 0.f;
+        for (int q = 0; q < SPW; ++q) acc[o][q] = 0.f;
     float nrm = 0.f;
 
     for (int kb = 0; kb < K; kb += KC) {
@@ -273,7 +276,7 @@ __global__ void __launch_bounds__(256, 1) mlp_head_kernel(LayerArgs a) {
         // stage w rows and activations of this chunk (zero beyond the layer's rows / samples / K)
         if (VEC) {
             // activations: asynchronous copies, in flight while the weights are formed
-            for (int t = threadIdx.x; t < 32 * (KC / 4); t += 256) {
+            for (int t = threadIdx.x; t < NS * (KC / 4); t += 256) {
                 const int j = t / (KC / 4), kk = (t % (KC / 4)) * 4;
                 const bool ok = j < a.n_r && kb + kk < K;
                 cp_async16(&hs[j][kk], ok ? hin + (int64_t)j * K + kb + kk : a.Hin, ok);
@@ -318,25 +321,25 @@ __global__ void __launch_bounds__(256, 1) mlp_head_kernel(LayerArgs a) {
                 }
                 ws[o][kk] = w;
             }
-            for (int t = threadIdx.x; t < 32 * KC; t += 256) {
+            for (int t = threadIdx.x; t < NS * KC; t += 256) {
                 const int j = t / KC, kk = t % KC;
                 hs[j][kk] = (j < a.n_r && kb + kk < K) ? __ldg(hin + (int64_t)j * K + kb + kk) : 0.f;
             }
         }
         __syncthreads();
-        // warp q: samples 4q..4q+3 against every row; lane l takes k = 4l + 128 i
+        // warp q: its SPW samples against every row; lane l takes k = 4l + 128 i
 #pragma unroll 1
         for (int i = 0; i < KC / 128; ++i) {
             if (kb + i * 128 >= K) break;
             const int kk = i * 128 + 4 * lane;
-            float4 h4[4];
+            float4 h4[SPW];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) h4[q] = *reinterpret_cast<const float4 *>(&hs[warp * 4 + q][kk]);
+            for (int q = 0; q < SPW; ++q) h4[q] = *reinterpret_cast<const float4 *>(&hs[warp * SPW + q][kk]);
 #pragma unroll
             for (int o = 0; o < OUT_T; ++o) {
                 const float4 w4 = *reinterpret_cast<const float4 *>(&ws[o][kk]);
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
+                for (int q = 0; q < SPW; ++q) {
                     acc[o][q] = fmaf(w4.x, h4[q].x, acc[o][q]);
                     acc[o][q] = fmaf(w4.y, h4[q].y, acc[o][q]);
                     acc[o][q] = fmaf(w4.z, h4[q].z, acc[o][q]);
@@ -347,15 +350,16 @@ __global__ void __launch_bounds__(256, 1) mlp_head_kernel(LayerArgs a) {
     }
 
     // lane totals: 32 (row, sample) pairs at a time; lane l receives pair l of the batch
+    constexpr int kRowsPerBatch = 32 / SPW;
 #pragma unroll
-    for (int ob = 0; ob < OUT_T; ob += 8) {
+    for (int ob = 0; ob < OUT_T; ob += kRowsPerBatch) {
         float v[32];
 #pragma unroll
-        for (int o = 0; o < 8; ++o)
+        for (int o = 0; o < kRowsPerBatch; ++o)
 #pragma unroll
-            for (int q = 0; q < 4; ++q) v[o * 4 + q] = acc[ob + o][q];
+            for (int q = 0; q < SPW; ++q) v[o * SPW + q] = acc[ob + o][q];
         float z = warp_transpose_reduce<32>(v, lane);
-        const int o = ob + (lane >> 2), j = warp * 4 + (lane & 3);
+        const int o = ob + lane / SPW, j = warp * SPW + lane % SPW;
         if (o < a.out && j < a.n_r) {
             if (a.offB >= 0) {
                 const float bx = load_elem(static_cast<const T *>(a.x) + a.offB + o);
@@ -379,14 +383,14 @@ __global__ void __launch_bounds__(256, 1) mlp_head_kernel(LayerArgs a) {
     if (has_v) block_norm_total(a.tail, c - 1);          // all layers' partials of this candidate
     if (warp == 0) {
         float l = 0.f;
-        if (lane < a.n_r) {
+        for (int j = lane; j < a.n_r; j += 32) {
             float zmax = -INFINITY;
-            for (int o = 0; o < a.out; ++o) zmax = fmaxf(zmax, zl[o][lane]);
+            for (int o = 0; o < a.out; ++o) zmax = fmaxf(zmax, zl[o][j]);
             float se = 0.f;
-            for (int o = 0; o < a.out; ++o) se += expf(zl[o][lane] - zmax);   // a NaN logit makes se NaN
-            int lab = a.labels[lane];
+            for (int o = 0; o < a.out; ++o) se += expf(zl[o][j] - zmax);   // a NaN logit makes se NaN
+            int lab = a.labels[j];
             if (lab < 0 || lab >= a.out) lab = 0;
-            l = zmax + logf(se) - zl[lab][lane];
+            l += zmax + logf(se) - zl[lab][j];
         }
         l = warp_sum(l);
         if (lane == 0) a.losses[c] = l / (float)a.n_r;
@@ -455,18 +459,19 @@ int mlp_norm_slots(int out) {
 
 // The cross-entropy can ride on the last layer's launch when one block sees all of a model's
 // logits: every output row in one block, every sample in one tile.
-bool mlp_can_fuse_loss(int out, int n_r) { return out <= kRowsPerWarp * kLayerWarps && n_r <= 32; }
+bool mlp_can_fuse_loss(int out, int n_r) { return (out <= 32 && n_r <= 32) || (out <= 16 && n_r <= 64); }
 
 template <typename T, bool VEC>
 cudaError_t launch_head(const LayerArgs &a, cudaStream_t s, bool overlap) {
-    auto go = [&](auto kernel, int out_t) {
-        const size_t smem = sizeof(float) * (size_t)(out_t + 32) * 512;
+    auto go = [&](auto kernel, int out_t, int ns) {
+        const size_t smem = sizeof(float) * (size_t)(out_t + ns) * 512;
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         return launch_chained(kernel, dim3(a.m + 1), dim3(256), smem, s, overlap, a);
     };
-    if (a.out <= 16) return go(mlp_head_kernel<T, 16, VEC>, 16);
-    return go(mlp_head_kernel<T, 32, VEC>, 32);
+    if (a.n_r > 32) return go(mlp_head_kernel<T, 16, 8, VEC>, 16, 64);
+    if (a.out <= 16) return go(mlp_head_kernel<T, 16, 4, VEC>, 16, 32);
+    return go(mlp_head_kernel<T, 32, 4, VEC>, 32, 32);
 }
 
 cudaError_t launch_mlp_layer(Context &c, const LayerArgs &a, bool aligned, cudaStream_t s,

@@ -270,6 +270,16 @@ __global__ void __launch_bounds__(256, 1) mlp_head_kernel(LayerArgs a) {
 #pragma unroll
         for (int q = 0; q < SPW; ++q) acc[o][q] = 0.f;
     float nrm = 0.f;
+    // bias of the rows this lane ends up with after the reduction: requested now, used at the end
+    constexpr int kBatches = OUT_T * SPW / 32;
+    float bias_x[kBatches], bias_v[kBatches];
+#pragma unroll
+    for (int bi = 0; bi < kBatches; ++bi) {
+        const int o = bi * (32 / SPW) + lane / SPW;
+        const bool ok = a.offB >= 0 && o < a.out;
+        bias_x[bi] = ok ? load_elem(static_cast<const T *>(a.x) + a.offB + o) : 0.f;
+        bias_v[bi] = ok && has_v ? load_elem(vbase + a.offB + o) : 0.f;
+    }
 
     for (int kb = 0; kb < K; kb += KC) {
         if (kb > 0) __syncthreads();
@@ -361,11 +371,7 @@ __global__ void __launch_bounds__(256, 1) mlp_head_kernel(LayerArgs a) {
         float z = warp_transpose_reduce<32>(v, lane);
         const int o = ob + lane / SPW, j = warp * SPW + lane % SPW;
         if (o < a.out && j < a.n_r) {
-            if (a.offB >= 0) {
-                const float bx = load_elem(static_cast<const T *>(a.x) + a.offB + o);
-                const float bv = has_v ? load_elem(vbase + a.offB + o) : 0.f;
-                z += candidate_param<T>(bx, bv, a.gamma);
-            }
+            if (a.offB >= 0) z += candidate_param<T>(bias_x[ob / kRowsPerBatch], bias_v[ob / kRowsPerBatch], a.gamma);
             if (a.relu) z = relu_keep_nan(z);
             zl[o][j] = z;
         }

@@ -522,9 +522,15 @@ __global__ void __launch_bounds__(256) stream_combine_kernel(const float *part, 
         const int64_t ic = cj * out + o;
         const int64_t i0 = linear ? (int64_t)j * out + o : ic;   // model 0 (linear), else the model itself
         const bool two = linear && c > 0;                        // a second set of partials to add
-        float z0[E], pc[E];
+        float z0[E], pc[E], xb[E], vb[E];
 #pragma unroll
-        for (int e = 0; e < E; ++e) z0[e] = pc[e] = 0.f;
+        for (int e = 0; e < E; ++e) {
+            z0[e] = pc[e] = 0.f;
+            // the bias entries come from HBM: ask for them before the partials, not after
+            const bool ok = offB >= 0 && o + e < out;
+            xb[e] = ok ? __ldg(x + offB + o + e) : 0.f;
+            vb[e] = ok && c > 0 ? __ldg(V + (int64_t)(c - 1) * ldv + offB + o + e) : 0.f;
+        }
         if (VEC4) {
             // twelve k-ranges at a time: all loads of a chunk are issued before they are added
             for (int r0 = 0; r0 < R; r0 += 12) {
@@ -552,13 +558,11 @@ __global__ void __launch_bounds__(256) stream_combine_kernel(const float *part, 
 #pragma unroll
         for (int e = 0; e < E; ++e) {
             if (offB >= 0 && o + e < out) {
-                const float xb = __ldg(x + offB + o + e);
-                const float vb = c > 0 ? __ldg(V + (int64_t)(c - 1) * ldv + offB + o + e) : 0.f;
                 if (linear) {
-                    z0[e] += xb;
-                    pc[e] += vb;
+                    z0[e] += xb[e];
+                    pc[e] += vb[e];
                 } else {
-                    z0[e] += fmaf(-gamma, vb, xb);
+                    z0[e] += fmaf(-gamma, vb[e], xb[e]);
                 }
             }
             float z = two ? fmaf(-gamma, pc[e], z0[e]) : z0[e];

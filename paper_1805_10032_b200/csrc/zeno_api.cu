@@ -147,15 +147,17 @@ zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv,
         zeno::StreamTcPlan plan;
         if (c->tc_ok[l] && aligned && !last_fused &&
             zeno::stream_tc_plan(c->sm_count, in_l, out_l, n_r, m, l > 0, &plan) && plan.R <= c->tc_r_max[l] &&
-            (l == 0 || getenv("ZENO_TC_ALL_LAYERS"))) {
+            (l == 0 || plan.fused || getenv("ZENO_TC_ALL_LAYERS"))) {
             const float *hin = l == 0 ? batch->features : c->act[(l - 1) & 1];
             e = zeno::launch_stream_tc(*c, plan, xf, Vf, ldv, c->offW[l], c->offB[l], in_l, out_l, hin,
                                        l == 0 ? 0 : (int64_t)n_r * in_l, gamma, n_r, m, c->tc_part,
-                                       c->np_base[l], s, launches);
+                                       c->act[l & 1], l + 1 < L, c->np_base[l], s, launches);
             if (e != cudaSuccess) return fail_cuda(c, e);
-            e = zeno::launch_stream_combine(*c, plan, c->tc_part, xf, Vf, ldv, c->offB[l], out_l, n_r, m, gamma,
-                                            l + 1 < L, c->act[l & 1], s, launches);
-            if (e != cudaSuccess) return fail_cuda(c, e);
+            if (!plan.fused) {
+                e = zeno::launch_stream_combine(*c, plan, c->tc_part, xf, Vf, ldv, c->offB[l], out_l, n_r, m,
+                                                gamma, l + 1 < L, c->act[l & 1], s, launches);
+                if (e != cudaSuccess) return fail_cuda(c, e);
+            }
             tail.used.base[l] = c->np_base[l];
             tail.used.count[l] = zeno::stream_tc_norm_slots(plan);
             continue;
@@ -286,8 +288,14 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
                                          &probe)) {
                     c->tc_ok[l] = true;
                     c->tc_r_max[l] = (int)((in + zeno::kStreamTcMinKR - 1) / zeno::kStreamTcMinKR);
+                    // the most slots any plan may use: the shortest k-ranges, or one k-range on a
+                    // pipeline that both converter sets share
                     probe.R = c->tc_r_max[l];
-                    const int tc_slots = zeno::stream_tc_norm_slots(probe);
+                    probe.pipes = 2;
+                    int tc_slots = zeno::stream_tc_norm_slots(probe);
+                    probe.R = 1;
+                    probe.pipes = 1;
+                    if (zeno::stream_tc_norm_slots(probe) > tc_slots) tc_slots = zeno::stream_tc_norm_slots(probe);
                     if (tc_slots > layer_slots) layer_slots = tc_slots;
                     const size_t need = (size_t)c->tc_r_max[l] * rows * (size_t)n_r_max * (size_t)o;
                     if (need > tc_elems) tc_elems = need;

@@ -21,8 +21,12 @@ constexpr int kMaxProfiled = ZENO_MAX_LAYERS + 8;
 constexpr int kProfileDepth = 64;
 
 // Launch shape of the tensor-core stream: k-range length, number of k-ranges, blocks per
-// k-range, padded sample count, 128-row tiles per model, dynamic shared memory.
-struct StreamTcPlan { int KR, R, G, n_pad, tiles_per_model, smem_bytes, stages, tile_groups, per_model; };
+// k-range, padded sample count, 128-row tiles per model, dynamic shared memory, pipelines in use
+// per block (1 or 2), and whether the block finishes the layer itself (one k-range: bias and
+// activation in the epilogue, no split-K partials).
+struct StreamTcPlan {
+    int KR, R, G, n_pad, tiles_per_model, smem_bytes, stages, tile_groups, per_model, pipes, fused;
+};
 constexpr int kStreamTcMinKR = 128;
 
 // Which norm-partial slots a call filled: per layer (first slot, count).
@@ -152,8 +156,8 @@ bool stream_tc_plan(int sms, int K, int out, int n_r, int m, bool per_model, Str
 int stream_tc_norm_slots(const StreamTcPlan &p);
 cudaError_t launch_stream_tc(Context &c, const StreamTcPlan &p, const float *x, const float *V, int64_t ldv,
                              int64_t offW, int64_t offB, int K, int out, const float *X, int64_t x_model_stride,
-                             float gamma, int n_r, int m, float *part, int np_base, cudaStream_t s,
-                             int *launches);
+                             float gamma, int n_r, int m, float *part, float *Hout, int relu, int np_base,
+                             cudaStream_t s, int *launches);
 cudaError_t launch_stream_combine(Context &c, const StreamTcPlan &p, const float *part, const float *x,
                                   const float *V, int64_t ldv, int64_t offB, int out, int n_r, int m,
                                   float gamma, int relu, float *H, cudaStream_t s, int *launches);

@@ -50,7 +50,7 @@ constexpr int kStageBytes = kTileRows * kBlockK * 4;
 constexpr int kMaxABufs = 2;            // TMEM A buffers per pipeline (hi 32 + lo 32 columns each)
 constexpr int kThreads = 32 * 16;
 constexpr int kTmemCols = 512;          // one accumulator set per pipeline, then the A buffers (see TmemLayout)
-constexpr int kSmemBudget = 220 * 1024;
+constexpr int kSmemBudget = 226 * 1024;      // dynamic; the static barriers and flags fit below the 227 KB limit
 constexpr uint32_t kSpinLimit = 1u << 22;
 
 // ---- PTX wrappers -------------------------------------------------------------------------
@@ -121,6 +121,11 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16]) {
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// a / b for small a (well below 2^20) with inv_b = 1.0f / b: no integer division in the pipelines' loops
+__device__ __forceinline__ uint32_t small_div(uint32_t a, float inv_b) {
+    return (uint32_t)__float2int_rd(((float)a + 0.5f) * inv_b);
+}
+
 // value rounded to tf32 (10 explicit mantissa bits), ties away from zero in magnitude
 __device__ __forceinline__ float tf32_hi(float a) {
     return __uint_as_float((__float_as_uint(a) + 0x1000u) & 0xffffe000u);
@@ -166,6 +171,13 @@ struct StreamArgs {
     int KR;                // floats of K per k-range (multiple of 32)
     int tiles_per_model;   // ceil(out / 128)
     int stages;            // depth of each pipeline's TMA ring (<= kMaxStages)
+    int pipes;             // pipelines in use (1 or 2); a block with one item at a time needs only one
+    int fused;             // one k-range: the epilogue adds the bias, activates and writes Hout
+    int early_loads;       // x and V were complete before the preceding kernel started: the
+                           // producers need not wait for it
+    const float *xparams;  // the parameter vector x (bias entries, fused epilogue)
+    float *Hout;           // [m+1][n_r][out] activations (fused epilogue)
+    int relu;
     int *status;           // device status word (raised on a wait that gave up)
 };
 
@@ -190,6 +202,9 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     __shared__ int issued[kPipes][kMaxStages];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // the descriptors are on their way while the barriers and TMEM are set up
+    if (tid == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
+    if (tid == 32) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
     const int r = blockIdx.x;                         // k-range
     const int k0 = r * a.KR;
     const int k_len = min(a.KR, a.K - k0);
@@ -209,6 +224,7 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     };
     const float *Xsrc = a.X + (PER_MODEL ? (int64_t)(blockIdx.y / a.tile_groups) * a.x_model_stride : 0);
     const int n_stages = a.stages;
+    const int pipes = a.pipes;
 
     // shared memory carve-up (dynamic part is 1024-byte aligned)
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -218,11 +234,20 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     uint8_t *stage_base = base + (uint32_t)nkb_max * xkb_bytes;   // pipeline p's ring at p * n_stages * kStage
     const TmemLayout tl(a.n_pad);
     const int n_abufs = tl.n_abufs;
+    // With one pipeline in use, it cycles through all the A buffers, and both converter sets feed
+    // it, taking alternate k-blocks (conversion, not the MMAs, bounds a lone pipeline).
+    const bool shared_pipe = pipes == 1;
+    const int n_abufs_eff = shared_pipe ? kPipes * n_abufs : n_abufs;
+    const float inv_stages = 1.0f / (float)n_stages, inv_abufs = 1.0f / (float)n_abufs_eff;
 
     auto bar_full = [&](int p, int s) { return smem_u32(&bars[p * kBarsPerPipe + s]); };
     auto bar_empty = [&](int p, int s) { return smem_u32(&bars[p * kBarsPerPipe + kMaxStages + s]); };
     auto bar_afull = [&](int p, int b) { return smem_u32(&bars[p * kBarsPerPipe + 2 * kMaxStages + b]); };
     auto bar_aempty = [&](int p, int b) { return smem_u32(&bars[p * kBarsPerPipe + 2 * kMaxStages + kMaxABufs + b]); };
+    // A buffer g of the block (pipeline p's buffers are g = p * n_abufs ..): barrier of its owner
+    const int ab_shift = n_abufs > 1 ? 1 : 0;           // n_abufs is 1 or 2
+    auto bar_afull_g = [&](int g) { return bar_afull(g >> ab_shift, g & (n_abufs - 1)); };
+    auto bar_aempty_g = [&](int g) { return bar_aempty(g >> ab_shift, g & (n_abufs - 1)); };
     auto bar_dfull = [&](int p) { return smem_u32(&bars[p * kBarsPerPipe + 2 * kMaxStages + 2 * kMaxABufs]); };
     auto bar_dempty = [&](int p) { return smem_u32(&bars[p * kBarsPerPipe + 2 * kMaxStages + 2 * kMaxABufs + 1]); };
 
@@ -251,7 +276,10 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     tc_fence_before();
     __syncthreads();                                   // barriers and the TMEM base are visible
     tc_fence_after();
-    pdl_wait();                                        // on-chip set-up done; global memory from here on
+    // On-chip set-up done; global memory from here on.  The weights are inputs of the whole call,
+    // so in a later kernel of the chain the producers may fetch them while the preceding kernel
+    // still runs; everything else (activations, partials, norm slots) waits for it.
+    if (!(a.early_loads && warp < kPipes)) pdl_wait();
     const uint32_t tmem = tmem_base_slot;
     volatile int *abortp = &abort_flag;
 
@@ -260,16 +288,31 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     // Everyone but the producer warps fills it while the first V tiles are already in flight.
     if (warp >= kPipes) {
         constexpr int kFillers = kThreads - 32 * kPipes;
-        for (int t = tid - 32 * kPipes; t < nkb_max * a.n_pad * 8; t += kFillers) {
-            const int c = t & 7, j = (t >> 3) % a.n_pad, kb = (t >> 3) / a.n_pad;
-            const int k = k0 + kb * kBlockK + c * 4;
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (j < a.n_r && k < a.K && kb < nkb) v = __ldg(reinterpret_cast<const float4 *>(Xsrc + (int64_t)j * a.K + k));
-            float4 hi = make_float4(tf32_hi(v.x), tf32_hi(v.y), tf32_hi(v.z), tf32_hi(v.w));
-            float4 lo = make_float4(v.x - hi.x, v.y - hi.y, v.z - hi.z, v.w - hi.w);
-            const uint32_t off = (uint32_t)kb * xkb_bytes + j * 128 + ((c ^ (j & 7)) << 4);
-            *reinterpret_cast<float4 *>(xs + off) = hi;
-            *reinterpret_cast<float4 *>(xs + off + a.n_pad * 128) = lo;   // n_pad % 8 == 0: same swizzle phase
+        constexpr int kFillBatch = 8;                    // loads of a thread in flight together
+        const int n_chunks = nkb_max * a.n_pad * 8;
+        const float inv_n_pad = 1.0f / (float)a.n_pad;   // row index / n_pad without an integer division
+        for (int t0 = tid - 32 * kPipes; t0 < n_chunks; t0 += kFillers * kFillBatch) {
+            float4 v[kFillBatch];
+#pragma unroll
+            for (int u = 0; u < kFillBatch; ++u) {
+                const int t = t0 + u * kFillers;
+                const int c = t & 7, kb = __float2int_rd(((t >> 3) + 0.5f) * inv_n_pad), j = (t >> 3) - kb * a.n_pad;
+                const int k = k0 + kb * kBlockK + c * 4;
+                v[u] = (t < n_chunks && j < a.n_r && k < a.K && kb < nkb)
+                           ? __ldg(reinterpret_cast<const float4 *>(Xsrc + (int64_t)j * a.K + k))
+                           : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int u = 0; u < kFillBatch; ++u) {
+                const int t = t0 + u * kFillers;
+                if (t >= n_chunks) break;
+                const int c = t & 7, kb = __float2int_rd(((t >> 3) + 0.5f) * inv_n_pad), j = (t >> 3) - kb * a.n_pad;
+                const float4 hi = make_float4(tf32_hi(v[u].x), tf32_hi(v[u].y), tf32_hi(v[u].z), tf32_hi(v[u].w));
+                const float4 lo = make_float4(v[u].x - hi.x, v[u].y - hi.y, v[u].z - hi.z, v[u].w - hi.w);
+                const uint32_t off = (uint32_t)kb * xkb_bytes + j * 128 + ((c ^ (j & 7)) << 4);
+                *reinterpret_cast<float4 *>(xs + off) = hi;
+                *reinterpret_cast<float4 *>(xs + off + a.n_pad * 128) = lo;   // n_pad % 8 == 0: same swizzle phase
+            }
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> tensor-core reads
         asm volatile("bar.sync 1, %0;" ::"n"(kFillers) : "memory");      // named barrier: all but the producers
@@ -279,56 +322,65 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     // matrix; pipeline p takes the items with li % kPipes == p.
     if (warp < kPipes) {
         // ------------------------------------------------------------------ TMA producers
+        // Lane w fetches operand w of a stage: the x tile (or the only tile), and in per-model mode
+        // the v tile, so that ONE instruction, at one issue site, requests the whole stage.
         const int p = warp;
-        if (lane == 0) {
+        const int w = lane;
+        constexpr int kOperands = PER_MODEL ? 2 : 1;
+        constexpr uint32_t kLanes = (1u << kOperands) - 1u;
+        if (w < kOperands && p < pipes) {
             uint8_t *ring = stage_base + (size_t)p * n_stages * kStage;
-            uint32_t it = 0;
+            int s = 0;                                 // stage, and how often the ring has wrapped
+            uint32_t round = 0;
             int model, tile;
-            for (int li = p; get_item(li, model, tile) && !*abortp; li += kPipes) {
-                const int c2 = max(model - 1, 0);
-                for (int kb = 0; kb < nkb; ++kb, ++it) {
-                    const int s = it % n_stages;
-                    if (!mbar_wait(bar_empty(p, s), ((it / n_stages) & 1) ^ 1, abortp)) break;
-                    const uint32_t dst = smem_u32(ring + s * kStage);
-                    if (PER_MODEL) {
-                        // x tile always, v tile for the candidates; both land on the same barrier
-                        const int n_loads = model > 0 ? 2 : 1;
+            for (int li = p; get_item(li, model, tile) && !*abortp; li += pipes) {
+                const int n_loads = (PER_MODEL && model > 0) ? 2 : 1;   // model 0 is x itself: no v tile
+                const bool from_v = PER_MODEL ? w > 0 : model > 0;      // x is a one-model stack
+                const CUtensorMap *map = from_v ? &map_v : &map_x;
+                const int c2 = from_v ? max(model - 1, 0) : 0;
+                bool ok = true;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    ok = mbar_wait(bar_empty(p, s), (round & 1) ^ 1, abortp);
+                    if (PER_MODEL) ok = __all_sync(kLanes, ok);
+                    if (!ok) break;
+                    if (w == 0) {
                         mbar_expect_tx(bar_full(p, s), n_loads * kStageBytes);
-#pragma unroll 1
-                        for (int w = 0; w < n_loads; ++w)       // kept as ONE issue site
-                            tma_load_3d(dst + w * kStageBytes, w ? &map_v : &map_x, k0 + kb * kBlockK,
-                                        tile * kTileRows, w ? c2 : 0, bar_full(p, s));
-                    } else {
-                        // one issue site for both operands: x is a one-model stack
-                        const CUtensorMap *map = model == 0 ? &map_x : &map_v;
-                        mbar_expect_tx(bar_full(p, s), kStageBytes);
-                        tma_load_3d(dst, map, k0 + kb * kBlockK, tile * kTileRows, c2, bar_full(p, s));
+                        issued[p][s] = (int)round + 1;
                     }
-                    issued[p][s] = (int)(it / n_stages) + 1;
+                    if (PER_MODEL) __syncwarp(kLanes);
+                    if (w < n_loads)
+                        tma_load_3d(smem_u32(ring + s * kStage) + w * kStageBytes, map, k0 + kb * kBlockK,
+                                    tile * kTileRows, c2, bar_full(p, s));
+                    if (++s == n_stages) {
+                        s = 0;
+                        ++round;
+                    }
                 }
+                if (!ok) break;
             }
         }
     } else if (warp < 2 * kPipes) {
         // ------------------------------------------------------------------ MMA issuers
         const int p = warp - kPipes;
-        if (lane == 0) {
+        if (lane == 0 && p < pipes) {
             // instruction descriptors: D fp32, A and B tf32, both K-major, M = 128, N = n_pad / 2 n_pad
             const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(a.n_pad >> 3) << 17) |
                                    ((uint32_t)(kTileRows >> 4) << 24);
             const uint32_t idesc2 = (idesc & ~(0x3fu << 17)) | ((uint32_t)((2 * a.n_pad) >> 3) << 17);
             const uint32_t d1 = tmem + p * tl.set_stride, d2 = d1 + tl.d2_off;
-            const uint32_t a_bufs = tmem + tl.a_base + p * n_abufs * 64;
+            const int g0 = shared_pipe ? 0 : p * n_abufs;       // first A buffer of this pipeline
             uint32_t it = 0, q = 0;
             int model, tile;
-            for (int li = p; get_item(li, model, tile) && !*abortp; li += kPipes, ++q) {
+            for (int li = p; get_item(li, model, tile) && !*abortp; li += pipes, ++q) {
                 if (!mbar_wait(bar_dempty(p), (q & 1) ^ 1, abortp)) break;    // accumulator drained
                 tc_fence_after();
                 bool ok = true;
                 for (int kb = 0; kb < nkb; ++kb, ++it) {
-                    const uint32_t ab = it % n_abufs;
-                    if (!mbar_wait(bar_afull(p, ab), (it / n_abufs) & 1, abortp)) { ok = false; break; }
+                    const uint32_t around = small_div(it, inv_abufs);          // uses of this A buffer so far
+                    const int g = g0 + (int)(it - around * n_abufs_eff);
+                    if (!mbar_wait(bar_afull_g(g), around & 1, abortp)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t a_tmem = a_bufs + ab * 64;
+                    const uint32_t a_tmem = tmem + tl.a_base + g * 64;
                     const uint32_t bx = smem_u32(xs) + (uint32_t)kb * xkb_bytes;
 #pragma unroll
                     for (int ks = 0; ks < kBlockK / 8; ++ks) {
@@ -336,7 +388,7 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                         tc_mma_tf32_ts(d1, a_tmem + ks * 8, db, idesc2, (kb | ks) != 0);       // a_hi [x_hi; x_lo]
                         tc_mma_tf32_ts(d2, a_tmem + 32 + ks * 8, db, idesc, (kb | ks) != 0);   // a_lo x_hi
                     }
-                    tc_commit(bar_aempty(p, ab));      // the A buffer may be overwritten once these finish
+                    tc_commit(bar_aempty_g(g));        // the A buffer may be overwritten once these finish
                 }
                 if (!ok) break;
                 tc_commit(bar_dfull(p));               // accumulators complete
@@ -344,20 +396,25 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         }
     } else if (warp < 2 * kPipes + 4 * kPipes) {
         // ------------------------------------------------------------------ converters
-        const int p = (warp - 2 * kPipes) >> 2;
+        const int cset = (warp - 2 * kPipes) >> 2;    // converter set
+        const int p = shared_pipe ? 0 : cset;
+        const int kstep = shared_pipe ? kPipes : 1;
+        const int g0 = shared_pipe ? 0 : p * n_abufs;
         const int quad = warp & 3;                    // TMEM lane quadrant this warp may access
         const int row = quad * 32 + lane;             // row of the tile = TMEM lane
         const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
         const uint8_t *ring = stage_base + (size_t)p * n_stages * kStage;
-        const uint32_t a_bufs = tmem + lane_addr + tl.a_base + p * n_abufs * 64;
-        uint32_t it = 0;
+        const uint32_t a_bufs = tmem + lane_addr + tl.a_base;
+        uint32_t it0 = 0;                             // k-blocks of this pipeline before the item
         int model, tile;
-        for (int li = p; get_item(li, model, tile) && !*abortp; li += kPipes) {
+        for (int li = p; get_item(li, model, tile) && !*abortp; li += pipes, it0 += nkb) {
             float nrm4[4] = {0.f, 0.f, 0.f, 0.f};
             bool ok = true;
-            for (int kb = 0; kb < nkb; ++kb, ++it) {
-                const int s = it % n_stages;
-                if (!mbar_wait(bar_full(p, s), (it / n_stages) & 1, abortp)) { ok = false; break; }
+            for (int kb = shared_pipe ? (int)((cset - it0) & 1u) : 0; kb < nkb; kb += kstep) {
+                const uint32_t it = it0 + kb;
+                const uint32_t sround = small_div(it, inv_stages);
+                const int s = (int)(it - sround * n_stages);
+                if (!mbar_wait(bar_full(p, s), sround & 1, abortp)) { ok = false; break; }
                 const uint8_t *src = ring + s * kStage + row * 128;
                 float4 v[8];
                 uint32_t hi[32], lo[32];
@@ -406,10 +463,11 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                         }
                     }
                 }
-                const uint32_t ab = it % n_abufs;
-                if (!mbar_wait(bar_aempty(p, ab), ((it / n_abufs) & 1) ^ 1, abortp)) { ok = false; break; }
+                const uint32_t around = small_div(it, inv_abufs);
+                const int g = g0 + (int)(it - around * n_abufs_eff);
+                if (!mbar_wait(bar_aempty_g(g), (around & 1) ^ 1, abortp)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t a_tmem = a_bufs + ab * 64;
+                const uint32_t a_tmem = a_bufs + g * 64;
                 tc_st16(a_tmem, reinterpret_cast<const uint32_t(&)[16]>(hi[0]));
                 tc_st16(a_tmem + 16, reinterpret_cast<const uint32_t(&)[16]>(hi[16]));
                 tc_st16(a_tmem + 32, reinterpret_cast<const uint32_t(&)[16]>(lo[0]));
@@ -417,7 +475,7 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar_afull(p, ab));
+                if (lane == 0) mbar_arrive(bar_afull_g(g));
             }
             if (!ok) break;
 
@@ -425,7 +483,7 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             if (model > 0) {
                 float nrm = (nrm4[0] + nrm4[1]) + (nrm4[2] + nrm4[3]);
                 const int o = tile * kTileRows + row;
-                if (r == 0 && a.offB >= 0 && o < a.out) {
+                if (r == 0 && a.offB >= 0 && o < a.out && (!shared_pipe || cset == 0)) {
                     const float bv = __ldg(a.V + (int64_t)(model - 1) * a.ldv + a.offB + o);
                     nrm = fmaf(bv, bv, nrm);
                 }
@@ -433,7 +491,8 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 for (int sft = 16; sft >= 1; sft >>= 1) nrm += __shfl_xor_sync(0xffffffffu, nrm, sft);
                 if (lane == 0)
                     a.normpart[(int64_t)(model - 1) * a.np_slots + a.np_base +
-                               (r * a.tiles_per_model + tile) * 4 + quad] = nrm;
+                               ((r * a.tiles_per_model + tile) * 4 + quad) * (shared_pipe ? kPipes : 1) +
+                               (shared_pipe ? cset : 0)] = nrm;
             }
         }
     } else {
@@ -443,12 +502,17 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
         int model, tile;
         for (uint32_t li = 0; get_item((int)li, model, tile) && !*abortp; ++li) {
-            const int p = li % kPipes;
-            const uint32_t q = li / kPipes;               // how many accumulators pipeline p has finished before
+            const int p = li % pipes;
+            const uint32_t q = li / pipes;                // how many accumulators pipeline p has finished before
             // thread = output row o, column = sample j
+            const int o = tile * kTileRows + row;
+            float bias = 0.f;
+            if (a.fused && a.offB >= 0 && o < a.out) {      // asked for before the accumulator is awaited
+                const float vb = model > 0 ? __ldg(a.V + (int64_t)(model - 1) * a.ldv + a.offB + o) : 0.f;
+                bias = fmaf(-a.gamma, vb, __ldg(a.xparams + a.offB + o));
+            }
             if (!mbar_wait(bar_dfull(p), q & 1, abortp)) break;
             tc_fence_after();
-            const int o = tile * kTileRows + row;
             float *dst = a.part + (((int64_t)r * (a.m + 1) + model) * a.n_r) * a.out + o;
             const uint32_t dset = tmem + lane_addr + p * tl.set_stride;
             for (int j0 = 0; j0 < a.n_pad; j0 += 16) {
@@ -462,12 +526,21 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_dempty(p));
                 }
-                if (o < a.out) {
+                if (o < a.out && !a.fused) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
                         if (j0 + j < a.n_r)
                             dst[(int64_t)(j0 + j) * a.out] =
                                 __uint_as_float(big[j]) + (__uint_as_float(s1[j]) + __uint_as_float(s2[j]));
+                } else if (o < a.out) {
+                    float *h = a.Hout + (int64_t)model * a.n_r * a.out + o;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        if (j0 + j < a.n_r) {
+                            float z = __uint_as_float(big[j]) + (__uint_as_float(s1[j]) + __uint_as_float(s2[j])) + bias;
+                            if (a.relu) z = (z > 0.f || z != z) ? z : 0.f;
+                            h[(int64_t)(j0 + j) * a.out] = z;
+                        }
                 }
             }
         }
@@ -606,6 +679,24 @@ bool stream_tc_plan(int sms, int K, int out, int n_r, int m, bool per_model, Str
     const int tiles = (out + kTileRows - 1) / kTileRows;
     const int stage_bytes = per_model ? 2 * kStageBytes : kStageBytes;
     const int items_all = (m + 1) * tiles;
+    p->pipes = kPipes;
+    p->fused = 0;
+    if (per_model) {
+        // The whole input range in one block: no split-K partials, bias and activation in the
+        // epilogue.  One row tile per block, so one pipeline, which leaves its ring the room the
+        // resident activations [X_hi; X_lo] do not take.
+        const int kr = (K + kBlockK - 1) / kBlockK * kBlockK;
+        const int xs = 2 * (kr / kBlockK) * n_pad * 128;
+        int stages = (kSmemBudget - 1024 - xs) / stage_bytes;
+        if (stages > kMaxStages) stages = kMaxStages;
+        if (xs < kSmemBudget && stages >= 3) {
+            p->KR = kr; p->R = 1; p->stages = stages; p->pipes = 1; p->fused = 1;
+            p->G = (m + 1) * tiles; p->tile_groups = tiles;
+            p->n_pad = n_pad; p->tiles_per_model = tiles; p->per_model = 1;
+            p->smem_bytes = xs + stages * stage_bytes + 1024;
+            return true;
+        }
+    }
     double best = 1e30;
     for (int kr = kStreamTcMinKR; kr <= 1024; kr += kBlockK) {
         const int xs = 2 * (kr / kBlockK) * n_pad * 128;            // [X_hi; X_lo]
@@ -642,15 +733,20 @@ bool stream_tc_plan(int sms, int K, int out, int n_r, int m, bool per_model, Str
     p->tiles_per_model = tiles;
     p->per_model = per_model ? 1 : 0;
     p->smem_bytes = 2 * (p->KR / kBlockK) * n_pad * 128 + kPipes * p->stages * stage_bytes + 1024;
+    p->pipes = kPipes;
+    p->fused = 0;
     return true;
 }
 
-int stream_tc_norm_slots(const StreamTcPlan &p) { return p.R * p.tiles_per_model * 4; }
+// one slot per (k-range, tile, warp of a converter set); both sets write when they share a pipeline
+int stream_tc_norm_slots(const StreamTcPlan &p) {
+    return p.R * p.tiles_per_model * 4 * (p.pipes == 1 ? kPipes : 1);
+}
 
 cudaError_t launch_stream_tc(Context &c, const StreamTcPlan &p, const float *x, const float *V, int64_t ldv,
                              int64_t offW, int64_t offB, int K, int out, const float *X, int64_t x_model_stride,
-                             float gamma, int n_r, int m, float *part, int np_base, cudaStream_t s,
-                             int *launches) {
+                             float gamma, int n_r, int m, float *part, float *Hout, int relu, int np_base,
+                             cudaStream_t s, int *launches) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return cudaErrorNotSupported;
     CUtensorMap map_x, map_v;
@@ -694,6 +790,12 @@ cudaError_t launch_stream_tc(Context &c, const StreamTcPlan &p, const float *x, 
     a.KR = p.KR;
     a.tiles_per_model = p.tiles_per_model;
     a.stages = p.stages;
+    a.pipes = p.pipes;
+    a.fused = p.fused;
+    a.early_loads = p.per_model;       // a later layer: the kernels before it in the chain are this call's own
+    a.xparams = x;
+    a.Hout = Hout;
+    a.relu = relu;
     a.status = c.dev_status;
     static bool attr_set = false;
     if (!attr_set) {

@@ -28,6 +28,10 @@ SHRUNK = {
     "cfg1_nr7": (1, dict(n_r=7, m=11, b=4, faults=[(4, "signflip")])),
     "cfg2_small": (2, dict(dims=(300, 72, 40, 10), n_r=9)),
     "cfg2_wide_k": (2, dict(dims=(1028, 36, 68, 10), n_r=33, m=7, b=3, faults=[(3, "noise200")])),
+    # hidden layers wide enough for the tensor-core stream: ragged row tiles and k tails in both
+    "cfg2_mid_layers": (2, dict(dims=(520, 200, 136, 10), n_r=21, m=6, b=2, faults=[(2, "noise200")])),
+    "cfg3_mid_layers": (3, dict(dims=(520, 136, 200, 10), m=11, b=4, n_r=40,
+                                faults=[(2, "signflip"), (2, "omniscient")])),
     "cfg3_small": (3, dict(dims=(260, 44, 36, 10), m=37, b=15, n_r=70,
                            faults=[(7, "signflip"), (8, "omniscient")])),
     "cfg4_small": (4, dict(dims=(264, 136, 72, 50), m=9, b=3, n_r=19, faults=[(3, "signflip")])),

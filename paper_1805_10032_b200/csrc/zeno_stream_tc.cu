@@ -285,37 +285,56 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
 
     // [X_hi; X_lo] of this k-range in the swizzled K-major layout: k-block kb at kb * xkb_bytes,
     // row j of X_hi at j * 128, of X_lo at (n_pad + j) * 128, 16-byte chunk c at c ^ (row & 7).
-    // Everyone but the producer warps fills it while the first V tiles are already in flight.
+    // Everyone but the producer warps fills it while the first tiles are in flight.
     if (warp >= kPipes) {
         constexpr int kFillers = kThreads - 32 * kPipes;
-        constexpr int kFillBatch = 8;                    // loads of a thread in flight together
+        const int fid = tid - 32 * kPipes;
         const int n_chunks = nkb_max * a.n_pad * 8;
         const float inv_n_pad = 1.0f / (float)a.n_pad;   // row index / n_pad without an integer division
-        for (int t0 = tid - 32 * kPipes; t0 < n_chunks; t0 += kFillers * kFillBatch) {
-            float4 v[kFillBatch];
+        // 16-byte chunk t of the slice: k-block, row and column chunk; where it lives; whether it exists
+        auto chunk = [&](int t, uint32_t &off, const float *&src) {
+            const int c = t & 7, kb = __float2int_rd(((t >> 3) + 0.5f) * inv_n_pad), j = (t >> 3) - kb * a.n_pad;
+            const int k = k0 + kb * kBlockK + c * 4;
+            off = (uint32_t)kb * xkb_bytes + j * 128 + ((c ^ (j & 7)) << 4);
+            src = Xsrc + (int64_t)j * a.K + k;
+            return j < a.n_r && k < a.K && kb < nkb;
+        };
+        // asynchronous copies of the raw values (zero fill where there is nothing), all in flight at
+        // once; then every thread splits the chunks it copied, in place
+        constexpr int kIlp = 4;                          // independent chunks per loop trip
+        for (int t0 = fid; t0 < n_chunks; t0 += kIlp * kFillers) {
 #pragma unroll
-            for (int u = 0; u < kFillBatch; ++u) {
+            for (int u = 0; u < kIlp; ++u) {
                 const int t = t0 + u * kFillers;
-                const int c = t & 7, kb = __float2int_rd(((t >> 3) + 0.5f) * inv_n_pad), j = (t >> 3) - kb * a.n_pad;
-                const int k = k0 + kb * kBlockK + c * 4;
-                v[u] = (t < n_chunks && j < a.n_r && k < a.K && kb < nkb)
-                           ? __ldg(reinterpret_cast<const float4 *>(Xsrc + (int64_t)j * a.K + k))
-                           : make_float4(0.f, 0.f, 0.f, 0.f);
+                uint32_t off;
+                const float *src;
+                const bool live = chunk(t, off, src);
+                if (t < n_chunks)
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;"
+                                 ::"r"(smem_u32(xs + off)), "l"(live ? src : Xsrc), "r"(live ? 16 : 0) : "memory");
+            }
+        }
+        asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
+        for (int t0 = fid; t0 < n_chunks; t0 += kIlp * kFillers) {
+            uint32_t off[kIlp];
+            float4 v[kIlp];
+#pragma unroll
+            for (int u = 0; u < kIlp; ++u) {
+                const float *src;
+                chunk(min(t0 + u * kFillers, n_chunks - 1), off[u], src);
+                v[u] = *reinterpret_cast<const float4 *>(xs + off[u]);
             }
 #pragma unroll
-            for (int u = 0; u < kFillBatch; ++u) {
-                const int t = t0 + u * kFillers;
-                if (t >= n_chunks) break;
-                const int c = t & 7, kb = __float2int_rd(((t >> 3) + 0.5f) * inv_n_pad), j = (t >> 3) - kb * a.n_pad;
+            for (int u = 0; u < kIlp; ++u) {
+                if (t0 + u * kFillers >= n_chunks) break;
                 const float4 hi = make_float4(tf32_hi(v[u].x), tf32_hi(v[u].y), tf32_hi(v[u].z), tf32_hi(v[u].w));
                 const float4 lo = make_float4(v[u].x - hi.x, v[u].y - hi.y, v[u].z - hi.z, v[u].w - hi.w);
-                const uint32_t off = (uint32_t)kb * xkb_bytes + j * 128 + ((c ^ (j & 7)) << 4);
-                *reinterpret_cast<float4 *>(xs + off) = hi;
-                *reinterpret_cast<float4 *>(xs + off + a.n_pad * 128) = lo;   // n_pad % 8 == 0: same swizzle phase
+                *reinterpret_cast<float4 *>(xs + off[u]) = hi;
+                *reinterpret_cast<float4 *>(xs + off[u] + a.n_pad * 128) = lo;   // n_pad % 8 == 0: same swizzle phase
             }
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> tensor-core reads
-        asm volatile("bar.sync 1, %0;" ::"n"(kFillers) : "memory");      // named barrier: all but the producers
+        asm volatile("bar.sync 1, %0;" ::"n"(kFillers) : "memory");      // named barrier of the filling warps
     }
 
     // Item li of this block (li = 0, 1, ..) is row tile blockIdx.y + li * gridDim.y of the stacked
@@ -382,11 +401,15 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                     tc_fence_after();
                     const uint32_t a_tmem = tmem + tl.a_base + g * 64;
                     const uint32_t bx = smem_u32(xs) + (uint32_t)kb * xkb_bytes;
+                    // A lone pipeline alternates between the two accumulator sets, so that consecutive
+                    // k-blocks do not wait for each other's adds; the epilogue sums the sets.
+                    const uint32_t dset = shared_pipe ? (uint32_t)(kb & 1) * tl.set_stride : 0u;
+                    const uint32_t fresh = shared_pipe ? (uint32_t)(kb >> 1) : (uint32_t)kb;   // 0: first use in the item
 #pragma unroll
                     for (int ks = 0; ks < kBlockK / 8; ++ks) {
                         const uint64_t db = smem_desc_sw128(bx + ks * 32);
-                        tc_mma_tf32_ts(d1, a_tmem + ks * 8, db, idesc2, (kb | ks) != 0);       // a_hi [x_hi; x_lo]
-                        tc_mma_tf32_ts(d2, a_tmem + 32 + ks * 8, db, idesc, (kb | ks) != 0);   // a_lo x_hi
+                        tc_mma_tf32_ts(d1 + dset, a_tmem + ks * 8, db, idesc2, fresh | ks);         // a_hi [x_hi; x_lo]
+                        tc_mma_tf32_ts(d2 + dset, a_tmem + 32 + ks * 8, db, idesc, fresh | ks);     // a_lo x_hi
                     }
                     tc_commit(bar_aempty_g(g));        // the A buffer may be overwritten once these finish
                 }
@@ -517,10 +540,23 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             const uint32_t dset = tmem + lane_addr + p * tl.set_stride;
             for (int j0 = 0; j0 < a.n_pad; j0 += 16) {
                 uint32_t big[16], s1[16], s2[16];
+                float acc[16];
                 tc_ld16(dset + j0, big);                       // a_hi x_hi
                 tc_ld16(dset + a.n_pad + j0, s1);              // a_hi x_lo
                 tc_ld16(dset + tl.d2_off + j0, s2);            // a_lo x_hi
                 tc_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    acc[j] = __uint_as_float(big[j]) + (__uint_as_float(s1[j]) + __uint_as_float(s2[j]));
+                if (shared_pipe && nkb > 1) {                  // the odd k-blocks went to the second set
+                    tc_ld16(dset + tl.set_stride + j0, big);
+                    tc_ld16(dset + tl.set_stride + a.n_pad + j0, s1);
+                    tc_ld16(dset + tl.set_stride + tl.d2_off + j0, s2);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        acc[j] += __uint_as_float(big[j]) + (__uint_as_float(s1[j]) + __uint_as_float(s2[j]));
+                }
                 if (j0 + 16 >= a.n_pad) {                      // everything is in registers: release the accumulator
                     tc_fence_before();
                     __syncwarp();
@@ -530,14 +566,13 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
                         if (j0 + j < a.n_r)
-                            dst[(int64_t)(j0 + j) * a.out] =
-                                __uint_as_float(big[j]) + (__uint_as_float(s1[j]) + __uint_as_float(s2[j]));
+                            dst[(int64_t)(j0 + j) * a.out] = acc[j];
                 } else if (o < a.out) {
                     float *h = a.Hout + (int64_t)model * a.n_r * a.out + o;
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
                         if (j0 + j < a.n_r) {
-                            float z = __uint_as_float(big[j]) + (__uint_as_float(s1[j]) + __uint_as_float(s2[j])) + bias;
+                            float z = acc[j] + bias;
                             if (a.relu) z = (z > 0.f || z != z) ? z : 0.f;
                             h[(int64_t)(j0 + j) * a.out] = z;
                         }

@@ -139,9 +139,60 @@ zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv,
     const float *Vf = static_cast<const float *>(V);
     const int classes = (int)c->desc.dims[L];
     const bool fuse_loss = zeno::mlp_can_fuse_loss(classes, n_r);
+    const size_t esz0 = elem_size(c->desc.param_dtype);
+    const bool tc_rows = aligned && is_aligned(x, 16) && is_aligned(V, 16) && (ldv * esz0) % 16 == 0 &&
+                         !getenv("ZENO_DISABLE_TENSOR_CORES");
+    // layers served by the streamed tensor-core kernel: every layer of a bfloat16 model it can take,
+    // the wide later layers of an fp32 model (the first one goes to the stream that shares the batch)
+    auto layer_tc_serves = [&](int l) {
+        if (l < 0 || l >= L || !tc_rows) return false;
+        const int in_l = (int)c->desc.dims[l], out_l = (int)c->desc.dims[l + 1];
+        if ((l + 1 == L) && fuse_loss) return false;
+        if (!zeno::layer_tc_usable((zeno_dtype)c->desc.param_dtype, in_l, out_l, n_r) || n_r > c->n_r_max) return false;
+        if ((c->offW[l] * esz0) % 16 != 0) return false;
+        if (c->desc.param_dtype == ZENO_BF16) return true;
+        if (l == 0 || in_l < 128 || out_l < 128) return false;
+        zeno::StreamTcPlan plan;          // a layer short enough for the fused stream keeps it
+        return !(c->tc_ok[l] && zeno::stream_tc_plan(c->sm_count, in_l, out_l, n_r, m, true, &plan) && plan.fused);
+    };
+    bool have_split = false;               // the previous layer left its output in the stacked form
     for (int l = 0; l < L; ++l) {
         const int in_l = (int)c->desc.dims[l], out_l = (int)c->desc.dims[l + 1];
         const bool last_fused = (l + 1 == L) && fuse_loss;
+        if (layer_tc_serves(l)) {
+            void *hs_in = c->act_split[(l + 1) & 1];
+            if (!have_split) {
+                const float *plain = l == 0 ? batch->features : c->act[(l - 1) & 1];
+                e = zeno::launch_split_acts(*c, plain, l == 0 ? 1 : m + 1, n_r, in_l, hs_in, s, launches);
+                if (e != cudaSuccess) return fail_cuda(c, e);
+            }
+            const bool next_tc = layer_tc_serves(l + 1);
+            zeno::LayerTcLaunch t;
+            t.x = x;
+            t.V = V;
+            t.ldv = ldv;
+            t.offW = c->offW[l];
+            t.offB = c->offB[l];
+            t.K = in_l;
+            t.out = out_l;
+            t.n_r = n_r;
+            t.n_pad = zeno::layer_tc_n_pad(n_r);
+            t.m = m;
+            t.h_shared = l == 0;
+            t.Hsplit_in = hs_in;
+            t.Hout = next_tc ? nullptr : c->act[l & 1];
+            t.Hsplit_out = next_tc ? c->act_split[l & 1] : nullptr;
+            t.relu = l + 1 < L;
+            t.gamma = gamma;
+            t.np_base = c->np_base[l];
+            e = zeno::launch_layer_tc(*c, t, s, launches);
+            if (e != cudaSuccess) return fail_cuda(c, e);
+            tail.used.base[l] = c->np_base[l];
+            tail.used.count[l] = zeno::layer_tc_norm_slots(out_l);
+            have_split = next_tc;
+            continue;
+        }
+        have_split = false;
         // fp32 layers on the tcgen05 stream when the shape and the alignment allow it: the first
         // layer against the shared batch, later layers against each model's own activations
         zeno::StreamTcPlan plan;
@@ -268,7 +319,7 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
     c->sm_count = prop.multiProcessorCount;
 
     const size_t rows = (size_t)m_max + 1;
-    size_t act_elems = 0, norm_elems = 0, lsq_elems = 0, tc_elems = 0, ticket_elems = 1;
+    size_t act_elems = 0, norm_elems = 0, lsq_elems = 0, tc_elems = 0, ticket_elems = 1, split_elems = 0;
     if (desc->kind == ZENO_LOSS_SOFTMAX_MLP) {
         int64_t off = 0, widest = 0;
         int slots = 0;
@@ -301,6 +352,13 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
                     if (need > tc_elems) tc_elems = need;
                 }
             }
+            if (zeno::layer_tc_usable((zeno_dtype)desc->param_dtype, (int)in, (int)o, n_r_max < 128 ? n_r_max : 128) &&
+                !getenv("ZENO_DISABLE_TENSOR_CORES")) {
+                if (zeno::layer_tc_norm_slots((int)o) > layer_slots) layer_slots = zeno::layer_tc_norm_slots((int)o);
+                const size_t need = (l == 0 ? 1 : rows) * 2 * (size_t)zeno::layer_tc_n_pad(n_r_max < 128 ? n_r_max : 128) *
+                                    (size_t)in;
+                if (need > split_elems) split_elems = need;
+            }
             slots += layer_slots;
             if (o > widest) widest = o;
         }
@@ -324,6 +382,7 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
     const size_t at_scores = reserve(m_max, 4), at_idx = reserve(m_max, 4);
     const size_t at_status = reserve(1, 4), at_tc = reserve(tc_elems, 4);
     const size_t at_tickets = reserve(ticket_elems, 4);
+    const size_t at_split0 = reserve(split_elems, 4), at_split1 = reserve(split_elems, 4);
 
     e = cudaMalloc(&c->arena, bytes);
     if (e != cudaSuccess) {
@@ -343,6 +402,8 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
     c->dev_status = reinterpret_cast<int *>(base + at_status);
     c->tc_part = reinterpret_cast<float *>(base + at_tc);
     c->tickets = reinterpret_cast<unsigned *>(base + at_tickets);
+    c->act_split[0] = base + at_split0;
+    c->act_split[1] = base + at_split1;
     e = cudaMemset(c->dev_status, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(c->tickets, 0, ticket_elems * sizeof(unsigned));
     if (e != cudaSuccess) {

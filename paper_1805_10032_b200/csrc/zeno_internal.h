@@ -44,6 +44,7 @@ struct Context {
     int np_slots;                   // norm-partial slots per candidate
     void *arena;                    // the one device allocation everything below is carved from
     float *act[2];                  // activations [m_max+1][n_r_max][widest layer output]
+    void *act_split[2];             // two-term stacked activations for the streamed tensor-core layers
     float *normpart;                // [m_max][np_slots] partial sums of v^2
     float *lsq_part;                // [slabs][m_max+1][n_r_max+1] partial A.v and v^2
     int lsq_slabs;
@@ -161,6 +162,28 @@ cudaError_t launch_stream_tc(Context &c, const StreamTcPlan &p, const float *x, 
 cudaError_t launch_stream_combine(Context &c, const StreamTcPlan &p, const float *part, const float *x,
                                   const float *V, int64_t ldv, int64_t offB, int out, int n_r, int m,
                                   float gamma, int relu, float *H, cudaStream_t s, int *launches);
+
+// Dense layer on the tensor cores with both operands streamed (any layer of a bfloat16 model, the
+// later layers of an fp32 model).  Its input activations come as the two-term stacked operand
+// [models][2 n_pad][K] that launch_split_acts, or a preceding layer of this kind, writes.
+struct LayerTcLaunch {
+    const void *x, *V;
+    int64_t ldv, offW, offB;
+    int K, out, n_r, n_pad, m;
+    int h_shared;            // first layer: one set of activations for every model
+    const void *Hsplit_in;
+    float *Hout;             // plain fp32 output [m+1][n_r][out], or NULL
+    void *Hsplit_out;        // stacked two-term output for a following layer of this kind, or NULL
+    int relu;
+    float gamma;
+    int np_base;
+};
+bool layer_tc_usable(zeno_dtype dtype, int K, int out, int n_r);
+int layer_tc_n_pad(int n_r);
+int layer_tc_norm_slots(int out);
+cudaError_t launch_layer_tc(Context &c, const LayerTcLaunch &l, cudaStream_t s, int *launches);
+cudaError_t launch_split_acts(Context &c, const float *H, int models, int n_r, int K, void *out, cudaStream_t s,
+                              int *launches);
 
 int lsq_slab_count(const Context &c);
 int mlp_norm_slots(int out);

@@ -1,0 +1,558 @@
+// Dense layers of all m+1 models on the 5th-generation tensor cores, both operands streamed.
+//
+// For every model c the layer is  Z_c = H_c (x - gamma v_c)^T + b_c  with H_c the model's own input
+// activations [n_r x K] (the shared server batch for the first layer).  A block takes whole
+// 128-row tiles of one model's weight matrix over the full input range K, so there are no split-K
+// partial sums: the epilogue adds the bias, applies the activation and writes the layer's output.
+//
+// Per k-block (128 bytes of every row: 32 floats or 64 bfloat16) ONE ring stage receives, by TMA,
+//   the x tile and the v tile (128 rows each, 128-byte swizzled), and
+//   the k-block of the activations, already split into two terms and stacked: rows 0..n_pad-1
+//   hold h_hi, rows n_pad..2 n_pad-1 hold h_lo, so that one MMA yields w h_hi and w h_lo side by side.
+// Converter warps form the candidate's weights w = x - gamma v from the two tiles (thread = row),
+// accumulate v^2 for the score's norm term, and put w into TMEM as the MMA's A operand; the
+// activations are the B operand, read from the stage by the tensor core itself.
+//
+//   fp32 storage : w is split too, w = w_hi + w_lo (tf32 + remainder); D1 += w_hi [h_hi; h_lo]^T,
+//                  D2 += w_lo h_hi^T (kind::tf32, K = 8 per MMA); result D1[j] + D1[n_pad + j] + D2[j].
+//   bf16 storage : the candidate is a bfloat16 model, w = RN_bf16(x - gamma v) is exact in the A
+//                  operand; the fp32 activations are carried as two bfloat16 terms;
+//                  D += w [h_hi; h_lo]^T (kind::f16, K = 16 per MMA); result D[j] + D[n_pad + j].
+//
+// Warp roles: warp 0 TMA producer, warp 1 MMA issuer and owner of TMEM (both stay converged and
+// issue from one elected lane), warps 4-11 two converter sets taking alternate k-blocks, warps
+// 12-15 epilogue.  Accumulator sets alternate between consecutive tiles when two fit in TMEM, so
+// a tile is drained while the next one is accumulated.  Every mbarrier wait is bounded; a wait that
+// gives up raises a status word and the block leaves through the common teardown.
+#include "zeno_internal.h"
+#include "zeno_tc.cuh"
+
+namespace zeno {
+
+namespace {
+
+constexpr int kRows = 128;                  // weight rows per tile = TMEM lanes
+constexpr int kRowBytes = 128;              // bytes of a row per k-block = one swizzle row
+constexpr int kTileBytes = kRows * kRowBytes;
+constexpr int kLThreads = 32 * 16;
+constexpr int kLMaxStages = 6;
+constexpr int kLMaxABufs = 8;
+constexpr int kLMaxSets = 2;
+constexpr int kLSmemBudget = 226 * 1024;
+constexpr int kLTmemCols = 512;
+
+template <typename T> struct TcTraits;
+template <> struct TcTraits<float> {
+    static constexpr int kBlockK = 32;      // elements per k-block
+    static constexpr int kACols = 64;       // TMEM columns of one A buffer: w_hi then w_lo
+    static constexpr int kAccPerPad = 3;    // accumulator columns per padded sample
+    static constexpr CUtensorMapDataType kMapType = CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+};
+template <> struct TcTraits<__nv_bfloat16> {
+    static constexpr int kBlockK = 64;
+    static constexpr int kACols = 32;
+    static constexpr int kAccPerPad = 2;
+    static constexpr CUtensorMapDataType kMapType = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+};
+
+__device__ __forceinline__ void tc_mma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+struct LayerTcArgs {
+    const void *xparams;   // the parameter vector x (bias entries)
+    const void *V;
+    int64_t ldv, offB;     // offB: element offset of the layer's bias inside a parameter vector, -1 if none
+    float gamma;
+    int K, out, n_r, n_pad, m;
+    int tiles;             // ceil(out / 128)
+    int h_shared;          // every model reads the same activations (first layer)
+    int stages, n_sets, n_abufs;
+    float *Hout;           // [m+1][n_r][out] fp32, or NULL
+    void *Hsplit;          // [m+1][2 n_pad][out] two-term activations for a following layer of this kind, or NULL
+    int relu;
+    float *normpart;
+    int np_slots, np_base;
+    int *status;
+};
+
+template <typename T>
+__global__ void __launch_bounds__(kLThreads, 1)
+layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_v,
+                const __grid_constant__ CUtensorMap map_h, LayerTcArgs a) {
+    using Tr = TcTraits<T>;
+    constexpr bool kBf16 = is_bf16<T>::value;
+    constexpr int kBlockK = Tr::kBlockK;
+    pdl_launch_dependents();
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    // full[kLMaxStages], empty[kLMaxStages], a_full[kLMaxABufs], a_empty[kLMaxABufs], d_full[2], d_empty[2]
+    constexpr int kBars = 2 * kLMaxStages + 2 * kLMaxABufs + 2 * kLMaxSets;
+    __shared__ __align__(8) uint64_t bars[kBars];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+    __shared__ int issued[kLMaxStages];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
+    if (tid == 32) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
+    if (tid == 64) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_h) : "memory");
+
+    const int nkb = (a.K + kBlockK - 1) / kBlockK;
+    const int n_items = (a.m + 1) * a.tiles;
+    const int n_stages = a.stages, n_abufs = a.n_abufs, n_sets = a.n_sets;
+    const int b_bytes = 2 * a.n_pad * kRowBytes;
+    const int stage_bytes = 2 * kTileBytes + b_bytes;          // x tile, v tile, activations
+    const int acc_cols = Tr::kAccPerPad * a.n_pad;
+    const int a_base = n_sets * acc_cols;                       // TMEM: accumulator sets, then the A buffers
+    const float inv_stages = 1.0f / (float)n_stages, inv_abufs = 1.0f / (float)n_abufs;
+    uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+
+    auto bar_full = [&](int s) { return smem_u32(&bars[s]); };
+    auto bar_empty = [&](int s) { return smem_u32(&bars[kLMaxStages + s]); };
+    auto bar_afull = [&](int g) { return smem_u32(&bars[2 * kLMaxStages + g]); };
+    auto bar_aempty = [&](int g) { return smem_u32(&bars[2 * kLMaxStages + kLMaxABufs + g]); };
+    auto bar_dfull = [&](int q) { return smem_u32(&bars[2 * kLMaxStages + 2 * kLMaxABufs + q]); };
+    auto bar_dempty = [&](int q) { return smem_u32(&bars[2 * kLMaxStages + 2 * kLMaxABufs + kLMaxSets + q]); };
+    // item li of this block -> (model, tile); neighbouring blocks share a model's activations in L2
+    auto get_item = [&](int li, int &model, int &tile) {
+        const int item = blockIdx.x + li * gridDim.x;
+        model = item / a.tiles;
+        tile = item - model * a.tiles;
+        return item < n_items;
+    };
+
+    if (tid == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < kLMaxStages; ++s) {
+            mbar_init(bar_full(s), 1);
+            mbar_init(bar_empty(s), 5);        // the four warps of a converter set and the MMAs' commit
+            issued[s] = 0;
+        }
+        for (int g = 0; g < kLMaxABufs; ++g) {
+            mbar_init(bar_afull(g), 4);
+            mbar_init(bar_aempty(g), 1);
+        }
+        for (int q = 0; q < kLMaxSets; ++q) {
+            mbar_init(bar_dfull(q), 1);
+            mbar_init(bar_dempty(q), 4);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {   // TMEM allocation by one full warp
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&tmem_base_slot)), "r"(kLTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    pdl_wait();                                        // the activations come from the preceding kernel
+    const uint32_t tmem = tmem_base_slot;
+    volatile int *abortp = &abort_flag;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        int s = 0;
+        uint32_t round = 0;
+        int model, tile;
+        for (int li = 0;; ++li) {
+            if (!__all_sync(0xffffffffu, get_item(li, model, tile) && !*abortp)) break;
+            const bool has_v = model > 0;                 // model 0 is x itself
+            bool ok = true;
+            for (int kb = 0; kb < nkb; ++kb) {
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_empty(s), (round & 1) ^ 1, abortp));
+                if (!ok) break;
+                if (elect_one()) {
+                    const uint32_t dst = smem_u32(ring + (size_t)s * stage_bytes);
+                    mbar_expect_tx(bar_full(s), (has_v ? 2 : 1) * kTileBytes + b_bytes);
+                    issued[s] = (int)round + 1;
+#pragma unroll 1
+                    for (int w = 0; w < 3; ++w) {         // x tile, v tile, activations: ONE issue site
+                        if (w == 1 && !has_v) continue;
+                        const CUtensorMap *map = w == 0 ? &map_x : w == 1 ? &map_v : &map_h;
+                        const int c1 = w == 2 ? 0 : tile * kRows;
+                        const int c2 = w == 0 ? 0 : w == 1 ? model - 1 : (a.h_shared ? 0 : model);
+                        tma_load_3d(dst + w * kTileBytes, map, kb * kBlockK, c1, c2, bar_full(s));
+                    }
+                }
+                __syncwarp();
+                if (++s == n_stages) {
+                    s = 0;
+                    ++round;
+                }
+            }
+            if (!ok) break;
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        // instruction descriptor: D fp32, A and B tf32 (2) or bf16 (1), both K-major, M = 128
+        const uint32_t fmt = kBf16 ? 1u : 2u;
+        const uint32_t idesc_base = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(kRows >> 4) << 24);
+        const uint32_t idesc_n = idesc_base | ((uint32_t)(a.n_pad >> 3) << 17);          // N = n_pad
+        const uint32_t idesc_2n = idesc_base | ((uint32_t)((2 * a.n_pad) >> 3) << 17);   // N = 2 n_pad
+        uint32_t it = 0;
+        int model, tile;
+        for (int li = 0;; ++li) {
+            if (!__all_sync(0xffffffffu, get_item(li, model, tile) && !*abortp)) break;
+            const int set = li % n_sets;
+            const uint32_t use = (uint32_t)(li / n_sets);        // earlier uses of this accumulator set
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_dempty(set), (use & 1) ^ 1, abortp))) break;
+            tc_fence_after();
+            const uint32_t d1 = tmem + set * acc_cols, d2 = d1 + 2 * a.n_pad;
+            bool ok = true;
+            for (int kb = 0; kb < nkb; ++kb, ++it) {
+                const uint32_t sround = small_div(it, inv_stages), around = small_div(it, inv_abufs);
+                const int s = (int)(it - sround * n_stages), g = (int)(it - around * n_abufs);
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_full(s), sround & 1, abortp) &&
+                                                 mbar_wait(bar_afull(g), around & 1, abortp));
+                if (!ok) break;
+                tc_fence_after();
+                if (elect_one()) {
+                    const uint32_t a_tmem = tmem + a_base + g * Tr::kACols;
+                    const uint32_t bx = smem_u32(ring + (size_t)s * stage_bytes + 2 * kTileBytes);
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) {            // 32 bytes of every row per MMA
+                        const uint64_t db = smem_desc_sw128(bx + ks * 32);
+                        if (kBf16) {
+                            tc_mma_bf16_ts(d1, a_tmem + ks * 8, db, idesc_2n, (uint32_t)(kb | ks));    // w [h_hi; h_lo]
+                        } else {
+                            tc_mma_tf32_ts(d1, a_tmem + ks * 8, db, idesc_2n, (uint32_t)(kb | ks));    // w_hi [h_hi; h_lo]
+                            tc_mma_tf32_ts(d2, a_tmem + 32 + ks * 8, db, idesc_n, (uint32_t)(kb | ks)); // w_lo h_hi
+                        }
+                    }
+                    tc_commit(bar_aempty(g));               // the A buffer and
+                    tc_commit(bar_empty(s));                // the stage's activations may be overwritten once these finish
+                    if (kb + 1 == nkb) tc_commit(bar_dfull(set));
+                }
+                __syncwarp();
+            }
+            if (!ok) break;
+        }
+    } else if (warp >= 4 && warp < 12) {
+        // ------------------------------------------------------------------ converters
+        const int cset = (warp - 4) >> 2;             // set 0 takes the even k-blocks of the stream, set 1 the odd
+        const int quad = warp & 3;                    // TMEM lane quadrant this warp may access
+        const int row = quad * 32 + lane;             // row of the tile = TMEM lane
+        const uint32_t a_bufs = tmem + ((uint32_t)(quad * 32) << 16) + a_base;
+        uint32_t it0 = 0;
+        int model, tile;
+        for (int li = 0; get_item(li, model, tile) && !*abortp; ++li, it0 += nkb) {
+            float nrm4[4] = {0.f, 0.f, 0.f, 0.f};
+            bool ok = true;
+            for (int kb = (int)((cset - it0) & 1u); kb < nkb; kb += 2) {
+                const uint32_t it = it0 + kb;
+                const uint32_t sround = small_div(it, inv_stages), around = small_div(it, inv_abufs);
+                const int s = (int)(it - sround * n_stages), g = (int)(it - around * n_abufs);
+                if (!mbar_wait(bar_full(s), sround & 1, abortp)) { ok = false; break; }
+                const uint8_t *src = ring + (size_t)s * stage_bytes + row * kRowBytes;
+                uint4 xq[8], vq[8];
+#pragma unroll
+                for (int c = 0; c < 8; ++c) xq[c] = *reinterpret_cast<const uint4 *>(src + ((c ^ (row & 7)) << 4));
+                if (model > 0) {
+#pragma unroll
+                    for (int c = 0; c < 8; ++c)
+                        vq[c] = *reinterpret_cast<const uint4 *>(src + kTileBytes + ((c ^ (row & 7)) << 4));
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) vq[c] = make_uint4(0u, 0u, 0u, 0u);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_empty(s));       // this set is done with the stage's weight tiles
+                uint32_t wa[32], wb[32];                        // bf16: wa = packed pairs; fp32: wa = hi, wb = lo
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const uint32_t xw[4] = {xq[c].x, xq[c].y, xq[c].z, xq[c].w};
+                    const uint32_t vw[4] = {vq[c].x, vq[c].y, vq[c].z, vq[c].w};
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        if (kBf16) {
+                            const float x0 = __uint_as_float(xw[u] << 16), x1 = __uint_as_float(xw[u] & 0xffff0000u);
+                            const float v0 = __uint_as_float(vw[u] << 16), v1 = __uint_as_float(vw[u] & 0xffff0000u);
+                            nrm4[u] = fmaf(v0, v0, nrm4[u]);
+                            nrm4[u] = fmaf(v1, v1, nrm4[u]);
+                            const __nv_bfloat162 pk = __floats2bfloat162_rn(fmaf(-a.gamma, v0, x0), fmaf(-a.gamma, v1, x1));
+                            wa[4 * c + u] = *reinterpret_cast<const uint32_t *>(&pk);
+                        } else {
+                            const float xv = __uint_as_float(xw[u]), vv = __uint_as_float(vw[u]);
+                            nrm4[u] = fmaf(vv, vv, nrm4[u]);
+                            const float w = fmaf(-a.gamma, vv, xv);
+                            const float h = tf32_hi(w);
+                            wa[4 * c + u] = __float_as_uint(h);
+                            wb[4 * c + u] = __float_as_uint(w - h);
+                        }
+                    }
+                }
+                if (!mbar_wait(bar_aempty(g), (around & 1) ^ 1, abortp)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t a_tmem = a_bufs + g * Tr::kACols;
+                tc_st32(a_tmem, wa);
+                if (!kBf16) tc_st32(a_tmem + 32, wb);
+                tc_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_afull(g));
+            }
+            if (!ok) break;
+            // partial sum of squares of this tile's rows (model 0 is x itself: not a candidate)
+            if (model > 0) {
+                float nrm = (nrm4[0] + nrm4[1]) + (nrm4[2] + nrm4[3]);
+                const int o = tile * kRows + row;
+                if (cset == 0 && a.offB >= 0 && o < a.out) {
+                    const float bv = load_elem(static_cast<const T *>(a.V) + (int64_t)(model - 1) * a.ldv + a.offB + o);
+                    nrm = fmaf(bv, bv, nrm);
+                }
+#pragma unroll
+                for (int sft = 16; sft >= 1; sft >>= 1) nrm += __shfl_xor_sync(0xffffffffu, nrm, sft);
+                if (lane == 0)
+                    a.normpart[(int64_t)(model - 1) * a.np_slots + a.np_base + (tile * 4 + quad) * 2 + cset] = nrm;
+            }
+        }
+    } else if (warp >= 12) {
+        // ------------------------------------------------------------------ epilogue
+        const int quad = warp & 3;
+        const int row = quad * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+        int model, tile;
+        for (int li = 0; get_item(li, model, tile) && !*abortp; ++li) {
+            const int set = li % n_sets;
+            const uint32_t use = (uint32_t)(li / n_sets);
+            const int o = tile * kRows + row;             // thread = output row o, column = sample j
+            float bias = 0.f;
+            if (a.offB >= 0 && o < a.out) {               // asked for before the accumulator is awaited
+                const float vb = model > 0 ? load_elem(static_cast<const T *>(a.V) + (int64_t)(model - 1) * a.ldv + a.offB + o) : 0.f;
+                bias = candidate_param<T>(load_elem(static_cast<const T *>(a.xparams) + a.offB + o), vb, a.gamma);
+            }
+            if (!mbar_wait(bar_dfull(set), use & 1, abortp)) break;
+            tc_fence_after();
+            const uint32_t dset = tmem + lane_addr + set * acc_cols;
+            for (int j0 = 0; j0 < a.n_pad; j0 += 16) {
+                uint32_t t0[16], t1[16];
+                float acc[16];
+                tc_ld16(dset + j0, t0);                       // w(_hi) h_hi
+                tc_ld16(dset + a.n_pad + j0, t1);             // w(_hi) h_lo
+                tc_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) acc[j] = __uint_as_float(t1[j]);
+                if (!kBf16) {
+                    tc_ld16(dset + 2 * a.n_pad + j0, t1);     // w_lo h_hi
+                    tc_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) acc[j] += __uint_as_float(t1[j]);
+                }
+#pragma unroll
+                for (int j = 0; j < 16; ++j) acc[j] += __uint_as_float(t0[j]);
+                if (j0 + 16 >= a.n_pad) {                     // everything is in registers: release the accumulator
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_dempty(set));
+                }
+                if (o < a.out) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int jj = j0 + j;
+                        float z = acc[j] + bias;
+                        if (a.relu) z = (z > 0.f || z != z) ? z : 0.f;
+                        if (jj >= a.n_r) z = 0.f;             // padded samples
+                        if (a.Hout && jj < a.n_r) a.Hout[((int64_t)model * a.n_r + jj) * a.out + o] = z;
+                        if (a.Hsplit) {
+                            T *hs = static_cast<T *>(a.Hsplit) + (int64_t)model * 2 * a.n_pad * a.out + o;
+                            if (kBf16) {
+                                const __nv_bfloat16 hi = __float2bfloat16_rn(z);
+                                const __nv_bfloat16 lo = __float2bfloat16_rn(z - __bfloat162float(hi));
+                                reinterpret_cast<__nv_bfloat16 *>(hs)[(int64_t)jj * a.out] = hi;
+                                reinterpret_cast<__nv_bfloat16 *>(hs)[(int64_t)(a.n_pad + jj) * a.out] = lo;
+                            } else {
+                                const float hi = tf32_hi(z);
+                                reinterpret_cast<float *>(hs)[(int64_t)jj * a.out] = hi;
+                                reinterpret_cast<float *>(hs)[(int64_t)(a.n_pad + jj) * a.out] = z - hi;
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (tid == 0 && abort_flag) {
+        // bulk copies still in flight (only after an aborted run) must land before the block exits
+        for (int s = 0; s < n_stages; ++s)
+            if (issued[s] > 0) {
+                for (uint32_t i = 0; i < kSpinLimit; ++i) {
+                    if (mbar_try_wait(bar_full(s), (uint32_t)(issued[s] - 1) & 1)) break;
+                    __nanosleep(64);
+                }
+            }
+        atomicMax(a.status, 1);
+    }
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kLTmemCols) : "memory");
+    }
+}
+
+// Activations [models][n_r][K] fp32 -> the two-term stacked operand [models][2 n_pad][K]:
+// rows 0..n_pad-1 the leading term, rows n_pad.. the remainder, zero rows for the padded samples.
+template <typename T>
+__global__ void __launch_bounds__(256) split_acts_kernel(const float *H, int models, int n_r, int n_pad, int K, T *out) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int64_t total = (int64_t)models * n_pad * K;
+    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
+        const int k = (int)(t % K);
+        const int64_t cj = t / K;
+        const int j = (int)(cj % n_pad);
+        const int64_t c = cj / n_pad;
+        const float h = j < n_r ? __ldg(H + (c * n_r + j) * K + k) : 0.f;
+        T *dst = out + (c * 2 * n_pad + j) * (int64_t)K + k;
+        if (is_bf16<T>::value) {
+            const __nv_bfloat16 hi = __float2bfloat16_rn(h);
+            reinterpret_cast<__nv_bfloat16 *>(dst)[0] = hi;
+            reinterpret_cast<__nv_bfloat16 *>(dst)[(int64_t)n_pad * K] = __float2bfloat16_rn(h - __bfloat162float(hi));
+        } else {
+            const float hi = tf32_hi(h);
+            reinterpret_cast<float *>(dst)[0] = hi;
+            reinterpret_cast<float *>(dst)[(int64_t)n_pad * K] = h - hi;
+        }
+    }
+}
+
+template <typename T>
+cudaError_t encode_maps(const LayerTcLaunch &l, CUtensorMap *map_x, CUtensorMap *map_v, CUtensorMap *map_h) {
+    using Tr = TcTraits<T>;
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return cudaErrorNotSupported;
+    const cuuint64_t es = sizeof(T);
+    cuuint32_t ones[3] = {1, 1, 1};
+    {
+        cuuint64_t dims[3] = {(cuuint64_t)l.K, (cuuint64_t)l.out, 1};
+        cuuint64_t strides[2] = {(cuuint64_t)l.K * es, (cuuint64_t)l.K * es * (cuuint64_t)l.out};
+        cuuint32_t box[3] = {(cuuint32_t)Tr::kBlockK, kRows, 1};
+        if (enc(map_x, Tr::kMapType, 3, const_cast<T *>(static_cast<const T *>(l.x) + l.offW), dims, strides, box, ones,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
+    {
+        cuuint64_t dims[3] = {(cuuint64_t)l.K, (cuuint64_t)l.out, (cuuint64_t)l.m};
+        cuuint64_t strides[2] = {(cuuint64_t)l.K * es, (cuuint64_t)l.ldv * es};
+        cuuint32_t box[3] = {(cuuint32_t)Tr::kBlockK, kRows, 1};
+        if (enc(map_v, Tr::kMapType, 3, const_cast<T *>(static_cast<const T *>(l.V) + l.offW), dims, strides, box, ones,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
+    {
+        const cuuint64_t rows = 2 * (cuuint64_t)l.n_pad, models = l.h_shared ? 1 : (cuuint64_t)l.m + 1;
+        cuuint64_t dims[3] = {(cuuint64_t)l.K, rows, models};
+        cuuint64_t strides[2] = {(cuuint64_t)l.K * es, (cuuint64_t)l.K * es * rows};
+        cuuint32_t box[3] = {(cuuint32_t)Tr::kBlockK, (cuuint32_t)rows, 1};
+        if (enc(map_h, Tr::kMapType, 3, const_cast<void *>(l.Hsplit_in), dims, strides, box, ones,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
+    return cudaSuccess;
+}
+
+template <typename T>
+cudaError_t launch_typed(Context &c, const LayerTcLaunch &l, cudaStream_t s) {
+    using Tr = TcTraits<T>;
+    CUtensorMap map_x, map_v, map_h;
+    cudaError_t e = encode_maps<T>(l, &map_x, &map_v, &map_h);
+    if (e != cudaSuccess) return e;
+    LayerTcArgs a;
+    a.xparams = l.x;
+    a.V = l.V;
+    a.ldv = l.ldv;
+    a.offB = l.offB;
+    a.gamma = l.gamma;
+    a.K = l.K;
+    a.out = l.out;
+    a.n_r = l.n_r;
+    a.n_pad = l.n_pad;
+    a.m = l.m;
+    a.tiles = (l.out + kRows - 1) / kRows;
+    a.h_shared = l.h_shared;
+    const int stage_bytes = 2 * kTileBytes + 2 * l.n_pad * kRowBytes;
+    a.stages = (kLSmemBudget - 1024) / stage_bytes;
+    if (a.stages > kLMaxStages) a.stages = kLMaxStages;
+    const int acc_cols = Tr::kAccPerPad * l.n_pad;
+    a.n_sets = 2 * acc_cols + 2 * Tr::kACols <= kLTmemCols ? 2 : 1;
+    a.n_abufs = (kLTmemCols - a.n_sets * acc_cols) / Tr::kACols;
+    if (a.n_abufs > kLMaxABufs) a.n_abufs = kLMaxABufs;
+    a.Hout = l.Hout;
+    a.Hsplit = l.Hsplit_out;
+    a.relu = l.relu;
+    a.normpart = c.normpart;
+    a.np_slots = c.np_slots;
+    a.np_base = l.np_base;
+    a.status = c.dev_status;
+    static bool attr_set = false;
+    if (!attr_set) {
+        e = cudaFuncSetAttribute(layer_tc_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLSmemBudget);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(layer_tc_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     kLSmemBudget);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    const int items = (l.m + 1) * a.tiles;
+    const int sms = c.sm_count > 0 ? c.sm_count : 148;
+    // equal shares: the fewest blocks that give the same number of rounds as one block per SM
+    const int rounds = (items + sms - 1) / sms;
+    const int blocks = (items + rounds - 1) / rounds;
+    return launch_chained(layer_tc_kernel<T>, dim3(blocks), dim3(kLThreads), (size_t)a.stages * stage_bytes + 1024, s,
+                          chain_launches(c), map_x, map_v, map_h, a);
+}
+
+}  // namespace
+
+// Shapes the kernel serves: rows of 16-byte multiples that a TMA box can step through, up to 128
+// samples (N = 2 n_pad <= 256), at least two ring stages and two A buffers.
+bool layer_tc_usable(zeno_dtype dtype, int K, int out, int n_r) {
+    const int per16 = dtype == ZENO_BF16 ? 8 : 4;
+    if (K % per16 != 0 || K < 64 || out < 32 || n_r < 1 || n_r > 128) return false;
+    const int n_pad = layer_tc_n_pad(n_r);
+    const int stage_bytes = 2 * kTileBytes + 2 * n_pad * kRowBytes;
+    if ((kLSmemBudget - 1024) / stage_bytes < 2) return false;
+    const int acc = (dtype == ZENO_BF16 ? 2 : 3) * n_pad, acols = dtype == ZENO_BF16 ? 32 : 64;
+    return (kLTmemCols - acc) / acols >= 2;
+}
+
+int layer_tc_n_pad(int n_r) { return (n_r + 15) / 16 * 16; }
+
+// one slot per (tile, warp of a converter set, converter set)
+int layer_tc_norm_slots(int out) { return (out + kRows - 1) / kRows * 8; }
+
+cudaError_t launch_layer_tc(Context &c, const LayerTcLaunch &l, cudaStream_t s, int *launches) {
+    ++*launches;
+    profile_mark(c, "layer_tc", s);
+    if (c.desc.param_dtype == ZENO_BF16) return launch_typed<__nv_bfloat16>(c, l, s);
+    return launch_typed<float>(c, l, s);
+}
+
+cudaError_t launch_split_acts(Context &c, const float *H, int models, int n_r, int K, void *out, cudaStream_t s,
+                              int *launches) {
+    ++*launches;
+    profile_mark(c, "split_acts", s);
+    const int n_pad = layer_tc_n_pad(n_r);
+    const int64_t total = (int64_t)models * n_pad * K;
+    int blocks = (int)((total + 255) / 256);
+    const int cap = (c.sm_count > 0 ? c.sm_count : 148) * 8;
+    if (blocks > cap) blocks = cap;
+    if (c.desc.param_dtype == ZENO_BF16)
+        return launch_chained(split_acts_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), 0, s, chain_launches(c), H,
+                              models, n_r, n_pad, K, static_cast<__nv_bfloat16 *>(out));
+    return launch_chained(split_acts_kernel<float>, dim3(blocks), dim3(256), 0, s, chain_launches(c), H, models, n_r,
+                          n_pad, K, static_cast<float *>(out));
+}
+
+}  // namespace zeno

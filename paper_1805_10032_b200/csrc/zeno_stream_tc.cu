@@ -37,6 +37,7 @@
 #include <cuda.h>
 
 #include "zeno_internal.h"
+#include "zeno_tc.cuh"
 
 namespace zeno {
 
@@ -51,97 +52,6 @@ constexpr int kMaxABufs = 2;            // TMEM A buffers per pipeline (hi 32 + 
 constexpr int kThreads = 32 * 16;
 constexpr int kTmemCols = 512;          // one accumulator set per pipeline, then the A buffers (see TmemLayout)
 constexpr int kSmemBudget = 226 * 1024;      // dynamic; the static barriers and flags fit below the 227 KB limit
-constexpr uint32_t kSpinLimit = 1u << 22;
-
-// ---- PTX wrappers -------------------------------------------------------------------------
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) {
-    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n.reg .pred p;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-        "selp.u32 %0, 1, 0, p;\n}\n"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait.  Returns false if it gave up (and raises *abort_flag) or if another thread did.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (i > 32) __nanosleep(40);
-        if ((i & 127u) == 127u && *abort_flag) return false;
-    }
-    *abort_flag = 1;
-    return false;
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2,
-                                            uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem]^T, tf32 inputs, fp32 accumulate
-__device__ __forceinline__ void tc_mma_tf32_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                               uint32_t accumulate) {
-    asm volatile(
-        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n}\n"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&v)[16]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
-          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]) : "memory");
-}
-__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-        : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// a / b for small a (well below 2^20) with inv_b = 1.0f / b: no integer division in the pipelines' loops
-__device__ __forceinline__ uint32_t small_div(uint32_t a, float inv_b) {
-    return (uint32_t)__float2int_rd(((float)a + 0.5f) * inv_b);
-}
-
-// value rounded to tf32 (10 explicit mantissa bits), ties away from zero in magnitude
-__device__ __forceinline__ float tf32_hi(float a) {
-    return __uint_as_float((__float_as_uint(a) + 0x1000u) & 0xffffe000u);
-}
-
-// K-major operand in the 128-byte swizzled layout: rows of 128 bytes, groups of 8 rows 1024
-// bytes apart (stride-dimension offset), descriptor version 1, swizzle mode 2 (128 B).
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr & 0x3ffffu) >> 4);
-    d |= (uint64_t)1 << 16;                 // leading-dimension offset: unused for swizzled K-major
-    d |= (uint64_t)(1024 >> 4) << 32;       // stride-dimension offset
-    d |= (uint64_t)1 << 46;                 // descriptor version
-    d |= (uint64_t)2 << 61;                 // 128-byte swizzle
-    return d;
-}
 
 // TMEM columns.  Pipeline p's accumulator set holds D1 = a_hi [x_hi; x_lo]^T (2 n_pad columns)
 // and D2 = a_lo x_hi^T (n_pad columns); the A buffers (64 columns each) follow the two sets,
@@ -341,35 +251,35 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     // matrix; pipeline p takes the items with li % kPipes == p.
     if (warp < kPipes) {
         // ------------------------------------------------------------------ TMA producers
-        // Lane w fetches operand w of a stage: the x tile (or the only tile), and in per-model mode
-        // the v tile, so that ONE instruction, at one issue site, requests the whole stage.
+        // The warp stays converged (every lane takes the waits); one elected lane arms the barrier
+        // and issues the stage's copies, at ONE issue site.
         const int p = warp;
-        const int w = lane;
-        constexpr int kOperands = PER_MODEL ? 2 : 1;
-        constexpr uint32_t kLanes = (1u << kOperands) - 1u;
-        if (w < kOperands && p < pipes) {
+        if (p < pipes) {
             uint8_t *ring = stage_base + (size_t)p * n_stages * kStage;
             int s = 0;                                 // stage, and how often the ring has wrapped
             uint32_t round = 0;
             int model, tile;
-            for (int li = p; get_item(li, model, tile) && !*abortp; li += pipes) {
+            for (int li = p;; li += pipes) {
+                if (!__all_sync(0xffffffffu, get_item(li, model, tile) && !*abortp)) break;
                 const int n_loads = (PER_MODEL && model > 0) ? 2 : 1;   // model 0 is x itself: no v tile
-                const bool from_v = PER_MODEL ? w > 0 : model > 0;      // x is a one-model stack
-                const CUtensorMap *map = from_v ? &map_v : &map_x;
-                const int c2 = from_v ? max(model - 1, 0) : 0;
+                const int c2 = max(model - 1, 0);
                 bool ok = true;
                 for (int kb = 0; kb < nkb; ++kb) {
-                    ok = mbar_wait(bar_empty(p, s), (round & 1) ^ 1, abortp);
-                    if (PER_MODEL) ok = __all_sync(kLanes, ok);
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar_empty(p, s), (round & 1) ^ 1, abortp));
                     if (!ok) break;
-                    if (w == 0) {
+                    if (elect_one()) {
+                        const uint32_t dst = smem_u32(ring + s * kStage);
                         mbar_expect_tx(bar_full(p, s), n_loads * kStageBytes);
                         issued[p][s] = (int)round + 1;
+#pragma unroll 1
+                        for (int w = 0; w < n_loads; ++w) {
+                            // first layer: x is a one-model stack, so both operands take the same path
+                            const bool from_v = PER_MODEL ? w > 0 : model > 0;
+                            tma_load_3d(dst + w * kStageBytes, from_v ? &map_v : &map_x, k0 + kb * kBlockK,
+                                        tile * kTileRows, from_v ? c2 : 0, bar_full(p, s));
+                        }
                     }
-                    if (PER_MODEL) __syncwarp(kLanes);
-                    if (w < n_loads)
-                        tma_load_3d(smem_u32(ring + s * kStage) + w * kStageBytes, map, k0 + kb * kBlockK,
-                                    tile * kTileRows, c2, bar_full(p, s));
+                    __syncwarp();
                     if (++s == n_stages) {
                         s = 0;
                         ++round;
@@ -380,8 +290,9 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         }
     } else if (warp < 2 * kPipes) {
         // ------------------------------------------------------------------ MMA issuers
+        // The warp stays converged; one elected lane issues the MMAs and their commits.
         const int p = warp - kPipes;
-        if (lane == 0 && p < pipes) {
+        if (p < pipes) {
             // instruction descriptors: D fp32, A and B tf32, both K-major, M = 128, N = n_pad / 2 n_pad
             const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(a.n_pad >> 3) << 17) |
                                    ((uint32_t)(kTileRows >> 4) << 24);
@@ -390,31 +301,36 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             const int g0 = shared_pipe ? 0 : p * n_abufs;       // first A buffer of this pipeline
             uint32_t it = 0, q = 0;
             int model, tile;
-            for (int li = p; get_item(li, model, tile) && !*abortp; li += pipes, ++q) {
-                if (!mbar_wait(bar_dempty(p), (q & 1) ^ 1, abortp)) break;    // accumulator drained
+            for (int li = p;; li += pipes, ++q) {
+                if (!__all_sync(0xffffffffu, get_item(li, model, tile) && !*abortp)) break;
+                if (!__all_sync(0xffffffffu, mbar_wait(bar_dempty(p), (q & 1) ^ 1, abortp))) break;   // accumulator drained
                 tc_fence_after();
                 bool ok = true;
                 for (int kb = 0; kb < nkb; ++kb, ++it) {
                     const uint32_t around = small_div(it, inv_abufs);          // uses of this A buffer so far
                     const int g = g0 + (int)(it - around * n_abufs_eff);
-                    if (!mbar_wait(bar_afull_g(g), around & 1, abortp)) { ok = false; break; }
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar_afull_g(g), around & 1, abortp));
+                    if (!ok) break;
                     tc_fence_after();
-                    const uint32_t a_tmem = tmem + tl.a_base + g * 64;
-                    const uint32_t bx = smem_u32(xs) + (uint32_t)kb * xkb_bytes;
-                    // A lone pipeline alternates between the two accumulator sets, so that consecutive
-                    // k-blocks do not wait for each other's adds; the epilogue sums the sets.
-                    const uint32_t dset = shared_pipe ? (uint32_t)(kb & 1) * tl.set_stride : 0u;
-                    const uint32_t fresh = shared_pipe ? (uint32_t)(kb >> 1) : (uint32_t)kb;   // 0: first use in the item
+                    if (elect_one()) {
+                        const uint32_t a_tmem = tmem + tl.a_base + g * 64;
+                        const uint32_t bx = smem_u32(xs) + (uint32_t)kb * xkb_bytes;
+                        // A lone pipeline alternates between the two accumulator sets, so that consecutive
+                        // k-blocks do not wait for each other's adds; the epilogue sums the sets.
+                        const uint32_t dset = shared_pipe ? (uint32_t)(kb & 1) * tl.set_stride : 0u;
+                        const uint32_t fresh = shared_pipe ? (uint32_t)(kb >> 1) : (uint32_t)kb;   // 0: first use in the item
 #pragma unroll
-                    for (int ks = 0; ks < kBlockK / 8; ++ks) {
-                        const uint64_t db = smem_desc_sw128(bx + ks * 32);
-                        tc_mma_tf32_ts(d1 + dset, a_tmem + ks * 8, db, idesc2, fresh | ks);         // a_hi [x_hi; x_lo]
-                        tc_mma_tf32_ts(d2 + dset, a_tmem + 32 + ks * 8, db, idesc, fresh | ks);     // a_lo x_hi
+                        for (int ks = 0; ks < kBlockK / 8; ++ks) {
+                            const uint64_t db = smem_desc_sw128(bx + ks * 32);
+                            tc_mma_tf32_ts(d1 + dset, a_tmem + ks * 8, db, idesc2, fresh | ks);         // a_hi [x_hi; x_lo]
+                            tc_mma_tf32_ts(d2 + dset, a_tmem + 32 + ks * 8, db, idesc, fresh | ks);     // a_lo x_hi
+                        }
+                        tc_commit(bar_aempty_g(g));        // the A buffer may be overwritten once these finish
+                        if (kb + 1 == nkb) tc_commit(bar_dfull(p));   // accumulators complete
                     }
-                    tc_commit(bar_aempty_g(g));        // the A buffer may be overwritten once these finish
+                    __syncwarp();
                 }
                 if (!ok) break;
-                tc_commit(bar_dfull(p));               // accumulators complete
             }
         }
     } else if (warp < 2 * kPipes + 4 * kPipes) {
@@ -491,10 +407,8 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 if (!mbar_wait(bar_aempty_g(g), (around & 1) ^ 1, abortp)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t a_tmem = a_bufs + g * 64;
-                tc_st16(a_tmem, reinterpret_cast<const uint32_t(&)[16]>(hi[0]));
-                tc_st16(a_tmem + 16, reinterpret_cast<const uint32_t(&)[16]>(hi[16]));
-                tc_st16(a_tmem + 32, reinterpret_cast<const uint32_t(&)[16]>(lo[0]));
-                tc_st16(a_tmem + 48, reinterpret_cast<const uint32_t(&)[16]>(lo[16]));
+                tc_st32(a_tmem, hi);                  // 32 columns of a_hi, then 32 of a_lo
+                tc_st32(a_tmem + 32, lo);
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
@@ -681,25 +595,6 @@ __global__ void __launch_bounds__(256) stream_combine_kernel(const float *part, 
 }
 
 // ---- host side ----------------------------------------------------------------------------
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
-                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                  CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_tiled_fn() {
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
-}
 
 }  // namespace
 

@@ -205,9 +205,14 @@ zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv,
                                        c->act[l & 1], l + 1 < L, c->np_base[l], s, launches);
             if (e != cudaSuccess) return fail_cuda(c, e);
             if (!plan.fused) {
+                // a following tensor-core layer takes its operand straight from the combine
+                const bool next_tc = layer_tc_serves(l + 1);
                 e = zeno::launch_stream_combine(*c, plan, c->tc_part, xf, Vf, ldv, c->offB[l], out_l, n_r, m,
-                                                gamma, l + 1 < L, c->act[l & 1], s, launches);
+                                                gamma, l + 1 < L, next_tc ? nullptr : c->act[l & 1],
+                                                next_tc ? static_cast<float *>(c->act_split[l & 1]) : nullptr, s,
+                                                launches);
                 if (e != cudaSuccess) return fail_cuda(c, e);
+                have_split = next_tc;
             }
             tail.used.base[l] = c->np_base[l];
             tail.used.count[l] = zeno::stream_tc_norm_slots(plan);
@@ -383,6 +388,7 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
     const size_t at_status = reserve(1, 4), at_tc = reserve(tc_elems, 4);
     const size_t at_tickets = reserve(ticket_elems, 4);
     const size_t at_split0 = reserve(split_elems, 4), at_split1 = reserve(split_elems, 4);
+    const size_t at_losspart = reserve(rows * 8, 4);
 
     e = cudaMalloc(&c->arena, bytes);
     if (e != cudaSuccess) {
@@ -402,6 +408,7 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
     c->dev_status = reinterpret_cast<int *>(base + at_status);
     c->tc_part = reinterpret_cast<float *>(base + at_tc);
     c->tickets = reinterpret_cast<unsigned *>(base + at_tickets);
+    c->loss_part = reinterpret_cast<float *>(base + at_losspart);
     c->act_split[0] = base + at_split0;
     c->act_split[1] = base + at_split1;
     e = cudaMemset(c->dev_status, 0, sizeof(int));

@@ -44,6 +44,7 @@ struct Context {
     int np_slots;                   // norm-partial slots per candidate
     void *arena;                    // the one device allocation everything below is carved from
     float *act[2];                  // activations [m_max+1][n_r_max][widest layer output]
+    float *loss_part;               // [m_max + 1][8] per-block sums of the sample losses
     void *act_split[2];             // two-term stacked activations for the streamed tensor-core layers
     float *normpart;                // [m_max][np_slots] partial sums of v^2
     float *lsq_part;                // [slabs][m_max+1][n_r_max+1] partial A.v and v^2
@@ -161,7 +162,7 @@ cudaError_t launch_stream_tc(Context &c, const StreamTcPlan &p, const float *x, 
                              cudaStream_t s, int *launches);
 cudaError_t launch_stream_combine(Context &c, const StreamTcPlan &p, const float *part, const float *x,
                                   const float *V, int64_t ldv, int64_t offB, int out, int n_r, int m,
-                                  float gamma, int relu, float *H, cudaStream_t s, int *launches);
+                                  float gamma, int relu, float *H, float *Hsplit, cudaStream_t s, int *launches);
 
 // Dense layer on the tensor cores with both operands streamed (any layer of a bfloat16 model, the
 // later layers of an fp32 model).  Its input activations come as the two-term stacked operand

@@ -404,17 +404,20 @@ __global__ void __launch_bounds__(256, 1) mlp_head_kernel(LayerArgs a) {
     if (take_last_ticket(a.tail.ticket, gridDim.x)) finalize_and_select(a.tail, a.losses);
 }
 
-// Per model: mean over the samples of log-sum-exp(z) - z[label].  One block per model, one
-// warp per sample, fixed summation order; the last block to finish runs the tail.
+// Per model: mean over the samples of log-sum-exp(z) - z[label].  G blocks per model (block g takes
+// the samples j = g, g + G, ..), one warp per sample, fixed summation order: the blocks leave their
+// sums in loss_part and the last block to finish adds them up, model by model, before it runs the
+// tail.  G = 1 for small problems: the block writes the model's loss itself.
 __global__ void __launch_bounds__(256) mlp_loss_kernel(const float *logits, const int32_t *labels,
-                                                        int n_r, int classes, float *losses, TailArgs tail) {
+                                                        int n_r, int classes, float *losses, float *loss_part,
+                                                        int G, TailArgs tail) {
     __shared__ float per_warp[8];
     pdl_launch_dependents();
     pdl_wait();
-    const int c = blockIdx.x;
+    const int c = blockIdx.x / G, g = blockIdx.x - c * G;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     float mine = 0.f;
-    for (int j = warp; j < n_r; j += 8) {
+    for (int j = g + warp * G; j < n_r; j += 8 * G) {
         const float *z = logits + ((int64_t)c * n_r + j) * classes;
         float zmax = -INFINITY;
         for (int q = lane; q < classes; q += 32) zmax = fmaxf(zmax, z[q]);
@@ -432,10 +435,22 @@ __global__ void __launch_bounds__(256) mlp_loss_kernel(const float *logits, cons
     if (threadIdx.x == 0) {
         float t = 0.f;
         for (int w = 0; w < 8; ++w) t += per_warp[w];
-        losses[c] = t / (float)n_r;
+        if (G == 1) losses[c] = t / (float)n_r;
+        else loss_part[blockIdx.x] = t;
     }
-    if (c > 0) block_norm_total(tail, c - 1);
-    if (take_last_ticket(tail.ticket, gridDim.x)) finalize_and_select(tail, losses);
+    if (c > 0 && g == 0) block_norm_total(tail, c - 1);
+    if (take_last_ticket(tail.ticket, gridDim.x)) {
+        if (G > 1) {
+            for (int i = threadIdx.x; i <= tail.m; i += blockDim.x) {
+                float t = 0.f;
+                for (int q = 0; q < G; ++q) t += __ldcg(loss_part + i * G + q);
+                losses[i] = t / (float)n_r;
+            }
+            __threadfence();
+            __syncthreads();
+        }
+        finalize_and_select(tail, losses);
+    }
 }
 
 template <typename T, bool VEC>
@@ -500,8 +515,11 @@ cudaError_t launch_mlp_loss(Context &c, const float *logits, const int32_t *labe
                             int *launches) {
     ++*launches;
     profile_mark(c, "mlp_loss_tail", s);
-    return launch_chained(mlp_loss_kernel, dim3(m + 1), dim3(256), 0, s, chain_launches(c), logits, labels, n_r,
-                          classes, losses, tail);
+    // enough blocks to spread a large batch of wide logits over the SMs
+    int G = 1;
+    if ((int64_t)n_r * classes >= 16384) G = n_r >= 64 ? 8 : n_r >= 32 ? 4 : 2;
+    return launch_chained(mlp_loss_kernel, dim3((m + 1) * G), dim3(256), 0, s, chain_launches(c), logits, labels, n_r,
+                          classes, losses, c.loss_part, G, tail);
 }
 
 }  // namespace zeno

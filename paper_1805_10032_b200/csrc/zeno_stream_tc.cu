@@ -529,19 +529,30 @@ template <bool VEC4>
 __global__ void __launch_bounds__(256) stream_combine_kernel(const float *part, int R, int m, int n_r, int out,
                                                              const float *x, const float *V, int64_t ldv,
                                                              int64_t offB, float gamma, int relu, int linear,
-                                                             float *H) {
+                                                             float *H, float *Hsplit, int n_pad) {
     constexpr int E = VEC4 ? 4 : 1;
     pdl_launch_dependents();
     pdl_wait();
+    // H: plain activations [m+1][n_r][out]; Hsplit: the same values as the two-term stacked operand
+    // [m+1][2 n_pad][out] of a following tensor-core layer (tf32 value, then remainder; zero rows for
+    // the padded samples).  Either may be NULL.
     const int og = (out + E - 1) / E;                       // output groups per row
-    const int64_t total = (int64_t)(m + 1) * n_r * og;
+    const int n_rows = Hsplit ? n_pad : n_r;
+    const int64_t total = (int64_t)(m + 1) * n_rows * og;
     const int64_t per_r = (int64_t)(m + 1) * n_r * out;
     for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total;
          t += (int64_t)gridDim.x * blockDim.x) {
         const int o = (int)(t % og) * E;
         const int64_t cj = t / og;
-        const int c = (int)(cj / n_r), j = (int)(cj % n_r);
-        const int64_t ic = cj * out + o;
+        const int c = (int)(cj / n_rows), j = (int)(cj % n_rows);
+        if (j >= n_r) {                                          // padded sample of the stacked operand
+            float *hs = Hsplit + ((int64_t)c * 2 * n_pad + j) * out + o;
+#pragma unroll
+            for (int e = 0; e < E; ++e)
+                if (o + e < out) hs[e] = hs[(int64_t)n_pad * out + e] = 0.f;
+            continue;
+        }
+        const int64_t ic = ((int64_t)c * n_r + j) * out + o;
         const int64_t i0 = linear ? (int64_t)j * out + o : ic;   // model 0 (linear), else the model itself
         const bool two = linear && c > 0;                        // a second set of partials to add
         float z0[E], pc[E], xb[E], vb[E];
@@ -589,7 +600,15 @@ __global__ void __launch_bounds__(256) stream_combine_kernel(const float *part, 
             }
             float z = two ? fmaf(-gamma, pc[e], z0[e]) : z0[e];
             if (relu) z = (z > 0.f || z != z) ? z : 0.f;
-            H[ic + e] = z;
+            if (o + e < out) {
+                if (H) H[ic + e] = z;
+                if (Hsplit) {
+                    float *hs = Hsplit + ((int64_t)c * 2 * n_pad + j) * out + o + e;
+                    const float hi = tf32_hi(z);
+                    hs[0] = hi;
+                    hs[(int64_t)n_pad * out] = z - hi;
+                }
+            }
         }
     }
 }
@@ -749,20 +768,21 @@ cudaError_t launch_stream_tc(Context &c, const StreamTcPlan &p, const float *x, 
 
 cudaError_t launch_stream_combine(Context &c, const StreamTcPlan &p, const float *part, const float *x,
                                   const float *V, int64_t ldv, int64_t offB, int out, int n_r, int m,
-                                  float gamma, int relu, float *H, cudaStream_t s, int *launches) {
+                                  float gamma, int relu, float *H, float *Hsplit, cudaStream_t s, int *launches) {
     const int linear = p.per_model ? 0 : 1;
     ++*launches;
     profile_mark(c, "stream_combine", s);
     const bool vec = out % 4 == 0;
-    const int64_t total = (int64_t)(m + 1) * n_r * (vec ? out / 4 : out);
+    const int n_pad = layer_tc_n_pad(n_r);
+    const int64_t total = (int64_t)(m + 1) * (Hsplit ? n_pad : n_r) * (vec ? out / 4 : out);
     int blocks = (int)((total + 255) / 256);
     const int cap = (c.sm_count > 0 ? c.sm_count : 148) * 16;
     if (blocks > cap) blocks = cap;
     if (vec)
         return launch_chained(stream_combine_kernel<true>, dim3(blocks), dim3(256), 0, s, chain_launches(c), part,
-                              p.R, m, n_r, out, x, V, ldv, offB, gamma, relu, linear, H);
+                              p.R, m, n_r, out, x, V, ldv, offB, gamma, relu, linear, H, Hsplit, n_pad);
     return launch_chained(stream_combine_kernel<false>, dim3(blocks), dim3(256), 0, s, chain_launches(c), part, p.R,
-                          m, n_r, out, x, V, ldv, offB, gamma, relu, linear, H);
+                          m, n_r, out, x, V, ldv, offB, gamma, relu, linear, H, Hsplit, n_pad);
 }
 
 }  // namespace zeno

@@ -151,9 +151,7 @@ zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv,
         if (!zeno::layer_tc_usable((zeno_dtype)c->desc.param_dtype, in_l, out_l, n_r) || n_r > c->n_r_max) return false;
         if ((c->offW[l] * esz0) % 16 != 0) return false;
         if (c->desc.param_dtype == ZENO_BF16) return true;
-        if (l == 0 || in_l < 128 || out_l < 128) return false;
-        zeno::StreamTcPlan plan;          // a layer short enough for the fused stream keeps it
-        return !(c->tc_ok[l] && zeno::stream_tc_plan(c->sm_count, in_l, out_l, n_r, m, true, &plan) && plan.fused);
+        return l > 0 && in_l >= 128 && out_l >= 128;
     };
     bool have_split = false;               // the previous layer left its output in the stacked form
     for (int l = 0; l < L; ++l) {
@@ -193,27 +191,22 @@ zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv,
             continue;
         }
         have_split = false;
-        // fp32 layers on the tcgen05 stream when the shape and the alignment allow it: the first
-        // layer against the shared batch, later layers against each model's own activations
+        // the first layer of an fp32 model on the tcgen05 stream against the shared batch, when the
+        // shape and the alignment allow it
         zeno::StreamTcPlan plan;
-        if (c->tc_ok[l] && aligned && !last_fused &&
-            zeno::stream_tc_plan(c->sm_count, in_l, out_l, n_r, m, l > 0, &plan) && plan.R <= c->tc_r_max[l] &&
-            (l == 0 || plan.fused || getenv("ZENO_TC_ALL_LAYERS"))) {
-            const float *hin = l == 0 ? batch->features : c->act[(l - 1) & 1];
-            e = zeno::launch_stream_tc(*c, plan, xf, Vf, ldv, c->offW[l], c->offB[l], in_l, out_l, hin,
-                                       l == 0 ? 0 : (int64_t)n_r * in_l, gamma, n_r, m, c->tc_part,
-                                       c->act[l & 1], l + 1 < L, c->np_base[l], s, launches);
+        if (l == 0 && c->tc_ok && aligned && !last_fused &&
+            zeno::stream_tc_plan(c->sm_count, in_l, out_l, n_r, m, &plan) && plan.R <= c->tc_r_max) {
+            e = zeno::launch_stream_tc(*c, plan, xf, Vf, ldv, c->offW[l], c->offB[l], in_l, out_l, batch->features,
+                                       n_r, m, c->tc_part, c->np_base[l], s, launches);
             if (e != cudaSuccess) return fail_cuda(c, e);
-            if (!plan.fused) {
-                // a following tensor-core layer takes its operand straight from the combine
-                const bool next_tc = layer_tc_serves(l + 1);
-                e = zeno::launch_stream_combine(*c, plan, c->tc_part, xf, Vf, ldv, c->offB[l], out_l, n_r, m,
-                                                gamma, l + 1 < L, next_tc ? nullptr : c->act[l & 1],
-                                                next_tc ? static_cast<float *>(c->act_split[l & 1]) : nullptr, s,
-                                                launches);
-                if (e != cudaSuccess) return fail_cuda(c, e);
-                have_split = next_tc;
-            }
+            // a following tensor-core layer takes its operand straight from the combine
+            const bool next_tc = layer_tc_serves(l + 1);
+            e = zeno::launch_stream_combine(*c, plan, c->tc_part, xf, Vf, ldv, c->offB[l], out_l, n_r, m, gamma,
+                                            l + 1 < L, next_tc ? nullptr : c->act[l & 1],
+                                            next_tc ? static_cast<float *>(c->act_split[l & 1]) : nullptr, s,
+                                            launches);
+            if (e != cudaSuccess) return fail_cuda(c, e);
+            have_split = next_tc;
             tail.used.base[l] = c->np_base[l];
             tail.used.count[l] = zeno::stream_tc_norm_slots(plan);
             continue;
@@ -336,24 +329,17 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
             if (desc->has_bias) off += o;
             c->np_base[l] = slots;
             int layer_slots = zeno::mlp_norm_slots((int)o);
-            if (desc->param_dtype == ZENO_F32 && !getenv("ZENO_DISABLE_TENSOR_CORES")) {
-                // the tensor-core stream may serve this layer: size its partials for the shortest
-                // k-range any plan may pick
+            if (l == 0 && desc->param_dtype == ZENO_F32 && !getenv("ZENO_DISABLE_TENSOR_CORES")) {
+                // the tensor-core stream may serve the first layer: size its partials and norm slots
+                // for the shortest k-range any plan may pick
                 zeno::StreamTcPlan probe;
-                if (zeno::stream_tc_plan(c->sm_count, (int)in, (int)o, n_r_max < 64 ? n_r_max : 64, m_max, l > 0,
-                                         &probe)) {
-                    c->tc_ok[l] = true;
-                    c->tc_r_max[l] = (int)((in + zeno::kStreamTcMinKR - 1) / zeno::kStreamTcMinKR);
-                    // the most slots any plan may use: the shortest k-ranges, or one k-range on a
-                    // pipeline that both converter sets share
-                    probe.R = c->tc_r_max[l];
-                    probe.pipes = 2;
-                    int tc_slots = zeno::stream_tc_norm_slots(probe);
-                    probe.R = 1;
-                    probe.pipes = 1;
-                    if (zeno::stream_tc_norm_slots(probe) > tc_slots) tc_slots = zeno::stream_tc_norm_slots(probe);
+                if (zeno::stream_tc_plan(c->sm_count, (int)in, (int)o, n_r_max < 64 ? n_r_max : 64, m_max, &probe)) {
+                    c->tc_ok = true;
+                    c->tc_r_max = (int)((in + zeno::kStreamTcMinKR - 1) / zeno::kStreamTcMinKR);
+                    probe.R = c->tc_r_max;
+                    const int tc_slots = zeno::stream_tc_norm_slots(probe);
                     if (tc_slots > layer_slots) layer_slots = tc_slots;
-                    const size_t need = (size_t)c->tc_r_max[l] * rows * (size_t)n_r_max * (size_t)o;
+                    const size_t need = (size_t)c->tc_r_max * rows * (size_t)n_r_max * (size_t)o;
                     if (need > tc_elems) tc_elems = need;
                 }
             }

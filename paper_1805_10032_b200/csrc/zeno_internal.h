@@ -21,12 +21,8 @@ constexpr int kMaxProfiled = ZENO_MAX_LAYERS + 8;
 constexpr int kProfileDepth = 64;
 
 // Launch shape of the tensor-core stream: k-range length, number of k-ranges, blocks per
-// k-range, padded sample count, 128-row tiles per model, dynamic shared memory, pipelines in use
-// per block (1 or 2), and whether the block finishes the layer itself (one k-range: bias and
-// activation in the epilogue, no split-K partials).
-struct StreamTcPlan {
-    int KR, R, G, n_pad, tiles_per_model, smem_bytes, stages, tile_groups, per_model, pipes, fused;
-};
+// k-range, padded sample count, 128-row tiles per model, dynamic shared memory, ring depth.
+struct StreamTcPlan { int KR, R, G, n_pad, tiles_per_model, smem_bytes, stages; };
 constexpr int kStreamTcMinKR = 128;
 
 // Which norm-partial slots a call filled: per layer (first slot, count).
@@ -54,8 +50,8 @@ struct Context {
     float *scores;                  // [m_max]
     int32_t *idx;                   // [m_max]
     int *dev_status;                // raised by a kernel whose bounded wait gave up
-    bool tc_ok[ZENO_MAX_LAYERS];    // the tensor-core stream can serve this layer (fp32 storage)
-    int tc_r_max[ZENO_MAX_LAYERS];  // most k-ranges any plan for the layer may use
+    bool tc_ok;                     // the tensor-core stream can serve the first layer (fp32 storage)
+    int tc_r_max;                   // most k-ranges any plan for it may use
     float *tc_part;                 // [R][m_max+1][n_r_max][dims[1]] split-K partials
     unsigned *tickets;              // the tail's arrival counter, zero between launches
     void *host_stage;               // device copies of host inputs (zeno_step_host), grown on demand
@@ -154,12 +150,11 @@ cudaError_t launch_aggregate(Context &c, const void *V, int64_t ldv, int m,
                              int *launches);
 
 // Tensor-core stream for the first layer (fp32 storage).
-bool stream_tc_plan(int sms, int K, int out, int n_r, int m, bool per_model, StreamTcPlan *p);
+bool stream_tc_plan(int sms, int K, int out, int n_r, int m, StreamTcPlan *p);
 int stream_tc_norm_slots(const StreamTcPlan &p);
 cudaError_t launch_stream_tc(Context &c, const StreamTcPlan &p, const float *x, const float *V, int64_t ldv,
-                             int64_t offW, int64_t offB, int K, int out, const float *X, int64_t x_model_stride,
-                             float gamma, int n_r, int m, float *part, float *Hout, int relu, int np_base,
-                             cudaStream_t s, int *launches);
+                             int64_t offW, int64_t offB, int K, int out, const float *X, int n_r, int m,
+                             float *part, int np_base, cudaStream_t s, int *launches);
 cudaError_t launch_stream_combine(Context &c, const StreamTcPlan &p, const float *part, const float *x,
                                   const float *V, int64_t ldv, int64_t offB, int out, int n_r, int m,
                                   float gamma, int relu, float *H, float *Hsplit, cudaStream_t s, int *launches);

@@ -8,9 +8,8 @@
 //
 // fp32 accuracy on tf32 tensor cores: both operands are split, a = a_hi + a_lo with a_hi the
 // value rounded to tf32, and the product is accumulated as a_hi b_hi + a_lo b_hi + a_hi b_lo
-// (the dropped a_lo b_lo term is below 2^-22 relative).  At these small N the MMA is bound by
-// fetching its A operand, so X_hi and X_lo are stacked along N: one MMA reads a_hi once and
-// yields a_hi x_hi and a_hi x_lo side by side; a second one adds a_lo x_hi.
+// (the dropped a_lo b_lo term is below 2^-22 relative).  X_hi and X_lo are stacked along N: one
+// MMA reads a_hi once and yields a_hi x_hi and a_hi x_lo side by side; a second one adds a_lo x_hi.
 //
 // The tensor core adds into its fp32 accumulator with truncation, so a long accumulation chain
 // drifts; the two small products go to an accumulator of their own (their truncation error is
@@ -18,22 +17,21 @@
 //
 // Per block (one SM): a k-range of the input index, whose X_hi / X_lo slices stay resident in
 // shared memory in the 128-byte-swizzled K-major layout the MMA reads, and a list of 128-row
-// tiles of the stacked matrix.  These MMAs are small (N = n_r), so one issuing thread cannot keep
-// the tensor pipe busy: its waits and commits would leave the pipe idle half of the time.  The
-// block therefore runs TWO independent pipelines side by side, each on its own row tiles, with
-// its own TMA ring, converter warps, MMA issuer, TMEM operand buffers and accumulator; the
-// tensor pipe interleaves their MMAs.  Warp roles (p = pipeline 0 / 1):
+// tiles of the stacked matrix.  The block runs TWO independent pipelines side by side, each on
+// its own row tiles, with its own TMA ring, converter warps, MMA issuer, TMEM operand buffers and
+// accumulator, so that one pipeline's waits are covered by the other's work.  Warp roles
+// (p = pipeline 0 / 1):
 //   warp p        TMA producer: 128 rows x 32 floats boxes of V (or x) into pipeline p's ring
 //   warp 2+p      MMA issuer (tcgen05.mma, A operand from TMEM, B from shared); warp 2 owns TMEM
 //   warps 4-7 / 8-11   converters of pipeline 0 / 1: thread t owns row t of the tile; reads its
 //                 128 bytes from the stage, accumulates v^2, splits into hi/lo and stores both
 //                 to TMEM (tcgen05.st) where the MMA picks them up
 //   warps 12-15   epilogue: drain finished accumulators (tcgen05.ld) into the split-K partial
-//                 output while both pipelines keep going.  The block that delivers the last
-//                 of a tile's R partials (a ticket per tile, no waiting) adds them up in
-//                 k-range order, so the sums do not depend on which block that is.
-// Every mbarrier wait is bounded; a wait that gives up raises a status word and the block leaves
-// through the common teardown (pending bulk copies awaited, TMEM freed).
+//                 output while both pipelines keep going; stream_combine_kernel adds the partials
+//                 in k-range order.
+// Producer and issuer warps stay converged and issue from one elected lane.  Every mbarrier wait
+// is bounded; a wait that gives up raises a status word and the block leaves through the common
+// teardown (pending bulk copies awaited, TMEM freed).
 #include <cuda.h>
 
 #include "zeno_internal.h"
@@ -67,10 +65,7 @@ struct TmemLayout {
 };
 
 struct StreamArgs {
-    const float *X;        // [n_r x K] the server batch, or the models' activations [m+1][n_r][K]
-    int64_t x_model_stride;   // 0 when every model shares X (first layer)
-    int tile_groups;       // per-model mode: blocks per model along y (each takes every tile_groups-th tile)
-    float gamma;           // per-model mode: A = x - gamma v is formed here
+    const float *X;        // [n_r x K] the server batch
     const float *V;        // for the bias entries' v^2
     int64_t ldv;
     int64_t offB;          // element offset of this layer's bias inside a row of V, -1 if none
@@ -81,27 +76,16 @@ struct StreamArgs {
     int KR;                // floats of K per k-range (multiple of 32)
     int tiles_per_model;   // ceil(out / 128)
     int stages;            // depth of each pipeline's TMA ring (<= kMaxStages)
-    int pipes;             // pipelines in use (1 or 2); a block with one item at a time needs only one
-    int fused;             // one k-range: the epilogue adds the bias, activates and writes Hout
-    int early_loads;       // x and V were complete before the preceding kernel started: the
-                           // producers need not wait for it
-    const float *xparams;  // the parameter vector x (bias entries, fused epilogue)
-    float *Hout;           // [m+1][n_r][out] activations (fused epilogue)
-    int relu;
     int *status;           // device status word (raised on a wait that gave up)
 };
 
-// PER_MODEL = false: the first layer.  B = the shared batch, A = raw rows of [x; V] (the layer is
-//   linear in its weights, the caller combines X W^T - gamma X V^T), a block's items are row tiles
-//   blockIdx.y, blockIdx.y + gridDim.y, .. of the stacked matrix.
-// PER_MODEL = true: a later layer.  B = model c's own activations, A = x - gamma v formed by the
-//   converters from an x tile and a v tile that arrive together in one stage; a block belongs to
-//   one model and takes every tile_groups-th row tile of it.
-template <bool PER_MODEL>
+// B = the shared batch, A = raw rows of [x; V] (the layer is linear in its weights, the combine
+// kernel forms X W^T - gamma X V^T); a block's items are row tiles blockIdx.y, blockIdx.y +
+// gridDim.y, .. of the stacked matrix.
 __global__ void __launch_bounds__(kThreads, 1)
 stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_v,
                      StreamArgs a) {
-    constexpr int kStage = PER_MODEL ? 2 * kStageBytes : kStageBytes;   // x tile then v tile, or one tile
+    constexpr int kStage = kStageBytes;
     pdl_launch_dependents();
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     // per pipeline: full[kMaxStages], empty[kMaxStages], a_full[kMaxABufs], a_empty[kMaxABufs], d_full, d_empty
@@ -122,19 +106,14 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     const int n_items_total = (a.m + 1) * a.tiles_per_model;
     // item li of this block -> (model, tile); false when the block has no such item
     auto get_item = [&](int li, int &model, int &tile) {
-        if (PER_MODEL) {
-            model = blockIdx.y / a.tile_groups;
-            tile = blockIdx.y % a.tile_groups + li * a.tile_groups;
-            return tile < a.tiles_per_model;
-        }
         const int item = blockIdx.y + li * gridDim.y;
         model = item / a.tiles_per_model;
         tile = item % a.tiles_per_model;
         return item < n_items_total;
     };
-    const float *Xsrc = a.X + (PER_MODEL ? (int64_t)(blockIdx.y / a.tile_groups) * a.x_model_stride : 0);
+    const float *Xsrc = a.X;
     const int n_stages = a.stages;
-    const int pipes = a.pipes;
+    constexpr int pipes = kPipes;
 
     // shared memory carve-up (dynamic part is 1024-byte aligned)
     uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -144,20 +123,12 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     uint8_t *stage_base = base + (uint32_t)nkb_max * xkb_bytes;   // pipeline p's ring at p * n_stages * kStage
     const TmemLayout tl(a.n_pad);
     const int n_abufs = tl.n_abufs;
-    // With one pipeline in use, it cycles through all the A buffers, and both converter sets feed
-    // it, taking alternate k-blocks (conversion, not the MMAs, bounds a lone pipeline).
-    const bool shared_pipe = pipes == 1;
-    const int n_abufs_eff = shared_pipe ? kPipes * n_abufs : n_abufs;
-    const float inv_stages = 1.0f / (float)n_stages, inv_abufs = 1.0f / (float)n_abufs_eff;
+    const float inv_stages = 1.0f / (float)n_stages, inv_abufs = 1.0f / (float)n_abufs;
 
     auto bar_full = [&](int p, int s) { return smem_u32(&bars[p * kBarsPerPipe + s]); };
     auto bar_empty = [&](int p, int s) { return smem_u32(&bars[p * kBarsPerPipe + kMaxStages + s]); };
     auto bar_afull = [&](int p, int b) { return smem_u32(&bars[p * kBarsPerPipe + 2 * kMaxStages + b]); };
     auto bar_aempty = [&](int p, int b) { return smem_u32(&bars[p * kBarsPerPipe + 2 * kMaxStages + kMaxABufs + b]); };
-    // A buffer g of the block (pipeline p's buffers are g = p * n_abufs ..): barrier of its owner
-    const int ab_shift = n_abufs > 1 ? 1 : 0;           // n_abufs is 1 or 2
-    auto bar_afull_g = [&](int g) { return bar_afull(g >> ab_shift, g & (n_abufs - 1)); };
-    auto bar_aempty_g = [&](int g) { return bar_aempty(g >> ab_shift, g & (n_abufs - 1)); };
     auto bar_dfull = [&](int p) { return smem_u32(&bars[p * kBarsPerPipe + 2 * kMaxStages + 2 * kMaxABufs]); };
     auto bar_dempty = [&](int p) { return smem_u32(&bars[p * kBarsPerPipe + 2 * kMaxStages + 2 * kMaxABufs + 1]); };
 
@@ -186,10 +157,7 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     tc_fence_before();
     __syncthreads();                                   // barriers and the TMEM base are visible
     tc_fence_after();
-    // On-chip set-up done; global memory from here on.  The weights are inputs of the whole call,
-    // so in a later kernel of the chain the producers may fetch them while the preceding kernel
-    // still runs; everything else (activations, partials, norm slots) waits for it.
-    if (!(a.early_loads && warp < kPipes)) pdl_wait();
+    pdl_wait();                                        // on-chip set-up done; global memory from here on
     const uint32_t tmem = tmem_base_slot;
     volatile int *abortp = &abort_flag;
 
@@ -254,165 +222,117 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         // The warp stays converged (every lane takes the waits); one elected lane arms the barrier
         // and issues the stage's copies, at ONE issue site.
         const int p = warp;
-        if (p < pipes) {
-            uint8_t *ring = stage_base + (size_t)p * n_stages * kStage;
-            int s = 0;                                 // stage, and how often the ring has wrapped
-            uint32_t round = 0;
-            int model, tile;
-            for (int li = p;; li += pipes) {
-                if (!__all_sync(0xffffffffu, get_item(li, model, tile) && !*abortp)) break;
-                const int n_loads = (PER_MODEL && model > 0) ? 2 : 1;   // model 0 is x itself: no v tile
-                const int c2 = max(model - 1, 0);
-                bool ok = true;
-                for (int kb = 0; kb < nkb; ++kb) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(bar_empty(p, s), (round & 1) ^ 1, abortp));
-                    if (!ok) break;
-                    if (elect_one()) {
-                        const uint32_t dst = smem_u32(ring + s * kStage);
-                        mbar_expect_tx(bar_full(p, s), n_loads * kStageBytes);
-                        issued[p][s] = (int)round + 1;
-#pragma unroll 1
-                        for (int w = 0; w < n_loads; ++w) {
-                            // first layer: x is a one-model stack, so both operands take the same path
-                            const bool from_v = PER_MODEL ? w > 0 : model > 0;
-                            tma_load_3d(dst + w * kStageBytes, from_v ? &map_v : &map_x, k0 + kb * kBlockK,
-                                        tile * kTileRows, from_v ? c2 : 0, bar_full(p, s));
-                        }
-                    }
-                    __syncwarp();
-                    if (++s == n_stages) {
-                        s = 0;
-                        ++round;
-                    }
-                }
+        uint8_t *ring = stage_base + (size_t)p * n_stages * kStage;
+        int s = 0;                                 // stage, and how often the ring has wrapped
+        uint32_t round = 0;
+        int model, tile;
+        for (int li = p;; li += pipes) {
+            if (!__all_sync(0xffffffffu, get_item(li, model, tile) && !*abortp)) break;
+            // x is a one-model stack, so both operands take the same path
+            const CUtensorMap *map = model > 0 ? &map_v : &map_x;
+            const int c2 = max(model - 1, 0);
+            bool ok = true;
+            for (int kb = 0; kb < nkb; ++kb) {
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_empty(p, s), (round & 1) ^ 1, abortp));
                 if (!ok) break;
+                if (elect_one()) {
+                    mbar_expect_tx(bar_full(p, s), kStageBytes);
+                    issued[p][s] = (int)round + 1;
+                    tma_load_3d(smem_u32(ring + s * kStage), map, k0 + kb * kBlockK, tile * kTileRows, c2,
+                                bar_full(p, s));
+                }
+                __syncwarp();
+                if (++s == n_stages) {
+                    s = 0;
+                    ++round;
+                }
             }
+            if (!ok) break;
         }
     } else if (warp < 2 * kPipes) {
         // ------------------------------------------------------------------ MMA issuers
         // The warp stays converged; one elected lane issues the MMAs and their commits.
         const int p = warp - kPipes;
-        if (p < pipes) {
-            // instruction descriptors: D fp32, A and B tf32, both K-major, M = 128, N = n_pad / 2 n_pad
-            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(a.n_pad >> 3) << 17) |
-                                   ((uint32_t)(kTileRows >> 4) << 24);
-            const uint32_t idesc2 = (idesc & ~(0x3fu << 17)) | ((uint32_t)((2 * a.n_pad) >> 3) << 17);
-            const uint32_t d1 = tmem + p * tl.set_stride, d2 = d1 + tl.d2_off;
-            const int g0 = shared_pipe ? 0 : p * n_abufs;       // first A buffer of this pipeline
-            uint32_t it = 0, q = 0;
-            int model, tile;
-            for (int li = p;; li += pipes, ++q) {
-                if (!__all_sync(0xffffffffu, get_item(li, model, tile) && !*abortp)) break;
-                if (!__all_sync(0xffffffffu, mbar_wait(bar_dempty(p), (q & 1) ^ 1, abortp))) break;   // accumulator drained
-                tc_fence_after();
-                bool ok = true;
-                for (int kb = 0; kb < nkb; ++kb, ++it) {
-                    const uint32_t around = small_div(it, inv_abufs);          // uses of this A buffer so far
-                    const int g = g0 + (int)(it - around * n_abufs_eff);
-                    ok = __all_sync(0xffffffffu, mbar_wait(bar_afull_g(g), around & 1, abortp));
-                    if (!ok) break;
-                    tc_fence_after();
-                    if (elect_one()) {
-                        const uint32_t a_tmem = tmem + tl.a_base + g * 64;
-                        const uint32_t bx = smem_u32(xs) + (uint32_t)kb * xkb_bytes;
-                        // A lone pipeline alternates between the two accumulator sets, so that consecutive
-                        // k-blocks do not wait for each other's adds; the epilogue sums the sets.
-                        const uint32_t dset = shared_pipe ? (uint32_t)(kb & 1) * tl.set_stride : 0u;
-                        const uint32_t fresh = shared_pipe ? (uint32_t)(kb >> 1) : (uint32_t)kb;   // 0: first use in the item
-#pragma unroll
-                        for (int ks = 0; ks < kBlockK / 8; ++ks) {
-                            const uint64_t db = smem_desc_sw128(bx + ks * 32);
-                            tc_mma_tf32_ts(d1 + dset, a_tmem + ks * 8, db, idesc2, fresh | ks);         // a_hi [x_hi; x_lo]
-                            tc_mma_tf32_ts(d2 + dset, a_tmem + 32 + ks * 8, db, idesc, fresh | ks);     // a_lo x_hi
-                        }
-                        tc_commit(bar_aempty_g(g));        // the A buffer may be overwritten once these finish
-                        if (kb + 1 == nkb) tc_commit(bar_dfull(p));   // accumulators complete
-                    }
-                    __syncwarp();
-                }
+        // instruction descriptors: D fp32, A and B tf32, both K-major, M = 128, N = n_pad / 2 n_pad
+        const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(a.n_pad >> 3) << 17) |
+                               ((uint32_t)(kTileRows >> 4) << 24);
+        const uint32_t idesc2 = (idesc & ~(0x3fu << 17)) | ((uint32_t)((2 * a.n_pad) >> 3) << 17);
+        const uint32_t d1 = tmem + p * tl.set_stride, d2 = d1 + tl.d2_off;
+        uint32_t it = 0, q = 0;
+        int model, tile;
+        for (int li = p;; li += pipes, ++q) {
+            if (!__all_sync(0xffffffffu, get_item(li, model, tile) && !*abortp)) break;
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_dempty(p), (q & 1) ^ 1, abortp))) break;   // accumulator drained
+            tc_fence_after();
+            bool ok = true;
+            for (int kb = 0; kb < nkb; ++kb, ++it) {
+                const uint32_t around = small_div(it, inv_abufs);          // uses of this A buffer so far
+                const int ab = (int)(it - around * n_abufs);
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_afull(p, ab), around & 1, abortp));
                 if (!ok) break;
+                tc_fence_after();
+                if (elect_one()) {
+                    const uint32_t a_tmem = tmem + tl.a_base + (p * n_abufs + ab) * 64;
+                    const uint32_t bx = smem_u32(xs) + (uint32_t)kb * xkb_bytes;
+#pragma unroll
+                    for (int ks = 0; ks < kBlockK / 8; ++ks) {
+                        const uint64_t db = smem_desc_sw128(bx + ks * 32);
+                        tc_mma_tf32_ts(d1, a_tmem + ks * 8, db, idesc2, (uint32_t)(kb | ks));        // a_hi [x_hi; x_lo]
+                        tc_mma_tf32_ts(d2, a_tmem + 32 + ks * 8, db, idesc, (uint32_t)(kb | ks));    // a_lo x_hi
+                    }
+                    tc_commit(bar_aempty(p, ab));          // the A buffer may be overwritten once these finish
+                    if (kb + 1 == nkb) tc_commit(bar_dfull(p));   // accumulators complete
+                }
+                __syncwarp();
             }
+            if (!ok) break;
         }
     } else if (warp < 2 * kPipes + 4 * kPipes) {
         // ------------------------------------------------------------------ converters
-        const int cset = (warp - 2 * kPipes) >> 2;    // converter set
-        const int p = shared_pipe ? 0 : cset;
-        const int kstep = shared_pipe ? kPipes : 1;
-        const int g0 = shared_pipe ? 0 : p * n_abufs;
+        const int p = (warp - 2 * kPipes) >> 2;
         const int quad = warp & 3;                    // TMEM lane quadrant this warp may access
         const int row = quad * 32 + lane;             // row of the tile = TMEM lane
         const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
         const uint8_t *ring = stage_base + (size_t)p * n_stages * kStage;
-        const uint32_t a_bufs = tmem + lane_addr + tl.a_base;
-        uint32_t it0 = 0;                             // k-blocks of this pipeline before the item
+        const uint32_t a_bufs = tmem + lane_addr + tl.a_base + p * n_abufs * 64;
+        uint32_t it = 0;
         int model, tile;
-        for (int li = p; get_item(li, model, tile) && !*abortp; li += pipes, it0 += nkb) {
+        for (int li = p; get_item(li, model, tile) && !*abortp; li += pipes) {
             float nrm4[4] = {0.f, 0.f, 0.f, 0.f};
             bool ok = true;
-            for (int kb = shared_pipe ? (int)((cset - it0) & 1u) : 0; kb < nkb; kb += kstep) {
-                const uint32_t it = it0 + kb;
+            for (int kb = 0; kb < nkb; ++kb, ++it) {
                 const uint32_t sround = small_div(it, inv_stages);
                 const int s = (int)(it - sround * n_stages);
                 if (!mbar_wait(bar_full(p, s), sround & 1, abortp)) { ok = false; break; }
                 const uint8_t *src = ring + s * kStage + row * 128;
                 float4 v[8];
                 uint32_t hi[32], lo[32];
-                if (PER_MODEL) {
-                    // stage = x tile then v tile: the candidate's weights are formed here
-                    float4 xv[8];
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) xv[c] = *reinterpret_cast<const float4 *>(src + ((c ^ (row & 7)) << 4));
-                    if (model > 0) {
+                for (int c = 0; c < 8; ++c) v[c] = *reinterpret_cast<const float4 *>(src + ((c ^ (row & 7)) << 4));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_empty(p, s));    // the stage may be refilled
 #pragma unroll
-                        for (int c = 0; c < 8; ++c)
-                            v[c] = *reinterpret_cast<const float4 *>(src + kStageBytes + ((c ^ (row & 7)) << 4));
-                    } else {
+                for (int c = 0; c < 8; ++c) {
+                    const float e[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
 #pragma unroll
-                        for (int c = 0; c < 8; ++c) v[c] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_empty(p, s));    // the stage may be refilled
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        const float ev[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
-                        const float ex[4] = {xv[c].x, xv[c].y, xv[c].z, xv[c].w};
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            nrm4[u] = fmaf(ev[u], ev[u], nrm4[u]);
-                            const float w = fmaf(-a.gamma, ev[u], ex[u]);
-                            const float h = tf32_hi(w);
-                            hi[4 * c + u] = __float_as_uint(h);
-                            lo[4 * c + u] = __float_as_uint(w - h);
-                        }
-                    }
-                } else {
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) v[c] = *reinterpret_cast<const float4 *>(src + ((c ^ (row & 7)) << 4));
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_empty(p, s));    // the stage may be refilled
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        const float e[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            nrm4[u] = fmaf(e[u], e[u], nrm4[u]);
-                            const float h = tf32_hi(e[u]);
-                            hi[4 * c + u] = __float_as_uint(h);
-                            lo[4 * c + u] = __float_as_uint(e[u] - h);
-                        }
+                    for (int u = 0; u < 4; ++u) {
+                        nrm4[u] = fmaf(e[u], e[u], nrm4[u]);
+                        const float h = tf32_hi(e[u]);
+                        hi[4 * c + u] = __float_as_uint(h);
+                        lo[4 * c + u] = __float_as_uint(e[u] - h);
                     }
                 }
                 const uint32_t around = small_div(it, inv_abufs);
-                const int g = g0 + (int)(it - around * n_abufs_eff);
-                if (!mbar_wait(bar_aempty_g(g), (around & 1) ^ 1, abortp)) { ok = false; break; }
+                const int ab = (int)(it - around * n_abufs);
+                if (!mbar_wait(bar_aempty(p, ab), (around & 1) ^ 1, abortp)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t a_tmem = a_bufs + g * 64;
+                const uint32_t a_tmem = a_bufs + ab * 64;
                 tc_st32(a_tmem, hi);                  // 32 columns of a_hi, then 32 of a_lo
                 tc_st32(a_tmem + 32, lo);
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar_afull_g(g));
+                if (lane == 0) mbar_arrive(bar_afull(p, ab));
             }
             if (!ok) break;
 
@@ -420,7 +340,7 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             if (model > 0) {
                 float nrm = (nrm4[0] + nrm4[1]) + (nrm4[2] + nrm4[3]);
                 const int o = tile * kTileRows + row;
-                if (r == 0 && a.offB >= 0 && o < a.out && (!shared_pipe || cset == 0)) {
+                if (r == 0 && a.offB >= 0 && o < a.out) {
                     const float bv = __ldg(a.V + (int64_t)(model - 1) * a.ldv + a.offB + o);
                     nrm = fmaf(bv, bv, nrm);
                 }
@@ -428,8 +348,7 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 for (int sft = 16; sft >= 1; sft >>= 1) nrm += __shfl_xor_sync(0xffffffffu, nrm, sft);
                 if (lane == 0)
                     a.normpart[(int64_t)(model - 1) * a.np_slots + a.np_base +
-                               ((r * a.tiles_per_model + tile) * 4 + quad) * (shared_pipe ? kPipes : 1) +
-                               (shared_pipe ? cset : 0)] = nrm;
+                               (r * a.tiles_per_model + tile) * 4 + quad] = nrm;
             }
         }
     } else {
@@ -443,53 +362,27 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             const uint32_t q = li / pipes;                // how many accumulators pipeline p has finished before
             // thread = output row o, column = sample j
             const int o = tile * kTileRows + row;
-            float bias = 0.f;
-            if (a.fused && a.offB >= 0 && o < a.out) {      // asked for before the accumulator is awaited
-                const float vb = model > 0 ? __ldg(a.V + (int64_t)(model - 1) * a.ldv + a.offB + o) : 0.f;
-                bias = fmaf(-a.gamma, vb, __ldg(a.xparams + a.offB + o));
-            }
             if (!mbar_wait(bar_dfull(p), q & 1, abortp)) break;
             tc_fence_after();
             float *dst = a.part + (((int64_t)r * (a.m + 1) + model) * a.n_r) * a.out + o;
             const uint32_t dset = tmem + lane_addr + p * tl.set_stride;
             for (int j0 = 0; j0 < a.n_pad; j0 += 16) {
                 uint32_t big[16], s1[16], s2[16];
-                float acc[16];
                 tc_ld16(dset + j0, big);                       // a_hi x_hi
                 tc_ld16(dset + a.n_pad + j0, s1);              // a_hi x_lo
                 tc_ld16(dset + tl.d2_off + j0, s2);            // a_lo x_hi
                 tc_wait_ld();
-#pragma unroll
-                for (int j = 0; j < 16; ++j)
-                    acc[j] = __uint_as_float(big[j]) + (__uint_as_float(s1[j]) + __uint_as_float(s2[j]));
-                if (shared_pipe && nkb > 1) {                  // the odd k-blocks went to the second set
-                    tc_ld16(dset + tl.set_stride + j0, big);
-                    tc_ld16(dset + tl.set_stride + a.n_pad + j0, s1);
-                    tc_ld16(dset + tl.set_stride + tl.d2_off + j0, s2);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int j = 0; j < 16; ++j)
-                        acc[j] += __uint_as_float(big[j]) + (__uint_as_float(s1[j]) + __uint_as_float(s2[j]));
-                }
                 if (j0 + 16 >= a.n_pad) {                      // everything is in registers: release the accumulator
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_dempty(p));
                 }
-                if (o < a.out && !a.fused) {
+                if (o < a.out) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
                         if (j0 + j < a.n_r)
-                            dst[(int64_t)(j0 + j) * a.out] = acc[j];
-                } else if (o < a.out) {
-                    float *h = a.Hout + (int64_t)model * a.n_r * a.out + o;
-#pragma unroll
-                    for (int j = 0; j < 16; ++j)
-                        if (j0 + j < a.n_r) {
-                            float z = acc[j] + bias;
-                            if (a.relu) z = (z > 0.f || z != z) ? z : 0.f;
-                            h[(int64_t)(j0 + j) * a.out] = z;
-                        }
+                            dst[(int64_t)(j0 + j) * a.out] =
+                                __uint_as_float(big[j]) + (__uint_as_float(s1[j]) + __uint_as_float(s2[j]));
                 }
             }
         }
@@ -523,12 +416,10 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
 //   z_0 = sum_r P[r][0] + b(x),   z_c = z_0 - gamma (sum_r P[r][c] + b(v_c)),   h = ReLU(z)
 // One thread per (model, sample, four outputs); the 2R loads of a thread are independent and
 // the partials are added in k-range order.
-// With linear = 0 (a layer whose products were already taken with x - gamma v) only the model's own
-// partials and its bias x_b - gamma v_b are added.
 template <bool VEC4>
 __global__ void __launch_bounds__(256) stream_combine_kernel(const float *part, int R, int m, int n_r, int out,
                                                              const float *x, const float *V, int64_t ldv,
-                                                             int64_t offB, float gamma, int relu, int linear,
+                                                             int64_t offB, float gamma, int relu,
                                                              float *H, float *Hsplit, int n_pad) {
     constexpr int E = VEC4 ? 4 : 1;
     pdl_launch_dependents();
@@ -553,8 +444,8 @@ __global__ void __launch_bounds__(256) stream_combine_kernel(const float *part, 
             continue;
         }
         const int64_t ic = ((int64_t)c * n_r + j) * out + o;
-        const int64_t i0 = linear ? (int64_t)j * out + o : ic;   // model 0 (linear), else the model itself
-        const bool two = linear && c > 0;                        // a second set of partials to add
+        const int64_t i0 = (int64_t)j * out + o;                 // the same entry of model 0
+        const bool two = c > 0;                                  // a candidate: a second set of partials to add
         float z0[E], pc[E], xb[E], vb[E];
 #pragma unroll
         for (int e = 0; e < E; ++e) {
@@ -591,12 +482,8 @@ __global__ void __launch_bounds__(256) stream_combine_kernel(const float *part, 
 #pragma unroll
         for (int e = 0; e < E; ++e) {
             if (offB >= 0 && o + e < out) {
-                if (linear) {
-                    z0[e] += xb[e];
-                    pc[e] += vb[e];
-                } else {
-                    z0[e] += fmaf(-gamma, vb[e], xb[e]);
-                }
+                z0[e] += xb[e];
+                pc[e] += vb[e];
             }
             float z = two ? fmaf(-gamma, pc[e], z0[e]) : z0[e];
             if (relu) z = (z > 0.f || z != z) ? z : 0.f;
@@ -622,80 +509,49 @@ __global__ void __launch_bounds__(256) stream_combine_kernel(const float *part, 
 // Cost model, in units of the time one k-block takes: the block that finishes last runs
 // ceil(items / 2) row tiles on its busier pipeline, nkb k-blocks each, plus a fixed start-up
 // and drain; every extra k-range adds split-K partials that have to be written and summed.
-bool stream_tc_plan(int sms, int K, int out, int n_r, int m, bool per_model, StreamTcPlan *p) {
-    if (n_r < 1 || n_r > 64 || K < (per_model ? 128 : 256) || K % 4 != 0 || out < 64) return false;
+bool stream_tc_plan(int sms, int K, int out, int n_r, int m, StreamTcPlan *p) {
+    if (n_r < 1 || n_r > 64 || K < 256 || K % 4 != 0 || out < 64) return false;
     const int n_pad = (n_r + 15) / 16 * 16;
     const int tiles = (out + kTileRows - 1) / kTileRows;
-    const int stage_bytes = per_model ? 2 * kStageBytes : kStageBytes;
     const int items_all = (m + 1) * tiles;
-    p->pipes = kPipes;
-    p->fused = 0;
-    if (per_model) {
-        // The whole input range in one block: no split-K partials, bias and activation in the
-        // epilogue.  One row tile per block, so one pipeline, which leaves its ring the room the
-        // resident activations [X_hi; X_lo] do not take.
-        const int kr = (K + kBlockK - 1) / kBlockK * kBlockK;
-        const int xs = 2 * (kr / kBlockK) * n_pad * 128;
-        int stages = (kSmemBudget - 1024 - xs) / stage_bytes;
-        if (stages > kMaxStages) stages = kMaxStages;
-        if (xs < kSmemBudget && stages >= 3) {
-            p->KR = kr; p->R = 1; p->stages = stages; p->pipes = 1; p->fused = 1;
-            p->G = (m + 1) * tiles; p->tile_groups = tiles;
-            p->n_pad = n_pad; p->tiles_per_model = tiles; p->per_model = 1;
-            p->smem_bytes = xs + stages * stage_bytes + 1024;
-            return true;
-        }
-    }
     double best = 1e30;
     for (int kr = kStreamTcMinKR; kr <= 1024; kr += kBlockK) {
         const int xs = 2 * (kr / kBlockK) * n_pad * 128;            // [X_hi; X_lo]
-        if (xs + kPipes * 2 * stage_bytes + 1024 > kSmemBudget) break;
-        int stages = (kSmemBudget - 1024 - xs) / (kPipes * stage_bytes);   // per pipeline
+        if (xs + kPipes * 2 * kStageBytes + 1024 > kSmemBudget) break;
+        int stages = (kSmemBudget - 1024 - xs) / (kPipes * kStageBytes);   // per pipeline
         if (stages > kMaxStages) stages = kMaxStages;
         const int R = (K + kr - 1) / kr;
         if (R > sms) continue;
         if (R > 1 && (R - 1) * kr >= K) continue;                    // same R as a shorter range
         const int nkb = kr / kBlockK;
-        const int g_hi = per_model ? tiles : (sms / R < items_all ? sms / R : items_all);
-        for (int g = 1; g <= g_hi; ++g) {
-            // g = blocks along y (first layer) or tile groups per model (later layers)
-            const int blocks = per_model ? R * (m + 1) * g : R * g;
-            const int items = per_model ? (tiles + g - 1) / g : (items_all + g - 1) / g;
-            const int waves = (blocks + sms - 1) / sms;
-            if (!per_model && waves > 1) continue;
+        const int g_hi = sms / R < items_all ? sms / R : items_all;
+        for (int g = 1; g <= g_hi; ++g) {                            // g = blocks along y: one wave
+            const int items = (items_all + g - 1) / g;
             // split-K partials are written and read back: 2 R n_r / K of the streamed bytes,
             // cheap while they stay in L2
             const double part_bytes = (double)R * (m + 1) * n_r * out * 4.0;
             const double part_cost = 2.0 * R * n_r / K * (part_bytes > 64e6 ? 1.0 : 0.35);
-            double est = (double)waves * ((items + 1) / 2 * nkb * (1.0 + part_cost) + 6.0) + 0.2 * R;
+            double est = (items + 1) / 2 * nkb * (1.0 + part_cost) + 6.0 + 0.2 * R;
             if (stages < 3) est *= 1.1;                             // a shallow ring hides less latency
             if (est < best) {
                 best = est;
-                p->KR = kr; p->R = R; p->stages = stages;
-                p->G = per_model ? (m + 1) * g : g;
-                p->tile_groups = per_model ? g : 1;
+                p->KR = kr; p->R = R; p->stages = stages; p->G = g;
             }
         }
     }
     if (best > 1e29) return false;
     p->n_pad = n_pad;
     p->tiles_per_model = tiles;
-    p->per_model = per_model ? 1 : 0;
-    p->smem_bytes = 2 * (p->KR / kBlockK) * n_pad * 128 + kPipes * p->stages * stage_bytes + 1024;
-    p->pipes = kPipes;
-    p->fused = 0;
+    p->smem_bytes = 2 * (p->KR / kBlockK) * n_pad * 128 + kPipes * p->stages * kStageBytes + 1024;
     return true;
 }
 
-// one slot per (k-range, tile, warp of a converter set); both sets write when they share a pipeline
-int stream_tc_norm_slots(const StreamTcPlan &p) {
-    return p.R * p.tiles_per_model * 4 * (p.pipes == 1 ? kPipes : 1);
-}
+// one slot per (k-range, tile, converter warp)
+int stream_tc_norm_slots(const StreamTcPlan &p) { return p.R * p.tiles_per_model * 4; }
 
 cudaError_t launch_stream_tc(Context &c, const StreamTcPlan &p, const float *x, const float *V, int64_t ldv,
-                             int64_t offW, int64_t offB, int K, int out, const float *X, int64_t x_model_stride,
-                             float gamma, int n_r, int m, float *part, float *Hout, int relu, int np_base,
-                             cudaStream_t s, int *launches) {
+                             int64_t offW, int64_t offB, int K, int out, const float *X, int n_r, int m,
+                             float *part, int np_base, cudaStream_t s, int *launches) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return cudaErrorNotSupported;
     CUtensorMap map_x, map_v;
@@ -721,9 +577,6 @@ cudaError_t launch_stream_tc(Context &c, const StreamTcPlan &p, const float *x, 
     }
     StreamArgs a;
     a.X = X;
-    a.x_model_stride = x_model_stride;
-    a.tile_groups = p.tile_groups;
-    a.gamma = gamma;
     a.V = V;
     a.ldv = ldv;
     a.offB = offB;
@@ -739,37 +592,23 @@ cudaError_t launch_stream_tc(Context &c, const StreamTcPlan &p, const float *x, 
     a.KR = p.KR;
     a.tiles_per_model = p.tiles_per_model;
     a.stages = p.stages;
-    a.pipes = p.pipes;
-    a.fused = p.fused;
-    a.early_loads = p.per_model;       // a later layer: the kernels before it in the chain are this call's own
-    a.xparams = x;
-    a.Hout = Hout;
-    a.relu = relu;
     a.status = c.dev_status;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(stream_tf32x3_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(stream_tf32x3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              kSmemBudget);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(stream_tf32x3_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     kSmemBudget);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
     ++*launches;
-    profile_mark(c, p.per_model ? "stream_tf32x3_layer" : "stream_tf32x3", s);
-    dim3 grid(p.R, p.G);
-    if (p.per_model)
-        return launch_chained(stream_tf32x3_kernel<true>, grid, dim3(kThreads), p.smem_bytes, s, chain_launches(c),
-                              map_x, map_v, a);
-    return launch_chained(stream_tf32x3_kernel<false>, grid, dim3(kThreads), p.smem_bytes, s, chain_launches(c),
+    profile_mark(c, "stream_tf32x3", s);
+    return launch_chained(stream_tf32x3_kernel, dim3(p.R, p.G), dim3(kThreads), p.smem_bytes, s, chain_launches(c),
                           map_x, map_v, a);
 }
 
 cudaError_t launch_stream_combine(Context &c, const StreamTcPlan &p, const float *part, const float *x,
                                   const float *V, int64_t ldv, int64_t offB, int out, int n_r, int m,
                                   float gamma, int relu, float *H, float *Hsplit, cudaStream_t s, int *launches) {
-    const int linear = p.per_model ? 0 : 1;
     ++*launches;
     profile_mark(c, "stream_combine", s);
     const bool vec = out % 4 == 0;
@@ -780,9 +619,9 @@ cudaError_t launch_stream_combine(Context &c, const StreamTcPlan &p, const float
     if (blocks > cap) blocks = cap;
     if (vec)
         return launch_chained(stream_combine_kernel<true>, dim3(blocks), dim3(256), 0, s, chain_launches(c), part,
-                              p.R, m, n_r, out, x, V, ldv, offB, gamma, relu, linear, H, Hsplit, n_pad);
+                              p.R, m, n_r, out, x, V, ldv, offB, gamma, relu, H, Hsplit, n_pad);
     return launch_chained(stream_combine_kernel<false>, dim3(blocks), dim3(256), 0, s, chain_launches(c), part, p.R,
-                          m, n_r, out, x, V, ldv, offB, gamma, relu, linear, H, Hsplit, n_pad);
+                          m, n_r, out, x, V, ldv, offB, gamma, relu, H, Hsplit, n_pad);
 }
 
 }  // namespace zeno

@@ -339,7 +339,7 @@ def run_ours(args, rank, world, local_rank):
     layer_of, layer = {}, 0
     for k in kern:
         name = k["kernel"].split(":")[1]
-        if name in ("stream_tf32x3", "stream_tf32x3_layer", "mlp_layer", "mlp_layer_mma", "mlp_head_loss_tail"):
+        if name in ("stream_tf32x3", "layer_tc", "mlp_layer", "mlp_layer_mma", "mlp_head_loss_tail"):
             layer_of[k["kernel"]] = layer
             layer += 1
     if top["kernel"] in layer_of:

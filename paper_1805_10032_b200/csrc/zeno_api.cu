@@ -151,7 +151,11 @@ zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv,
         if (!zeno::layer_tc_usable((zeno_dtype)c->desc.param_dtype, in_l, out_l, n_r) || n_r > c->n_r_max) return false;
         if ((c->offW[l] * esz0) % 16 != 0) return false;
         if (c->desc.param_dtype == ZENO_BF16) return true;
-        return l > 0 && in_l >= 128 && out_l >= 128;
+        if (in_l < 128 || out_l < 128) return false;
+        if (l > 0) return true;
+        // first layer: the stream that shares the batch reads V once and nothing else, but it needs
+        // split-K partials to fill the SMs; with enough whole tiles for every SM this kernel wins
+        return (m + 1) * ((out_l + 127) / 128) >= 2 * c->sm_count;
     };
     bool have_split = false;               // the previous layer left its output in the stacked form
     for (int l = 0; l < L; ++l) {

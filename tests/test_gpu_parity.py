@@ -32,6 +32,13 @@ SHRUNK = {
     "cfg2_mid_layers": (2, dict(dims=(520, 200, 136, 10), n_r=21, m=6, b=2, faults=[(2, "noise200")])),
     "cfg3_mid_layers": (3, dict(dims=(520, 136, 200, 10), m=11, b=4, n_r=40,
                                 faults=[(2, "signflip"), (2, "omniscient")])),
+    # the streamed tensor-core layer kernel: 128 samples (N = 256) on a bfloat16 model, a padded
+    # sample count above 64 on an fp32 model, and an fp32 first layer with a tile for every SM
+    "cfg4_128_samples": (4, dict(dims=(136, 200, 72, 50), m=4, b=1, n_r=128, faults=[(1, "signflip")])),
+    "cfg3_100_samples": (3, dict(dims=(200, 136, 130, 10), m=7, b=2, n_r=100,
+                                 faults=[(1, "signflip"), (1, "omniscient")])),
+    "cfg3_many_tiles": (3, dict(dims=(132, 384, 10), m=100, b=40, n_r=5,
+                                faults=[(20, "signflip"), (20, "omniscient")])),
     "cfg3_small": (3, dict(dims=(260, 44, 36, 10), m=37, b=15, n_r=70,
                            faults=[(7, "signflip"), (8, "omniscient")])),
     "cfg4_small": (4, dict(dims=(264, 136, 72, 50), m=9, b=3, n_r=19, faults=[(3, "signflip")])),
@@ -47,6 +54,28 @@ def test_step_matches_oracle_on_shrunk_workloads(oracle, name):
     w = syn.make_config(index, **ov)
     res = P.run_step_parity(oracle, w)
     assert res["launches"] >= 2
+
+
+def kernels_of_a_step(w):
+    """Names of the kernels one zeno_step launches on this workload, in launch order."""
+    x, V, feats, tgt = P.to_device(w)
+    with zeno.from_workload(w) as z:
+        z.profile(True)
+        z.step(x, V, feats, tgt, w.gamma, w.rho, w.b)
+        torch.cuda.synchronize()
+        return [name for name, _ in z.profile_read(0)]
+
+
+@pytest.mark.parametrize("name,expected", [
+    ("cfg2_mid_layers", ["stream_tf32x3", "stream_combine", "layer_tc", "mlp_head_loss_tail", "aggregate"]),
+    ("cfg3_many_tiles", ["split_acts", "layer_tc", "mlp_head_loss_tail", "aggregate"]),
+    ("cfg4_128_samples", ["split_acts", "layer_tc", "layer_tc", "layer_tc", "mlp_loss_tail", "aggregate"]),
+    ("cfg4_small", ["split_acts", "layer_tc", "layer_tc", "layer_tc", "mlp_loss_tail", "aggregate"]),
+])
+def test_which_kernels_serve_a_workload(name, expected):
+    """The parity cases above exercise the kernels they were written for (no quiet detour)."""
+    index, ov = SHRUNK[name]
+    assert kernels_of_a_step(syn.make_config(index, **ov)) == expected
 
 
 def test_config2_full_size(oracle):

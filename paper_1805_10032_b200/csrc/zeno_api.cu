@@ -181,14 +181,26 @@ zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv,
             t.n_pad = zeno::layer_tc_n_pad(n_r);
             t.m = m;
             t.h_shared = l == 0;
+            // an fp32 first layer is linear in its weights and shares its activations: raw products,
+            // then the combine kernel (one k-range) forms z_0 - gamma (P_c + b(v_c))
+            t.linear = l == 0 && c->desc.param_dtype == ZENO_F32 && c->tc_part != nullptr;
             t.Hsplit_in = hs_in;
-            t.Hout = next_tc ? nullptr : c->act[l & 1];
-            t.Hsplit_out = next_tc ? c->act_split[l & 1] : nullptr;
+            t.Hout = t.linear ? c->tc_part : next_tc ? nullptr : c->act[l & 1];
+            t.Hsplit_out = next_tc && !t.linear ? c->act_split[l & 1] : nullptr;
             t.relu = l + 1 < L;
             t.gamma = gamma;
             t.np_base = c->np_base[l];
             e = zeno::launch_layer_tc(*c, t, s, launches);
             if (e != cudaSuccess) return fail_cuda(c, e);
+            if (t.linear) {
+                zeno::StreamTcPlan one;
+                one.R = 1;
+                e = zeno::launch_stream_combine(*c, one, c->tc_part, xf, Vf, ldv, c->offB[l], out_l, n_r, m, gamma,
+                                                l + 1 < L, next_tc ? nullptr : c->act[l & 1],
+                                                next_tc ? static_cast<float *>(c->act_split[l & 1]) : nullptr, s,
+                                                launches);
+                if (e != cudaSuccess) return fail_cuda(c, e);
+            }
             tail.used.base[l] = c->np_base[l];
             tail.used.count[l] = zeno::layer_tc_norm_slots(out_l);
             have_split = next_tc;
@@ -353,6 +365,9 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
                 const size_t need = (l == 0 ? 1 : rows) * 2 * (size_t)zeno::layer_tc_n_pad(n_r_max < 128 ? n_r_max : 128) *
                                     (size_t)in;
                 if (need > split_elems) split_elems = need;
+                // an fp32 first layer leaves its raw products where the stream leaves its partials
+                const size_t raw = rows * (size_t)n_r_max * (size_t)o;
+                if (l == 0 && desc->param_dtype == ZENO_F32 && raw > tc_elems) tc_elems = raw;
             }
             slots += layer_slots;
             if (o > widest) widest = o;

@@ -167,6 +167,7 @@ struct LayerTcLaunch {
     int64_t ldv, offW, offB;
     int K, out, n_r, n_pad, m;
     int h_shared;            // first layer: one set of activations for every model
+    int linear;              // fp32 first layer: raw products H v_c^T into Hout, finished by the combine kernel
     const void *Hsplit_in;
     float *Hout;             // plain fp32 output [m+1][n_r][out], or NULL
     void *Hsplit_out;        // stacked two-term output for a following layer of this kind, or NULL

@@ -80,7 +80,11 @@ struct LayerTcArgs {
     int *status;
 };
 
-template <typename T>
+// LINEAR (fp32 first layer): the layer is linear in its weights and every model reads the same
+// activations, so the tile of model c is the raw rows of v_c (of x for model 0): no x tile is fetched
+// for the candidates, the epilogue writes the raw products H v_c^T, and the combine kernel forms
+// z_c = z_0 - gamma (H v_c^T + b(v_c)).
+template <typename T, bool LINEAR>
 __global__ void __launch_bounds__(kLThreads, 1)
 layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_v,
                 const __grid_constant__ CUtensorMap map_h, LayerTcArgs a) {
@@ -105,7 +109,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     const int n_items = (a.m + 1) * a.tiles;
     const int n_stages = a.stages, n_abufs = a.n_abufs, n_sets = a.n_sets;
     const int b_bytes = 2 * a.n_pad * kRowBytes;
-    const int stage_bytes = 2 * kTileBytes + b_bytes;          // x tile, v tile, activations
+    constexpr int kWTiles = LINEAR ? 1 : 2;                     // weight tiles per stage
+    const int stage_bytes = kWTiles * kTileBytes + b_bytes;     // x tile, v tile, activations
     const int acc_cols = Tr::kAccPerPad * a.n_pad;
     const int a_base = n_sets * acc_cols;                       // TMEM: accumulator sets, then the A buffers
     const float inv_stages = 1.0f / (float)n_stages, inv_abufs = 1.0f / (float)n_abufs;
@@ -168,15 +173,17 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 if (!ok) break;
                 if (elect_one()) {
                     const uint32_t dst = smem_u32(ring + (size_t)s * stage_bytes);
-                    mbar_expect_tx(bar_full(s), (has_v ? 2 : 1) * kTileBytes + b_bytes);
+                    mbar_expect_tx(bar_full(s), (has_v && !LINEAR ? 2 : 1) * kTileBytes + b_bytes);
                     issued[s] = (int)round + 1;
 #pragma unroll 1
                     for (int w = 0; w < 3; ++w) {         // x tile, v tile, activations: ONE issue site
-                        if (w == 1 && !has_v) continue;
+                        // LINEAR: the only weight tile is x's for model 0, v's otherwise
+                        if (LINEAR ? w == (has_v ? 0 : 1) : (w == 1 && !has_v)) continue;
                         const CUtensorMap *map = w == 0 ? &map_x : w == 1 ? &map_v : &map_h;
                         const int c1 = w == 2 ? 0 : tile * kRows;
                         const int c2 = w == 0 ? 0 : w == 1 ? model - 1 : (a.h_shared ? 0 : model);
-                        tma_load_3d(dst + w * kTileBytes, map, kb * kBlockK, c1, c2, bar_full(s));
+                        const int slot = w == 2 ? kWTiles : (LINEAR ? 0 : w);
+                        tma_load_3d(dst + slot * kTileBytes, map, kb * kBlockK, c1, c2, bar_full(s));
                     }
                 }
                 __syncwarp();
@@ -213,7 +220,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 tc_fence_after();
                 if (elect_one()) {
                     const uint32_t a_tmem = tmem + a_base + g * Tr::kACols;
-                    const uint32_t bx = smem_u32(ring + (size_t)s * stage_bytes + 2 * kTileBytes);
+                    const uint32_t bx = smem_u32(ring + (size_t)s * stage_bytes + kWTiles * kTileBytes);
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {            // 32 bytes of every row per MMA
                         const uint64_t db = smem_desc_sw128(bx + ks * 32);
@@ -252,7 +259,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 uint4 xq[8], vq[8];
 #pragma unroll
                 for (int c = 0; c < 8; ++c) xq[c] = *reinterpret_cast<const uint4 *>(src + ((c ^ (row & 7)) << 4));
-                if (model > 0) {
+                if (model > 0 && !LINEAR) {
 #pragma unroll
                     for (int c = 0; c < 8; ++c)
                         vq[c] = *reinterpret_cast<const uint4 *>(src + kTileBytes + ((c ^ (row & 7)) << 4));
@@ -278,8 +285,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                             wa[4 * c + u] = *reinterpret_cast<const uint32_t *>(&pk);
                         } else {
                             const float xv = __uint_as_float(xw[u]), vv = __uint_as_float(vw[u]);
-                            nrm4[u] = fmaf(vv, vv, nrm4[u]);
-                            const float w = fmaf(-a.gamma, vv, xv);
+                            nrm4[u] = LINEAR ? fmaf(xv, xv, nrm4[u]) : fmaf(vv, vv, nrm4[u]);   // LINEAR: the tile is v itself
+                            const float w = LINEAR ? xv : fmaf(-a.gamma, vv, xv);
                             const float h = tf32_hi(w);
                             wa[4 * c + u] = __float_as_uint(h);
                             wb[4 * c + u] = __float_as_uint(w - h);
@@ -322,7 +329,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             const uint32_t use = (uint32_t)(li / n_sets);
             const int o = tile * kRows + row;             // thread = output row o, column = sample j
             float bias = 0.f;
-            if (a.offB >= 0 && o < a.out) {               // asked for before the accumulator is awaited
+            if (!LINEAR && a.offB >= 0 && o < a.out) {    // asked for before the accumulator is awaited
                 const float vb = model > 0 ? load_elem(static_cast<const T *>(a.V) + (int64_t)(model - 1) * a.ldv + a.offB + o) : 0.f;
                 bias = candidate_param<T>(load_elem(static_cast<const T *>(a.xparams) + a.offB + o), vb, a.gamma);
             }
@@ -462,7 +469,7 @@ cudaError_t encode_maps(const LayerTcLaunch &l, CUtensorMap *map_x, CUtensorMap 
     return cudaSuccess;
 }
 
-template <typename T>
+template <typename T, bool LINEAR>
 cudaError_t launch_typed(Context &c, const LayerTcLaunch &l, cudaStream_t s) {
     using Tr = TcTraits<T>;
     CUtensorMap map_x, map_v, map_h;
@@ -481,7 +488,7 @@ cudaError_t launch_typed(Context &c, const LayerTcLaunch &l, cudaStream_t s) {
     a.m = l.m;
     a.tiles = (l.out + kRows - 1) / kRows;
     a.h_shared = l.h_shared;
-    const int stage_bytes = 2 * kTileBytes + 2 * l.n_pad * kRowBytes;
+    const int stage_bytes = (LINEAR ? 1 : 2) * kTileBytes + 2 * l.n_pad * kRowBytes;
     a.stages = (kLSmemBudget - 1024) / stage_bytes;
     if (a.stages > kLMaxStages) a.stages = kLMaxStages;
     const int acc_cols = Tr::kAccPerPad * l.n_pad;
@@ -490,16 +497,18 @@ cudaError_t launch_typed(Context &c, const LayerTcLaunch &l, cudaStream_t s) {
     if (a.n_abufs > kLMaxABufs) a.n_abufs = kLMaxABufs;
     a.Hout = l.Hout;
     a.Hsplit = l.Hsplit_out;
-    a.relu = l.relu;
+    a.relu = LINEAR ? 0 : l.relu;          // LINEAR: raw products, the combine kernel activates
     a.normpart = c.normpart;
     a.np_slots = c.np_slots;
     a.np_base = l.np_base;
     a.status = c.dev_status;
     static bool attr_set = false;
     if (!attr_set) {
-        e = cudaFuncSetAttribute(layer_tc_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLSmemBudget);
+        e = cudaFuncSetAttribute(layer_tc_kernel<float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLSmemBudget);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(layer_tc_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            e = cudaFuncSetAttribute(layer_tc_kernel<float, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLSmemBudget);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(layer_tc_kernel<__nv_bfloat16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      kLSmemBudget);
         if (e != cudaSuccess) return e;
         attr_set = true;
@@ -509,7 +518,7 @@ cudaError_t launch_typed(Context &c, const LayerTcLaunch &l, cudaStream_t s) {
     // equal shares: the fewest blocks that give the same number of rounds as one block per SM
     const int rounds = (items + sms - 1) / sms;
     const int blocks = (items + rounds - 1) / rounds;
-    return launch_chained(layer_tc_kernel<T>, dim3(blocks), dim3(kLThreads), (size_t)a.stages * stage_bytes + 1024, s,
+    return launch_chained(layer_tc_kernel<T, LINEAR>, dim3(blocks), dim3(kLThreads), (size_t)a.stages * stage_bytes + 1024, s,
                           chain_launches(c), map_x, map_v, map_h, a);
 }
 
@@ -535,8 +544,9 @@ int layer_tc_norm_slots(int out) { return (out + kRows - 1) / kRows * 8; }
 cudaError_t launch_layer_tc(Context &c, const LayerTcLaunch &l, cudaStream_t s, int *launches) {
     ++*launches;
     profile_mark(c, "layer_tc", s);
-    if (c.desc.param_dtype == ZENO_BF16) return launch_typed<__nv_bfloat16>(c, l, s);
-    return launch_typed<float>(c, l, s);
+    if (c.desc.param_dtype == ZENO_BF16) return launch_typed<__nv_bfloat16, false>(c, l, s);
+    if (l.linear) return launch_typed<float, true>(c, l, s);
+    return launch_typed<float, false>(c, l, s);
 }
 
 cudaError_t launch_split_acts(Context &c, const float *H, int models, int n_r, int K, void *out, cudaStream_t s,

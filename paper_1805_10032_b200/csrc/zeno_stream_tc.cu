@@ -412,10 +412,14 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     }
 }
 
-// Split-K reduction and activation after the streamed first layer:
+// Split-K reduction and activation after a first layer whose products were taken against raw rows:
 //   z_0 = sum_r P[r][0] + b(x),   z_c = z_0 - gamma (sum_r P[r][c] + b(v_c)),   h = ReLU(z)
-// One thread per (model, sample, four outputs); the 2R loads of a thread are independent and
-// the partials are added in k-range order.
+// Block row blockIdx.y = model c; one thread per (sample, four outputs).  The partials are added in
+// k-range order, four k-ranges' loads in flight at a time (few registers: several blocks per SM hide
+// the latency instead).
+// H: plain activations [m+1][n_r][out]; Hsplit: the same values as the two-term stacked operand
+// [m+1][2 n_pad][out] of a following tensor-core layer (tf32 value, then remainder; zero rows for the
+// padded samples).  Either may be NULL.
 template <bool VEC4>
 __global__ void __launch_bounds__(256) stream_combine_kernel(const float *part, int R, int m, int n_r, int out,
                                                              const float *x, const float *V, int64_t ldv,
@@ -424,23 +428,20 @@ __global__ void __launch_bounds__(256) stream_combine_kernel(const float *part, 
     constexpr int E = VEC4 ? 4 : 1;
     pdl_launch_dependents();
     pdl_wait();
-    // H: plain activations [m+1][n_r][out]; Hsplit: the same values as the two-term stacked operand
-    // [m+1][2 n_pad][out] of a following tensor-core layer (tf32 value, then remainder; zero rows for
-    // the padded samples).  Either may be NULL.
     const int og = (out + E - 1) / E;                       // output groups per row
     const int n_rows = Hsplit ? n_pad : n_r;
-    const int64_t total = (int64_t)(m + 1) * n_rows * og;
+    const int c = blockIdx.y;
     const int64_t per_r = (int64_t)(m + 1) * n_r * out;
-    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total;
-         t += (int64_t)gridDim.x * blockDim.x) {
-        const int o = (int)(t % og) * E;
-        const int64_t cj = t / og;
-        const int c = (int)(cj / n_rows), j = (int)(cj % n_rows);
+    for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < n_rows * og; t += gridDim.x * blockDim.x) {
+        const int j = t / og, o = (t - j * og) * E;
+        float *hs = Hsplit ? Hsplit + ((int64_t)c * 2 * n_pad + j) * out + o : nullptr;
         if (j >= n_r) {                                          // padded sample of the stacked operand
-            float *hs = Hsplit + ((int64_t)c * 2 * n_pad + j) * out + o;
-#pragma unroll
-            for (int e = 0; e < E; ++e)
-                if (o + e < out) hs[e] = hs[(int64_t)n_pad * out + e] = 0.f;
+            if (VEC4) {
+                *reinterpret_cast<float4 *>(hs) = make_float4(0.f, 0.f, 0.f, 0.f);
+                *reinterpret_cast<float4 *>(hs + (int64_t)n_pad * out) = make_float4(0.f, 0.f, 0.f, 0.f);
+            } else {
+                hs[0] = hs[(int64_t)n_pad * out] = 0.f;
+            }
             continue;
         }
         const int64_t ic = ((int64_t)c * n_r + j) * out + o;
@@ -453,14 +454,13 @@ __global__ void __launch_bounds__(256) stream_combine_kernel(const float *part, 
             // the bias entries come from HBM: ask for them before the partials, not after
             const bool ok = offB >= 0 && o + e < out;
             xb[e] = ok ? __ldg(x + offB + o + e) : 0.f;
-            vb[e] = ok && c > 0 ? __ldg(V + (int64_t)(c - 1) * ldv + offB + o + e) : 0.f;
+            vb[e] = ok && two ? __ldg(V + (int64_t)(c - 1) * ldv + offB + o + e) : 0.f;
         }
-        if (VEC4) {
-            // twelve k-ranges at a time: all loads of a chunk are issued before they are added
-            for (int r0 = 0; r0 < R; r0 += 12) {
-                float4 a4[12], b4[12];
+        for (int r0 = 0; r0 < R; r0 += 4) {
+            if (VEC4) {
+                float4 a4[4], b4[4];
 #pragma unroll
-                for (int u = 0; u < 12; ++u) {
+                for (int u = 0; u < 4; ++u) {
                     const bool ok = r0 + u < R;
                     a4[u] = ok ? __ldcg(reinterpret_cast<const float4 *>(part + (r0 + u) * per_r + i0))
                                : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -468,33 +468,36 @@ __global__ void __launch_bounds__(256) stream_combine_kernel(const float *part, 
                                         : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
 #pragma unroll
-                for (int u = 0; u < 12; ++u) {
+                for (int u = 0; u < 4; ++u) {
                     z0[0] += a4[u].x; z0[1] += a4[u].y; z0[2] += a4[u].z; z0[3] += a4[u].w;
                     pc[0] += b4[u].x; pc[1] += b4[u].y; pc[2] += b4[u].z; pc[3] += b4[u].w;
                 }
-            }
-        } else {
-            for (int r = 0; r < R; ++r) {
-                z0[0] += __ldcg(part + r * per_r + i0);
-                if (two) pc[0] += __ldcg(part + r * per_r + ic);
+            } else {
+                for (int r = r0; r < min(r0 + 4, R); ++r) {
+                    z0[0] += __ldcg(part + r * per_r + i0);
+                    if (two) pc[0] += __ldcg(part + r * per_r + ic);
+                }
             }
         }
 #pragma unroll
         for (int e = 0; e < E; ++e) {
-            if (offB >= 0 && o + e < out) {
-                z0[e] += xb[e];
-                pc[e] += vb[e];
-            }
-            float z = two ? fmaf(-gamma, pc[e], z0[e]) : z0[e];
+            float z = two ? fmaf(-gamma, pc[e] + vb[e], z0[e] + xb[e]) : z0[e] + xb[e];
             if (relu) z = (z > 0.f || z != z) ? z : 0.f;
-            if (o + e < out) {
-                if (H) H[ic + e] = z;
-                if (Hsplit) {
-                    float *hs = Hsplit + ((int64_t)c * 2 * n_pad + j) * out + o + e;
-                    const float hi = tf32_hi(z);
-                    hs[0] = hi;
-                    hs[(int64_t)n_pad * out] = z - hi;
-                }
+            z0[e] = z;                                           // the activation
+            pc[e] = tf32_hi(z);                                  // its leading term
+        }
+        if (VEC4) {                                              // out % 4 == 0: whole 16-byte groups
+            if (H) *reinterpret_cast<float4 *>(H + ic) = make_float4(z0[0], z0[1], z0[2], z0[3]);
+            if (hs) {
+                *reinterpret_cast<float4 *>(hs) = make_float4(pc[0], pc[1], pc[2], pc[3]);
+                *reinterpret_cast<float4 *>(hs + (int64_t)n_pad * out) =
+                    make_float4(z0[0] - pc[0], z0[1] - pc[1], z0[2] - pc[2], z0[3] - pc[3]);
+            }
+        } else {
+            if (H) H[ic] = z0[0];
+            if (hs) {
+                hs[0] = pc[0];
+                hs[(int64_t)n_pad * out] = z0[0] - pc[0];
             }
         }
     }
@@ -613,15 +616,16 @@ cudaError_t launch_stream_combine(Context &c, const StreamTcPlan &p, const float
     profile_mark(c, "stream_combine", s);
     const bool vec = out % 4 == 0;
     const int n_pad = layer_tc_n_pad(n_r);
-    const int64_t total = (int64_t)(m + 1) * (Hsplit ? n_pad : n_r) * (vec ? out / 4 : out);
-    int blocks = (int)((total + 255) / 256);
-    const int cap = (c.sm_count > 0 ? c.sm_count : 148) * 16;
-    if (blocks > cap) blocks = cap;
+    const int per_model = (Hsplit ? n_pad : n_r) * (vec ? out / 4 : out);
+    int bx = (per_model + 255) / 256;
+    const int cap = ((c.sm_count > 0 ? c.sm_count : 148) * 16 + m) / (m + 1);   // about 16 blocks per SM in all
+    if (bx > cap) bx = cap > 0 ? cap : 1;
+    const dim3 grid(bx, m + 1);
     if (vec)
-        return launch_chained(stream_combine_kernel<true>, dim3(blocks), dim3(256), 0, s, chain_launches(c), part,
-                              p.R, m, n_r, out, x, V, ldv, offB, gamma, relu, H, Hsplit, n_pad);
-    return launch_chained(stream_combine_kernel<false>, dim3(blocks), dim3(256), 0, s, chain_launches(c), part, p.R,
-                          m, n_r, out, x, V, ldv, offB, gamma, relu, H, Hsplit, n_pad);
+        return launch_chained(stream_combine_kernel<true>, grid, dim3(256), 0, s, chain_launches(c), part, p.R, m,
+                              n_r, out, x, V, ldv, offB, gamma, relu, H, Hsplit, n_pad);
+    return launch_chained(stream_combine_kernel<false>, grid, dim3(256), 0, s, chain_launches(c), part, p.R, m, n_r,
+                          out, x, V, ldv, offB, gamma, relu, H, Hsplit, n_pad);
 }
 
 }  // namespace zeno

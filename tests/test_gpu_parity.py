@@ -68,7 +68,7 @@ def kernels_of_a_step(w):
 
 @pytest.mark.parametrize("name,expected", [
     ("cfg2_mid_layers", ["stream_tf32x3", "stream_combine", "layer_tc", "mlp_head_loss_tail", "aggregate"]),
-    ("cfg3_many_tiles", ["split_acts", "layer_tc", "mlp_head_loss_tail", "aggregate"]),
+    ("cfg3_many_tiles", ["split_acts", "layer_tc", "stream_combine", "mlp_head_loss_tail", "aggregate"]),
     ("cfg4_128_samples", ["split_acts", "layer_tc", "layer_tc", "layer_tc", "mlp_loss_tail", "aggregate"]),
     ("cfg4_small", ["split_acts", "layer_tc", "layer_tc", "layer_tc", "mlp_loss_tail", "aggregate"]),
 ])

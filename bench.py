@@ -47,14 +47,19 @@ def measured_peaks():
 # DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum) from one ncu capture of
 # the kernel on the named configuration, valid only while the kernel's source is unchanged.
 NCU_TRAFFIC = {
-    ("stream_tf32x3", 2): {"bytes": 137.1e6, "source": "paper_1805_10032_b200/csrc/zeno_stream_tc.cu",
-                           "sha256_16": "ee74b5709fd49649"},
+    ("0:stream_tf32x3", 2): {"bytes": 136.9e6, "source": "paper_1805_10032_b200/csrc/zeno_stream_tc.cu",
+                             "sha256_16": "051ef066a4b567be"},
+    ("1:layer_tc", 4): {"bytes": 1421.3e6, "source": "paper_1805_10032_b200/csrc/zeno_layer_tc.cu",
+                        "sha256_16": "fc9edef7ec0d2f6d"},
+    ("2:layer_tc", 4): {"bytes": 1486.7e6, "source": "paper_1805_10032_b200/csrc/zeno_layer_tc.cu",
+                        "sha256_16": "fc9edef7ec0d2f6d"},
 }
 
 
-def measured_traffic(kernel_name, config):
+def measured_traffic(kernel_key, config):
+    """kernel_key: position in the step and name, as in the per-kernel list ("0:stream_tf32x3")."""
     import hashlib
-    ent = NCU_TRAFFIC.get((kernel_name, config))
+    ent = NCU_TRAFFIC.get((kernel_key, config))
     if not ent:
         return None
     try:
@@ -354,7 +359,7 @@ def run_ours(args, rank, world, local_rank):
     step_bytes = score_b + agg_b
     roofline = {
         "bound": "hbm", "kernel": top["kernel"], "achieved": achieved, "peak": peak,
-        "unit": "GB/s", "frac": achieved / peak, "traffic": measured_traffic(top_name, args.config),
+        "unit": "GB/s", "frac": achieved / peak, "traffic": measured_traffic(top["kernel"], args.config),
         "peak_source": peak_kind,
         "bytes_per_launch": top_bytes, "avg_us": top["avg_us"],
         "timed": "second pass over the same K steps, enqueued back to back with a CUDA event around every kernel",

@@ -246,6 +246,7 @@ zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv,
         a.np_slots = c->np_slots;
         a.np_base = c->np_base[l];
         a.fuse_loss = (l + 1 == L) && fuse_loss;
+        a.first_in_call = l == 0;
         // 16-byte aligned rows of eight-parameter multiples take the warp-MMA kernel
         const size_t esz = elem_size(c->desc.param_dtype);
         const bool mma = !a.fuse_loss && aligned && !getenv("ZENO_DISABLE_TENSOR_CORES") &&

@@ -113,6 +113,9 @@ struct LayerArgs {
     int np_slots, np_base;
     // last layer only: fold the cross-entropy (and the tail) into this launch
     int fuse_loss;
+    // this launch is the first of the call: whatever precedes it on the stream is the caller's and may
+    // be producing x or V, so nothing is read before the preceding kernel has completed
+    int first_in_call;
     const int32_t *labels;
     float *losses;
     TailArgs tail;

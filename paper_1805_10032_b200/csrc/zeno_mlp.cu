@@ -254,7 +254,6 @@ __global__ void __launch_bounds__(256, 1) mlp_head_kernel(LayerArgs a) {
     __shared__ float zl[32][NS + 1];
 
     pdl_launch_dependents();
-    pdl_wait();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int c = blockIdx.x;
     const int K = a.in;
@@ -281,18 +280,10 @@ __global__ void __launch_bounds__(256, 1) mlp_head_kernel(LayerArgs a) {
         bias_v[bi] = ok && has_v ? load_elem(vbase + a.offB + o) : 0.f;
     }
 
-    for (int kb = 0; kb < K; kb += KC) {
-        if (kb > 0) __syncthreads();
-        // stage w rows and activations of this chunk (zero beyond the layer's rows / samples / K)
+    // w = x - gamma v of the layer's rows for the chunk starting at kb (zero beyond the rows / K)
+    auto stage_weights = [&](int kb) {
         if (VEC) {
-            // activations: asynchronous copies, in flight while the weights are formed
-            for (int t = threadIdx.x; t < NS * (KC / 4); t += 256) {
-                const int j = t / (KC / 4), kk = (t % (KC / 4)) * 4;
-                const bool ok = j < a.n_r && kb + kk < K;
-                cp_async16(&hs[j][kk], ok ? hin + (int64_t)j * K + kb + kk : a.Hin, ok);
-            }
-            cp_async_commit();
-            // weights: all of a thread's loads are issued before the first is used
+            // all of a thread's loads are issued before the first is used
             constexpr int kPerThread = OUT_T * (KC / 4) / 256;
             float xv[kPerThread][4], vv[kPerThread][4];
 #pragma unroll
@@ -318,7 +309,6 @@ __global__ void __launch_bounds__(256, 1) mlp_head_kernel(LayerArgs a) {
                 }
                 *reinterpret_cast<float4 *>(&ws[o][kk]) = make_float4(w4[0], w4[1], w4[2], w4[3]);
             }
-            cp_async_wait<0>();
         } else {
             for (int t = threadIdx.x; t < OUT_T * KC; t += 256) {
                 const int o = t / KC, kk = t % KC;
@@ -331,11 +321,35 @@ __global__ void __launch_bounds__(256, 1) mlp_head_kernel(LayerArgs a) {
                 }
                 ws[o][kk] = w;
             }
+        }
+    };
+    // the model's input activations for the chunk (asynchronous copies on the vector path)
+    auto stage_acts = [&](int kb) {
+        if (VEC) {
+            for (int t = threadIdx.x; t < NS * (KC / 4); t += 256) {
+                const int j = t / (KC / 4), kk = (t % (KC / 4)) * 4;
+                const bool ok = j < a.n_r && kb + kk < K;
+                cp_async16(&hs[j][kk], ok ? hin + (int64_t)j * K + kb + kk : a.Hin, ok);
+            }
+            cp_async_commit();
+        } else {
             for (int t = threadIdx.x; t < NS * KC; t += 256) {
                 const int j = t / KC, kk = t % KC;
                 hs[j][kk] = (j < a.n_r && kb + kk < K) ? __ldg(hin + (int64_t)j * K + kb + kk) : 0.f;
             }
         }
+    };
+
+    // The weights are inputs of the whole call: the first chunk is formed while the kernel that
+    // produces the activations may still be running.
+    if (a.first_in_call) pdl_wait();    // unless x and V may still be in the making (see LayerArgs)
+    stage_weights(0);
+    pdl_wait();
+    for (int kb = 0; kb < K; kb += KC) {
+        if (kb > 0) __syncthreads();
+        stage_acts(kb);                 // in flight while the weights are formed
+        if (kb > 0) stage_weights(kb);
+        if (VEC) cp_async_wait<0>();
         __syncthreads();
         // warp q: its SPW samples against every row; lane l takes k = 4l + 128 i
 #pragma unroll 1

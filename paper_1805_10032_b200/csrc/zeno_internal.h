@@ -186,6 +186,9 @@ cudaError_t launch_split_acts(Context &c, const float *H, int models, int n_r, i
                               int *launches);
 
 int lsq_slab_count(const Context &c);
+// Tensor-core version of the least-squares stream (zeno_lsq_tc.cu): one slab per block into a.part.
+bool lsq_tc_usable(const LsqArgs &a, bool aligned);
+cudaError_t launch_lsq_tc(Context &c, const LsqArgs &a, int max_slabs, int *slabs, cudaStream_t s);
 int mlp_norm_slots(int out);
 
 // ---- device helpers shared by the kernels ------------------------------------------------

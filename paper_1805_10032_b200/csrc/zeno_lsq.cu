@@ -264,13 +264,19 @@ cudaError_t launch_lsq_score(Context &c, const LsqArgs &a_in, const float *y, fl
     a.slabs = slabs;
     cudaError_t e;
     ++*launches;
-    profile_mark(c, "lsq_stream", s);
-    if (nrt == 8)
-        e = aligned ? launch_stream<8, 8, true>(a, s) : launch_stream<8, 8, false>(a, s);
-    else if (nrt == 16)
-        e = aligned ? launch_stream<16, 6, true>(a, s) : launch_stream<16, 6, false>(a, s);
-    else
-        e = aligned ? launch_stream<32, 4, true>(a, s) : launch_stream<32, 4, false>(a, s);
+    if (lsq_tc_usable(a, aligned) && !getenv("ZENO_DISABLE_TENSOR_CORES")) {
+        // up to 64 candidates on aligned rows: the tensor-core stream (one slab per block)
+        profile_mark(c, "lsq_tc", s);
+        e = launch_lsq_tc(c, a, lsq_slab_count(c), &slabs, s);
+    } else {
+        profile_mark(c, "lsq_stream", s);
+        if (nrt == 8)
+            e = aligned ? launch_stream<8, 8, true>(a, s) : launch_stream<8, 8, false>(a, s);
+        else if (nrt == 16)
+            e = aligned ? launch_stream<16, 6, true>(a, s) : launch_stream<16, 6, false>(a, s);
+        else
+            e = aligned ? launch_stream<32, 4, true>(a, s) : launch_stream<32, 4, false>(a, s);
+    }
     if (e != cudaSuccess) return e;
     ++*launches;
     profile_mark(c, "lsq_finish", s);

@@ -1,0 +1,409 @@
+// Least-squares scoring pass on the 5th-generation tensor cores.
+//
+// The residual of candidate i is linear in the parameters, A (x - gamma v_i) - y = A x - gamma A v_i - y,
+// so one pass over V, A and x yields everything: the products A v_i^T for all candidates (a skinny
+// GEMM of the rows of V against the n_r rows of A over the parameter index k), A x, and the sums of
+// squares of the rows of V.  All three operands are streamed from HBM exactly once; a block owns a
+// contiguous range of k and leaves its partial sums in a slab that lsq_finish_kernel adds up in double.
+//
+// A tile of the MMA has 128 rows but there are at most 64 candidates, so a block works on TWO halves of
+// its k-range at once: TMEM lanes 0-63 hold the candidates' entries of a k-block of the first half,
+// lanes 64-127 those of the matching k-block of the second half.  Each k-block takes two groups of MMAs
+// on the same A operand, one against the first half's rows of A (whose result is meaningful in lanes
+// 0-63), one against the second half's (lanes 64-127), into different accumulator columns.
+//
+// fp32 accuracy on tf32 tensor cores as in the first-layer stream: both operands are split,
+// a = a_hi + a_lo, and a_hi b_hi + a_hi b_lo + a_lo b_hi is accumulated, the small products in columns of
+// their own.  The tensor core adds into its accumulator with truncation, so the accumulator is drained
+// into fp32 registers every kFlush k-blocks (two sets alternate: one is drained while the other adds).
+//
+// Warp roles (every producer / issuer warp stays converged and issues from one elected lane):
+//   warp 0       TMA producer: per stage two 64-row boxes of V, two boxes of A, two 128-byte pieces of x
+//   warp 1       MMA issuer, owner of TMEM
+//   warp 2       splits the stage's rows of A into [a_hi; a_lo] (the MMA's B operand, 128-byte swizzled)
+//                and takes A x from the same registers
+//   warps 4-11   two converter sets on alternate k-blocks: thread = TMEM lane; reads its 128 bytes of V,
+//                accumulates v^2, stores v_hi / v_lo to TMEM as the A operand
+//   warps 12-15  drain the accumulator sets into registers; at the end write the slab
+// Every mbarrier wait is bounded; a wait that gives up raises a status word and the block leaves through
+// the common teardown.
+#include "zeno_internal.h"
+#include "zeno_tc.cuh"
+
+namespace zeno {
+
+namespace {
+
+constexpr int kHalfRows = 64;               // candidates per half tile
+constexpr int kQBlockK = 32;                // floats per k-block = one 128-byte swizzle row
+constexpr int kVHalfBytes = kHalfRows * 128;
+constexpr int kQThreads = 32 * 16;
+constexpr int kQMaxStages = 8;
+constexpr int kQMaxABufs = 5;
+constexpr int kQSmem = 200 * 1024;          // dynamic; the result exchange below is static
+constexpr int kQTmemCols = 512;
+constexpr int kFlush = 32;                  // k-blocks accumulated in TMEM before a drain
+
+struct LsqTcArgs {
+    int m, n_r, n_pad;                      // n_pad: 16 or 32
+    int nkb;                                // k-blocks per half of a block's k-range
+    int stages, n_abufs;
+    float *part;                            // [blocks][m+1][n_r+1]
+    int *status;
+};
+
+// bytes of a stage: V halves | [a_hi; a_lo] halves | raw A halves | x pieces (padded to 1 KB)
+__host__ __device__ inline int lsq_stage_bytes(int n_pad) { return 2 * kVHalfBytes + 2 * (2 * n_pad * 128) + 2 * (n_pad * 128) + 1024; }
+
+__global__ void __launch_bounds__(kQThreads, 1)
+lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_a,
+              const __grid_constant__ CUtensorMap map_x, LsqTcArgs a) {
+    pdl_launch_dependents();
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    // full, empty, bready [stages]; afull, aempty [A buffers]; dfull, dempty [2 sets]
+    constexpr int kBars = 3 * kQMaxStages + 2 * kQMaxABufs + 4;
+    __shared__ __align__(8) uint64_t bars[kBars];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+    __shared__ int issued[kQMaxStages];
+    __shared__ float res[128][33];          // drained products per TMEM lane
+    __shared__ float nrm_s[2][128];         // sums of squares per lane and converter set
+    __shared__ float z0_s[32];              // A x
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
+    if (tid == 32) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
+    if (tid == 64) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
+
+    const int n_pad = a.n_pad, nkb = a.nkb, n_stages = a.stages, n_abufs = a.n_abufs;
+    const int b_bytes = 2 * n_pad * 128;                   // [a_hi; a_lo] of one half
+    const int raw_bytes = n_pad * 128;
+    const int stage_bytes = lsq_stage_bytes(n_pad);
+    const int off_b = 2 * kVHalfBytes, off_raw = off_b + 2 * b_bytes, off_x = off_raw + 2 * raw_bytes;
+    const int set_cols = 6 * n_pad;                        // per half: D1 (2 n_pad) and D2 (n_pad)
+    const int a_base = 2 * set_cols;
+    const int n_flush = (nkb + kFlush - 1) / kFlush;
+    const int64_t kb0 = (int64_t)blockIdx.x * 2 * nkb;     // first k-block of the block's range
+    const float inv_stages = 1.0f / (float)n_stages, inv_abufs = 1.0f / (float)n_abufs;
+    uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+
+    auto bar_full = [&](int s) { return smem_u32(&bars[s]); };
+    auto bar_empty = [&](int s) { return smem_u32(&bars[kQMaxStages + s]); };
+    auto bar_bready = [&](int s) { return smem_u32(&bars[2 * kQMaxStages + s]); };
+    auto bar_afull = [&](int g) { return smem_u32(&bars[3 * kQMaxStages + g]); };
+    auto bar_aempty = [&](int g) { return smem_u32(&bars[3 * kQMaxStages + kQMaxABufs + g]); };
+    auto bar_dfull = [&](int q) { return smem_u32(&bars[3 * kQMaxStages + 2 * kQMaxABufs + q]); };
+    auto bar_dempty = [&](int q) { return smem_u32(&bars[3 * kQMaxStages + 2 * kQMaxABufs + 2 + q]); };
+
+    if (tid == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < kQMaxStages; ++s) {
+            mbar_init(bar_full(s), 1);
+            mbar_init(bar_empty(s), 5);        // the four warps of a converter set and the MMAs' commit
+            mbar_init(bar_bready(s), 1);
+            issued[s] = 0;
+        }
+        for (int g = 0; g < kQMaxABufs; ++g) {
+            mbar_init(bar_afull(g), 4);
+            mbar_init(bar_aempty(g), 1);
+        }
+        for (int q = 0; q < 2; ++q) {
+            mbar_init(bar_dfull(q), 1);
+            mbar_init(bar_dempty(q), 4);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&tmem_base_slot)), "r"(kQTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    pdl_wait();
+    const uint32_t tmem = tmem_base_slot;
+    volatile int *abortp = &abort_flag;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        int s = 0;
+        uint32_t round = 0;
+        for (int kb = 0; kb < nkb; ++kb) {
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_empty(s), (round & 1) ^ 1, abortp))) break;
+            if (elect_one()) {
+                const uint32_t dst = smem_u32(ring + (size_t)s * stage_bytes);
+                mbar_expect_tx(bar_full(s), 2 * kVHalfBytes + 2 * raw_bytes + 2 * 128);
+                issued[s] = (int)round + 1;
+#pragma unroll 1
+                for (int w = 0; w < 6; ++w) {          // V, A, x of the two halves: ONE issue site
+                    const int h = w & 1, what = w >> 1;
+                    const CUtensorMap *map = what == 0 ? &map_v : what == 1 ? &map_a : &map_x;
+                    const uint32_t off = what == 0 ? h * kVHalfBytes : what == 1 ? off_raw + h * raw_bytes : off_x + h * 128;
+                    const int64_t k = (kb0 + (int64_t)h * nkb + kb) * kQBlockK;
+                    tma_load_3d(dst + off, map, (int)k, 0, 0, bar_full(s));
+                }
+            }
+            __syncwarp();
+            if (++s == n_stages) {
+                s = 0;
+                ++round;
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        const uint32_t idesc_base = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(128 >> 4) << 24);
+        const uint32_t idesc_n = idesc_base | ((uint32_t)(n_pad >> 3) << 17);
+        const uint32_t idesc_2n = idesc_base | ((uint32_t)((2 * n_pad) >> 3) << 17);
+        for (int kb = 0; kb < nkb; ++kb) {
+            const int fl = kb / kFlush, in_fl = kb - fl * kFlush;
+            const int set = fl & 1;
+            if (in_fl == 0) {                          // a fresh accumulator set: wait until it was drained
+                if (!__all_sync(0xffffffffu, mbar_wait(bar_dempty(set), (((uint32_t)fl >> 1) & 1) ^ 1, abortp))) break;
+                tc_fence_after();
+            }
+            const uint32_t it = (uint32_t)kb;
+            const uint32_t sround = small_div(it, inv_stages), around = small_div(it, inv_abufs);
+            const int s = (int)(it - sround * n_stages), g = (int)(it - around * n_abufs);
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_bready(s), sround & 1, abortp) &&
+                                             mbar_wait(bar_afull(g), around & 1, abortp)))
+                break;
+            tc_fence_after();
+            if (elect_one()) {
+                const uint32_t a_tmem = tmem + a_base + g * 64;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint32_t d1 = tmem + set * set_cols + h * 3 * n_pad, d2 = d1 + 2 * n_pad;
+                    const uint32_t bx = smem_u32(ring + (size_t)s * stage_bytes + off_b + h * b_bytes);
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) {
+                        const uint64_t db = smem_desc_sw128(bx + ks * 32);
+                        tc_mma_tf32_ts(d1, a_tmem + ks * 8, db, idesc_2n, (uint32_t)(in_fl | ks));        // v_hi [a_hi; a_lo]
+                        tc_mma_tf32_ts(d2, a_tmem + 32 + ks * 8, db, idesc_n, (uint32_t)(in_fl | ks));    // v_lo a_hi
+                    }
+                }
+                tc_commit(bar_aempty(g));
+                tc_commit(bar_empty(s));
+                if (in_fl == kFlush - 1 || kb + 1 == nkb) tc_commit(bar_dfull(set));
+            }
+            __syncwarp();
+        }
+    } else if (warp == 2) {
+        // ------------------------------------------------------------------ rows of A: split for the MMA, and A x
+        float accx[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};    // rows 4 u + lane / 8 (u < n_pad / 4)
+        bool ok = true;
+        for (int kb = 0; kb < nkb && ok; ++kb) {
+            const uint32_t sround = small_div((uint32_t)kb, inv_stages);
+            const int s = kb - (int)sround * n_stages;
+            ok = mbar_wait(bar_full(s), sround & 1, abortp);
+            if (!ok) break;
+            uint8_t *st = ring + (size_t)s * stage_bytes;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const float4 x4 = *reinterpret_cast<const float4 *>(st + off_x + h * 128 + (lane & 7) * 16);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    if (4 * u >= n_pad) break;
+                    const int j = 4 * u + (lane >> 3), c = lane & 7;
+                    const uint32_t sw = (uint32_t)j * 128 + ((c ^ (j & 7)) << 4);
+                    const float4 v = *reinterpret_cast<const float4 *>(st + off_raw + h * raw_bytes + sw);
+                    accx[u] = fmaf(v.x, x4.x, fmaf(v.y, x4.y, fmaf(v.z, x4.z, fmaf(v.w, x4.w, accx[u]))));
+                    const float4 hi = make_float4(tf32_hi(v.x), tf32_hi(v.y), tf32_hi(v.z), tf32_hi(v.w));
+                    *reinterpret_cast<float4 *>(st + off_b + h * b_bytes + sw) = hi;
+                    *reinterpret_cast<float4 *>(st + off_b + h * b_bytes + n_pad * 128 + sw) =
+                        make_float4(v.x - hi.x, v.y - hi.y, v.z - hi.z, v.w - hi.w);     // n_pad % 8 == 0: same swizzle phase
+                }
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> tensor-core reads
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_bready(s));
+        }
+        // A x: the eight lanes of a row add up
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            float t = accx[u];
+            t += __shfl_xor_sync(0xffffffffu, t, 1);
+            t += __shfl_xor_sync(0xffffffffu, t, 2);
+            t += __shfl_xor_sync(0xffffffffu, t, 4);
+            if ((lane & 7) == 0 && 4 * u + (lane >> 3) < 32) z0_s[4 * u + (lane >> 3)] = t;
+        }
+    } else if (warp >= 4 && warp < 12) {
+        // ------------------------------------------------------------------ converters
+        const int cset = (warp - 4) >> 2;             // set 0 takes the even k-blocks, set 1 the odd
+        const int quad = warp & 3;
+        const int row = quad * 32 + lane;             // TMEM lane: candidate row (half 0), row - 64 (half 1)
+        const uint32_t a_bufs = tmem + ((uint32_t)(quad * 32) << 16) + a_base;
+        float nrm4[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int kb = cset; kb < nkb; kb += 2) {
+            const uint32_t it = (uint32_t)kb;
+            const uint32_t sround = small_div(it, inv_stages), around = small_div(it, inv_abufs);
+            const int s = (int)(it - sround * n_stages), g = (int)(it - around * n_abufs);
+            if (!mbar_wait(bar_full(s), sround & 1, abortp)) break;
+            const uint8_t *src = ring + (size_t)s * stage_bytes + row * 128;     // the two V boxes are contiguous
+            float4 v[8];
+            uint32_t hi[32], lo[32];
+#pragma unroll
+            for (int c = 0; c < 8; ++c) v[c] = *reinterpret_cast<const float4 *>(src + ((c ^ (row & 7)) << 4));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_empty(s));
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const float e[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    nrm4[u] = fmaf(e[u], e[u], nrm4[u]);
+                    const float h = tf32_hi(e[u]);
+                    hi[4 * c + u] = __float_as_uint(h);
+                    lo[4 * c + u] = __float_as_uint(e[u] - h);
+                }
+            }
+            if (!mbar_wait(bar_aempty(g), (around & 1) ^ 1, abortp)) break;
+            tc_fence_after();
+            tc_st32(a_bufs + g * 64, hi);
+            tc_st32(a_bufs + g * 64 + 32, lo);
+            tc_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_afull(g));
+        }
+        nrm_s[cset][row] = (nrm4[0] + nrm4[1]) + (nrm4[2] + nrm4[3]);
+    } else if (warp >= 12) {
+        // ------------------------------------------------------------------ drains
+        const int quad = warp & 3;
+        const int row = quad * 32 + lane;
+        const int h = row >> 6;                       // which half's columns are meaningful in this lane
+        const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+        float acc[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) acc[j] = 0.f;
+        for (int fl = 0; fl < n_flush; ++fl) {
+            const int set = fl & 1;
+            if (!mbar_wait(bar_dfull(set), ((uint32_t)fl >> 1) & 1, abortp)) break;
+            tc_fence_after();
+            const uint32_t d = tmem + lane_addr + set * set_cols + h * 3 * n_pad;
+#pragma unroll
+            for (int j0 = 0; j0 < 32; j0 += 16) {
+                if (j0 >= n_pad) break;
+                uint32_t big[16], s1[16], s2[16];
+                tc_ld16(d + j0, big);                           // v_hi a_hi
+                tc_ld16(d + n_pad + j0, s1);                    // v_hi a_lo
+                tc_ld16(d + 2 * n_pad + j0, s2);                // v_lo a_hi
+                tc_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    acc[j0 + j] += __uint_as_float(big[j]) + (__uint_as_float(s1[j]) + __uint_as_float(s2[j]));
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_dempty(set));
+        }
+#pragma unroll
+        for (int j = 0; j < 32; ++j) res[row][j] = acc[j];
+    }
+
+    // ---------------------------------------------------------------------- teardown and the slab
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (tid == 0 && abort_flag) {
+        for (int s = 0; s < n_stages; ++s)
+            if (issued[s] > 0) {
+                for (uint32_t i = 0; i < kSpinLimit; ++i) {
+                    if (mbar_try_wait(bar_full(s), (uint32_t)(issued[s] - 1) & 1)) break;
+                    __nanosleep(64);
+                }
+            }
+        atomicMax(a.status, 1);
+    }
+    // slab [m+1][n_r+1]: row 0 = A x, row 1+c = A v_c^T (both halves of the k-range), last column = sum of squares
+    const int stride = a.n_r + 1;
+    float *slab = a.part + (int64_t)blockIdx.x * (a.m + 1) * stride;
+    for (int t = tid; t < (a.m + 1) * stride; t += kQThreads) {
+        const int r = t / stride, j = t - r * stride;
+        float v;
+        if (r == 0) {
+            v = j < a.n_r ? z0_s[j] : 0.f;
+        } else {
+            const int c = r - 1;
+            v = j < a.n_r ? res[c][j] + res[c + kHalfRows][j]
+                          : (nrm_s[0][c] + nrm_s[1][c]) + (nrm_s[0][c + kHalfRows] + nrm_s[1][c + kHalfRows]);
+        }
+        slab[t] = v;
+    }
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kQTmemCols) : "memory");
+    }
+}
+
+}  // namespace
+
+// Rows a TMA box can step through (16-byte multiples), at most 64 candidates (one half tile) and
+// 32 samples.
+bool lsq_tc_usable(const LsqArgs &a, bool aligned) {
+    return aligned && a.m >= 1 && a.m <= kHalfRows && a.n_r >= 1 && a.n_r <= 32 && a.d % 4 == 0 && a.ldv % 4 == 0 &&
+           a.d >= 4096 && encode_tiled_fn() != nullptr;
+}
+
+// Fills a.part with one slab per block; *slabs = the number of slabs written.
+cudaError_t launch_lsq_tc(Context &c, const LsqArgs &a, int max_slabs, int *slabs, cudaStream_t s) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return cudaErrorNotSupported;
+    const int n_pad = a.n_r <= 16 ? 16 : 32;
+    CUtensorMap map_v, map_a, map_x;
+    cuuint32_t ones[3] = {1, 1, 1};
+    {
+        cuuint64_t dims[3] = {(cuuint64_t)a.d, (cuuint64_t)a.m, 1};
+        cuuint64_t strides[2] = {(cuuint64_t)a.ldv * 4, (cuuint64_t)a.ldv * 4 * (cuuint64_t)a.m};
+        cuuint32_t box[3] = {kQBlockK, kHalfRows, 1};
+        if (enc(&map_v, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(a.V), dims, strides, box, ones,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
+    {
+        cuuint64_t dims[3] = {(cuuint64_t)a.d, (cuuint64_t)a.n_r, 1};
+        cuuint64_t strides[2] = {(cuuint64_t)a.d * 4, (cuuint64_t)a.d * 4 * (cuuint64_t)a.n_r};
+        cuuint32_t box[3] = {kQBlockK, (cuuint32_t)n_pad, 1};
+        if (enc(&map_a, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(a.A), dims, strides, box, ones,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
+    {
+        cuuint64_t dims[3] = {(cuuint64_t)a.d, 1, 1};
+        cuuint64_t strides[2] = {(cuuint64_t)a.d * 4, (cuuint64_t)a.d * 4};
+        cuuint32_t box[3] = {kQBlockK, 1, 1};
+        if (enc(&map_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(a.x), dims, strides, box, ones,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
+    const int64_t n_kblocks = (a.d + kQBlockK - 1) / kQBlockK;
+    int blocks = c.sm_count > 0 ? c.sm_count : 148;
+    if (blocks > max_slabs) blocks = max_slabs;
+    if ((int64_t)blocks > (n_kblocks + 1) / 2) blocks = (int)((n_kblocks + 1) / 2);
+    LsqTcArgs t;
+    t.m = a.m;
+    t.n_r = a.n_r;
+    t.n_pad = n_pad;
+    t.nkb = (int)((n_kblocks + 2 * (int64_t)blocks - 1) / (2 * (int64_t)blocks));
+    const int stage_bytes = lsq_stage_bytes(n_pad);
+    t.stages = (kQSmem - 1024) / stage_bytes;
+    if (t.stages > kQMaxStages) t.stages = kQMaxStages;
+    t.n_abufs = (kQTmemCols - 2 * 6 * n_pad) / 64;
+    if (t.n_abufs > kQMaxABufs) t.n_abufs = kQMaxABufs;
+    t.part = a.part;
+    t.status = c.dev_status;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(lsq_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kQSmem);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    *slabs = blocks;
+    return launch_chained(lsq_tc_kernel, dim3(blocks), dim3(kQThreads), (size_t)t.stages * stage_bytes + 1024, s,
+                          chain_launches(c), map_v, map_a, map_x, t);
+}
+
+}  // namespace zeno

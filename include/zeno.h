@@ -203,6 +203,11 @@ int32_t zeno_last_launch_count(zeno_handle h);
 /* The cudaError_t (as int) behind the most recent ZENO_ERR_CUDA on this handle. */
 int32_t zeno_last_cuda_error(zeno_handle h);
 
+/* Which device-side wait was behind the most recent ZENO_ERR_TIMEOUT on this handle (0 if none): the
+ * kernel in bits 24-27 (1 first-layer stream, 2 layer, 3 least squares), the index of the barrier in
+ * that kernel's barrier array in bits 1-16, the awaited phase parity in bit 0.  For bug reports. */
+int32_t zeno_last_wait_code(zeno_handle h);
+
 const char *zeno_status_string(zeno_status s);
 
 #ifdef __cplusplus

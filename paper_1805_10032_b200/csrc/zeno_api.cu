@@ -575,6 +575,7 @@ zeno_status zeno_step_host(zeno_handle h, const void *x, const void *V, int64_t 
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return fail_cuda(h, e);
     h->last_launches = launches;
+    if (dev_status) h->last_wait_code = dev_status;
     return dev_status ? ZENO_ERR_TIMEOUT : ZENO_OK;
 }
 
@@ -587,6 +588,7 @@ zeno_status zeno_device_status(zeno_handle h, void *stream) {
     cudaError_t e = cudaMemcpyAsync(&dev_status, h->dev_status, sizeof(int), cudaMemcpyDeviceToHost, s);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return fail_cuda(h, e);
+    if (dev_status) h->last_wait_code = dev_status;
     return dev_status ? ZENO_ERR_TIMEOUT : ZENO_OK;
 }
 
@@ -635,6 +637,8 @@ int32_t zeno_profile_read(zeno_handle h, int32_t back, float *ms, const char **n
 int32_t zeno_last_launch_count(zeno_handle h) { return h ? h->last_launches : 0; }
 
 int32_t zeno_last_cuda_error(zeno_handle h) { return h ? h->last_cuda_error : 0; }
+
+int32_t zeno_last_wait_code(zeno_handle h) { return h ? h->last_wait_code : 0; }
 
 const char *zeno_status_string(zeno_status s) {
     switch (s) {

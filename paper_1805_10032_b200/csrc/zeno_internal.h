@@ -58,6 +58,7 @@ struct Context {
     size_t host_stage_bytes;
     int last_launches;
     int last_cuda_error;
+    int last_wait_code;             // status word read back after a kernel gave up on a bounded wait
     // optional per-kernel timing (zeno_profile): a ring of the last kProfileDepth calls; in a
     // call's slot events[i] is recorded before kernel i and events[n] after the last one
     bool chain;                     // chain a step's kernels with programmatic dependent launch

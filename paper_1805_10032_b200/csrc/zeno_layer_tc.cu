@@ -397,7 +397,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                     __nanosleep(64);
                 }
             }
-        atomicMax(a.status, 1);
+        atomicCAS(a.status, 0, wait_code(2, abort_flag, smem_u32(bars)));   // the first block to give up is kept
     }
     __syncthreads();
     if (warp == 1) {

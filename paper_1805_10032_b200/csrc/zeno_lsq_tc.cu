@@ -313,7 +313,7 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
                     __nanosleep(64);
                 }
             }
-        atomicMax(a.status, 1);
+        atomicCAS(a.status, 0, wait_code(3, abort_flag, smem_u32(bars)));   // the first block to give up is kept
     }
     // slab [m+1][n_r+1]: row 0 = A x, row 1+c = A v_c^T (both halves of the k-range), last column = sum of squares
     const int stride = a.n_r + 1;

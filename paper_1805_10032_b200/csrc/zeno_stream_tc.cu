@@ -403,7 +403,7 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                             __nanosleep(64);
                         }
                     }
-            atomicMax(a.status, 1);
+            atomicCAS(a.status, 0, wait_code(1, abort_flag, smem_u32(bars)));   // the first block to give up is kept
         }
     }
     __syncthreads();

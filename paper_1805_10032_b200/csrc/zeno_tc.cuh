@@ -31,15 +31,24 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false if it gave up (and raises *abort_flag) or if another thread did.
+// Bounded wait.  Returns false if it gave up or if another thread did.  The thread that gives up
+// leaves in *abort_flag which wait it was: bit 30, the parity in bit 20, the barrier's shared-memory
+// address in the low 20 bits (wait_code() turns that into the word the host reads).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if (i > 32) __nanosleep(40);
         if ((i & 127u) == 127u && *abort_flag) return false;
     }
-    *abort_flag = 1;
+    *abort_flag = (int)(0x40000000u | ((parity & 1u) << 20) | (bar & 0xfffffu));
     return false;
+}
+// Status word of a block that gave up: kernel id (1 first-layer stream, 2 layer, 3 least squares) in
+// bits 24-27, the index of the barrier within the block's barrier array in bits 1-16, the awaited
+// parity in bit 0.  Never zero.
+__device__ __forceinline__ int wait_code(int kernel_id, int flag, uint32_t bars_base) {
+    const uint32_t index = (((uint32_t)flag & 0xfffffu) - (bars_base & 0xfffffu)) >> 3;
+    return (kernel_id << 24) | (int)((index & 0xffffu) << 1) | ((flag >> 20) & 1);
 }
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int c0, int c1, int c2,
                                             uint32_t bar) {

@@ -28,7 +28,7 @@ EXPORTS = (
     "zeno_aggregate", "zeno_step", "zeno_step_host", "zeno_device_status", "zeno_score_lsq_static",
     "zeno_profile", "zeno_profile_read",
     "zeno_last_launch_count",
-    "zeno_last_cuda_error", "zeno_status_string",
+    "zeno_last_cuda_error", "zeno_last_wait_code", "zeno_status_string",
 )
 
 
@@ -91,6 +91,8 @@ def load_library() -> ctypes.CDLL:
     lib.zeno_last_launch_count.argtypes = [vp]
     lib.zeno_last_cuda_error.restype = i32
     lib.zeno_last_cuda_error.argtypes = [vp]
+    lib.zeno_last_wait_code.restype = i32
+    lib.zeno_last_wait_code.argtypes = [vp]
     lib.zeno_status_string.restype = ctypes.c_char_p
     lib.zeno_status_string.argtypes = [i32]
     _lib = lib
@@ -173,6 +175,8 @@ class Zeno:
             detail = ""
             if st == ERR_CUDA:
                 detail = f" [cudaError {self._lib.zeno_last_cuda_error(self._h)}]"
+            if st == ERR_TIMEOUT:
+                detail = f" [wait code {self._lib.zeno_last_wait_code(self._h):#x}]"
             raise ZenoError(st, what, detail)
 
     def _batch(self, features: torch.Tensor, targets: torch.Tensor) -> Batch:

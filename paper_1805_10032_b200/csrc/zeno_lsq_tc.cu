@@ -6,11 +6,11 @@
 // squares of the rows of V.  All three operands are streamed from HBM exactly once; a block owns a
 // contiguous range of k and leaves its partial sums in a slab that lsq_finish_kernel adds up in double.
 //
-// A tile of the MMA has 128 rows but there are at most 64 candidates, so a block works on TWO halves of
-// its k-range at once: TMEM lanes 0-63 hold the candidates' entries of a k-block of the first half,
-// lanes 64-127 those of the matching k-block of the second half.  Each k-block takes two groups of MMAs
-// on the same A operand, one against the first half's rows of A (whose result is meaningful in lanes
-// 0-63), one against the second half's (lanes 64-127), into different accumulator columns.
+// A tile of the MMA has 128 rows but there are at most 64 candidates, so a block works on TWO neighbouring
+// k-blocks at once (every row of V, A and x is then read 256 contiguous bytes at a time): TMEM lanes 0-63
+// hold the candidates' entries of the even k-block, lanes 64-127 those of the odd one.  Each pair takes two
+// groups of MMAs on the same A operand, one against the even k-block's rows of A (whose result is meaningful
+// in lanes 0-63), one against the odd one's (lanes 64-127), into different accumulator columns.
 //
 // fp32 accuracy on tf32 tensor cores as in the first-layer stream: both operands are split,
 // a = a_hi + a_lo, and a_hi b_hi + a_hi b_lo + a_lo b_hi is accumulated, the small products in columns of
@@ -46,7 +46,7 @@ constexpr int kFlush = 32;                  // k-blocks accumulated in TMEM befo
 
 struct LsqTcArgs {
     int m, n_r, n_pad;                      // n_pad: 16 or 32
-    int nkb;                                // k-blocks per half of a block's k-range
+    int nkb;                                // pairs of k-blocks in a block's k-range
     int stages, n_abufs;
     float *part;                            // [blocks][m+1][n_r+1]
     int *status;
@@ -140,7 +140,7 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
                     const int h = w & 1, what = w >> 1;
                     const CUtensorMap *map = what == 0 ? &map_v : what == 1 ? &map_a : &map_x;
                     const uint32_t off = what == 0 ? h * kVHalfBytes : what == 1 ? off_raw + h * raw_bytes : off_x + h * 128;
-                    const int64_t k = (kb0 + (int64_t)h * nkb + kb) * kQBlockK;
+                    const int64_t k = (kb0 + 2 * (int64_t)kb + h) * kQBlockK;     // neighbouring k-blocks: 256 contiguous bytes of every row
                     tma_load_3d(dst + off, map, (int)k, 0, 0, bar_full(s));
                 }
             }

@@ -347,10 +347,13 @@ def run_ours(args, rank, world, local_rank):
     for k in kern:
         name = k["kernel"].split(":")[1]
         if name in ("stream_tf32x3", "layer_tc", "mlp_layer", "mlp_layer_mma", "mlp_head_loss_tail"):
-            layer_of[k["kernel"]] = layer
+            layer_of[k["kernel"]] = [layer]
             layer += 1
+        elif name == "layer_tc_head":           # a hidden layer with the small last layer folded in
+            layer_of[k["kernel"]] = [layer, layer + 1]
+            layer += 2
     if top["kernel"] in layer_of:
-        top_bytes = layer_bytes(w0, layer_of[top["kernel"]])
+        top_bytes = sum(layer_bytes(w0, l) for l in layer_of[top["kernel"]])
     elif top_name in ("lsq_stream", "lsq_tc"):
         top_bytes = score_b
     elif top_name == "aggregate":

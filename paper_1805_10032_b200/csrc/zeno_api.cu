@@ -157,11 +157,23 @@ zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv,
         // split-K partials to fill the SMs; with enough whole tiles for every SM this kernel wins
         return (m + 1) * ((out_l + 127) / 128) >= 2 * c->sm_count;
     };
+    // the layer before a small last layer takes that layer, the loss and the tail along
+    auto head_folds_into = [&](int l) {
+        if (l + 2 != L || c->head_zpart == nullptr || classes > zeno::kHeadMaxClasses || !layer_tc_serves(l)) return false;
+        if (c->desc.dims[l] < 128) return false;     // at least two k-blocks: both converter sets take part in every tile
+        // measured: the finish costs each tile about 9 us of its epilogue warps' time (two rounds of
+        // fence, ticket and reads); that is cheaper than a further launch while every block has one
+        // tile, and dearer once blocks take several tiles in a row
+        if ((m + 1) * ((int)((c->desc.dims[l + 1] + 127) / 128)) > c->sm_count) return false;
+        return !(l == 0 && c->desc.param_dtype == ZENO_F32 && c->tc_part != nullptr);      // not the linear first layer
+    };
     bool have_split = false;               // the previous layer left its output in the stacked form
     for (int l = 0; l < L; ++l) {
         const int in_l = (int)c->desc.dims[l], out_l = (int)c->desc.dims[l + 1];
         const bool last_fused = (l + 1 == L) && fuse_loss;
         if (layer_tc_serves(l)) {
+            const bool with_head = head_folds_into(l);
+            zeno::HeadFuse hf;
             void *hs_in = c->act_split[(l + 1) & 1];
             if (!have_split) {
                 const float *plain = l == 0 ? batch->features : c->act[(l - 1) & 1];
@@ -190,8 +202,31 @@ zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv,
             t.relu = l + 1 < L;
             t.gamma = gamma;
             t.np_base = c->np_base[l];
+            t.head = nullptr;
+            tail.used.base[l] = c->np_base[l];
+            tail.used.count[l] = zeno::layer_tc_norm_slots(out_l);
+            if (with_head) {
+                tail.used.base[l + 1] = c->np_base[l + 1];
+                tail.used.count[l + 1] = zeno::layer_tc_head_slots(out_l);
+                hf.classes = classes;
+                hf.offW = c->offW[l + 1];
+                hf.offB = c->offB[l + 1];
+                hf.zpart = c->head_zpart;
+                hf.model_ticket = c->head_tickets;
+                hf.labels = static_cast<const int32_t *>(batch->targets);
+                hf.losses = loss_buf;
+                hf.np_base = c->np_base[l + 1];
+                hf.tail = tail;                          // complete: this is the last launch of the pass
+                t.head = &hf;
+                t.Hout = nullptr;
+                t.Hsplit_out = nullptr;
+            }
             e = zeno::launch_layer_tc(*c, t, s, launches);
             if (e != cudaSuccess) return fail_cuda(c, e);
+            if (with_head) {
+                *ranked = keep > 0;
+                return ZENO_OK;
+            }
             if (t.linear) {
                 zeno::StreamTcPlan one;
                 one.R = 1;
@@ -335,6 +370,7 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
 
     const size_t rows = (size_t)m_max + 1;
     size_t act_elems = 0, norm_elems = 0, lsq_elems = 0, tc_elems = 0, ticket_elems = 1, split_elems = 0;
+    size_t head_elems = 0;
     if (desc->kind == ZENO_LOSS_SOFTMAX_MLP) {
         int64_t off = 0, widest = 0;
         int slots = 0;
@@ -370,6 +406,15 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
                 const size_t raw = rows * (size_t)n_r_max * (size_t)o;
                 if (l == 0 && desc->param_dtype == ZENO_F32 && raw > tc_elems) tc_elems = raw;
             }
+            // a small last layer may be folded into a tensor-core layer before it: partial logits and
+            // norm partials per (128-row tile of that layer, epilogue warp)
+            if (l >= 1 && l + 1 == desc->n_layers && o <= zeno::kHeadMaxClasses && !getenv("ZENO_DISABLE_TENSOR_CORES") &&
+                zeno::layer_tc_usable((zeno_dtype)desc->param_dtype, (int)desc->dims[l - 1], (int)in,
+                                      n_r_max < 128 ? n_r_max : 128)) {
+                const int hs = zeno::layer_tc_head_slots((int)in);
+                if (hs > layer_slots) layer_slots = hs;
+                head_elems = rows * (size_t)(hs / 4) * zeno::kHeadMaxClasses * (size_t)zeno::layer_tc_n_pad(n_r_max < 128 ? n_r_max : 128);
+            }
             slots += layer_slots;
             if (o > widest) widest = o;
         }
@@ -395,6 +440,7 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
     const size_t at_tickets = reserve(ticket_elems, 4);
     const size_t at_split0 = reserve(split_elems, 4), at_split1 = reserve(split_elems, 4);
     const size_t at_losspart = reserve(rows * 8, 4);
+    const size_t at_headz = reserve(head_elems, 4), at_headt = reserve(rows, 4);
 
     e = cudaMalloc(&c->arena, bytes);
     if (e != cudaSuccess) {
@@ -417,8 +463,11 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
     c->loss_part = reinterpret_cast<float *>(base + at_losspart);
     c->act_split[0] = base + at_split0;
     c->act_split[1] = base + at_split1;
+    c->head_zpart = head_elems ? reinterpret_cast<float *>(base + at_headz) : nullptr;
+    c->head_tickets = reinterpret_cast<unsigned *>(base + at_headt);
     e = cudaMemset(c->dev_status, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(c->tickets, 0, ticket_elems * sizeof(unsigned));
+    if (e == cudaSuccess) e = cudaMemset(c->head_tickets, 0, rows * sizeof(unsigned));
     if (e != cudaSuccess) {
         cudaFree(c->arena);
         delete c;

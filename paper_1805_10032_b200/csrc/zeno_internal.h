@@ -54,6 +54,8 @@ struct Context {
     int tc_r_max;                   // most k-ranges any plan for it may use
     float *tc_part;                 // [R][m_max+1][n_r_max][dims[1]] split-K partials
     unsigned *tickets;              // the tail's arrival counter, zero between launches
+    float *head_zpart;              // partial logits of a last layer folded into the layer before it, or NULL
+    unsigned *head_tickets;         // [m_max + 1] per-model arrival counters of that mode, zero between launches
     void *host_stage;               // device copies of host inputs (zeno_step_host), grown on demand
     size_t host_stage_bytes;
     int last_launches;
@@ -163,6 +165,25 @@ cudaError_t launch_stream_combine(Context &c, const StreamTcPlan &p, const float
                                   const float *V, int64_t ldv, int64_t offB, int out, int n_r, int m,
                                   float gamma, int relu, float *H, float *Hsplit, cudaStream_t s, int *launches);
 
+// A small last layer (at most kHeadMaxClasses outputs) folded into the tensor-core layer before it:
+// that layer's epilogue multiplies its activations, still in registers, against the last layer's
+// weights and leaves per-tile partial logits; the block that completes a model (a ticket per
+// model) adds them up and takes the cross-entropy, and the block that completes the last model
+// runs the scoring tail.  Neither the hidden activations nor the logits of that pair of layers
+// are written out in full, and no further kernel is launched.
+constexpr int kHeadMaxClasses = 16;
+struct HeadFuse {
+    int classes;             // outputs of the last layer; 0: not fused
+    int64_t offW, offB;      // element offsets of its weights [classes][out] and bias (-1: none)
+    float *zpart;            // [m+1][tiles][kHeadMaxClasses][n_pad] partial logits, one set per 128-row tile
+    unsigned *model_ticket;  // [m+1], zero between launches
+    const int32_t *labels;
+    float *losses;           // [m+1]
+    int np_base;             // first norm-partial slot of the last layer (one per tile and epilogue warp)
+    TailArgs tail;
+};
+int layer_tc_head_slots(int out);
+
 // Dense layer on the tensor cores with both operands streamed (any layer of a bfloat16 model, the
 // later layers of an fp32 model).  Its input activations come as the two-term stacked operand
 // [models][2 n_pad][K] that launch_split_acts, or a preceding layer of this kind, writes.
@@ -178,6 +199,7 @@ struct LayerTcLaunch {
     int relu;
     float gamma;
     int np_base;
+    const HeadFuse *head;    // the last layer folded in (Hout and Hsplit_out are then unused), or NULL
 };
 bool layer_tc_usable(zeno_dtype dtype, int K, int out, int n_r);
 int layer_tc_n_pad(int n_r);

@@ -24,7 +24,17 @@
 // 12-15 epilogue.  Accumulator sets alternate between consecutive tiles when two fit in TMEM, so
 // a tile is drained while the next one is accumulated.  Every mbarrier wait is bounded; a wait that
 // gives up raises a status word and the block leaves through the common teardown.
+//
+// HEAD mode (the layer before a small last layer): the epilogue thread of output row o holds that
+// row's activations of all samples in registers, so it multiplies them against column o of the
+// last layer's weights (formed as x - gamma v on the spot, v^2 accumulated); the four epilogue
+// warps add their 128 rows up through shared memory and leave one set of partial logits per tile.
+// The epilogue group then takes a ticket for the model: the group that completes a model sums the
+// tiles' partial logits in tile order, takes the cross-entropy and the candidate's norm total, and
+// takes the pass's ticket; the block that completes the last model forms the scores and the
+// ranking after its teardown.  All of it runs beside the main loop of the block's next tile.
 #include "zeno_internal.h"
+#include "zeno_tail.cuh"
 #include "zeno_tc.cuh"
 
 namespace zeno {
@@ -78,13 +88,112 @@ struct LayerTcArgs {
     float *normpart;
     int np_slots, np_base;
     int *status;
+    HeadFuse head;         // used by the HEAD instantiations only
 };
 
-// LINEAR (fp32 first layer): the layer is linear in its weights and every model reads the same
-// activations, so the tile of model c is the raw rows of v_c (of x for model 0): no x tile is fetched
-// for the candidates, the epilogue writes the raw products H v_c^T, and the combine kernel forms
-// z_c = z_0 - gamma (H v_c^T + b(v_c)).
-template <typename T, bool LINEAR>
+// Sum over the 32 lanes of each of 32 per-lane values; lane j ends up with the total of value j
+// (recursive halving: 31 shuffles).
+__device__ __forceinline__ float lane_transpose_sum32(float (&v)[32], int lane) {
+#pragma unroll
+    for (int s = 16; s >= 1; s >>= 1) {
+        const bool upper = (lane & s) != 0;
+#pragma unroll
+        for (int i = 0; i < s; ++i) {
+            const float send = upper ? v[i] : v[i + s];
+            const float keep = upper ? v[i + s] : v[i];
+            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, s);
+        }
+    }
+    return v[0];
+}
+
+constexpr int kEpiThreads = 128;            // the four epilogue warps
+constexpr int kEpiBarrier = 1;              // their named barrier
+
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync %0, %1;" ::"n"(kEpiBarrier), "n"(kEpiThreads) : "memory"); }
+// true iff `ok` holds in every thread of the epilogue group (a barrier as well)
+__device__ __forceinline__ bool epi_all(bool ok) {
+    uint32_t r;
+    asm volatile(
+        "{\n.reg .pred p, q;\nsetp.ne.b32 p, %1, 0;\n"
+        "bar.red.and.pred q, %2, %3, p;\nselp.u32 %0, 1, 0, q;\n}\n"
+        : "=r"(r) : "r"((uint32_t)ok), "n"(kEpiBarrier), "n"(kEpiThreads) : "memory");
+    return r != 0;
+}
+
+// HEAD mode, the 128 threads of the epilogue group that completed `model` (g = thread within the
+// group): the model's logits from the tiles' partial sums in tile order plus the last layer's bias;
+// then one warp takes the mean cross-entropy into losses[model] while another adds up the
+// candidate's norm partials of all layers.  `zl` is group-shared scratch of classes x n_pad floats.
+template <typename T>
+__device__ __forceinline__ void head_finish_model(const LayerTcArgs &a, int model, float *zl, int g) {
+    const HeadFuse &h = a.head;
+    const int n_pad = a.n_pad, lane = g & 31, gw = g >> 5;
+    const float *zp = h.zpart + (int64_t)model * a.tiles * kHeadMaxClasses * n_pad;
+    for (int t = g; t < h.classes * n_pad; t += kEpiThreads) {
+        const int cls = t / n_pad, j = t - cls * n_pad;
+        const float *src = zp + (int64_t)cls * n_pad + j;
+        const int64_t tstride = (int64_t)kHeadMaxClasses * n_pad;
+        float z = 0.f;
+        for (int t0 = 0; t0 < a.tiles; t0 += 4) {          // four loads in flight, added in tile order
+            float part[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) part[u] = t0 + u < a.tiles ? __ldcg(src + (t0 + u) * tstride) : 0.f;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) z += part[u];
+        }
+        if (h.offB >= 0) {
+            const float bv = model > 0 ? load_elem(static_cast<const T *>(a.V) + (int64_t)(model - 1) * a.ldv + h.offB + cls) : 0.f;
+            z += candidate_param<T>(load_elem(static_cast<const T *>(a.xparams) + h.offB + cls), bv, a.gamma);
+        }
+        zl[cls * n_pad + j] = z;
+    }
+    epi_sync();
+    if (gw == 0) {
+        float l = 0.f;
+        for (int j = lane; j < a.n_r; j += 32) {
+            float zmax = -INFINITY;
+            for (int o = 0; o < h.classes; ++o) zmax = fmaxf(zmax, zl[o * n_pad + j]);
+            float se = 0.f;
+            for (int o = 0; o < h.classes; ++o) se += expf(zl[o * n_pad + j] - zmax);   // a NaN logit makes se NaN
+            int lab = h.labels[j];
+            if (lab < 0 || lab >= h.classes) lab = 0;
+            l += zmax + logf(se) - zl[lab * n_pad + j];
+        }
+#pragma unroll
+        for (int sft = 16; sft >= 1; sft >>= 1) l += __shfl_xor_sync(0xffffffffu, l, sft);
+        if (lane == 0) {
+            h.losses[model] = l / (float)a.n_r;
+            __threadfence();
+        }
+    } else if (gw == 1 && model > 0) {
+        // the candidate's ||v||^2: the partial sums of every layer, eight loads per lane in flight
+        float nv = 0.f;
+        for (int l = 0; l < h.tail.used.layers; ++l) {
+            const float *src = h.tail.normpart + (int64_t)(model - 1) * h.tail.np_slots + h.tail.used.base[l];
+            const int count = h.tail.used.count[l];
+            for (int s0 = 0; s0 < count; s0 += 256) {
+                float v[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int sl = s0 + u * 32 + lane;
+                    v[u] = sl < count ? __ldcg(src + sl) : 0.f;
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) nv += v[u];
+            }
+        }
+#pragma unroll
+        for (int sft = 16; sft >= 1; sft >>= 1) nv += __shfl_xor_sync(0xffffffffu, nv, sft);
+        if (lane == 0) {
+            h.tail.norm_tot[model - 1] = nv;
+            __threadfence();
+        }
+    }
+    epi_sync();
+}
+
+template <typename T, bool LINEAR, bool HEAD>
 __global__ void __launch_bounds__(kLThreads, 1)
 layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_v,
                 const __grid_constant__ CUtensorMap map_h, LayerTcArgs a) {
@@ -99,6 +208,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
     __shared__ int issued[kLMaxStages];
+    __shared__ int head_last;                  // HEAD: the epilogue group's ticket result
+    __shared__ int head_final;                 // HEAD: this block completed the last model
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
@@ -115,6 +226,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     const int a_base = n_sets * acc_cols;                       // TMEM: accumulator sets, then the A buffers
     const float inv_stages = 1.0f / (float)n_stages, inv_abufs = 1.0f / (float)n_abufs;
     uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    // HEAD: behind the ring, the epilogue warps' partial logits [4][classes rounded up to even][n_pad]
+    float *zq = reinterpret_cast<float *>(ring + (size_t)n_stages * stage_bytes);
 
     auto bar_full = [&](int s) { return smem_u32(&bars[s]); };
     auto bar_empty = [&](int s) { return smem_u32(&bars[kLMaxStages + s]); };
@@ -132,6 +245,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
 
     if (tid == 0) {
         abort_flag = 0;
+        head_final = 0;
         for (int s = 0; s < kLMaxStages; ++s) {
             mbar_init(bar_full(s), 1);
             mbar_init(bar_empty(s), 5);        // the four warps of a converter set and the MMAs' commit
@@ -247,6 +361,23 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         const uint32_t a_bufs = tmem + ((uint32_t)(quad * 32) << 16) + a_base;
         uint32_t it0 = 0;
         int model, tile;
+        // partial sum of squares of this tile's rows (model 0 is x itself: not a candidate)
+        auto store_norm = [&](const float (&n4)[4]) {
+            if (model > 0) {
+                float nrm = (n4[0] + n4[1]) + (n4[2] + n4[3]);
+                const int o = tile * kRows + row;
+                if (cset == 0 && a.offB >= 0 && o < a.out) {
+                    const float bv = load_elem(static_cast<const T *>(a.V) + (int64_t)(model - 1) * a.ldv + a.offB + o);
+                    nrm = fmaf(bv, bv, nrm);
+                }
+#pragma unroll
+                for (int sft = 16; sft >= 1; sft >>= 1) nrm += __shfl_xor_sync(0xffffffffu, nrm, sft);
+                if (lane == 0) {
+                    a.normpart[(int64_t)(model - 1) * a.np_slots + a.np_base + (tile * 4 + quad) * 2 + cset] = nrm;
+                    if (HEAD) __threadfence();
+                }
+            }
+        };
         for (int li = 0; get_item(li, model, tile) && !*abortp; ++li, it0 += nkb) {
             float nrm4[4] = {0.f, 0.f, 0.f, 0.f};
             bool ok = true;
@@ -293,6 +424,9 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                         }
                     }
                 }
+                // HEAD: the norm partial must be in global memory before the epilogue group takes the
+                // model's ticket, so it is written ahead of the set's last A buffer of the tile
+                if (HEAD && kb + 2 >= nkb) store_norm(nrm4);
                 if (!mbar_wait(bar_aempty(g), (around & 1) ^ 1, abortp)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t a_tmem = a_bufs + g * Tr::kACols;
@@ -304,19 +438,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 if (lane == 0) mbar_arrive(bar_afull(g));
             }
             if (!ok) break;
-            // partial sum of squares of this tile's rows (model 0 is x itself: not a candidate)
-            if (model > 0) {
-                float nrm = (nrm4[0] + nrm4[1]) + (nrm4[2] + nrm4[3]);
-                const int o = tile * kRows + row;
-                if (cset == 0 && a.offB >= 0 && o < a.out) {
-                    const float bv = load_elem(static_cast<const T *>(a.V) + (int64_t)(model - 1) * a.ldv + a.offB + o);
-                    nrm = fmaf(bv, bv, nrm);
-                }
-#pragma unroll
-                for (int sft = 16; sft >= 1; sft >>= 1) nrm += __shfl_xor_sync(0xffffffffu, nrm, sft);
-                if (lane == 0)
-                    a.normpart[(int64_t)(model - 1) * a.np_slots + a.np_base + (tile * 4 + quad) * 2 + cset] = nrm;
-            }
+            if (!HEAD) store_norm(nrm4);          // HEAD: already written (every set has a k-block: K >= 2 k-blocks)
         }
     } else if (warp >= 12) {
         // ------------------------------------------------------------------ epilogue
@@ -324,7 +446,10 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         const int row = quad * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
         int model, tile;
-        for (int li = 0; get_item(li, model, tile) && !*abortp; ++li) {
+        const int g = tid - (kLThreads - kEpiThreads);    // thread within the epilogue group
+        const int cls_even = (a.head.classes + 1) & ~1;
+        // HEAD: the group leaves the loop together (its named barrier needs all four warps)
+        for (int li = 0; get_item(li, model, tile) && (HEAD || !*abortp); ++li) {
             const int set = li % n_sets;
             const uint32_t use = (uint32_t)(li / n_sets);
             const int o = tile * kRows + row;             // thread = output row o, column = sample j
@@ -333,7 +458,34 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 const float vb = model > 0 ? load_elem(static_cast<const T *>(a.V) + (int64_t)(model - 1) * a.ldv + a.offB + o) : 0.f;
                 bias = candidate_param<T>(load_elem(static_cast<const T *>(a.xparams) + a.offB + o), vb, a.gamma);
             }
-            if (!mbar_wait(bar_dfull(set), use & 1, abortp)) break;
+            // HEAD: column o of the last layer's weights for this model, and their share of ||v||^2
+            float w3[kHeadMaxClasses];
+            if (HEAD) {
+                float nrm3 = 0.f;
+                const T *x3 = static_cast<const T *>(a.xparams) + a.head.offW + o;
+                const T *v3 = static_cast<const T *>(a.V) + (int64_t)(model > 0 ? model - 1 : 0) * a.ldv + a.head.offW + o;
+#pragma unroll
+                for (int cls = 0; cls < kHeadMaxClasses; ++cls) {
+                    w3[cls] = 0.f;
+                    if (cls < a.head.classes && o < a.out) {
+                        const float vv = model > 0 ? load_elem(v3 + (int64_t)cls * a.out) : 0.f;
+                        w3[cls] = candidate_param<T>(load_elem(x3 + (int64_t)cls * a.out), vv, a.gamma);
+                        nrm3 = fmaf(vv, vv, nrm3);
+                    }
+                }
+                if (model > 0) {
+                    if (tile == 0 && quad == 0 && a.head.offB >= 0 && lane < a.head.classes) {
+                        const float bv = load_elem(static_cast<const T *>(a.V) + (int64_t)(model - 1) * a.ldv + a.head.offB + lane);
+                        nrm3 = fmaf(bv, bv, nrm3);
+                    }
+#pragma unroll
+                    for (int sft = 16; sft >= 1; sft >>= 1) nrm3 += __shfl_xor_sync(0xffffffffu, nrm3, sft);
+                    if (lane == 0) a.normpart[(int64_t)(model - 1) * a.np_slots + a.head.np_base + tile * 4 + quad] = nrm3;
+                }
+            }
+            bool got = mbar_wait(bar_dfull(set), use & 1, abortp);
+            if (HEAD) got = epi_all(got);
+            if (!got) break;
             tc_fence_after();
             const uint32_t dset = tmem + lane_addr + set * acc_cols;
             for (int j0 = 0; j0 < a.n_pad; j0 += 16) {
@@ -357,7 +509,29 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bar_dempty(set));
                 }
-                if (o < a.out) {
+                if (HEAD) {
+                    // partial logits of this warp's 32 rows: lane l ends up with class cb + l / 16, sample j0 + l % 16
+                    float zz[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        float z = acc[j] + bias;
+                        if (a.relu) z = (z > 0.f || z != z) ? z : 0.f;
+                        zz[j] = (j0 + j < a.n_r) ? z : 0.f;
+                    }
+                    float *zq_w = zq + (int64_t)quad * cls_even * a.n_pad;
+#pragma unroll
+                    for (int cb = 0; cb < kHeadMaxClasses; cb += 2) {
+                        if (cb >= a.head.classes) break;
+                        float pv[32];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            pv[j] = w3[cb] * zz[j];
+                            pv[16 + j] = w3[cb + 1] * zz[j];
+                        }
+                        const float r = lane_transpose_sum32(pv, lane);
+                        zq_w[(cb + (lane >> 4)) * a.n_pad + j0 + (lane & 15)] = r;
+                    }
+                } else if (o < a.out) {
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
                         const int jj = j0 + j;
@@ -381,6 +555,34 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                     }
                 }
             }
+            if (HEAD) {
+                // the four warps' partial logits added in warp order: one set per tile in global memory
+                epi_sync();
+                const int n_out = cls_even * a.n_pad;
+                float *zp = a.head.zpart + ((int64_t)model * a.tiles + tile) * kHeadMaxClasses * a.n_pad;
+                for (int t = g; t < n_out; t += kEpiThreads)
+                    zp[t] = (zq[t] + zq[n_out + t]) + (zq[2 * n_out + t] + zq[3 * n_out + t]);
+                __threadfence();
+                epi_sync();
+                if (g == 0) {
+                    const unsigned tk = atomicAdd(a.head.model_ticket + model, 1u);
+                    head_last = tk == (unsigned)a.tiles - 1;
+                    if (head_last) a.head.model_ticket[model] = 0;       // ready for the next launch
+                }
+                epi_sync();
+                if (head_last) {                       // uniform in the group; rewritten only after the barriers below
+                    __threadfence();
+                    head_finish_model<T>(a, model, zq, g);
+                    if (g == 0) {
+                        const unsigned tk = atomicAdd(a.head.tail.ticket, 1u);
+                        if (tk == (unsigned)a.m) {
+                            *a.head.tail.ticket = 0;
+                            head_final = 1;
+                        }
+                    }
+                }
+                epi_sync();                            // zq and head_last may be reused
+            }
         }
     }
 
@@ -402,6 +604,10 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     __syncthreads();
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kLTmemCols) : "memory");
+    }
+    if (HEAD && head_final) {               // block-uniform: written before the teardown's barrier
+        __threadfence();
+        finalize_and_select(a.head.tail, a.head.losses);
     }
 }
 
@@ -469,7 +675,7 @@ cudaError_t encode_maps(const LayerTcLaunch &l, CUtensorMap *map_x, CUtensorMap 
     return cudaSuccess;
 }
 
-template <typename T, bool LINEAR>
+template <typename T, bool LINEAR, bool HEAD>
 cudaError_t launch_typed(Context &c, const LayerTcLaunch &l, cudaStream_t s) {
     using Tr = TcTraits<T>;
     CUtensorMap map_x, map_v, map_h;
@@ -489,7 +695,11 @@ cudaError_t launch_typed(Context &c, const LayerTcLaunch &l, cudaStream_t s) {
     a.tiles = (l.out + kRows - 1) / kRows;
     a.h_shared = l.h_shared;
     const int stage_bytes = (LINEAR ? 1 : 2) * kTileBytes + 2 * l.n_pad * kRowBytes;
-    a.stages = (kLSmemBudget - 1024) / stage_bytes;
+    // HEAD: the ranking holds 9 KB of static shared memory, and the epilogue warps' partial logits
+    // sit behind the ring
+    const int zq_bytes = HEAD ? 4 * ((l.head->classes + 1) & ~1) * l.n_pad * 4 : 0;
+    const int budget = HEAD ? kLSmemBudget - 10 * 1024 : kLSmemBudget;
+    a.stages = (budget - 1024 - zq_bytes) / stage_bytes;
     if (a.stages > kLMaxStages) a.stages = kLMaxStages;
     const int acc_cols = Tr::kAccPerPad * l.n_pad;
     a.n_sets = 2 * acc_cols + 2 * Tr::kACols <= kLTmemCols ? 2 : 1;
@@ -502,14 +712,10 @@ cudaError_t launch_typed(Context &c, const LayerTcLaunch &l, cudaStream_t s) {
     a.np_slots = c.np_slots;
     a.np_base = l.np_base;
     a.status = c.dev_status;
-    static bool attr_set = false;
+    if (HEAD) a.head = *l.head; else a.head = HeadFuse{};
+    static bool attr_set = false;       // per instantiation
     if (!attr_set) {
-        e = cudaFuncSetAttribute(layer_tc_kernel<float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLSmemBudget);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(layer_tc_kernel<float, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kLSmemBudget);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(layer_tc_kernel<__nv_bfloat16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     kLSmemBudget);
+        e = cudaFuncSetAttribute(layer_tc_kernel<T, LINEAR, HEAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, budget);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
@@ -518,7 +724,7 @@ cudaError_t launch_typed(Context &c, const LayerTcLaunch &l, cudaStream_t s) {
     // equal shares: the fewest blocks that give the same number of rounds as one block per SM
     const int rounds = (items + sms - 1) / sms;
     const int blocks = (items + rounds - 1) / rounds;
-    return launch_chained(layer_tc_kernel<T, LINEAR>, dim3(blocks), dim3(kLThreads), (size_t)a.stages * stage_bytes + 1024, s,
+    return launch_chained(layer_tc_kernel<T, LINEAR, HEAD>, dim3(blocks), dim3(kLThreads), (size_t)a.stages * stage_bytes + 1024 + zq_bytes, s,
                           chain_launches(c), map_x, map_v, map_h, a);
 }
 
@@ -541,12 +747,17 @@ int layer_tc_n_pad(int n_r) { return (n_r + 15) / 16 * 16; }
 // one slot per (tile, warp of a converter set, converter set)
 int layer_tc_norm_slots(int out) { return (out + kRows - 1) / kRows * 8; }
 
+// HEAD mode: partial logits and the last layer's norm partials, one slot per (tile, epilogue warp)
+int layer_tc_head_slots(int out) { return (out + kRows - 1) / kRows * 4; }
+
 cudaError_t launch_layer_tc(Context &c, const LayerTcLaunch &l, cudaStream_t s, int *launches) {
     ++*launches;
-    profile_mark(c, "layer_tc", s);
-    if (c.desc.param_dtype == ZENO_BF16) return launch_typed<__nv_bfloat16, false>(c, l, s);
-    if (l.linear) return launch_typed<float, true>(c, l, s);
-    return launch_typed<float, false>(c, l, s);
+    const bool head = l.head != nullptr && l.head->classes > 0 && !l.linear;
+    profile_mark(c, head ? "layer_tc_head" : "layer_tc", s);
+    if (c.desc.param_dtype == ZENO_BF16)
+        return head ? launch_typed<__nv_bfloat16, false, true>(c, l, s) : launch_typed<__nv_bfloat16, false, false>(c, l, s);
+    if (l.linear) return launch_typed<float, true, false>(c, l, s);
+    return head ? launch_typed<float, false, true>(c, l, s) : launch_typed<float, false, false>(c, l, s);
 }
 
 cudaError_t launch_split_acts(Context &c, const float *H, int models, int n_r, int K, void *out, cudaStream_t s,

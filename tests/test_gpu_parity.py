@@ -42,6 +42,10 @@ SHRUNK = {
     "cfg3_small": (3, dict(dims=(260, 44, 36, 10), m=37, b=15, n_r=70,
                            faults=[(7, "signflip"), (8, "omniscient")])),
     "cfg4_small": (4, dict(dims=(264, 136, 72, 50), m=9, b=3, n_r=19, faults=[(3, "signflip")])),
+    # a small last layer folded into the tensor-core layer before it, bfloat16 and fp32 (ragged tiles,
+    # several tiles per model, an odd number of classes)
+    "cfg4_ten_classes": (4, dict(dims=(264, 136, 200, 10), m=9, b=3, n_r=19, faults=[(3, "signflip")])),
+    "cfg2_seven_classes": (2, dict(dims=(520, 200, 300, 7), n_r=30, m=12, b=5, faults=[(5, "noise200")])),
     "cfg5_small": (5, dict(d=70000, m=13, b=5, n_r=16, n_noise=5)),
     "cfg5_nr5": (5, dict(d=33333 * 4, m=70, b=30, n_r=5, n_noise=30)),
     "cfg5_nr40": (5, dict(d=9000, m=6, b=2, n_r=40, n_noise=2)),
@@ -67,7 +71,8 @@ def kernels_of_a_step(w):
 
 
 @pytest.mark.parametrize("name,expected", [
-    ("cfg2_mid_layers", ["stream_tf32x3", "stream_combine", "layer_tc", "mlp_head_loss_tail", "aggregate"]),
+    ("cfg2_mid_layers", ["stream_tf32x3", "stream_combine", "layer_tc_head", "aggregate"]),
+    ("cfg4_ten_classes", ["split_acts", "layer_tc", "layer_tc_head", "aggregate"]),
     ("cfg3_many_tiles", ["split_acts", "layer_tc", "stream_combine", "mlp_head_loss_tail", "aggregate"]),
     ("cfg4_128_samples", ["split_acts", "layer_tc", "layer_tc", "layer_tc", "mlp_loss_tail", "aggregate"]),
     ("cfg4_small", ["split_acts", "layer_tc", "layer_tc", "layer_tc", "mlp_loss_tail", "aggregate"]),

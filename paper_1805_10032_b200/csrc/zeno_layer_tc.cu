@@ -45,11 +45,19 @@ constexpr int kRows = 128;                  // weight rows per tile = TMEM lanes
 constexpr int kRowBytes = 128;              // bytes of a row per k-block = one swizzle row
 constexpr int kTileBytes = kRows * kRowBytes;
 constexpr int kLThreads = 32 * 16;
-constexpr int kLMaxStages = 6;
+constexpr int kLMaxStages = 12;               // weight ring (x and v tiles)
+constexpr int kLMaxBStages = 6;               // activation ring
 constexpr int kLMaxABufs = 8;
 constexpr int kLMaxSets = 2;
 constexpr int kLSmemBudget = 226 * 1024;
 constexpr int kLTmemCols = 512;
+
+// Depth of the activation ring: 96 KB worth of stages, three to six (measured: a copy from L2 takes
+// two to three microseconds under load, and the MMAs consume a stage in well under one).
+inline int layer_tc_b_stages(int n_pad) {
+    const int fit = 96 * 1024 / (2 * n_pad * kRowBytes);
+    return fit < 3 ? 3 : fit > kLMaxBStages ? kLMaxBStages : fit;
+}
 
 template <typename T> struct TcTraits;
 template <> struct TcTraits<float> {
@@ -81,7 +89,7 @@ struct LayerTcArgs {
     int K, out, n_r, n_pad, m;
     int tiles;             // ceil(out / 128)
     int h_shared;          // every model reads the same activations (first layer)
-    int stages, n_sets, n_abufs;
+    int stages, b_stages, n_sets, n_abufs;   // stages: weight ring; b_stages: activation ring
     float *Hout;           // [m+1][n_r][out] fp32, or NULL
     void *Hsplit;          // [m+1][2 n_pad][out] two-term activations for a following layer of this kind, or NULL
     int relu;
@@ -202,12 +210,13 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     constexpr int kBlockK = Tr::kBlockK;
     pdl_launch_dependents();
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    // full[kLMaxStages], empty[kLMaxStages], a_full[kLMaxABufs], a_empty[kLMaxABufs], d_full[2], d_empty[2]
-    constexpr int kBars = 2 * kLMaxStages + 2 * kLMaxABufs + 2 * kLMaxSets;
+    // full, empty [kLMaxStages] (weight ring); bfull, bempty [kLMaxBStages] (activation ring);
+    // a_full, a_empty [kLMaxABufs]; d_full, d_empty [2]
+    constexpr int kBars = 2 * kLMaxStages + 2 * kLMaxBStages + 2 * kLMaxABufs + 2 * kLMaxSets;
     __shared__ __align__(8) uint64_t bars[kBars];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
-    __shared__ int issued[kLMaxStages];
+    __shared__ int issued[kLMaxStages + kLMaxBStages];     // last round a copy was issued into a stage, plus one
     __shared__ int head_last;                  // HEAD: the epilogue group's ticket result
     __shared__ int head_final;                 // HEAD: this block completed the last model
 
@@ -218,23 +227,27 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
 
     const int nkb = (a.K + kBlockK - 1) / kBlockK;
     const int n_items = (a.m + 1) * a.tiles;
-    const int n_stages = a.stages, n_abufs = a.n_abufs, n_sets = a.n_sets;
-    const int b_bytes = 2 * a.n_pad * kRowBytes;
+    const int n_stages = a.stages, n_bstages = a.b_stages, n_abufs = a.n_abufs, n_sets = a.n_sets;
+    const int b_bytes = 2 * a.n_pad * kRowBytes;                // a stage of the activation ring
     constexpr int kWTiles = LINEAR ? 1 : 2;                     // weight tiles per stage
-    const int stage_bytes = kWTiles * kTileBytes + b_bytes;     // x tile, v tile, activations
+    constexpr int stage_bytes = kWTiles * kTileBytes;           // a stage of the weight ring: x tile, v tile
     const int acc_cols = Tr::kAccPerPad * a.n_pad;
     const int a_base = n_sets * acc_cols;                       // TMEM: accumulator sets, then the A buffers
-    const float inv_stages = 1.0f / (float)n_stages, inv_abufs = 1.0f / (float)n_abufs;
+    const float inv_stages = 1.0f / (float)n_stages, inv_bstages = 1.0f / (float)n_bstages, inv_abufs = 1.0f / (float)n_abufs;
     uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     // HEAD: behind the ring, the epilogue warps' partial logits [4][classes rounded up to even][n_pad]
-    float *zq = reinterpret_cast<float *>(ring + (size_t)n_stages * stage_bytes);
+    uint8_t *bring = ring + (size_t)n_stages * stage_bytes;     // the activation ring follows the weight ring
+    float *zq = reinterpret_cast<float *>(bring + (size_t)n_bstages * b_bytes);
 
     auto bar_full = [&](int s) { return smem_u32(&bars[s]); };
     auto bar_empty = [&](int s) { return smem_u32(&bars[kLMaxStages + s]); };
-    auto bar_afull = [&](int g) { return smem_u32(&bars[2 * kLMaxStages + g]); };
-    auto bar_aempty = [&](int g) { return smem_u32(&bars[2 * kLMaxStages + kLMaxABufs + g]); };
-    auto bar_dfull = [&](int q) { return smem_u32(&bars[2 * kLMaxStages + 2 * kLMaxABufs + q]); };
-    auto bar_dempty = [&](int q) { return smem_u32(&bars[2 * kLMaxStages + 2 * kLMaxABufs + kLMaxSets + q]); };
+    constexpr int kBarB = 2 * kLMaxStages, kBarA = kBarB + 2 * kLMaxBStages, kBarD = kBarA + 2 * kLMaxABufs;
+    auto bar_bfull = [&](int s) { return smem_u32(&bars[kBarB + s]); };
+    auto bar_bempty = [&](int s) { return smem_u32(&bars[kBarB + kLMaxBStages + s]); };
+    auto bar_afull = [&](int g) { return smem_u32(&bars[kBarA + g]); };
+    auto bar_aempty = [&](int g) { return smem_u32(&bars[kBarA + kLMaxABufs + g]); };
+    auto bar_dfull = [&](int q) { return smem_u32(&bars[kBarD + q]); };
+    auto bar_dempty = [&](int q) { return smem_u32(&bars[kBarD + kLMaxSets + q]); };
     // item li of this block -> (model, tile); neighbouring blocks share a model's activations in L2
     auto get_item = [&](int li, int &model, int &tile) {
         const int item = blockIdx.x + li * gridDim.x;
@@ -248,8 +261,13 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         head_final = 0;
         for (int s = 0; s < kLMaxStages; ++s) {
             mbar_init(bar_full(s), 1);
-            mbar_init(bar_empty(s), 5);        // the four warps of a converter set and the MMAs' commit
+            mbar_init(bar_empty(s), 4);        // the four warps of the converter set that read the tiles
             issued[s] = 0;
+        }
+        for (int s = 0; s < kLMaxBStages; ++s) {
+            mbar_init(bar_bfull(s), 1);
+            mbar_init(bar_bempty(s), 1);       // the commit of the MMAs that read the activations
+            issued[kLMaxStages + s] = 0;
         }
         for (int g = 0; g < kLMaxABufs; ++g) {
             mbar_init(bar_afull(g), 4);
@@ -273,8 +291,13 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     const uint32_t tmem = tmem_base_slot;
     volatile int *abortp = &abort_flag;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
+    if (warp == 0 || warp == 2) {
+        // ------------------------------------------------------------------ TMA producers
+        // warp 0 feeds the weight ring (x tile, v tile), warp 2 the activation ring; the two rings
+        // have their own depths because their stages live for different times: a weight stage is free
+        // as soon as a converter set has read it, an activation stage only when its MMAs have finished.
+        const bool acts = warp == 2;
+        const int ring_stages = acts ? n_bstages : n_stages;
         int s = 0;
         uint32_t round = 0;
         int model, tile;
@@ -283,25 +306,26 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             const bool has_v = model > 0;                 // model 0 is x itself
             bool ok = true;
             for (int kb = 0; kb < nkb; ++kb) {
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_empty(s), (round & 1) ^ 1, abortp));
+                const uint32_t empty = acts ? bar_bempty(s) : bar_empty(s), full = acts ? bar_bfull(s) : bar_full(s);
+                ok = __all_sync(0xffffffffu, mbar_wait(empty, (round & 1) ^ 1, abortp));
                 if (!ok) break;
                 if (elect_one()) {
-                    const uint32_t dst = smem_u32(ring + (size_t)s * stage_bytes);
-                    mbar_expect_tx(bar_full(s), (has_v && !LINEAR ? 2 : 1) * kTileBytes + b_bytes);
-                    issued[s] = (int)round + 1;
+                    const uint32_t dst = acts ? smem_u32(bring + (size_t)s * b_bytes) : smem_u32(ring + (size_t)s * stage_bytes);
+                    mbar_expect_tx(full, acts ? b_bytes : (has_v && !LINEAR ? 2 : 1) * kTileBytes);
+                    issued[acts ? kLMaxStages + s : s] = (int)round + 1;
 #pragma unroll 1
-                    for (int w = 0; w < 3; ++w) {         // x tile, v tile, activations: ONE issue site
+                    for (int w = acts ? 2 : 0; w < (acts ? 3 : 2); ++w) {     // x tile, v tile | activations: ONE issue site
                         // LINEAR: the only weight tile is x's for model 0, v's otherwise
                         if (LINEAR ? w == (has_v ? 0 : 1) : (w == 1 && !has_v)) continue;
                         const CUtensorMap *map = w == 0 ? &map_x : w == 1 ? &map_v : &map_h;
                         const int c1 = w == 2 ? 0 : tile * kRows;
                         const int c2 = w == 0 ? 0 : w == 1 ? model - 1 : (a.h_shared ? 0 : model);
-                        const int slot = w == 2 ? kWTiles : (LINEAR ? 0 : w);
-                        tma_load_3d(dst + slot * kTileBytes, map, kb * kBlockK, c1, c2, bar_full(s));
+                        const int slot = w == 2 ? 0 : (LINEAR ? 0 : w);
+                        tma_load_3d(dst + slot * kTileBytes, map, kb * kBlockK, c1, c2, full);
                     }
                 }
                 __syncwarp();
-                if (++s == n_stages) {
+                if (++s == ring_stages) {
                     s = 0;
                     ++round;
                 }
@@ -326,15 +350,15 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             const uint32_t d1 = tmem + set * acc_cols, d2 = d1 + 2 * a.n_pad;
             bool ok = true;
             for (int kb = 0; kb < nkb; ++kb, ++it) {
-                const uint32_t sround = small_div(it, inv_stages), around = small_div(it, inv_abufs);
-                const int s = (int)(it - sround * n_stages), g = (int)(it - around * n_abufs);
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_full(s), sround & 1, abortp) &&
+                const uint32_t sround = small_div(it, inv_bstages), around = small_div(it, inv_abufs);
+                const int s = (int)(it - sround * n_bstages), g = (int)(it - around * n_abufs);
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_bfull(s), sround & 1, abortp) &&
                                                  mbar_wait(bar_afull(g), around & 1, abortp));
                 if (!ok) break;
                 tc_fence_after();
                 if (elect_one()) {
                     const uint32_t a_tmem = tmem + a_base + g * Tr::kACols;
-                    const uint32_t bx = smem_u32(ring + (size_t)s * stage_bytes + kWTiles * kTileBytes);
+                    const uint32_t bx = smem_u32(bring + (size_t)s * b_bytes);
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {            // 32 bytes of every row per MMA
                         const uint64_t db = smem_desc_sw128(bx + ks * 32);
@@ -346,7 +370,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                         }
                     }
                     tc_commit(bar_aempty(g));               // the A buffer and
-                    tc_commit(bar_empty(s));                // the stage's activations may be overwritten once these finish
+                    tc_commit(bar_bempty(s));               // the stage's activations may be overwritten once these finish
                     if (kb + 1 == nkb) tc_commit(bar_dfull(set));
                 }
                 __syncwarp();
@@ -592,10 +616,11 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     tc_fence_after();
     if (tid == 0 && abort_flag) {
         // bulk copies still in flight (only after an aborted run) must land before the block exits
-        for (int s = 0; s < n_stages; ++s)
+        for (int s = 0; s < kLMaxStages + kLMaxBStages; ++s)
             if (issued[s] > 0) {
+                const uint32_t bar = s < kLMaxStages ? bar_full(s) : bar_bfull(s - kLMaxStages);
                 for (uint32_t i = 0; i < kSpinLimit; ++i) {
-                    if (mbar_try_wait(bar_full(s), (uint32_t)(issued[s] - 1) & 1)) break;
+                    if (mbar_try_wait(bar, (uint32_t)(issued[s] - 1) & 1)) break;
                     __nanosleep(64);
                 }
             }
@@ -694,13 +719,16 @@ cudaError_t launch_typed(Context &c, const LayerTcLaunch &l, cudaStream_t s) {
     a.m = l.m;
     a.tiles = (l.out + kRows - 1) / kRows;
     a.h_shared = l.h_shared;
-    const int stage_bytes = (LINEAR ? 1 : 2) * kTileBytes + 2 * l.n_pad * kRowBytes;
+    const int stage_bytes = (LINEAR ? 1 : 2) * kTileBytes, b_bytes = 2 * l.n_pad * kRowBytes;
     // HEAD: the ranking holds 9 KB of static shared memory, and the epilogue warps' partial logits
     // sit behind the ring
     const int zq_bytes = HEAD ? 4 * ((l.head->classes + 1) & ~1) * l.n_pad * 4 : 0;
     const int budget = HEAD ? kLSmemBudget - 10 * 1024 : kLSmemBudget;
-    a.stages = (budget - 1024 - zq_bytes) / stage_bytes;
+    // the activation ring gets kBStages stages, the weight ring (whose tiles come from HBM) the rest
+    a.b_stages = layer_tc_b_stages(l.n_pad);
+    a.stages = (budget - 1024 - zq_bytes - a.b_stages * b_bytes) / stage_bytes;
     if (a.stages > kLMaxStages) a.stages = kLMaxStages;
+    if (a.stages < 2) return cudaErrorInvalidConfiguration;
     const int acc_cols = Tr::kAccPerPad * l.n_pad;
     a.n_sets = 2 * acc_cols + 2 * Tr::kACols <= kLTmemCols ? 2 : 1;
     a.n_abufs = (kLTmemCols - a.n_sets * acc_cols) / Tr::kACols;
@@ -724,7 +752,7 @@ cudaError_t launch_typed(Context &c, const LayerTcLaunch &l, cudaStream_t s) {
     // equal shares: the fewest blocks that give the same number of rounds as one block per SM
     const int rounds = (items + sms - 1) / sms;
     const int blocks = (items + rounds - 1) / rounds;
-    return launch_chained(layer_tc_kernel<T, LINEAR, HEAD>, dim3(blocks), dim3(kLThreads), (size_t)a.stages * stage_bytes + 1024 + zq_bytes, s,
+    return launch_chained(layer_tc_kernel<T, LINEAR, HEAD>, dim3(blocks), dim3(kLThreads), (size_t)a.stages * stage_bytes + (size_t)a.b_stages * b_bytes + 1024 + zq_bytes, s,
                           chain_launches(c), map_x, map_v, map_h, a);
 }
 
@@ -736,8 +764,9 @@ bool layer_tc_usable(zeno_dtype dtype, int K, int out, int n_r) {
     const int per16 = dtype == ZENO_BF16 ? 8 : 4;
     if (K % per16 != 0 || K < 64 || out < 32 || n_r < 1 || n_r > 128) return false;
     const int n_pad = layer_tc_n_pad(n_r);
-    const int stage_bytes = 2 * kTileBytes + 2 * n_pad * kRowBytes;
-    if ((kLSmemBudget - 1024) / stage_bytes < 2) return false;
+    // two stages of the weight ring beside the activation ring, in the smallest budget any mode leaves
+    const int head_room = 10 * 1024 + 4 * kHeadMaxClasses * n_pad * 4;
+    if (kLSmemBudget - head_room - 1024 - layer_tc_b_stages(n_pad) * 2 * n_pad * kRowBytes < 2 * 2 * kTileBytes) return false;
     const int acc = (dtype == ZENO_BF16 ? 2 : 3) * n_pad, acols = dtype == ZENO_BF16 ? 32 : 64;
     return (kLTmemCols - acc) / acols >= 2;
 }

@@ -243,12 +243,13 @@ def run_ours(args, rank, world, local_rank):
 
     # inputs: enough distinct sets that the rotation exceeds 4x the L2 capacity
     gen_device = "cuda" if args.config >= 3 else "cpu"      # the large workloads are generated on the device
-    w0 = syn.make_config(args.config, device=gen_device)
+    shrink = {"d": args.lsq_d} if (args.config == 5 and args.lsq_d > 0) else {}
+    w0 = syn.make_config(args.config, device=gen_device, **shrink)
     score_b, agg_b = algorithmic_bytes(w0)
     set_bytes = w0.V.numel() * w0.V.element_size() + w0.features.numel() * 4
     n_sets = max(1, min(8, -(-4 * L2_BYTES // set_bytes)))
     sets = [w0] + [syn.make_config(args.config, seed=syn.BASE_SEED + args.config + 1000 * (i + 1),
-                                   device=gen_device) for i in range(n_sets - 1)]
+                                   device=gen_device, **shrink) for i in range(n_sets - 1)]
     dsets = [(s.x.cuda(), s.V.cuda(), s.features.cuda(), s.targets.cuda()) for s in sets]
     z = zeno.from_workload(w0, device=dev)
     out = torch.empty(w0.d, dtype=torch.float32, device="cuda")
@@ -414,6 +415,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--config", type=int, default=2, help="benchmark configuration 1..5 (default 2)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--lsq-d", type=int, default=0,
+                    help="configuration 5 only: a smaller parameter count, for profiler captures of the "
+                         "least-squares kernels on a case that holds a few GB (not a benchmark line)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", "0"))

@@ -31,10 +31,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false if it gave up or if another thread did.  The thread that gives up
-// leaves in *abort_flag which wait it was: bit 30, the parity in bit 20, the barrier's shared-memory
-// address in the low 20 bits (wait_code() turns that into the word the host reads).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+// The polling part of a bounded wait, kept out of line so that the common case below stays a single
+// probe (with the loop inlined, a wait on the MMA-issuing warp cost about 190 cycles even when the
+// barrier's phase had already completed; a bare probe costs 15 to 20).
+static __device__ __noinline__ bool mbar_wait_poll(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if (i > 32) __nanosleep(40);
@@ -42,6 +42,13 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
     *abort_flag = (int)(0x40000000u | ((parity & 1u) << 20) | (bar & 0xfffffu));
     return false;
+}
+// Bounded wait.  Returns false if it gave up or if another thread did.  The thread that gives up
+// leaves in *abort_flag which wait it was: bit 30, the parity in bit 20, the barrier's shared-memory
+// address in the low 20 bits (wait_code() turns that into the word the host reads).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_poll(bar, parity, abort_flag);
 }
 // Status word of a block that gave up: kernel id (1 first-layer stream, 2 layer, 3 least squares) in
 // bits 24-27, the index of the barrier within the block's barrier array in bits 1-16, the awaited

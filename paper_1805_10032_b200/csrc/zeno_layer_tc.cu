@@ -5,10 +5,12 @@
 // 128-row tiles of one model's weight matrix over the full input range K, so there are no split-K
 // partial sums: the epilogue adds the bias, applies the activation and writes the layer's output.
 //
-// Per k-block (128 bytes of every row: 32 floats or 64 bfloat16) ONE ring stage receives, by TMA,
-//   the x tile and the v tile (128 rows each, 128-byte swizzled), and
-//   the k-block of the activations, already split into two terms and stacked: rows 0..n_pad-1
-//   hold h_hi, rows n_pad..2 n_pad-1 hold h_lo, so that one MMA yields w h_hi and w h_lo side by side.
+// Per k-block (128 bytes of every row: 32 floats or 64 bfloat16) TMA fills a stage of each of two rings:
+//   the weight ring: the x tile and the v tile (128 rows each, 128-byte swizzled), free again as soon
+//   as a converter set has read them, and
+//   the activation ring: the k-block of the activations, already split into two terms and stacked --
+//   rows 0..n_pad-1 hold h_hi, rows n_pad..2 n_pad-1 hold h_lo, so that one MMA yields w h_hi and
+//   w h_lo side by side -- free once the MMAs that read it have finished.
 // Converter warps form the candidate's weights w = x - gamma v from the two tiles (thread = row),
 // accumulate v^2 for the score's norm term, and put w into TMEM as the MMA's A operand; the
 // activations are the B operand, read from the stage by the tensor core itself.
@@ -19,8 +21,8 @@
 //                  operand; the fp32 activations are carried as two bfloat16 terms;
 //                  D += w [h_hi; h_lo]^T (kind::f16, K = 16 per MMA); result D[j] + D[n_pad + j].
 //
-// Warp roles: warp 0 TMA producer, warp 1 MMA issuer and owner of TMEM (both stay converged and
-// issue from one elected lane), warps 4-11 two converter sets taking alternate k-blocks, warps
+// Warp roles: warps 0 and 2 TMA producers (weight ring, activation ring), warp 1 MMA issuer and owner of
+// TMEM (all three stay converged and issue from one elected lane; the issuer takes two k-blocks per turn), warps 4-11 two converter sets taking alternate k-blocks, warps
 // 12-15 epilogue.  Accumulator sets alternate between consecutive tiles when two fit in TMEM, so
 // a tile is drained while the next one is accumulated.  Every mbarrier wait is bounded; a wait that
 // gives up raises a status word and the block leaves through the common teardown.
@@ -233,7 +235,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     constexpr int stage_bytes = kWTiles * kTileBytes;           // a stage of the weight ring: x tile, v tile
     const int acc_cols = Tr::kAccPerPad * a.n_pad;
     const int a_base = n_sets * acc_cols;                       // TMEM: accumulator sets, then the A buffers
-    const float inv_stages = 1.0f / (float)n_stages, inv_bstages = 1.0f / (float)n_bstages, inv_abufs = 1.0f / (float)n_abufs;
+    const float inv_stages = 1.0f / (float)n_stages, inv_abufs = 1.0f / (float)n_abufs;
     uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     // HEAD: behind the ring, the epilogue warps' partial logits [4][classes rounded up to even][n_pad]
     uint8_t *bring = ring + (size_t)n_stages * stage_bytes;     // the activation ring follows the weight ring
@@ -339,7 +341,9 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         const uint32_t idesc_base = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(kRows >> 4) << 24);
         const uint32_t idesc_n = idesc_base | ((uint32_t)(a.n_pad >> 3) << 17);          // N = n_pad
         const uint32_t idesc_2n = idesc_base | ((uint32_t)((2 * a.n_pad) >> 3) << 17);   // N = 2 n_pad
-        uint32_t it = 0;
+        const int kb_step = n_bstages >= 4 ? 2 : 1;
+        int bs = 0, ag = 0;                              // activation stage and A buffer of the next k-block
+        uint32_t bph = 0, aph = 0;                       // and the phases their full barriers are awaited in
         int model, tile;
         for (int li = 0;; ++li) {
             if (!__all_sync(0xffffffffu, get_item(li, model, tile) && !*abortp)) break;
@@ -349,31 +353,53 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             tc_fence_after();
             const uint32_t d1 = tmem + set * acc_cols, d2 = d1 + 2 * a.n_pad;
             bool ok = true;
-            for (int kb = 0; kb < nkb; ++kb, ++it) {
-                const uint32_t sround = small_div(it, inv_bstages), around = small_div(it, inv_abufs);
-                const int s = (int)(it - sround * n_bstages), g = (int)(it - around * n_abufs);
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_bfull(s), sround & 1, abortp) &&
-                                                 mbar_wait(bar_afull(g), around & 1, abortp));
+            // Two k-blocks per turn of the loop: by the time this warp gets there the operands of both
+            // are long in place (cycle stamps put them ~800 cycles ahead), and the waits, the vote, the
+            // fence, the election and the loop's own arithmetic cost this warp -- the one every other
+            // role ends up waiting for -- as much as the sixteen MMAs it issues.  Only with an activation ring
+            // of four stages or more: with three (128 samples), holding two back at a time measured slower.
+            for (int kb = 0; kb < nkb; kb += kb_step) {
+                const bool two = kb_step == 2 && kb + 1 < nkb;
+                int s1 = bs + 1, g1 = ag + 1;
+                uint32_t sph1 = bph, gph1 = aph;
+                if (s1 == n_bstages) { s1 = 0; sph1 ^= 1; }
+                if (g1 == n_abufs) { g1 = 0; gph1 ^= 1; }
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_bfull(bs), bph, abortp) && mbar_wait(bar_afull(ag), aph, abortp) &&
+                                                 (!two || (mbar_wait(bar_bfull(s1), sph1, abortp) &&
+                                                           mbar_wait(bar_afull(g1), gph1, abortp))));
                 if (!ok) break;
                 tc_fence_after();
                 if (elect_one()) {
-                    const uint32_t a_tmem = tmem + a_base + g * Tr::kACols;
-                    const uint32_t bx = smem_u32(bring + (size_t)s * b_bytes);
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) {            // 32 bytes of every row per MMA
-                        const uint64_t db = smem_desc_sw128(bx + ks * 32);
-                        if (kBf16) {
-                            tc_mma_bf16_ts(d1, a_tmem + ks * 8, db, idesc_2n, (uint32_t)(kb | ks));    // w [h_hi; h_lo]
-                        } else {
-                            tc_mma_tf32_ts(d1, a_tmem + ks * 8, db, idesc_2n, (uint32_t)(kb | ks));    // w_hi [h_hi; h_lo]
-                            tc_mma_tf32_ts(d2, a_tmem + 32 + ks * 8, db, idesc_n, (uint32_t)(kb | ks)); // w_lo h_hi
+                    for (int h = 0; h < 2; ++h) {
+                        if (h == 1 && !two) break;
+                        const int s = h ? s1 : bs, g = h ? g1 : ag;
+                        const uint32_t a_tmem = tmem + a_base + g * Tr::kACols;
+                        const uint32_t bx = smem_u32(bring + (size_t)s * b_bytes);
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks) {            // 32 bytes of every row per MMA
+                            const uint64_t db = smem_desc_sw128(bx + ks * 32);
+                            const uint32_t acc = (uint32_t)(kb | h | ks);
+                            if (kBf16) {
+                                tc_mma_bf16_ts(d1, a_tmem + ks * 8, db, idesc_2n, acc);          // w [h_hi; h_lo]
+                            } else {
+                                tc_mma_tf32_ts(d1, a_tmem + ks * 8, db, idesc_2n, acc);          // w_hi [h_hi; h_lo]
+                                tc_mma_tf32_ts(d2, a_tmem + 32 + ks * 8, db, idesc_n, acc);      // w_lo h_hi
+                            }
                         }
+                        tc_commit(bar_aempty(g));               // the A buffer and
+                        tc_commit(bar_bempty(s));               // the stage's activations may be overwritten once these finish
                     }
-                    tc_commit(bar_aempty(g));               // the A buffer and
-                    tc_commit(bar_bempty(s));               // the stage's activations may be overwritten once these finish
-                    if (kb + 1 == nkb) tc_commit(bar_dfull(set));
+                    if (kb + kb_step >= nkb) tc_commit(bar_dfull(set));
                 }
                 __syncwarp();
+                // advance both rings by the k-blocks taken
+                bs = two ? s1 + 1 : s1;
+                bph = sph1;
+                if (two && bs == n_bstages) { bs = 0; bph ^= 1; }
+                ag = two ? g1 + 1 : g1;
+                aph = gph1;
+                if (two && ag == n_abufs) { ag = 0; aph ^= 1; }
             }
             if (!ok) break;
         }

@@ -8,9 +8,10 @@
 //
 // A tile of the MMA has 128 rows but there are at most 64 candidates, so a block works on TWO neighbouring
 // k-blocks at once (every row of V, A and x is then read 256 contiguous bytes at a time): TMEM lanes 0-63
-// hold the candidates' entries of the even k-block, lanes 64-127 those of the odd one.  Each pair takes two
-// groups of MMAs on the same A operand, one against the even k-block's rows of A (whose result is meaningful
-// in lanes 0-63), one against the odd one's (lanes 64-127), into different accumulator columns.
+// hold the candidates' entries of the even k-block, lanes 64-127 those of the odd one.  The rows of A of both
+// k-blocks are stacked into ONE B operand, [a_hi(even); a_hi(odd); a_lo(even); a_lo(odd)], so a pair takes one
+// group of MMAs: every lane gets the products against all four blocks, and a lane's meaningful columns are
+// those of its own k-block (the others multiply entries of one k-block with rows of the other and are never read).
 //
 // fp32 accuracy on tf32 tensor cores as in the first-layer stream: both operands are split,
 // a = a_hi + a_lo, and a_hi b_hi + a_hi b_lo + a_lo b_hi is accumulated, the small products in columns of
@@ -80,7 +81,7 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
     const int raw_bytes = n_pad * 128;
     const int stage_bytes = lsq_stage_bytes(n_pad);
     const int off_b = 2 * kVHalfBytes, off_raw = off_b + 2 * b_bytes, off_x = off_raw + 2 * raw_bytes;
-    const int set_cols = 6 * n_pad;                        // per half: D1 (2 n_pad) and D2 (n_pad)
+    const int set_cols = 6 * n_pad;                        // D1 (4 n_pad) and D2 (2 n_pad), both halves side by side
     const int a_base = 2 * set_cols;
     const int n_flush = (nkb + kFlush - 1) / kFlush;
     const int64_t kb0 = (int64_t)blockIdx.x * 2 * nkb;     // first k-block of the block's range
@@ -153,40 +154,60 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         const uint32_t idesc_base = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(128 >> 4) << 24);
-        const uint32_t idesc_n = idesc_base | ((uint32_t)(n_pad >> 3) << 17);
         const uint32_t idesc_2n = idesc_base | ((uint32_t)((2 * n_pad) >> 3) << 17);
-        for (int kb = 0; kb < nkb; ++kb) {
+        const uint32_t idesc_4n = idesc_base | ((uint32_t)((4 * n_pad) >> 3) << 17);
+        int rs = 0, ag = 0;                              // ring stage and A buffer of the next k-block pair
+        uint32_t rph = 0, aph = 0;                       // and the phases their barriers are awaited in
+        // Two stages per turn of the loop (the operands are in place well ahead of this warp, and its
+        // waits, vote, fence and election cost as much as the MMAs it issues).  kFlush is even, so the two
+        // stages of a turn always add into the same accumulator set.
+        for (int kb = 0; kb < nkb; kb += 2) {
+            const bool two = kb + 1 < nkb;
             const int fl = kb / kFlush, in_fl = kb - fl * kFlush;
             const int set = fl & 1;
             if (in_fl == 0) {                          // a fresh accumulator set: wait until it was drained
                 if (!__all_sync(0xffffffffu, mbar_wait(bar_dempty(set), (((uint32_t)fl >> 1) & 1) ^ 1, abortp))) break;
                 tc_fence_after();
             }
-            const uint32_t it = (uint32_t)kb;
-            const uint32_t sround = small_div(it, inv_stages), around = small_div(it, inv_abufs);
-            const int s = (int)(it - sround * n_stages), g = (int)(it - around * n_abufs);
-            if (!__all_sync(0xffffffffu, mbar_wait(bar_bready(s), sround & 1, abortp) &&
-                                             mbar_wait(bar_afull(g), around & 1, abortp)))
+            int s1 = rs + 1, g1 = ag + 1;
+            uint32_t rph1 = rph, aph1 = aph;
+            if (s1 == n_stages) { s1 = 0; rph1 ^= 1; }
+            if (g1 == n_abufs) { g1 = 0; aph1 ^= 1; }
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_bready(rs), rph, abortp) && mbar_wait(bar_afull(ag), aph, abortp) &&
+                                             (!two || (mbar_wait(bar_bready(s1), rph1, abortp) &&
+                                                       mbar_wait(bar_afull(g1), aph1, abortp)))))
                 break;
             tc_fence_after();
             if (elect_one()) {
-                const uint32_t a_tmem = tmem + a_base + g * 64;
+                // D1 = v_hi [a_hi(even); a_hi(odd); a_lo(even); a_lo(odd)]^T, D2 = v_lo [a_hi(even); a_hi(odd)]^T:
+                // lanes 0-63 use the even k-block's columns, lanes 64-127 the odd one's
+                const uint32_t d1 = tmem + set * set_cols, d2 = d1 + 4 * n_pad;
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const uint32_t d1 = tmem + set * set_cols + h * 3 * n_pad, d2 = d1 + 2 * n_pad;
-                    const uint32_t bx = smem_u32(ring + (size_t)s * stage_bytes + off_b + h * b_bytes);
+                for (int q = 0; q < 2; ++q) {
+                    if (q == 1 && !two) break;
+                    const int s = q ? s1 : rs, g = q ? g1 : ag;
+                    const uint32_t a_tmem = tmem + a_base + g * 64;
+                    const uint32_t bx = smem_u32(ring + (size_t)s * stage_bytes + off_b);
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {
                         const uint64_t db = smem_desc_sw128(bx + ks * 32);
-                        tc_mma_tf32_ts(d1, a_tmem + ks * 8, db, idesc_2n, (uint32_t)(in_fl | ks));        // v_hi [a_hi; a_lo]
-                        tc_mma_tf32_ts(d2, a_tmem + 32 + ks * 8, db, idesc_n, (uint32_t)(in_fl | ks));    // v_lo a_hi
+                        const uint32_t acc = (uint32_t)(in_fl | q | ks);
+                        tc_mma_tf32_ts(d1, a_tmem + ks * 8, db, idesc_4n, acc);
+                        tc_mma_tf32_ts(d2, a_tmem + 32 + ks * 8, db, idesc_2n, acc);
                     }
+                    tc_commit(bar_aempty(g));
+                    tc_commit(bar_empty(s));
                 }
-                tc_commit(bar_aempty(g));
-                tc_commit(bar_empty(s));
-                if (in_fl == kFlush - 1 || kb + 1 == nkb) tc_commit(bar_dfull(set));
+                const int last = two ? kb + 1 : kb;
+                if (last - fl * kFlush == kFlush - 1 || last + 1 == nkb) tc_commit(bar_dfull(set));
             }
             __syncwarp();
+            rs = two ? s1 + 1 : s1;
+            rph = rph1;
+            if (two && rs == n_stages) { rs = 0; rph ^= 1; }
+            ag = two ? g1 + 1 : g1;
+            aph = aph1;
+            if (two && ag == n_abufs) { ag = 0; aph ^= 1; }
         }
     } else if (warp == 2) {
         // ------------------------------------------------------------------ rows of A: split for the MMA, and A x
@@ -209,9 +230,11 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
                     const float4 v = *reinterpret_cast<const float4 *>(st + off_raw + h * raw_bytes + sw);
                     accx[u] = fmaf(v.x, x4.x, fmaf(v.y, x4.y, fmaf(v.z, x4.z, fmaf(v.w, x4.w, accx[u]))));
                     const float4 hi = make_float4(tf32_hi(v.x), tf32_hi(v.y), tf32_hi(v.z), tf32_hi(v.w));
-                    *reinterpret_cast<float4 *>(st + off_b + h * b_bytes + sw) = hi;
-                    *reinterpret_cast<float4 *>(st + off_b + h * b_bytes + n_pad * 128 + sw) =
-                        make_float4(v.x - hi.x, v.y - hi.y, v.z - hi.z, v.w - hi.w);     // n_pad % 8 == 0: same swizzle phase
+                    // B operand rows: a_hi of the even k-block, a_hi of the odd one, then the two a_lo blocks
+                    // (n_pad % 8 == 0: every block starts in the same swizzle phase)
+                    *reinterpret_cast<float4 *>(st + off_b + h * n_pad * 128 + sw) = hi;
+                    *reinterpret_cast<float4 *>(st + off_b + (2 + h) * n_pad * 128 + sw) =
+                        make_float4(v.x - hi.x, v.y - hi.y, v.z - hi.z, v.w - hi.w);
                 }
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> tensor-core reads
@@ -280,14 +303,14 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
             const int set = fl & 1;
             if (!mbar_wait(bar_dfull(set), ((uint32_t)fl >> 1) & 1, abortp)) break;
             tc_fence_after();
-            const uint32_t d = tmem + lane_addr + set * set_cols + h * 3 * n_pad;
+            const uint32_t d = tmem + lane_addr + set * set_cols + h * n_pad;    // this lane's k-block's columns
 #pragma unroll
             for (int j0 = 0; j0 < 32; j0 += 16) {
                 if (j0 >= n_pad) break;
                 uint32_t big[16], s1[16], s2[16];
                 tc_ld16(d + j0, big);                           // v_hi a_hi
-                tc_ld16(d + n_pad + j0, s1);                    // v_hi a_lo
-                tc_ld16(d + 2 * n_pad + j0, s2);                // v_lo a_hi
+                tc_ld16(d + 2 * n_pad + j0, s1);                // v_hi a_lo
+                tc_ld16(d + 4 * n_pad + j0, s2);                // v_lo a_hi
                 tc_wait_ld();
 #pragma unroll
                 for (int j = 0; j < 16; ++j)

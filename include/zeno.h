@@ -140,10 +140,23 @@ zeno_status zeno_aggregate(zeno_handle h, const void *V, int64_t ldv, int32_t m,
 
 /* Zeno_b({v_i}) = score -> select -> aggregate on one stream, no host round trip.
  * out: float[d] (required); scores: float[m] or NULL; idx: int32[m-b] or NULL.
- * The SGD update x <- x - gamma * out (Algorithm 1) is left to the caller. */
+ * The SGD update x <- x - gamma * out (Algorithm 1) is left to the caller; zeno_step_update
+ * applies it in the same call. */
 zeno_status zeno_step(zeno_handle h, const void *x, const void *V, int64_t ldv, int32_t m,
                       const zeno_batch *batch, float gamma, float rho, int32_t b, float *out,
                       float *scores, int32_t *idx, void *stream);
+
+/* Algorithm 1's server lines v = Zeno_b({v_i}) and x <- x - gamma v in one call: zeno_step, and
+ * in the pass that forms the average the parameter vector takes the update,
+ *     x[j] <- RN(x[j] - gamma out[j])    (one fused multiply-add in binary32, rounded to the
+ *                                          storage type of x: binary32, or bfloat16 to nearest even),
+ * so the update costs no further pass over x.  gamma is the same learning rate that the score
+ * uses (Definition 2).  x is read by the scoring pass and overwritten in place afterwards; out
+ * (the average itself, [d] binary32) may be NULL when only the new x is wanted; scores and idx as
+ * in zeno_step.  Same argument checks and errors as zeno_step. */
+zeno_status zeno_step_update(zeno_handle h, void *x, const void *V, int64_t ldv, int32_t m,
+                             const zeno_batch *batch, float gamma, float rho, int32_t b, float *out,
+                             float *scores, int32_t *idx, void *stream);
 
 /* The same step for a caller whose data lives in HOST memory (Algorithm 1's server receiving the
  * candidates over the network): x, V, features, targets, out, scores and idx are HOST pointers

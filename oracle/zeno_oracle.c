@@ -311,6 +311,23 @@ int zo_aggregate(int dtype, const void *V, int64_t ldv, int64_t d, int m,
     return ZO_OK;
 }
 
+/* ---- Algorithm 1, the server's update line -------------------------------- */
+
+/* xnew[j] = x[j] - gamma * vbar[j] with vbar the aggregated vector (the line after
+ * v = Zeno_b({v_i}) in Algorithm 1).  float32 storage: the exact double value.
+ * bfloat16 storage: the new parameter is a bfloat16 number, the difference rounded
+ * once to binary32 and then to bfloat16, the same rule as for a candidate's parameters. */
+void zo_update(const void *x, const double *vbar, int64_t d, int dtype, double gamma,
+               double *xnew)
+{
+    for (int64_t j = 0; j < d; ++j) {
+        double diff = zo_load(x, j, dtype) - gamma * vbar[j];
+        if (dtype == ZO_BF16)
+            diff = zo_round_to_bf16((float)diff);
+        xnew[j] = diff;
+    }
+}
+
 /* ---- the whole step: Zeno_b({v_i}) ---------------------------------------- */
 
 int zo_step(int kind, int dtype, int n_layers, const int64_t *dims, int has_bias,

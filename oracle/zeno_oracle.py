@@ -60,6 +60,8 @@ def _load():
         lib.zo_select.argtypes = [vp, i32, i32, vp]
         lib.zo_aggregate.restype = i32
         lib.zo_aggregate.argtypes = [i32, vp, i64, i64, i32, vp, i32, vp]
+        lib.zo_update.restype = None
+        lib.zo_update.argtypes = [vp, vp, i64, i32, dbl, vp]
         lib.zo_step.restype = i32
         lib.zo_step.argtypes = [i32, i32, i32, vp, i32, vp, vp, i64, i32, vp, vp, i32,
                                 dbl, dbl, i32, vp, vp, vp]
@@ -184,6 +186,16 @@ def aggregate(dtype, V, ldv, d, m, idx):
     _check(_load().zo_aggregate(dtype, _ptr(V), int(ldv), int(d), int(m), _ptr(idx),
                                 idx.shape[0], _ptr(out)), "zo_aggregate")
     return out
+
+
+def update(dtype, x, vbar, gamma):
+    """Algorithm 1's server update: x - gamma * vbar, element by element (float64; a bfloat16
+    parameter vector is rounded back to bfloat16)."""
+    x = _params(x, dtype)
+    vbar = np.ascontiguousarray(vbar, dtype=np.float64)
+    xnew = np.empty(vbar.shape[0], dtype=np.float64)
+    _load().zo_update(_ptr(x), _ptr(vbar), vbar.shape[0], dtype, float(gamma), _ptr(xnew))
+    return xnew
 
 
 def step(kind, dtype, dims, has_bias, x, V, ldv, m, features, targets, gamma, rho, b):

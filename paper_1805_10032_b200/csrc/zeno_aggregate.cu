@@ -4,6 +4,10 @@
 // loads when the rows allow it.  A thread owns one 16-byte column group and walks the k rows,
 // so k independent loads are in flight per thread and consecutive threads read consecutive
 // addresses of the same row.  Rows are added in rank order, in binary32.
+//
+// With xu != NULL the same pass applies Algorithm 1's server update, xu[j] <- xu[j] - gamma out[j]
+// (one fused multiply-add in binary32, rounded to the storage type of x), so that the step costs no
+// further pass over x; out may then be NULL.
 #include "zeno_internal.h"
 
 namespace zeno {
@@ -17,9 +21,22 @@ template <> struct Group<float> {
         float4 t = __ldcs(reinterpret_cast<const float4 *>(p));
         o[0] = t.x; o[1] = t.y; o[2] = t.z; o[3] = t.w;
     }
+    __device__ static void store(float *p, const float (&v)[4]) {
+        *reinterpret_cast<float4 *>(p) = make_float4(v[0], v[1], v[2], v[3]);
+    }
 };
 template <> struct Group<__nv_bfloat16> {
     static constexpr int kElems = 8;
+    __device__ static void store(__nv_bfloat16 *p, const float (&v)[8]) {
+        uint4 t;
+        unsigned *w = &t.x;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const __nv_bfloat162 pk = __floats2bfloat162_rn(v[2 * q], v[2 * q + 1]);
+            w[q] = *reinterpret_cast<const unsigned *>(&pk);
+        }
+        *reinterpret_cast<uint4 *>(p) = t;
+    }
     __device__ static void load(const __nv_bfloat16 *p, float (&o)[8]) {
         uint4 t = __ldcs(reinterpret_cast<const uint4 *>(p));
         const unsigned w[4] = {t.x, t.y, t.z, t.w};
@@ -41,9 +58,13 @@ __device__ __forceinline__ void stage_rows(const int32_t *idx, int k, int m, int
     __syncthreads();
 }
 
+__device__ __forceinline__ void store_param(float *p, float v) { *p = v; }
+__device__ __forceinline__ void store_param(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
+
 template <typename T>
 __global__ void __launch_bounds__(256) aggregate_vec_kernel(const T *V, int64_t ldv, int64_t d, int m,
-                                                             const int32_t *idx, int k, float *out) {
+                                                             const int32_t *idx, int k, float *out, T *xu,
+                                                             float gamma) {
     constexpr int E = Group<T>::kElems;
     __shared__ int64_t rows_s[ZENO_MAX_CANDIDATES];
     pdl_launch_dependents();
@@ -81,11 +102,20 @@ __global__ void __launch_bounds__(256) aggregate_vec_kernel(const T *V, int64_t 
 #pragma unroll
             for (int e = 0; e < E; ++e) acc[e] += v[e];
         }
-        float4 *o = reinterpret_cast<float4 *>(out + g * E);
 #pragma unroll
-        for (int q = 0; q < E / 4; ++q)
-            o[q] = make_float4(acc[4 * q] / (float)k, acc[4 * q + 1] / (float)k,
-                               acc[4 * q + 2] / (float)k, acc[4 * q + 3] / (float)k);
+        for (int e = 0; e < E; ++e) acc[e] = acc[e] / (float)k;
+        if (out) {
+            float4 *o = reinterpret_cast<float4 *>(out + g * E);
+#pragma unroll
+            for (int q = 0; q < E / 4; ++q) o[q] = make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
+        }
+        if (xu) {                                // 16-byte aligned like the rows of V
+            float xv[E];
+            Group<T>::load(xu + g * E, xv);
+#pragma unroll
+            for (int e = 0; e < E; ++e) xv[e] = fmaf(-gamma, acc[e], xv[e]);
+            Group<T>::store(xu + g * E, xv);
+        }
     }
     // tail columns (fewer than one group), one per thread of block 0
     if (blockIdx.x == 0) {
@@ -96,7 +126,9 @@ __global__ void __launch_bounds__(256) aggregate_vec_kernel(const T *V, int64_t 
                 int64_t off = rows_s[r];
                 if (off >= 0) acc += load_elem(V + off + j);
             }
-            out[j] = acc / (float)k;
+            acc = acc / (float)k;
+            if (out) out[j] = acc;
+            if (xu) store_param(xu + j, fmaf(-gamma, acc, load_elem(xu + j)));
         }
     }
 }
@@ -105,7 +137,7 @@ __global__ void __launch_bounds__(256) aggregate_vec_kernel(const T *V, int64_t 
 template <typename T>
 __global__ void __launch_bounds__(256) aggregate_scalar_kernel(const T *V, int64_t ldv, int64_t d,
                                                                 int m, const int32_t *idx, int k,
-                                                                float *out) {
+                                                                float *out, T *xu, float gamma) {
     __shared__ int64_t rows_s[ZENO_MAX_CANDIDATES];
     pdl_launch_dependents();
     pdl_wait();
@@ -117,13 +149,15 @@ __global__ void __launch_bounds__(256) aggregate_scalar_kernel(const T *V, int64
             int64_t off = rows_s[r];
             if (off >= 0) acc += load_elem(V + off + j);
         }
-        out[j] = acc / (float)k;
+        acc = acc / (float)k;
+        if (out) out[j] = acc;
+        if (xu) store_param(xu + j, fmaf(-gamma, acc, load_elem(xu + j)));
     }
 }
 
 template <typename T>
 cudaError_t launch_typed(const Context &c, const T *V, int64_t ldv, int m, const int32_t *idx, int k,
-                         float *out, bool aligned, cudaStream_t s) {
+                         float *out, T *xu, float gamma, bool aligned, cudaStream_t s) {
     const int sms = c.sm_count > 0 ? c.sm_count : 148;
     const int64_t d = c.d;
     constexpr int E = Group<T>::kElems;
@@ -133,13 +167,13 @@ cudaError_t launch_typed(const Context &c, const T *V, int64_t ldv, int m, const
         int64_t cap = (int64_t)sms * 8;
         int blocks = (int)(want < cap ? want : cap);
         if (blocks < 1) blocks = 1;
-        e = launch_chained(aggregate_vec_kernel<T>, dim3(blocks), dim3(256), 0, s, chain_launches(c), V, ldv, d, m, idx, k, out);
+        e = launch_chained(aggregate_vec_kernel<T>, dim3(blocks), dim3(256), 0, s, chain_launches(c), V, ldv, d, m, idx, k, out, xu, gamma);
     } else {
         int64_t want = (d + 255) / 256;
         int64_t cap = (int64_t)sms * 8;
         int blocks = (int)(want < cap ? want : cap);
         if (blocks < 1) blocks = 1;
-        e = launch_chained(aggregate_scalar_kernel<T>, dim3(blocks), dim3(256), 0, s, chain_launches(c), V, ldv, d, m, idx, k, out);
+        e = launch_chained(aggregate_scalar_kernel<T>, dim3(blocks), dim3(256), 0, s, chain_launches(c), V, ldv, d, m, idx, k, out, xu, gamma);
     }
     return e;
 }
@@ -147,13 +181,14 @@ cudaError_t launch_typed(const Context &c, const T *V, int64_t ldv, int m, const
 }  // namespace
 
 cudaError_t launch_aggregate(Context &c, const void *V, int64_t ldv, int m,
-                             const int32_t *idx, int k, float *out, bool aligned, cudaStream_t s,
-                             int *launches) {
+                             const int32_t *idx, int k, float *out, void *xu, float gamma, bool aligned,
+                             cudaStream_t s, int *launches) {
     ++*launches;
     profile_mark(c, "aggregate", s);
     if (c.desc.param_dtype == ZENO_BF16)
-        return launch_typed(c, static_cast<const __nv_bfloat16 *>(V), ldv, m, idx, k, out, aligned, s);
-    return launch_typed(c, static_cast<const float *>(V), ldv, m, idx, k, out, aligned, s);
+        return launch_typed(c, static_cast<const __nv_bfloat16 *>(V), ldv, m, idx, k, out, static_cast<__nv_bfloat16 *>(xu),
+                            gamma, aligned, s);
+    return launch_typed(c, static_cast<const float *>(V), ldv, m, idx, k, out, static_cast<float *>(xu), gamma, aligned, s);
 }
 
 }  // namespace zeno

@@ -77,8 +77,9 @@ bool score_rows_aligned(const Context &c, const void *x, const void *V, int64_t 
     return true;
 }
 
-bool aggregate_rows_aligned(const Context &c, const void *V, int64_t ldv, const float *out) {
-    return is_aligned(V, 16) && is_aligned(out, 16) && (ldv * elem_size(c.desc.param_dtype)) % 16 == 0;
+bool aggregate_rows_aligned(const Context &c, const void *V, int64_t ldv, const float *out, const void *xu) {
+    return is_aligned(V, 16) && is_aligned(out, 16) && is_aligned(xu, 16) &&
+           (ldv * elem_size(c.desc.param_dtype)) % 16 == 0;
 }
 
 zeno_status check_common(const Context *c, const void *V, int64_t ldv, int32_t m) {
@@ -312,13 +313,14 @@ zeno_status enqueue_select(Context *c, const float *scores, int32_t m, int32_t b
     return e == cudaSuccess ? ZENO_OK : fail_cuda(c, e);
 }
 
+// xu: NULL, or the parameter vector that takes Algorithm 1's update in the same pass (out may then be NULL)
 zeno_status enqueue_aggregate(Context *c, const void *V, int64_t ldv, int32_t m, const int32_t *idx,
-                              int32_t k, float *out, cudaStream_t s, int *launches) {
+                              int32_t k, float *out, void *xu, float gamma, cudaStream_t s, int *launches) {
     zeno_status st = check_common(c, V, ldv, m);
     if (st != ZENO_OK) return st;
-    if (!idx || !out || k < 1 || k > m) return ZENO_ERR_INVALID_ARG;
-    cudaError_t e = zeno::launch_aggregate(*c, V, ldv, m, idx, k, out,
-                                           aggregate_rows_aligned(*c, V, ldv, out), s, launches);
+    if (!idx || (!out && !xu) || k < 1 || k > m) return ZENO_ERR_INVALID_ARG;
+    cudaError_t e = zeno::launch_aggregate(*c, V, ldv, m, idx, k, out, xu, gamma,
+                                           aggregate_rows_aligned(*c, V, ldv, out, xu), s, launches);
     return e == cudaSuccess ? ZENO_OK : fail_cuda(c, e);
 }
 
@@ -525,7 +527,7 @@ zeno_status zeno_aggregate(zeno_handle h, const void *V, int64_t ldv, int32_t m,
     if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
     int launches = 0;
     profile_begin(h);
-    zeno_status st = enqueue_aggregate(h, V, ldv, m, idx, k, out, static_cast<cudaStream_t>(stream),
+    zeno_status st = enqueue_aggregate(h, V, ldv, m, idx, k, out, nullptr, 0.f, static_cast<cudaStream_t>(stream),
                                        &launches);
     profile_end(h, static_cast<cudaStream_t>(stream));
     h->last_launches = st == ZENO_OK ? launches : 0;
@@ -548,7 +550,30 @@ zeno_status zeno_step(zeno_handle h, const void *x, const void *V, int64_t ldv, 
     zeno_status st = enqueue_score(h, x, V, ldv, m, batch, gamma, rho, score_buf, nullptr, nullptr, m - b,
                                    idx_buf, &ranked, s, &launches);
     if (st == ZENO_OK && !ranked) st = enqueue_select(h, score_buf, m, b, idx_buf, s, &launches);
-    if (st == ZENO_OK) st = enqueue_aggregate(h, V, ldv, m, idx_buf, m - b, out, s, &launches);
+    if (st == ZENO_OK) st = enqueue_aggregate(h, V, ldv, m, idx_buf, m - b, out, nullptr, 0.f, s, &launches);
+    profile_end(h, s);
+    h->last_launches = st == ZENO_OK ? launches : 0;
+    return st;
+}
+
+zeno_status zeno_step_update(zeno_handle h, void *x, const void *V, int64_t ldv, int32_t m,
+                             const zeno_batch *batch, float gamma, float rho, int32_t b, float *out,
+                             float *scores, int32_t *idx, void *stream) {
+    if (!h || !x) return ZENO_ERR_INVALID_ARG;
+    if (m < 1 || m > h->m_max || b < 0 || b >= m) return ZENO_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    float *score_buf = scores ? scores : h->scores;
+    int32_t *idx_buf = idx ? idx : h->idx;
+    int launches = 0;
+    profile_begin(h);
+    bool ranked = false;
+    zeno_status st = enqueue_score(h, x, V, ldv, m, batch, gamma, rho, score_buf, nullptr, nullptr, m - b,
+                                   idx_buf, &ranked, s, &launches);
+    if (st == ZENO_OK && !ranked) st = enqueue_select(h, score_buf, m, b, idx_buf, s, &launches);
+    // the scoring pass has read x by the time the average is formed: the update goes in place
+    if (st == ZENO_OK) st = enqueue_aggregate(h, V, ldv, m, idx_buf, m - b, out, x, gamma, s, &launches);
     profile_end(h, s);
     h->last_launches = st == ZENO_OK ? launches : 0;
     return st;
@@ -608,7 +633,7 @@ zeno_status zeno_step_host(zeno_handle h, const void *x, const void *V, int64_t 
     zeno_status st = enqueue_score(h, dx, dV, ldv, m, &batch, gamma, rho, h->scores, nullptr, nullptr, m - b,
                                    h->idx, &ranked, s, &launches);
     if (st == ZENO_OK && !ranked) st = enqueue_select(h, h->scores, m, b, h->idx, s, &launches);
-    if (st == ZENO_OK) st = enqueue_aggregate(h, dV, ldv, m, h->idx, m - b, dout, s, &launches);
+    if (st == ZENO_OK) st = enqueue_aggregate(h, dV, ldv, m, h->idx, m - b, dout, nullptr, 0.f, s, &launches);
     profile_end(h, s);
     if (st != ZENO_OK) {
         h->last_launches = 0;

@@ -151,9 +151,10 @@ cudaError_t launch_lsq_score(Context &c, const LsqArgs &a, const float *y, float
                              cudaStream_t s, int *launches);
 cudaError_t launch_select(Context &c, const float *scores, int m, int b, int32_t *idx, cudaStream_t s,
                           int *launches);
+// xu != NULL: the parameter vector to update in the same pass, xu <- xu - gamma out (out may be NULL)
 cudaError_t launch_aggregate(Context &c, const void *V, int64_t ldv, int m,
-                             const int32_t *idx, int k, float *out, bool aligned, cudaStream_t s,
-                             int *launches);
+                             const int32_t *idx, int k, float *out, void *xu, float gamma, bool aligned,
+                             cudaStream_t s, int *launches);
 
 // Tensor-core stream for the first layer (fp32 storage).
 bool stream_tc_plan(int sms, int K, int out, int n_r, int m, StreamTcPlan *p);

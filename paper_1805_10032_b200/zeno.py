@@ -25,7 +25,7 @@ F32, BF16 = 0, 1
 
 EXPORTS = (
     "zeno_param_count", "zeno_create", "zeno_destroy", "zeno_score", "zeno_select",
-    "zeno_aggregate", "zeno_step", "zeno_step_host", "zeno_device_status", "zeno_score_lsq_static",
+    "zeno_aggregate", "zeno_step", "zeno_step_update", "zeno_step_host", "zeno_device_status", "zeno_score_lsq_static",
     "zeno_profile", "zeno_profile_read",
     "zeno_last_launch_count",
     "zeno_last_cuda_error", "zeno_last_wait_code", "zeno_status_string",
@@ -77,6 +77,8 @@ def load_library() -> ctypes.CDLL:
     lib.zeno_aggregate.argtypes = [vp, vp, i64, i32, vp, i32, vp, vp]
     lib.zeno_step.restype = i32
     lib.zeno_step.argtypes = [vp, vp, vp, i64, i32, ctypes.POINTER(Batch), f32, f32, i32, vp, vp, vp, vp]
+    lib.zeno_step_update.restype = i32
+    lib.zeno_step_update.argtypes = [vp, vp, vp, i64, i32, ctypes.POINTER(Batch), f32, f32, i32, vp, vp, vp, vp]
     lib.zeno_step_host.restype = i32
     lib.zeno_step_host.argtypes = [vp, vp, vp, i64, i32, vp, vp, i32, f32, f32, i32, vp, vp, vp, vp]
     lib.zeno_score_lsq_static.restype = i32
@@ -263,6 +265,25 @@ class Zeno:
                                  float(gamma), float(rho), int(b), _ptr(out), _ptr(scores), _ptr(idx),
                                  _stream_ptr(stream))
         self._check(st, "zeno_step")
+        return out, scores, idx
+
+    def step_update(self, x, V, features, targets, gamma, rho, b, m=None, ldv=None, out=None,
+                    scores=None, idx=None, want_out=True, want_scores=True, want_idx=True, stream=None):
+        """Zeno_b followed by the server update x <- x - gamma * average, in place and in the pass that
+        forms the average.  Returns (out[d] or None, scores[m] or None, idx[m-b] or None)."""
+        m = V.shape[0] if m is None else m
+        ldv = V.stride(0) if ldv is None else ldv
+        if out is None and want_out:
+            out = torch.empty(self.d, dtype=torch.float32, device=self._dev())
+        if scores is None and want_scores:
+            scores = torch.empty(m, dtype=torch.float32, device=self._dev())
+        if idx is None and want_idx:
+            idx = torch.empty(max(m - b, 0), dtype=torch.int32, device=self._dev())
+        bt = self._batch(features, targets)
+        st = self._lib.zeno_step_update(self._h, _ptr(x), _ptr(V), int(ldv), int(m), ctypes.byref(bt),
+                                        float(gamma), float(rho), int(b), _ptr(out), _ptr(scores),
+                                        _ptr(idx), _stream_ptr(stream))
+        self._check(st, "zeno_step_update")
         return out, scores, idx
 
     def step_host(self, x, V, features, targets, gamma, rho, b, out, scores=None, idx=None,

@@ -367,6 +367,41 @@ def test_aggregate_bf16_rows_with_library_mean(oracle):
     assert np.allclose(out, t.double().numpy()[[4, 0, 2], :37].mean(0), rtol=1e-14)
 
 
+# ---------------------------------------------------------------- Algorithm 1's server update
+
+def test_update_hand_values_and_gamma_zero(oracle):
+    """x - gamma * vbar on numbers worked by hand; gamma = 0 leaves x as it is."""
+    x = np.array([1.0, 2.0, -3.0], np.float32)
+    vbar = np.array([0.5, -4.0, 8.0])
+    assert np.allclose(oracle.update(F32, x, vbar, 0.1), [0.95, 2.4, -3.8], rtol=1e-15)
+    assert np.array_equal(oracle.update(F32, x, vbar, 0.0), x.astype(np.float64))
+    xb = torch.tensor([1.5, -0.3125, 96.0]).to(torch.bfloat16)
+    assert np.array_equal(oracle.update(BF16, syn.to_numpy_params(xb), vbar, 0.0), xb.double().numpy())
+
+
+def test_update_of_bf16_parameters_rounds_to_nearest_even(oracle):
+    """1 - 2^-9 lies halfway between the bfloat16 neighbours 255/256 and 1: the tie goes to 1 (even);
+    1 - 3 * 2^-10 is nearer to 255/256; library route for random values."""
+    one = syn.to_numpy_params(torch.tensor([1.0, 1.0]).to(torch.bfloat16))
+    got = oracle.update(BF16, one, np.array([2.0 ** -9, 3 * 2.0 ** -10]), 1.0)
+    assert got.tolist() == [1.0, 255.0 / 256.0]
+    g = torch.Generator().manual_seed(31)
+    x = torch.randn(2000, generator=g).to(torch.bfloat16)
+    vbar = torch.randn(2000, generator=g, dtype=torch.float64) * 3
+    gamma = float(np.float32(0.05))
+    want = (x.double() - gamma * vbar).float().to(torch.bfloat16).double().numpy()
+    assert np.array_equal(oracle.update(BF16, syn.to_numpy_params(x), vbar.numpy(), gamma), want)
+
+
+def test_update_after_step_is_x_minus_gamma_times_mean_of_kept_rows(oracle):
+    dims = (7, 5, 4, 3)
+    d, ldv, x, V, feats, labels = _random_mlp_problem(23, m=6)
+    out, s, idx = oracle.step(MLP, F32, dims, True, x, V, ldv, 6, feats, labels, 0.1, 5e-4, 2)
+    kept = np.argsort(-s, kind="stable")[:4]
+    want = x.astype(np.float64) - 0.1 * V[kept, :d].astype(np.float64).mean(0)
+    assert np.allclose(oracle.update(F32, x, out, 0.1), want, rtol=1e-13, atol=1e-16)
+
+
 def test_aggregate_rejects_out_of_range_index(oracle):
     V = np.zeros((3, 4), np.float32)
     with pytest.raises(RuntimeError):

@@ -3,8 +3,9 @@
 // The residual of candidate i is linear in the parameters, A (x - gamma v_i) - y = A x - gamma A v_i - y,
 // so one pass over V, A and x yields everything: the products A v_i^T for all candidates (a skinny
 // GEMM of the rows of V against the n_r rows of A over the parameter index k), A x, and the sums of
-// squares of the rows of V.  All three operands are streamed from HBM exactly once; a block owns a
-// contiguous range of k and leaves its partial sums in a slab that lsq_finish_kernel adds up in double.
+// squares of the rows of V.  All three operands are streamed from HBM exactly once; the k-blocks are dealt
+// to the blocks round robin, and a block leaves its partial sums in a slab that lsq_finish_kernel adds up in
+// double.
 //
 // A tile of the MMA has 128 rows but there are at most 64 candidates, so a block works on TWO neighbouring
 // k-blocks at once (every row of V, A and x is then read 256 contiguous bytes at a time): TMEM lanes 0-63
@@ -21,8 +22,8 @@
 // Warp roles (every producer / issuer warp stays converged and issues from one elected lane):
 //   warp 0       TMA producer: per stage two 64-row boxes of V, two boxes of A, two 128-byte pieces of x
 //   warp 1       MMA issuer, owner of TMEM
-//   warp 2       splits the stage's rows of A into [a_hi; a_lo] (the MMA's B operand, 128-byte swizzled)
-//                and takes A x from the same registers
+//   warps 2, 3   split the stage's rows of A (warp 2 the even k-block's, warp 3 the odd one's) into hi and lo
+//                terms (the MMA's B operand, 128-byte swizzled) and take A x from the same registers
 //   warps 4-11   two converter sets on alternate k-blocks: thread = TMEM lane; reads its 128 bytes of V,
 //                accumulates v^2, stores v_hi / v_lo to TMEM as the A operand
 //   warps 12-15  drain the accumulator sets into registers; at the end write the slab
@@ -41,7 +42,7 @@ constexpr int kVHalfBytes = kHalfRows * 128;
 constexpr int kQThreads = 32 * 16;
 constexpr int kQMaxStages = 8;
 constexpr int kQMaxABufs = 5;
-constexpr int kQSmem = 200 * 1024;          // dynamic; the result exchange below is static
+constexpr int kQSmem = 217 * 1024;          // dynamic: the ring, reused for the result exchange at the end
 constexpr int kQTmemCols = 512;
 constexpr int kFlush = 32;                  // k-blocks accumulated in TMEM before a drain
 
@@ -67,9 +68,8 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
     __shared__ int issued[kQMaxStages];
-    __shared__ float res[128][33];          // drained products per TMEM lane
     __shared__ float nrm_s[2][128];         // sums of squares per lane and converter set
-    __shared__ float z0_s[32];              // A x
+    __shared__ float z0_s[2][32];           // A x, per splitter warp
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
@@ -84,9 +84,11 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
     const int set_cols = 6 * n_pad;                        // D1 (4 n_pad) and D2 (2 n_pad), both halves side by side
     const int a_base = 2 * set_cols;
     const int n_flush = (nkb + kFlush - 1) / kFlush;
-    const int64_t kb0 = (int64_t)blockIdx.x * 2 * nkb;     // first k-block of the block's range
     const float inv_stages = 1.0f / (float)n_stages, inv_abufs = 1.0f / (float)n_abufs;
     uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    // drained products per TMEM lane; written once the last accumulator set has been drained, when every
+    // stage of the ring has been consumed
+    float(*res)[33] = reinterpret_cast<float(*)[33]>(ring);
 
     auto bar_full = [&](int s) { return smem_u32(&bars[s]); };
     auto bar_empty = [&](int s) { return smem_u32(&bars[kQMaxStages + s]); };
@@ -101,7 +103,7 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
         for (int s = 0; s < kQMaxStages; ++s) {
             mbar_init(bar_full(s), 1);
             mbar_init(bar_empty(s), 5);        // the four warps of a converter set and the MMAs' commit
-            mbar_init(bar_bready(s), 1);
+            mbar_init(bar_bready(s), 2);        // the two warps that split the rows of A
             issued[s] = 0;
         }
         for (int g = 0; g < kQMaxABufs; ++g) {
@@ -141,7 +143,10 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
                     const int h = w & 1, what = w >> 1;
                     const CUtensorMap *map = what == 0 ? &map_v : what == 1 ? &map_a : &map_x;
                     const uint32_t off = what == 0 ? h * kVHalfBytes : what == 1 ? off_raw + h * raw_bytes : off_x + h * 128;
-                    const int64_t k = (kb0 + 2 * (int64_t)kb + h) * kQBlockK;     // neighbouring k-blocks: 256 contiguous bytes of every row
+                    // Pairs of neighbouring k-blocks (256 contiguous bytes of every row) are dealt round robin:
+                    // at any moment the blocks read neighbouring addresses of the same ~80 rows, a few hundred
+                    // pages in all; with one contiguous k-range per block it was ~12,000 pages of 2 MB at once
+                    const int64_t k = (2 * ((int64_t)blockIdx.x + (int64_t)kb * gridDim.x) + h) * kQBlockK;
                     tma_load_3d(dst + off, map, (int)k, 0, 0, bar_full(s));
                 }
             }
@@ -209,8 +214,12 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
             aph = aph1;
             if (two && ag == n_abufs) { ag = 0; aph ^= 1; }
         }
-    } else if (warp == 2) {
+    } else if (warp == 2 || warp == 3) {
         // ------------------------------------------------------------------ rows of A: split for the MMA, and A x
+        // Warp 2 takes the even k-block's rows of every stage, warp 3 the odd one's.  All of a lane's rows
+        // are loaded before the first store: the stores go to the same shared array, so loads placed after
+        // them would wait for them, and the stage would reach the MMAs ~1,000 cycles later (cycle stamps).
+        const int h = warp - 2;
         float accx[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};    // rows 4 u + lane / 8 (u < n_pad / 4)
         bool ok = true;
         for (int kb = 0; kb < nkb && ok; ++kb) {
@@ -219,23 +228,26 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
             ok = mbar_wait(bar_full(s), sround & 1, abortp);
             if (!ok) break;
             uint8_t *st = ring + (size_t)s * stage_bytes;
+            const float4 x4 = *reinterpret_cast<const float4 *>(st + off_x + h * 128 + (lane & 7) * 16);
+            float4 v[8];
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const float4 x4 = *reinterpret_cast<const float4 *>(st + off_x + h * 128 + (lane & 7) * 16);
+            for (int u = 0; u < 8; ++u) {
+                const int j = 4 * u + (lane >> 3), c = lane & 7;
+                v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (4 * u < n_pad) v[u] = *reinterpret_cast<const float4 *>(st + off_raw + h * raw_bytes + j * 128 + ((c ^ (j & 7)) << 4));
+            }
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    if (4 * u >= n_pad) break;
-                    const int j = 4 * u + (lane >> 3), c = lane & 7;
-                    const uint32_t sw = (uint32_t)j * 128 + ((c ^ (j & 7)) << 4);
-                    const float4 v = *reinterpret_cast<const float4 *>(st + off_raw + h * raw_bytes + sw);
-                    accx[u] = fmaf(v.x, x4.x, fmaf(v.y, x4.y, fmaf(v.z, x4.z, fmaf(v.w, x4.w, accx[u]))));
-                    const float4 hi = make_float4(tf32_hi(v.x), tf32_hi(v.y), tf32_hi(v.z), tf32_hi(v.w));
-                    // B operand rows: a_hi of the even k-block, a_hi of the odd one, then the two a_lo blocks
-                    // (n_pad % 8 == 0: every block starts in the same swizzle phase)
-                    *reinterpret_cast<float4 *>(st + off_b + h * n_pad * 128 + sw) = hi;
-                    *reinterpret_cast<float4 *>(st + off_b + (2 + h) * n_pad * 128 + sw) =
-                        make_float4(v.x - hi.x, v.y - hi.y, v.z - hi.z, v.w - hi.w);
-                }
+            for (int u = 0; u < 8; ++u) {
+                if (4 * u >= n_pad) break;
+                const int j = 4 * u + (lane >> 3), c = lane & 7;
+                const uint32_t sw = (uint32_t)j * 128 + ((c ^ (j & 7)) << 4);
+                accx[u] = fmaf(v[u].x, x4.x, fmaf(v[u].y, x4.y, fmaf(v[u].z, x4.z, fmaf(v[u].w, x4.w, accx[u]))));
+                const float4 hi = make_float4(tf32_hi(v[u].x), tf32_hi(v[u].y), tf32_hi(v[u].z), tf32_hi(v[u].w));
+                // B operand rows: a_hi of the even k-block, a_hi of the odd one, then the two a_lo blocks
+                // (n_pad % 8 == 0: every block starts in the same swizzle phase)
+                *reinterpret_cast<float4 *>(st + off_b + h * n_pad * 128 + sw) = hi;
+                *reinterpret_cast<float4 *>(st + off_b + (2 + h) * n_pad * 128 + sw) =
+                    make_float4(v[u].x - hi.x, v[u].y - hi.y, v[u].z - hi.z, v[u].w - hi.w);
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> tensor-core reads
             __syncwarp();
@@ -248,7 +260,7 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
             t += __shfl_xor_sync(0xffffffffu, t, 1);
             t += __shfl_xor_sync(0xffffffffu, t, 2);
             t += __shfl_xor_sync(0xffffffffu, t, 4);
-            if ((lane & 7) == 0 && 4 * u + (lane >> 3) < 32) z0_s[4 * u + (lane >> 3)] = t;
+            if ((lane & 7) == 0 && 4 * u + (lane >> 3) < 32) z0_s[warp - 2][4 * u + (lane >> 3)] = t;
         }
     } else if (warp >= 4 && warp < 12) {
         // ------------------------------------------------------------------ converters
@@ -345,7 +357,7 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
         const int r = t / stride, j = t - r * stride;
         float v;
         if (r == 0) {
-            v = j < a.n_r ? z0_s[j] : 0.f;
+            v = j < a.n_r ? z0_s[0][j] + z0_s[1][j] : 0.f;
         } else {
             const int c = r - 1;
             v = j < a.n_r ? res[c][j] + res[c + kHalfRows][j]

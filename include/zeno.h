@@ -12,8 +12,9 @@
  *
  * Conventions for every call
  *   - All data pointers are DEVICE pointers owned by the caller (x, V, the batch,
- *     and every output).  Inputs are never written; outputs are overwritten in
- *     full.  The library allocates device memory only inside zeno_create.
+ *     and every output).  Inputs are never written (the one exception is x in
+ *     zeno_step_update, which is that call's output too); outputs are overwritten
+ *     in full.  The library allocates device memory only inside zeno_create.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
  *     Calls are asynchronous on it: they enqueue kernels and return; there is
  *     no host synchronisation and no device-to-host copy inside a call.

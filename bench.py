@@ -321,6 +321,21 @@ def run_ours(args, rank, world, local_rank):
     value, ms_total = whole_job_rate(ms_total, args.steps, world, dist, "cuda")
     ms_per_step = ms_total / args.steps
 
+    # ---- launch floor: as many of the library's smallest kernel (the one-block ranking of m scores)
+    # back to back as a step has launches -- what the step would cost if its kernels did no work
+    lib = zeno.load_library()
+    floor_calls = 200
+    def floor_pass():
+        for _ in range(floor_calls * launches_per_step):
+            lib.zeno_select(z._h, scores.data_ptr(), w0.m, w0.b, idx.data_ptr(), None)
+    floor_pass()
+    barrier()
+    e0.record()
+    floor_pass()
+    e1.record()
+    barrier()
+    launch_floor_us = e0.elapsed_time(e1) * 1e3 / floor_calls
+
     # ---- end to end through the host-memory entry point (copies inside the timed region)
     hx, hV = sets[0].x.cpu().pin_memory(), sets[0].V.cpu().pin_memory()
     hf, ht = sets[0].features.cpu().pin_memory(), sets[0].targets.cpu().pin_memory()
@@ -381,6 +396,7 @@ def run_ours(args, rank, world, local_rank):
         "peak_source": peak_kind,
         "bytes_per_launch": top_bytes, "avg_us": top["avg_us"],
         "timed": "second pass over the same K steps, enqueued back to back with a CUDA event around every kernel",
+        "launch_floor_us": launch_floor_us,
         "step": {"algorithmic_bytes": step_bytes,
                  "achieved_GBs": step_bytes / (ms_per_step * 1e-3) / 1e9,
                  "frac_of_hbm_peak": step_bytes / (ms_per_step * 1e-3) / 1e9 / peak,

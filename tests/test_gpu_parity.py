@@ -49,6 +49,11 @@ SHRUNK = {
     "cfg5_small": (5, dict(d=70000, m=13, b=5, n_r=16, n_noise=5)),
     "cfg5_nr5": (5, dict(d=33333 * 4, m=70, b=30, n_r=5, n_noise=30)),
     "cfg5_nr40": (5, dict(d=9000, m=6, b=2, n_r=40, n_noise=2)),
+    # the tensor-core least-squares stream with 32 padded samples (N = 128) and all 64 candidate lanes in use,
+    # a parameter count that leaves a ragged last k-block pair
+    # (gamma = 0.1: with 0.01 one honest score is a 1e-6 difference of terms near 0.6, a condition number
+    # of 1e6 that no binary32 loss can carry to 1e-4 relative)
+    "cfg5_nr24_m64": (5, dict(d=50004, m=64, b=20, n_r=24, n_noise=20, gamma=0.1)),
 }
 
 
@@ -76,6 +81,8 @@ def kernels_of_a_step(w):
     ("cfg3_many_tiles", ["split_acts", "layer_tc", "stream_combine", "mlp_head_loss_tail", "aggregate"]),
     ("cfg4_128_samples", ["split_acts", "layer_tc", "layer_tc", "layer_tc", "mlp_loss_tail", "aggregate"]),
     ("cfg4_small", ["split_acts", "layer_tc", "layer_tc", "layer_tc", "mlp_loss_tail", "aggregate"]),
+    ("cfg5_nr24_m64", ["lsq_tc", "lsq_finish", "select", "aggregate"]),
+    ("cfg5_small", ["lsq_tc", "lsq_finish", "select", "aggregate"]),
 ])
 def test_which_kernels_serve_a_workload(name, expected):
     """The parity cases above exercise the kernels they were written for (no quiet detour)."""

@@ -50,6 +50,7 @@ struct LsqTcArgs {
     int m, n_r, n_pad;                      // n_pad: 16 or 32
     int nkb;                                // pairs of k-blocks in a block's k-range
     int stages, n_abufs;
+    int wide;                               // the tensor maps fetch both k-blocks of a pair in one copy (d % 32 == 0)
     float *part;                            // [blocks][m+1][n_r+1]
     int *status;
 };
@@ -138,16 +139,24 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
                 const uint32_t dst = smem_u32(ring + (size_t)s * stage_bytes);
                 mbar_expect_tx(bar_full(s), 2 * kVHalfBytes + 2 * raw_bytes + 2 * 128);
                 issued[s] = (int)round + 1;
+                // Pairs of neighbouring k-blocks (256 contiguous bytes of every row) are dealt round robin:
+                // at any moment the blocks read neighbouring addresses of the same ~80 rows, a few hundred
+                // pages in all; with one contiguous k-range per block it was ~12,000 pages of 2 MB at once
+                const int64_t pair = (int64_t)blockIdx.x + (int64_t)kb * gridDim.x;
+                // Issuing a copy costs this lane well over a hundred cycles, and with six per stage the producer
+                // was what the ring waited for (cycle stamps: stages re-armed 1,400-2,200 cycles after they were
+                // free).  When d and ldv are multiples of 32 the maps see V and A as [row][k-block][32] and one box
+                // takes both k-blocks of the pair (a row's two 128-byte pieces then lie side by side in the stage),
+                // x comes as one 256-byte piece: three copies per stage.
+                const int n_loads = a.wide ? 3 : 6;
 #pragma unroll 1
-                for (int w = 0; w < 6; ++w) {          // V, A, x of the two halves: ONE issue site
-                    const int h = w & 1, what = w >> 1;
+                for (int w = 0; w < n_loads; ++w) {    // V, A, x (of the two halves): ONE issue site
+                    const int h = a.wide ? 0 : (w & 1), what = a.wide ? w : (w >> 1);
                     const CUtensorMap *map = what == 0 ? &map_v : what == 1 ? &map_a : &map_x;
                     const uint32_t off = what == 0 ? h * kVHalfBytes : what == 1 ? off_raw + h * raw_bytes : off_x + h * 128;
-                    // Pairs of neighbouring k-blocks (256 contiguous bytes of every row) are dealt round robin:
-                    // at any moment the blocks read neighbouring addresses of the same ~80 rows, a few hundred
-                    // pages in all; with one contiguous k-range per block it was ~12,000 pages of 2 MB at once
-                    const int64_t k = (2 * ((int64_t)blockIdx.x + (int64_t)kb * gridDim.x) + h) * kQBlockK;
-                    tma_load_3d(dst + off, map, (int)k, 0, 0, bar_full(s));
+                    const int64_t k = (2 * pair + h) * kQBlockK;
+                    const bool blocked = a.wide && what < 2;          // coordinates (0, k-block, row 0)
+                    tma_load_3d(dst + off, map, blocked ? 0 : (int)k, blocked ? (int)(2 * pair) : 0, 0, bar_full(s));
                 }
             }
             __syncwarp();
@@ -234,7 +243,8 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
             for (int u = 0; u < 8; ++u) {
                 const int j = 4 * u + (lane >> 3), c = lane & 7;
                 v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (4 * u < n_pad) v[u] = *reinterpret_cast<const float4 *>(st + off_raw + h * raw_bytes + j * 128 + ((c ^ (j & 7)) << 4));
+                const int piece = a.wide ? 2 * j + h : h * n_pad + j;        // where row j of this warp's k-block landed
+                if (4 * u < n_pad) v[u] = *reinterpret_cast<const float4 *>(st + off_raw + piece * 128 + ((c ^ (piece & 7)) << 4));
             }
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
@@ -274,11 +284,13 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
             const uint32_t sround = small_div(it, inv_stages), around = small_div(it, inv_abufs);
             const int s = (int)(it - sround * n_stages), g = (int)(it - around * n_abufs);
             if (!mbar_wait(bar_full(s), sround & 1, abortp)) break;
-            const uint8_t *src = ring + (size_t)s * stage_bytes + row * 128;     // the two V boxes are contiguous
+            // this lane's 128 bytes: box h, row r (two boxes one after the other), or row r, piece h (one box)
+            const int piece = a.wide ? (((row & 63) << 1) | (row >> 6)) : row;
+            const uint8_t *src = ring + (size_t)s * stage_bytes + piece * 128;
             float4 v[8];
             uint32_t hi[32], lo[32];
 #pragma unroll
-            for (int c = 0; c < 8; ++c) v[c] = *reinterpret_cast<const float4 *>(src + ((c ^ (row & 7)) << 4));
+            for (int c = 0; c < 8; ++c) v[c] = *reinterpret_cast<const float4 *>(src + ((c ^ (piece & 7)) << 4));
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_empty(s));
 #pragma unroll
@@ -387,6 +399,38 @@ cudaError_t launch_lsq_tc(Context &c, const LsqArgs &a, int max_slabs, int *slab
     const int n_pad = a.n_r <= 16 ? 16 : 32;
     CUtensorMap map_v, map_a, map_x;
     cuuint32_t ones[3] = {1, 1, 1};
+    const bool wide = a.d % kQBlockK == 0 && a.ldv % kQBlockK == 0;
+    if (wide) {
+        // [row][k-block][32]: the k-blocks of a row are 128 bytes apart, the rows ldv (or d) elements
+        const cuuint64_t nkb_all = (cuuint64_t)(a.d / kQBlockK);
+        {
+            cuuint64_t dims[3] = {kQBlockK, nkb_all, (cuuint64_t)a.m};
+            cuuint64_t strides[2] = {128, (cuuint64_t)a.ldv * 4};
+            cuuint32_t box[3] = {kQBlockK, 2, kHalfRows};
+            if (enc(&map_v, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(a.V), dims, strides, box, ones,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                return cudaErrorInvalidValue;
+        }
+        {
+            cuuint64_t dims[3] = {kQBlockK, nkb_all, (cuuint64_t)a.n_r};
+            cuuint64_t strides[2] = {128, (cuuint64_t)a.d * 4};
+            cuuint32_t box[3] = {kQBlockK, 2, (cuuint32_t)n_pad};
+            if (enc(&map_a, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(a.A), dims, strides, box, ones,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                return cudaErrorInvalidValue;
+        }
+        {
+            cuuint64_t dims[3] = {(cuuint64_t)a.d, 1, 1};
+            cuuint64_t strides[2] = {(cuuint64_t)a.d * 4, (cuuint64_t)a.d * 4};
+            cuuint32_t box[3] = {2 * kQBlockK, 1, 1};
+            if (enc(&map_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(a.x), dims, strides, box, ones,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                return cudaErrorInvalidValue;
+        }
+    } else {
     {
         cuuint64_t dims[3] = {(cuuint64_t)a.d, (cuuint64_t)a.m, 1};
         cuuint64_t strides[2] = {(cuuint64_t)a.ldv * 4, (cuuint64_t)a.ldv * 4 * (cuuint64_t)a.m};
@@ -414,6 +458,7 @@ cudaError_t launch_lsq_tc(Context &c, const LsqArgs &a, int max_slabs, int *slab
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return cudaErrorInvalidValue;
     }
+    }
     const int64_t n_kblocks = (a.d + kQBlockK - 1) / kQBlockK;
     int blocks = c.sm_count > 0 ? c.sm_count : 148;
     if (blocks > max_slabs) blocks = max_slabs;
@@ -422,6 +467,7 @@ cudaError_t launch_lsq_tc(Context &c, const LsqArgs &a, int max_slabs, int *slab
     t.m = a.m;
     t.n_r = a.n_r;
     t.n_pad = n_pad;
+    t.wide = wide ? 1 : 0;
     t.nkb = (int)((n_kblocks + 2 * (int64_t)blocks - 1) / (2 * (int64_t)blocks));
     const int stage_bytes = lsq_stage_bytes(n_pad);
     t.stages = (kQSmem - 1024) / stage_bytes;

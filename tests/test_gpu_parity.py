@@ -48,6 +48,9 @@ SHRUNK = {
     "cfg2_seven_classes": (2, dict(dims=(520, 200, 300, 7), n_r=30, m=12, b=5, faults=[(5, "noise200")])),
     "cfg5_small": (5, dict(d=70000, m=13, b=5, n_r=16, n_noise=5)),
     "cfg5_nr5": (5, dict(d=33333 * 4, m=70, b=30, n_r=5, n_noise=30)),
+    # d a multiple of 32: the tensor-core stream fetches both k-blocks of a pair with one copy per operand
+    "cfg5_d_mult_32": (5, dict(d=69632 + 32, m=37, b=12, n_r=16, n_noise=12)),
+    "cfg5_d_mult_32_nr30": (5, dict(d=40960, m=64, b=20, n_r=30, n_noise=20, gamma=0.1)),
     "cfg5_nr40": (5, dict(d=9000, m=6, b=2, n_r=40, n_noise=2)),
     # the tensor-core least-squares stream with 32 padded samples (N = 128) and all 64 candidate lanes in use,
     # a parameter count that leaves a ragged last k-block pair

@@ -171,7 +171,9 @@ zeno_status zeno_step_host(zeno_handle h, const void *x, const void *V, int64_t 
                            void *stream);
 
 /* Least-squares scores for callers that must not allocate.  (The paper has no counterpart: this
- * is a packaging variant of zeno_score for the least-squares loss, same arithmetic, same kernels.)
+ * is a packaging variant of zeno_score for the least-squares loss.  It always runs the CUDA-core
+ * streaming kernel, whereas a handle takes the tensor-core stream for aligned shapes of up to 64
+ * candidates: the two agree to the tolerances the tests use, not bit for bit.)
  * Some users of this library cannot call cudaMalloc at the point where they need a score: a
  * serving loop that promised its host framework not to touch the allocator after start-up
  * (cudaMalloc synchronises the whole device and would stall every other stream), or a process
@@ -180,13 +182,17 @@ zeno_status zeno_step_host(zeno_handle h, const void *x, const void *V, int64_t 
  * products, about 1.4 MB) is a fixed array inside the library image, present on every GPU that
  * loads the library for the life of the process.
  *   - All pointers are device pointers on `device`; x [d], V [m x ldv], A [n_r x d], y [n_r];
- *     scores[m] required, losses[m+1] and norms[m] optional (NULL).  Same results as
- *     zeno_score on a least-squares handle.
+ *     scores[m] required, losses[m+1] and norms[m] optional (NULL).  Same quantities as
+ *     zeno_score on a least-squares handle (equal within 1e-4 relative on the scores, see above).
  *   - m <= ZENO_STATIC_MAX_M and n_r <= ZENO_STATIC_MAX_N_R, else ZENO_ERR_WORKSPACE (the scratch
  *     is fixed).  Other argument errors: ZENO_ERR_INVALID_ARG, as for zeno_score.
- *   - The first call on a device looks up the array's device address (no allocation, but a
- *     runtime query): make that first call before any stream capture begins.
- *   - No cudaMalloc / cudaFree / allocating routine is called, ever.
+ *   - The first call on a device looks up the array's device address, which makes the CUDA
+ *     runtime load the library's code and data (this array included) onto that device if it has
+ *     not done so yet -- the one moment at which device memory is claimed on the caller's behalf.
+ *     Make that first call at start-up: before the process hands the rest of the device's memory
+ *     to its own pool, and before any stream capture begins.  Later calls only launch kernels.
+ *     First calls from several host threads are serialised inside the library.
+ *   - The call itself invokes no cudaMalloc / cudaFree / allocating routine, ever.
  *   - All calls on a device share the one array and nothing in it needs clearing between calls
  *     (each call rewrites every partial it later reads), but two calls whose kernels overlap on
  *     the GPU (different streams, no ordering) race on it: order them. */

@@ -133,6 +133,8 @@ zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv,
     tail.scores = scores;
     tail.norms_out = norms;
     tail.norm_tot = c->norms;
+    tail.loss_sum = c->loss_sum;
+    tail.n_r = n_r;
     tail.idx = idx;
     tail.keep = keep;
     tail.ticket = c->tickets;
@@ -142,7 +144,7 @@ zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv,
     const bool fuse_loss = zeno::mlp_can_fuse_loss(classes, n_r);
     const size_t esz0 = elem_size(c->desc.param_dtype);
     const bool tc_rows = aligned && is_aligned(x, 16) && is_aligned(V, 16) && (ldv * esz0) % 16 == 0 &&
-                         !getenv("ZENO_DISABLE_TENSOR_CORES");
+                         c->use_tc;
     // layers served by the streamed tensor-core kernel: every layer of a bfloat16 model it can take,
     // the wide later layers of an fp32 model (the first one goes to the stream that shares the batch)
     auto layer_tc_serves = [&](int l) {
@@ -285,7 +287,7 @@ zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv,
         a.first_in_call = l == 0;
         // 16-byte aligned rows of eight-parameter multiples take the warp-MMA kernel
         const size_t esz = elem_size(c->desc.param_dtype);
-        const bool mma = !a.fuse_loss && aligned && !getenv("ZENO_DISABLE_TENSOR_CORES") &&
+        const bool mma = !a.fuse_loss && aligned && c->use_tc &&
                          zeno::mlp_mma_usable(a.in, a.out) && is_aligned(x, 16) && is_aligned(V, 16) &&
                          (ldv * esz) % 16 == 0 && (a.offW * esz) % 16 == 0;
         tail.used.base[l] = c->np_base[l];
@@ -359,7 +361,9 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
     c->device = device;
     c->m_max = m_max;
     c->n_r_max = n_r_max;
+    // the environment switches are read here, once: no call on the handle looks at them again
     c->chain = getenv("ZENO_DISABLE_PDL") == nullptr;
+    c->use_tc = getenv("ZENO_DISABLE_TENSOR_CORES") == nullptr;
 
     DeviceGuard guard(device);
     cudaDeviceProp prop;
@@ -384,7 +388,7 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
             if (desc->has_bias) off += o;
             c->np_base[l] = slots;
             int layer_slots = zeno::mlp_norm_slots((int)o);
-            if (l == 0 && desc->param_dtype == ZENO_F32 && !getenv("ZENO_DISABLE_TENSOR_CORES")) {
+            if (l == 0 && desc->param_dtype == ZENO_F32 && c->use_tc) {
                 // the tensor-core stream may serve the first layer: size its partials and norm slots
                 // for the shortest k-range any plan may pick
                 zeno::StreamTcPlan probe;
@@ -399,7 +403,7 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
                 }
             }
             if (zeno::layer_tc_usable((zeno_dtype)desc->param_dtype, (int)in, (int)o, n_r_max < 128 ? n_r_max : 128) &&
-                !getenv("ZENO_DISABLE_TENSOR_CORES")) {
+                c->use_tc) {
                 if (zeno::layer_tc_norm_slots((int)o) > layer_slots) layer_slots = zeno::layer_tc_norm_slots((int)o);
                 const size_t need = (l == 0 ? 1 : rows) * 2 * (size_t)zeno::layer_tc_n_pad(n_r_max < 128 ? n_r_max : 128) *
                                     (size_t)in;
@@ -410,7 +414,7 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
             }
             // a small last layer may be folded into a tensor-core layer before it: partial logits and
             // norm partials per (128-row tile of that layer, epilogue warp)
-            if (l >= 1 && l + 1 == desc->n_layers && o <= zeno::kHeadMaxClasses && !getenv("ZENO_DISABLE_TENSOR_CORES") &&
+            if (l >= 1 && l + 1 == desc->n_layers && o <= zeno::kHeadMaxClasses && c->use_tc &&
                 zeno::layer_tc_usable((zeno_dtype)desc->param_dtype, (int)desc->dims[l - 1], (int)in,
                                       n_r_max < 128 ? n_r_max : 128)) {
                 const int hs = zeno::layer_tc_head_slots((int)in);
@@ -441,7 +445,7 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
     const size_t at_status = reserve(1, 4), at_tc = reserve(tc_elems, 4);
     const size_t at_tickets = reserve(ticket_elems, 4);
     const size_t at_split0 = reserve(split_elems, 4), at_split1 = reserve(split_elems, 4);
-    const size_t at_losspart = reserve(rows * 8, 4);
+    const size_t at_losspart = reserve(rows * 8, 8), at_losssum = reserve(rows, 8);
     const size_t at_headz = reserve(head_elems, 4), at_headt = reserve(rows, 4);
 
     e = cudaMalloc(&c->arena, bytes);
@@ -462,7 +466,8 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
     c->dev_status = reinterpret_cast<int *>(base + at_status);
     c->tc_part = reinterpret_cast<float *>(base + at_tc);
     c->tickets = reinterpret_cast<unsigned *>(base + at_tickets);
-    c->loss_part = reinterpret_cast<float *>(base + at_losspart);
+    c->loss_part = reinterpret_cast<double *>(base + at_losspart);
+    c->loss_sum = reinterpret_cast<double *>(base + at_losssum);
     c->act_split[0] = base + at_split0;
     c->act_split[1] = base + at_split1;
     c->head_zpart = head_elems ? reinterpret_cast<float *>(base + at_headz) : nullptr;

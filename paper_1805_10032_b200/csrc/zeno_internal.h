@@ -20,6 +20,15 @@ constexpr int kMaxProfiled = ZENO_MAX_LAYERS + 8;
 // Calls whose per-kernel events are kept for zeno_profile_read.
 constexpr int kProfileDepth = 64;
 
+// cudaFuncSetAttribute acts on the current device only, so "already done" is remembered per device
+// (one of these per kernel instantiation; devices beyond the table are simply set again each time).
+constexpr int kMaxDevices = 64;
+struct PerDeviceOnce {
+    bool done[kMaxDevices] = {};
+    bool need(int device) const { return device < 0 || device >= kMaxDevices || !done[device]; }
+    void mark(int device) { if (device >= 0 && device < kMaxDevices) done[device] = true; }
+};
+
 // Launch shape of the tensor-core stream: k-range length, number of k-ranges, blocks per
 // k-range, padded sample count, 128-row tiles per model, dynamic shared memory, ring depth.
 struct StreamTcPlan { int KR, R, G, n_pad, tiles_per_model, smem_bytes, stages; };
@@ -40,7 +49,8 @@ struct Context {
     int np_slots;                   // norm-partial slots per candidate
     void *arena;                    // the one device allocation everything below is carved from
     float *act[2];                  // activations [m_max+1][n_r_max][widest layer output]
-    float *loss_part;               // [m_max + 1][8] per-block sums of the sample losses
+    double *loss_part;              // [m_max + 1][8] per-block sums of the sample losses
+    double *loss_sum;               // [m_max + 1] per-model sums of the sample losses
     void *act_split[2];             // two-term stacked activations for the streamed tensor-core layers
     float *normpart;                // [m_max][np_slots] partial sums of v^2
     float *lsq_part;                // [slabs][m_max+1][n_r_max+1] partial A.v and v^2
@@ -63,6 +73,7 @@ struct Context {
     int last_wait_code;             // status word read back after a kernel gave up on a bounded wait
     // optional per-kernel timing (zeno_profile): a ring of the last kProfileDepth calls; in a
     // call's slot events[i] is recorded before kernel i and events[n] after the last one
+    bool use_tc;                    // tensor-core kernels allowed (ZENO_DISABLE_TENSOR_CORES unset at zeno_create)
     bool chain;                     // chain a step's kernels with programmatic dependent launch
     bool profile;
     cudaEvent_t events[kProfileDepth][kMaxProfiled + 1];
@@ -94,6 +105,8 @@ struct TailArgs {
     float *scores;
     float *norms_out;   // may be NULL
     float *norm_tot;    // [m] workspace: ||v_i||^2 summed over the layers' partials
+    double *loss_sum;   // [m+1] workspace: each model's sample losses added up in double (not yet divided by n_r)
+    int n_r;
     int32_t *idx;       // used if keep > 0
     int keep;           // m - b, or 0: no ranking wanted
     unsigned *ticket;   // zero between launches
@@ -263,6 +276,22 @@ __device__ __forceinline__ void load_vec4(const __nv_bfloat16 *p, float (&o)[4])
     o[1] = __uint_as_float(t.x & 0xffff0000u);
     o[2] = __uint_as_float(t.y << 16);
     o[3] = __uint_as_float(t.y & 0xffff0000u);
+}
+
+// value rounded to tf32 (10 explicit mantissa bits), ties away from zero in magnitude
+__device__ __forceinline__ float tf32_hi(float a) {
+    return __uint_as_float((__float_as_uint(a) + 0x1000u) & 0xffffe000u);
+}
+
+// (score, index) packed so that unsigned order is "higher score first, then lower index":
+// the score's bits mapped to an order-preserving unsigned integer (NaN ranks with minus
+// infinity, -0 is folded into +0), the index stored complemented in the low half.
+__device__ __forceinline__ unsigned long long rank_key(float s, int index) {
+    if (s != s) s = -INFINITY;   // a NaN score ranks with minus infinity
+    s += 0.0f;                   // -0 -> +0
+    unsigned u = __float_as_uint(s);
+    u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+    return ((unsigned long long)u << 32) | (unsigned)(0xffffffffu - (unsigned)index);
 }
 
 template <typename T> struct is_bf16 { static constexpr bool value = false; };

@@ -160,7 +160,7 @@ __device__ __forceinline__ void head_finish_model(const LayerTcArgs &a, int mode
     }
     epi_sync();
     if (gw == 0) {
-        float l = 0.f;
+        double l = 0.0;
         for (int j = lane; j < a.n_r; j += 32) {
             float zmax = -INFINITY;
             for (int o = 0; o < h.classes; ++o) zmax = fmaxf(zmax, zl[o * n_pad + j]);
@@ -168,12 +168,13 @@ __device__ __forceinline__ void head_finish_model(const LayerTcArgs &a, int mode
             for (int o = 0; o < h.classes; ++o) se += expf(zl[o * n_pad + j] - zmax);   // a NaN logit makes se NaN
             int lab = h.labels[j];
             if (lab < 0 || lab >= h.classes) lab = 0;
-            l += zmax + logf(se) - zl[lab * n_pad + j];
+            l += (double)((zmax - zl[lab * n_pad + j]) + logf(se));
         }
 #pragma unroll
         for (int sft = 16; sft >= 1; sft >>= 1) l += __shfl_xor_sync(0xffffffffu, l, sft);
         if (lane == 0) {
-            h.losses[model] = l / (float)a.n_r;
+            h.tail.loss_sum[model] = l;
+            h.losses[model] = (float)(l / (double)a.n_r);
             __threadfence();
         }
     } else if (gw == 1 && model > 0) {
@@ -658,7 +659,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     }
     if (HEAD && head_final) {               // block-uniform: written before the teardown's barrier
         __threadfence();
-        finalize_and_select(a.head.tail, a.head.losses);
+        finalize_and_select(a.head.tail);
     }
 }
 
@@ -767,11 +768,11 @@ cudaError_t launch_typed(Context &c, const LayerTcLaunch &l, cudaStream_t s) {
     a.np_base = l.np_base;
     a.status = c.dev_status;
     if (HEAD) a.head = *l.head; else a.head = HeadFuse{};
-    static bool attr_set = false;       // per instantiation
-    if (!attr_set) {
+    static PerDeviceOnce attr_set;      // per instantiation and device
+    if (attr_set.need(c.device)) {
         e = cudaFuncSetAttribute(layer_tc_kernel<T, LINEAR, HEAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, budget);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_set.mark(c.device);
     }
     const int items = (l.m + 1) * a.tiles;
     const int sms = c.sm_count > 0 ? c.sm_count : 148;

@@ -8,6 +8,8 @@
 // against it with per-lane register accumulators.  Per-slab partial sums are written out and
 // combined in a fixed order (in double) by a one-block finishing kernel, which also forms the
 // losses and the scores.
+#include <mutex>
+
 #include "zeno_internal.h"
 
 namespace zeno {
@@ -264,7 +266,7 @@ cudaError_t launch_lsq_score(Context &c, const LsqArgs &a_in, const float *y, fl
     a.slabs = slabs;
     cudaError_t e;
     ++*launches;
-    if (lsq_tc_usable(a, aligned) && !getenv("ZENO_DISABLE_TENSOR_CORES")) {
+    if (lsq_tc_usable(a, aligned) && c.use_tc) {
         // up to 64 candidates on aligned rows: the tensor-core stream (one slab per block)
         profile_mark(c, "lsq_tc", s);
         e = launch_lsq_tc(c, a, lsq_slab_count(c), &slabs, s);
@@ -303,14 +305,16 @@ constexpr size_t kStaticScratchFloats =
 
 static __device__ __align__(256) float g_static_scratch[kStaticScratchFloats];
 
-constexpr int kMaxDevices = 64;
+using zeno::kMaxDevices;
 float *g_static_scratch_ptr[kMaxDevices];      // device address of the array, per device
 int g_static_sms[kMaxDevices];
 bool g_static_ready[kMaxDevices];
+std::mutex g_static_mutex;                     // host threads may make their first calls at the same time
 
 // In host code `g_static_scratch` is only a handle for the runtime, not an address a kernel can
 // use: the device address is asked for once per device, with that device current.
 cudaError_t static_scratch_setup(int device) {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
     if (g_static_ready[device]) return cudaSuccess;
     float *ptr = nullptr;
     cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void **>(&ptr), g_static_scratch);

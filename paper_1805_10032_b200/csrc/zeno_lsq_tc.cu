@@ -386,10 +386,11 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
 }  // namespace
 
 // Rows a TMA box can step through (16-byte multiples), at most 64 candidates (one half tile) and
-// 32 samples.
+// 32 samples; the copies take the parameter index as a signed 32-bit coordinate, so d stays below 2^31
+// (longer vectors go to the CUDA-core stream, which indexes in 64 bits).
 bool lsq_tc_usable(const LsqArgs &a, bool aligned) {
     return aligned && a.m >= 1 && a.m <= kHalfRows && a.n_r >= 1 && a.n_r <= 32 && a.d % 4 == 0 && a.ldv % 4 == 0 &&
-           a.d >= 4096 && encode_tiled_fn() != nullptr;
+           a.d >= 4096 && a.d < (int64_t(1) << 31) && encode_tiled_fn() != nullptr;
 }
 
 // Fills a.part with one slab per block; *slabs = the number of slabs written.
@@ -476,11 +477,11 @@ cudaError_t launch_lsq_tc(Context &c, const LsqArgs &a, int max_slabs, int *slab
     if (t.n_abufs > kQMaxABufs) t.n_abufs = kQMaxABufs;
     t.part = a.part;
     t.status = c.dev_status;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceOnce attr_set;
+    if (attr_set.need(c.device)) {
         cudaError_t e = cudaFuncSetAttribute(lsq_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kQSmem);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_set.mark(c.device);
     }
     *slabs = blocks;
     return launch_chained(lsq_tc_kernel, dim3(blocks), dim3(kQThreads), (size_t)t.stages * stage_bytes + 1024, s,

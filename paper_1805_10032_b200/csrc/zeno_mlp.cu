@@ -58,6 +58,11 @@ __device__ __forceinline__ float warp_sum(float v) {
     for (int s = 16; s >= 1; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
     return v;
 }
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int s = 16; s >= 1; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
+    return v;
+}
 
 __device__ __forceinline__ float relu_keep_nan(float z) { return (z > 0.f || z != z) ? z : 0.f; }
 
@@ -402,7 +407,7 @@ __global__ void __launch_bounds__(256, 1) mlp_head_kernel(LayerArgs a) {
     __syncthreads();
     if (has_v) block_norm_total(a.tail, c - 1);          // all layers' partials of this candidate
     if (warp == 0) {
-        float l = 0.f;
+        double l = 0.0;
         for (int j = lane; j < a.n_r; j += 32) {
             float zmax = -INFINITY;
             for (int o = 0; o < a.out; ++o) zmax = fmaxf(zmax, zl[o][j]);
@@ -410,12 +415,15 @@ __global__ void __launch_bounds__(256, 1) mlp_head_kernel(LayerArgs a) {
             for (int o = 0; o < a.out; ++o) se += expf(zl[o][j] - zmax);   // a NaN logit makes se NaN
             int lab = a.labels[j];
             if (lab < 0 || lab >= a.out) lab = 0;
-            l += zmax + logf(se) - zl[lab][j];
+            l += (double)((zmax - zl[lab][j]) + logf(se));
         }
         l = warp_sum(l);
-        if (lane == 0) a.losses[c] = l / (float)a.n_r;
+        if (lane == 0) {
+            a.tail.loss_sum[c] = l;
+            a.losses[c] = (float)(l / (double)a.n_r);
+        }
     }
-    if (take_last_ticket(a.tail.ticket, gridDim.x)) finalize_and_select(a.tail, a.losses);
+    if (take_last_ticket(a.tail.ticket, gridDim.x)) finalize_and_select(a.tail);
 }
 
 // Per model: mean over the samples of log-sum-exp(z) - z[label].  G blocks per model (block g takes
@@ -423,14 +431,14 @@ __global__ void __launch_bounds__(256, 1) mlp_head_kernel(LayerArgs a) {
 // sums in loss_part and the last block to finish adds them up, model by model, before it runs the
 // tail.  G = 1 for small problems: the block writes the model's loss itself.
 __global__ void __launch_bounds__(256) mlp_loss_kernel(const float *logits, const int32_t *labels,
-                                                        int n_r, int classes, float *losses, float *loss_part,
+                                                        int n_r, int classes, float *losses, double *loss_part,
                                                         int G, TailArgs tail) {
-    __shared__ float per_warp[8];
+    __shared__ double per_warp[8];
     pdl_launch_dependents();
     pdl_wait();
     const int c = blockIdx.x / G, g = blockIdx.x - c * G;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    float mine = 0.f;
+    double mine = 0.0;
     for (int j = g + warp * G; j < n_r; j += 8 * G) {
         const float *z = logits + ((int64_t)c * n_r + j) * classes;
         float zmax = -INFINITY;
@@ -442,28 +450,33 @@ __global__ void __launch_bounds__(256) mlp_loss_kernel(const float *logits, cons
         se = warp_sum(se);
         int lab = labels[j];
         if (lab < 0 || lab >= classes) lab = 0;
-        mine += zmax + logf(se) - z[lab];   // identical in every lane of the warp
+        mine += (double)((zmax - z[lab]) + logf(se));   // identical in every lane of the warp
     }
     if (lane == 0) per_warp[warp] = mine;
     __syncthreads();
     if (threadIdx.x == 0) {
-        float t = 0.f;
+        double t = 0.0;
         for (int w = 0; w < 8; ++w) t += per_warp[w];
-        if (G == 1) losses[c] = t / (float)n_r;
-        else loss_part[blockIdx.x] = t;
+        if (G == 1) {
+            tail.loss_sum[c] = t;
+            losses[c] = (float)(t / (double)n_r);
+        } else {
+            loss_part[blockIdx.x] = t;
+        }
     }
     if (c > 0 && g == 0) block_norm_total(tail, c - 1);
     if (take_last_ticket(tail.ticket, gridDim.x)) {
         if (G > 1) {
             for (int i = threadIdx.x; i <= tail.m; i += blockDim.x) {
-                float t = 0.f;
+                double t = 0.0;
                 for (int q = 0; q < G; ++q) t += __ldcg(loss_part + i * G + q);
-                losses[i] = t / (float)n_r;
+                tail.loss_sum[i] = t;
+                losses[i] = (float)(t / (double)n_r);
             }
             __threadfence();
             __syncthreads();
         }
-        finalize_and_select(tail, losses);
+        finalize_and_select(tail);
     }
 }
 

@@ -44,9 +44,6 @@ template <bool BF16> __device__ __forceinline__ int swizzle_slot(int slot) {
     return BF16 ? slot : slot ^ (((slot >> 3) & 1) << 1);
 }
 
-__device__ __forceinline__ float tf32_hi(float a) {
-    return __uint_as_float((__float_as_uint(a) + 0x1000u) & 0xffffe000u);
-}
 __device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm volatile(
         "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"

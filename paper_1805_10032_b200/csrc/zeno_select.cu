@@ -12,14 +12,6 @@ namespace zeno {
 
 namespace {
 
-__device__ __forceinline__ unsigned long long rank_key(float s, int index) {
-    if (s != s) s = -INFINITY;   // a NaN score ranks with minus infinity
-    s += 0.0f;                   // -0 -> +0
-    unsigned u = __float_as_uint(s);
-    u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-    return ((unsigned long long)u << 32) | (unsigned)(0xffffffffu - (unsigned)index);
-}
-
 __global__ void __launch_bounds__(1024) select_kernel(const float *scores, int m, int keep,
                                                        int32_t *idx) {
     __shared__ unsigned long long keys[ZENO_MAX_CANDIDATES];

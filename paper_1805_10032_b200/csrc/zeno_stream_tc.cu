@@ -596,12 +596,12 @@ cudaError_t launch_stream_tc(Context &c, const StreamTcPlan &p, const float *x, 
     a.tiles_per_model = p.tiles_per_model;
     a.stages = p.stages;
     a.status = c.dev_status;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceOnce attr_set;
+    if (attr_set.need(c.device)) {
         cudaError_t e = cudaFuncSetAttribute(stream_tf32x3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              kSmemBudget);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_set.mark(c.device);
     }
     ++*launches;
     profile_mark(c, "stream_tf32x3", s);

@@ -6,17 +6,6 @@
 
 namespace zeno {
 
-// (score, index) packed so that unsigned order is "higher score first, then lower index":
-// the score's bits mapped to an order-preserving unsigned integer (NaN ranks with minus
-// infinity, -0 is folded into +0), the index stored complemented in the low half.
-__device__ __forceinline__ unsigned long long rank_key(float s, int index) {
-    if (s != s) s = -INFINITY;
-    s += 0.0f;
-    unsigned u = __float_as_uint(s);
-    u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-    return ((unsigned long long)u << 32) | (unsigned)(0xffffffffu - (unsigned)index);
-}
-
 // Called by ALL threads of a block.  Returns true in the block that took the last ticket, after
 // making the other blocks' global writes visible to it.
 __device__ __forceinline__ bool take_last_ticket(unsigned *ticket, unsigned n_blocks) {
@@ -69,16 +58,20 @@ __device__ __forceinline__ void block_norm_total(const TailArgs &t, int i) {
 // One block, any size.  norms[i] = the per-candidate totals left by block_norm_total;
 // scores[i] = f_0 - f_i - rho norms[i]; if keep > 0, idx[0..keep) = the candidates with the
 // highest scores in rank order (bitonic sort of the packed keys in shared memory).
-__device__ __forceinline__ void finalize_and_select(const TailArgs &t, const float *losses) {
+// The loss difference is formed in double from the models' loss sums (t.loss_sum), so that the
+// score of a candidate whose loss is close to f_0 is not rounded twice to binary32 before the
+// terms cancel; only the finished score is rounded.
+__device__ __forceinline__ void finalize_and_select(const TailArgs &t) {
     __shared__ unsigned long long keys[ZENO_MAX_CANDIDATES];
     int n = 32;
     while (n < t.m) n <<= 1;
-    const float f0 = __ldcg(losses);
+    const double s0 = __ldcg(t.loss_sum);
+    const double inv_n = 1.0 / (double)t.n_r;
     for (int i = threadIdx.x; i < n; i += blockDim.x)
         if (i >= t.m) keys[i] = 0ull;      // padding: below every real key
     for (int i = threadIdx.x; i < t.m; i += blockDim.x) {
         const float nv = __ldcg(t.norm_tot + i);
-        const float sc = f0 - __ldcg(losses + 1 + i) - t.rho * nv;
+        const float sc = (float)((s0 - __ldcg(t.loss_sum + 1 + i)) * inv_n - (double)t.rho * (double)nv);
         if (t.norms_out) t.norms_out[i] = nv;
         t.scores[i] = sc;
         keys[i] = rank_key(sc, i);

@@ -114,11 +114,6 @@ __device__ __forceinline__ uint32_t small_div(uint32_t a, float inv_b) {
     return (uint32_t)__float2int_rd(((float)a + 0.5f) * inv_b);
 }
 
-// value rounded to tf32 (10 explicit mantissa bits), ties away from zero in magnitude
-__device__ __forceinline__ float tf32_hi(float a) {
-    return __uint_as_float((__float_as_uint(a) + 0x1000u) & 0xffffe000u);
-}
-
 // K-major operand in the 128-byte swizzled layout: rows of 128 bytes, groups of 8 rows 1024
 // bytes apart (stride-dimension offset), descriptor version 1, swizzle mode 2 (128 B).
 __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {

@@ -39,14 +39,19 @@ def _reference(w):
     return s.cpu().numpy(), losses.cpu().numpy(), norms.cpu().numpy()
 
 
-def _static(w, with_optional):
+def _static(w, with_optional, check_memory=False):
     x, V, A, y = P.to_device(w)
     # every buffer comes from the caller; the call itself allocates nothing
     scores = torch.full((w.m,), float("nan"), dtype=torch.float32, device="cuda")
     losses = torch.full((w.m + 1,), float("nan"), dtype=torch.float32, device="cuda") if with_optional else None
     norms = torch.full((w.m,), float("nan"), dtype=torch.float32, device="cuda") if with_optional else None
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
     zeno.score_lsq_static(x, V, A, y, w.gamma, w.rho, scores, losses, norms, ldv=w.ldv)
     torch.cuda.synchronize()
+    if check_memory:
+        # not the first call in this process: the device's free memory is what it was before the call
+        assert torch.cuda.mem_get_info()[0] == free_before
     return (scores.cpu().numpy(), None if losses is None else losses.cpu().numpy(),
             None if norms is None else norms.cpu().numpy())
 
@@ -54,9 +59,9 @@ def _static(w, with_optional):
 def test_two_calls_in_a_row_match_the_handle_based_scores(oracle):
     first = syn.make_config(5, d=70000, m=13, b=5, n_r=16, n_noise=5)
     second = syn.make_config(5, d=33333 * 4, m=40, b=12, n_r=5, n_noise=12, seed=77)
-    for w, with_optional in ((first, True), (second, False)):
+    for call, (w, with_optional) in enumerate(((first, True), (second, False))):
         want_s, want_f, want_n = _reference(w)
-        got_s, got_f, got_n = _static(w, with_optional)
+        got_s, got_f, got_n = _static(w, with_optional, check_memory=call > 0)
         assert np.all(np.abs(got_s - want_s) <= P.SCORE_RTOL * np.abs(want_s))
         if with_optional:
             assert np.allclose(got_f, want_f, rtol=1e-5, atol=1e-7)
@@ -64,6 +69,20 @@ def test_two_calls_in_a_row_match_the_handle_based_scores(oracle):
         # and both agree with the float64 oracle
         s_orc, _, _ = P.oracle_score(oracle, w)
         P.assert_scores_close(got_s, s_orc)
+
+
+@pytest.mark.parametrize("shape", [
+    dict(d=4099, m=5, b=2, n_r=3, n_noise=2, ldv=4101),          # rows that are not 16-byte aligned: scalar loads
+    dict(d=50000, m=64, b=20, n_r=24, n_noise=20),               # 17..32 samples, every candidate slot in use
+    dict(d=20004, m=7, b=2, n_r=32, n_noise=2, gamma=0.1),       # the largest sample count the scratch holds
+])
+def test_other_kernel_instantiations(oracle, shape):
+    w = syn.make_config(5, **shape)
+    _static(w, False)                                            # whatever ran before, this is not the first call
+    got_s, got_f, got_n = _static(w, True, check_memory=True)
+    s_orc, f_orc, n_orc = P.oracle_score(oracle, w)
+    P.assert_scores_close(got_s, s_orc, f_orc, n_orc, float(np.float32(w.rho)))
+    assert np.allclose(got_n, n_orc, rtol=1e-5)
 
 
 def test_sizes_beyond_the_fixed_scratch_are_refused():

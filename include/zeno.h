@@ -205,6 +205,17 @@ zeno_status zeno_score_lsq_static(int32_t device, const float *x, const float *V
  * ZENO_OK.  The condition is sticky for the life of the handle. */
 zeno_status zeno_device_status(zeno_handle h, void *stream);
 
+/* Test hook for the give-up path of the bounded device-side waits.  Every wait a tensor-core kernel
+ * makes on one of its barriers polls at most `polls` times (default 2^22, a few tenths of a second)
+ * before it gives up, raises the status word that zeno_device_status reads and lets the block leave
+ * through its teardown (copies in flight awaited, tensor memory freed) -- the context stays usable.
+ * polls = 0 makes every wait that is not already satisfied give up, and makes every block begin by
+ * waiting, as briefly, for an arrival that never comes -- which is how the tests reach that path for
+ * certain without anything going wrong on the device; the waits of the teardown itself keep the
+ * default.  The outputs of a call that gave up are undefined and the handle's workspace may be left
+ * inconsistent: destroy the handle afterwards. */
+zeno_status zeno_debug_set_wait_limit(zeno_handle h, uint32_t polls);
+
 /* Per-kernel timing for benchmarks.  zeno_profile(h, 1) makes every later call on the handle
  * record a CUDA event on the call's stream before each of its kernels and after the last one
  * (a few microseconds of overhead per call) and keeps the events of the last 64 calls;

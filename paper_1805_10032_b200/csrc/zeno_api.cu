@@ -364,6 +364,7 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
     // the environment switches are read here, once: no call on the handle looks at them again
     c->chain = getenv("ZENO_DISABLE_PDL") == nullptr;
     c->use_tc = getenv("ZENO_DISABLE_TENSOR_CORES") == nullptr;
+    c->spin_limit = zeno::kSpinLimit;
 
     DeviceGuard guard(device);
     cudaDeviceProp prop;
@@ -711,6 +712,12 @@ int32_t zeno_profile_read(zeno_handle h, int32_t back, float *ms, const char **n
         if (names) names[i] = h->kernel_names[slot][i];
     }
     return n;
+}
+
+zeno_status zeno_debug_set_wait_limit(zeno_handle h, uint32_t polls) {
+    if (!h) return ZENO_ERR_INVALID_ARG;
+    h->spin_limit = polls;
+    return ZENO_OK;
 }
 
 int32_t zeno_last_launch_count(zeno_handle h) { return h ? h->last_launches : 0; }

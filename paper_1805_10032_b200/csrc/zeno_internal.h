@@ -29,6 +29,10 @@ struct PerDeviceOnce {
     void mark(int device) { if (device >= 0 && device < kMaxDevices) done[device] = true; }
 };
 
+// Polls of a barrier before a bounded device-side wait gives up: the default of a handle, and the
+// limit of the waits a block's teardown makes after an abort whatever the handle says.
+constexpr uint32_t kSpinLimit = 1u << 22;
+
 // Launch shape of the tensor-core stream: k-range length, number of k-ranges, blocks per
 // k-range, padded sample count, 128-row tiles per model, dynamic shared memory, ring depth.
 struct StreamTcPlan { int KR, R, G, n_pad, tiles_per_model, smem_bytes, stages; };
@@ -60,6 +64,7 @@ struct Context {
     float *scores;                  // [m_max]
     int32_t *idx;                   // [m_max]
     int *dev_status;                // raised by a kernel whose bounded wait gave up
+    uint32_t spin_limit;            // polls a bounded device-side wait may take before it gives up
     bool tc_ok;                     // the tensor-core stream can serve the first layer (fp32 storage)
     int tc_r_max;                   // most k-ranges any plan for it may use
     float *tc_part;                 // [R][m_max+1][n_r_max][dims[1]] split-K partials

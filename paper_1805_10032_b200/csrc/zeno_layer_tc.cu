@@ -98,6 +98,7 @@ struct LayerTcArgs {
     float *normpart;
     int np_slots, np_base;
     int *status;
+    uint32_t spin_limit;   // polls a bounded wait may take
     HeadFuse head;         // used by the HEAD instantiations only
 };
 
@@ -217,8 +218,11 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     // a_full, a_empty [kLMaxABufs]; d_full, d_empty [2]
     constexpr int kBars = 2 * kLMaxStages + 2 * kLMaxBStages + 2 * kLMaxABufs + 2 * kLMaxSets;
     __shared__ __align__(8) uint64_t bars[kBars];
+    __shared__ __align__(8) uint64_t drain_bar;   // teardown after an abort: the issuer's last commit
+    __shared__ __align__(8) uint64_t never_bar;   // nothing arrives here (test hook, see wait_for_nothing)
     __shared__ uint32_t tmem_base_slot;
-    __shared__ int abort_flag;
+    __shared__ int abort_state[kAbortWords];
+    int &abort_flag = abort_state[0];
     __shared__ int issued[kLMaxStages + kLMaxBStages];     // last round a copy was issued into a stage, plus one
     __shared__ int head_last;                  // HEAD: the epilogue group's ticket result
     __shared__ int head_final;                 // HEAD: this block completed the last model
@@ -261,6 +265,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
 
     if (tid == 0) {
         abort_flag = 0;
+        abort_state[1] = (int)a.spin_limit;
         head_final = 0;
         for (int s = 0; s < kLMaxStages; ++s) {
             mbar_init(bar_full(s), 1);
@@ -280,6 +285,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             mbar_init(bar_dfull(q), 1);
             mbar_init(bar_dempty(q), 4);
         }
+        mbar_init(smem_u32(&drain_bar), 1);
+        mbar_init(smem_u32(&never_bar), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {   // TMEM allocation by one full warp
@@ -294,6 +301,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     const uint32_t tmem = tmem_base_slot;
     volatile int *abortp = &abort_flag;
 
+    if (warp == 0) wait_for_nothing(smem_u32(&never_bar), abortp);
     if (warp == 0 || warp == 2) {
         // ------------------------------------------------------------------ TMA producers
         // warp 0 feeds the weight ring (x tile, v tile), warp 2 the activation ring; the two rings
@@ -641,6 +649,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    if (warp == 1 && abort_flag) drain_mmas(smem_u32(&drain_bar));
     if (tid == 0 && abort_flag) {
         // bulk copies still in flight (only after an aborted run) must land before the block exits
         for (int s = 0; s < kLMaxStages + kLMaxBStages; ++s)
@@ -767,6 +776,7 @@ cudaError_t launch_typed(Context &c, const LayerTcLaunch &l, cudaStream_t s) {
     a.np_slots = c.np_slots;
     a.np_base = l.np_base;
     a.status = c.dev_status;
+    a.spin_limit = c.spin_limit;
     if (HEAD) a.head = *l.head; else a.head = HeadFuse{};
     static PerDeviceOnce attr_set;      // per instantiation and device
     if (attr_set.need(c.device)) {

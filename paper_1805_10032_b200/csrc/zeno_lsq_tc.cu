@@ -53,6 +53,7 @@ struct LsqTcArgs {
     int wide;                               // the tensor maps fetch both k-blocks of a pair in one copy (d % 32 == 0)
     float *part;                            // [blocks][m+1][n_r+1]
     int *status;
+    uint32_t spin_limit;                    // polls a bounded wait may take
 };
 
 // bytes of a stage: V halves | [a_hi; a_lo] halves | raw A halves | x pieces (padded to 1 KB)
@@ -66,8 +67,11 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
     // full, empty, bready [stages]; afull, aempty [A buffers]; dfull, dempty [2 sets]
     constexpr int kBars = 3 * kQMaxStages + 2 * kQMaxABufs + 4;
     __shared__ __align__(8) uint64_t bars[kBars];
+    __shared__ __align__(8) uint64_t drain_bar;   // teardown after an abort: the issuer's last commit
+    __shared__ __align__(8) uint64_t never_bar;   // nothing arrives here (test hook, see wait_for_nothing)
     __shared__ uint32_t tmem_base_slot;
-    __shared__ int abort_flag;
+    __shared__ int abort_state[kAbortWords];
+    int &abort_flag = abort_state[0];
     __shared__ int issued[kQMaxStages];
     __shared__ float nrm_s[2][128];         // sums of squares per lane and converter set
     __shared__ float z0_s[2][32];           // A x, per splitter warp
@@ -101,6 +105,7 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
 
     if (tid == 0) {
         abort_flag = 0;
+        abort_state[1] = (int)a.spin_limit;
         for (int s = 0; s < kQMaxStages; ++s) {
             mbar_init(bar_full(s), 1);
             mbar_init(bar_empty(s), 5);        // the four warps of a converter set and the MMAs' commit
@@ -115,6 +120,8 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
             mbar_init(bar_dfull(q), 1);
             mbar_init(bar_dempty(q), 4);
         }
+        mbar_init(smem_u32(&drain_bar), 1);
+        mbar_init(smem_u32(&never_bar), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -131,6 +138,7 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
+        wait_for_nothing(smem_u32(&never_bar), abortp);
         int s = 0;
         uint32_t round = 0;
         for (int kb = 0; kb < nkb; ++kb) {
@@ -352,6 +360,7 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    if (warp == 1 && abort_flag) drain_mmas(smem_u32(&drain_bar));
     if (tid == 0 && abort_flag) {
         for (int s = 0; s < n_stages; ++s)
             if (issued[s] > 0) {
@@ -477,6 +486,7 @@ cudaError_t launch_lsq_tc(Context &c, const LsqArgs &a, int max_slabs, int *slab
     if (t.n_abufs > kQMaxABufs) t.n_abufs = kQMaxABufs;
     t.part = a.part;
     t.status = c.dev_status;
+    t.spin_limit = c.spin_limit;
     static PerDeviceOnce attr_set;
     if (attr_set.need(c.device)) {
         cudaError_t e = cudaFuncSetAttribute(lsq_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kQSmem);

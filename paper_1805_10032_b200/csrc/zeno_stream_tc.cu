@@ -77,6 +77,7 @@ struct StreamArgs {
     int tiles_per_model;   // ceil(out / 128)
     int stages;            // depth of each pipeline's TMA ring (<= kMaxStages)
     int *status;           // device status word (raised on a wait that gave up)
+    uint32_t spin_limit;   // polls a bounded wait may take
 };
 
 // B = the shared batch, A = raw rows of [x; V] (the layer is linear in its weights, the combine
@@ -91,8 +92,11 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     // per pipeline: full[kMaxStages], empty[kMaxStages], a_full[kMaxABufs], a_empty[kMaxABufs], d_full, d_empty
     constexpr int kBarsPerPipe = 2 * kMaxStages + 2 * kMaxABufs + 2;
     __shared__ __align__(8) uint64_t bars[kPipes * kBarsPerPipe];
+    __shared__ __align__(8) uint64_t drain_bar[kPipes];   // teardown after an abort: each issuer's last commit
+    __shared__ __align__(8) uint64_t never_bar;           // nothing arrives here (test hook, see wait_for_nothing)
     __shared__ uint32_t tmem_base_slot;
-    __shared__ int abort_flag;
+    __shared__ int abort_state[kAbortWords];
+    int &abort_flag = abort_state[0];
     __shared__ int issued[kPipes][kMaxStages];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -134,6 +138,7 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
 
     if (tid == 0) {
         abort_flag = 0;
+        abort_state[1] = (int)a.spin_limit;
         for (int p = 0; p < kPipes; ++p) {
             for (int s = 0; s < kMaxStages; ++s) {
                 mbar_init(bar_full(p, s), 1);
@@ -146,7 +151,9 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             }
             mbar_init(bar_dfull(p), 1);
             mbar_init(bar_dempty(p), 4);
+            mbar_init(smem_u32(&drain_bar[p]), 1);
         }
+        mbar_init(smem_u32(&never_bar), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 2) {   // TMEM allocation by one full warp
@@ -222,6 +229,7 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         // The warp stays converged (every lane takes the waits); one elected lane arms the barrier
         // and issues the stage's copies, at ONE issue site.
         const int p = warp;
+        if (p == 0) wait_for_nothing(smem_u32(&never_bar), abortp);
         uint8_t *ring = stage_base + (size_t)p * n_stages * kStage;
         int s = 0;                                 // stage, and how often the ring has wrapped
         uint32_t round = 0;
@@ -392,6 +400,7 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    if (abort_flag && warp >= kPipes && warp < 2 * kPipes) drain_mmas(smem_u32(&drain_bar[warp - kPipes]));
     if (tid == 0) {
         // bulk copies still in flight (only after an aborted run) must land before the block exits
         if (abort_flag) {
@@ -596,6 +605,7 @@ cudaError_t launch_stream_tc(Context &c, const StreamTcPlan &p, const float *x, 
     a.tiles_per_model = p.tiles_per_model;
     a.stages = p.stages;
     a.status = c.dev_status;
+    a.spin_limit = c.spin_limit;
     static PerDeviceOnce attr_set;
     if (attr_set.need(c.device)) {
         cudaError_t e = cudaFuncSetAttribute(stream_tf32x3_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,

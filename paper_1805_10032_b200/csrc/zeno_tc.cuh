@@ -8,7 +8,10 @@
 
 namespace zeno {
 
-constexpr uint32_t kSpinLimit = 1u << 22;   // polls of a barrier before a wait gives up
+// A block's abort state in shared memory: word 0 is the flag (zero until a wait gives up), word 1 the
+// number of polls a wait may take, copied from the launch arguments.  The bounded waits get a pointer
+// to word 0.
+constexpr int kAbortWords = 2;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -35,7 +38,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // probe (with the loop inlined, a wait on the MMA-issuing warp cost about 190 cycles even when the
 // barrier's phase had already completed; a bare probe costs 15 to 20).
 static __device__ __noinline__ bool mbar_wait_poll(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    const uint32_t limit = (uint32_t)abort_flag[1];
+    for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if (i > 32) __nanosleep(40);
         if ((i & 127u) == 127u && *abort_flag) return false;
@@ -49,6 +53,27 @@ static __device__ __noinline__ bool mbar_wait_poll(uint32_t bar, uint32_t parity
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
     if (mbar_try_wait(bar, parity)) return true;
     return mbar_wait_poll(bar, parity, abort_flag);
+}
+// After an aborted run the MMAs a warp issued before the abort may still be running (they read the
+// ring and write TMEM).  Called by that whole warp, converged, before TMEM is freed: one more commit
+// from the lane that issued them, then a bounded wait for it.  `bar` is a barrier of count 1 used
+// for nothing else.
+__device__ __forceinline__ void tc_commit(uint32_t bar);
+__device__ __forceinline__ bool elect_one();
+__device__ __forceinline__ void drain_mmas(uint32_t bar) {
+    if (elect_one()) tc_commit(bar);
+    __syncwarp();
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        if (mbar_try_wait(bar, 0)) break;
+        __nanosleep(64);
+    }
+    __syncwarp();
+}
+// Test hook (a wait limit of zero): the calling warp waits, bounded, for an arrival on a barrier that
+// nothing ever arrives at, so that the block is certain to take its give-up path -- on a small problem
+// every real wait may well be satisfied at its first probe.  `bar` is a barrier used for nothing else.
+__device__ __forceinline__ void wait_for_nothing(uint32_t bar, volatile int *abort_flag) {
+    if (abort_flag[1] == 0) (void)__all_sync(0xffffffffu, mbar_wait(bar, 0, abort_flag));
 }
 // Status word of a block that gave up: kernel id (1 first-layer stream, 2 layer, 3 least squares) in
 // bits 24-27, the index of the barrier within the block's barrier array in bits 1-16, the awaited

@@ -210,30 +210,44 @@ def make_lsq_workload(name, seed, d, m, b, n_r, gamma, rho, honest_std, n_noise,
                     targets=y, honest=honest, seed=seed)
 
 
+# The five benchmark configurations (1-based): recipe parameters only, no tensors.
+CONFIGS = {
+    1: dict(dims=(784, 10), dtype="f32", m=20, b=8, n_r=4, gamma=0.1, rho=5e-4,
+            honest_std=0.1, faults=[(8, "signflip")], x_init="normal0.1"),
+    2: dict(dims=(3072, 512, 512, 10), dtype="f32", m=20, b=8, n_r=32, gamma=0.1, rho=5e-4,
+            honest_std=0.1, faults=[(8, "noise200")]),
+    3: dict(dims=(3072, 512, 512, 10), dtype="f32", m=100, b=40, n_r=64, gamma=0.05,
+            rho=1e-3, honest_std=0.1, faults=[(20, "signflip"), (20, "omniscient")]),
+    4: dict(dims=(4096, 4096, 4096, 1000), dtype="bf16", m=32, b=12, n_r=128, gamma=0.1,
+            rho=5e-4, honest_std=0.05, faults=[(12, "signflip")]),
+    5: dict(d=1 << 26, m=64, b=24, n_r=16, gamma=0.01, rho=1e-4, honest_std=0.01,
+            n_noise=24, noise_std=100.0),
+}
+
+
+def describe_config(index: int) -> dict:
+    """Shape of a benchmark configuration without generating it: kind, dims, dtype, m, b, n_r,
+    gamma, rho, d, ldv (the default row pitch)."""
+    p = CONFIGS[index]
+    if index == 5:
+        kind, dims, dtype = "lsq", (p["d"], 1), "f32"
+    else:
+        kind, dims, dtype = "mlp", tuple(p["dims"]), p["dtype"]
+    d = param_count(kind, dims)
+    return dict(kind=kind, dims=dims, dtype=dtype, m=p["m"], b=p["b"], n_r=p["n_r"], gamma=p["gamma"],
+                rho=p["rho"], d=d, ldv=round_up(d, 32))
+
+
 def make_config(index: int, device="cpu", **ov) -> Workload:
     """The five benchmark configurations (1-based).  Keyword overrides shrink a
     configuration for tests (e.g. dims=(96, 40, 24, 10), m=9, b=3, n_r=5)."""
     seed = ov.pop("seed", BASE_SEED + index)
-    if index == 1:
-        p = dict(dims=(784, 10), dtype="f32", m=20, b=8, n_r=4, gamma=0.1, rho=5e-4,
-                 honest_std=0.1, faults=[(8, "signflip")], x_init="normal0.1")
-    elif index == 2:
-        p = dict(dims=(3072, 512, 512, 10), dtype="f32", m=20, b=8, n_r=32, gamma=0.1, rho=5e-4,
-                 honest_std=0.1, faults=[(8, "noise200")])
-    elif index == 3:
-        p = dict(dims=(3072, 512, 512, 10), dtype="f32", m=100, b=40, n_r=64, gamma=0.05,
-                 rho=1e-3, honest_std=0.1, faults=[(20, "signflip"), (20, "omniscient")])
-    elif index == 4:
-        p = dict(dims=(4096, 4096, 4096, 1000), dtype="bf16", m=32, b=12, n_r=128, gamma=0.1,
-                 rho=5e-4, honest_std=0.05, faults=[(12, "signflip")])
-    elif index == 5:
-        p = dict(d=1 << 26, m=64, b=24, n_r=16, gamma=0.01, rho=1e-4, honest_std=0.01,
-                 n_noise=24, noise_std=100.0)
-        p.update(ov)
-        return make_lsq_workload(f"config5", seed, device=device, **p)
-    else:
+    if index not in CONFIGS:
         raise ValueError("config index must be 1..5")
+    p = dict(CONFIGS[index])
     p.update(ov)
+    if index == 5:
+        return make_lsq_workload("config5", seed, device=device, **p)
     return make_mlp_workload(f"config{index}", seed, device=device, **p)
 
 

@@ -26,6 +26,7 @@ F32, BF16 = 0, 1
 EXPORTS = (
     "zeno_param_count", "zeno_create", "zeno_destroy", "zeno_score", "zeno_select",
     "zeno_aggregate", "zeno_step", "zeno_step_update", "zeno_step_host", "zeno_device_status", "zeno_score_lsq_static",
+    "zeno_debug_set_wait_limit",
     "zeno_profile", "zeno_profile_read",
     "zeno_last_launch_count",
     "zeno_last_cuda_error", "zeno_last_wait_code", "zeno_status_string",
@@ -85,6 +86,8 @@ def load_library() -> ctypes.CDLL:
     lib.zeno_score_lsq_static.argtypes = [i32, vp, vp, i64, i64, i32, vp, vp, i32, f32, f32, vp, vp, vp, vp]
     lib.zeno_device_status.restype = i32
     lib.zeno_device_status.argtypes = [vp, vp]
+    lib.zeno_debug_set_wait_limit.restype = i32
+    lib.zeno_debug_set_wait_limit.argtypes = [vp, ctypes.c_uint32]
     lib.zeno_profile.restype = i32
     lib.zeno_profile.argtypes = [vp, i32]
     lib.zeno_profile_read.restype = i32
@@ -198,6 +201,14 @@ class Zeno:
     def check_device_status(self, stream=None):
         """Synchronises and raises if a kernel gave up on a bounded device-side wait."""
         self._check(self._lib.zeno_device_status(self._h, _stream_ptr(stream)), "zeno_device_status")
+
+    def debug_set_wait_limit(self, polls: int):
+        """Test hook: polls a bounded device-side wait may take before it gives up (see zeno.h)."""
+        self._check(self._lib.zeno_debug_set_wait_limit(self._h, int(polls)), "zeno_debug_set_wait_limit")
+
+    @property
+    def last_wait_code(self) -> int:
+        return int(self._lib.zeno_last_wait_code(self._h))
 
     def profile(self, enable: bool = True):
         self._check(self._lib.zeno_profile(self._h, int(enable)), "zeno_profile")

@@ -159,6 +159,22 @@ zeno_status zeno_step_update(zeno_handle h, void *x, const void *V, int64_t ldv,
                              const zeno_batch *batch, float gamma, float rho, int32_t b, float *out,
                              float *scores, int32_t *idx, void *stream);
 
+/* Algorithm 1's server loop for `steps` iterations on one stream with no host synchronisation in between:
+ * iteration t scores the candidates V_t against the batch z_t at the current x, ranks them, and applies
+ * x <- x - gamma Zeno_b(V_t) in the pass that forms the average (zeno_step_update without the out vector).
+ * The candidates and batches of all iterations are laid out one after the other:
+ *   V:        iteration t's [m x ldv] matrix starts step_stride_v elements after iteration t - 1's
+ *             (step_stride_v >= m * ldv);
+ *   features: [steps][n_r x dims[0]] binary32, contiguous;   targets: [steps][n_r] (int32 or float);
+ *   scores:   [steps][m] or NULL;   idx: [steps][m - b] or NULL.
+ * x is read and updated in place by every iteration.  The candidates are inputs: they are what the workers
+ * sent for these iterations, however the caller obtained them.  The profiler (zeno_profile) sees the whole
+ * run as one call and keeps only the kernels that fit its per-call list.
+ * INVALID_ARG: as zeno_step_update, or steps < 1, or step_stride_v < m * ldv. */
+zeno_status zeno_run(zeno_handle h, void *x, const void *V, int64_t ldv, int64_t step_stride_v, int32_t m,
+                     const float *features, const void *targets, int32_t n_r, int32_t steps, float gamma,
+                     float rho, int32_t b, float *scores, int32_t *idx, void *stream);
+
 /* The same step for a caller whose data lives in HOST memory (Algorithm 1's server receiving the
  * candidates over the network): x, V, features, targets, out, scores and idx are HOST pointers
  * (pinned memory makes the copies asynchronous).  The call copies the inputs to a device staging

@@ -349,3 +349,94 @@ int zo_step(int kind, int dtype, int n_layers, const int64_t *dims, int has_bias
     if (!idx) free(ix);
     return rc;
 }
+
+/* ---- the baseline aggregation rules on the same candidates ----------------
+ *
+ * Experiments, "Baselines": the marginal median (Definition "Median") and Krum
+ * (Definition "Krum"), written out as their definitions. */
+
+static int zo_cmp_double(const void *a, const void *b)
+{
+    double x = *(const double *)a, y = *(const double *)b;
+    return (x > y) - (x < y);
+}
+
+/* Marginal median: out[j] = the one-dimensional median of the j-th entries of the m
+ * candidates -- the middle one of the sorted values for odd m, the mean of the two
+ * middle ones for even m.  Reading where the paper is silent: a NaN entry (a faulty
+ * worker may send anything) counts as plus infinity. */
+int zo_median(int dtype, const void *V, int64_t ldv, int64_t d, int m, double *out)
+{
+    if (m < 1 || d < 1 || ldv < d) return ZO_BAD_ARG;
+    const size_t esz = dtype == ZO_BF16 ? 2 : 4;
+    int rc = ZO_OK;
+#pragma omp parallel
+    {
+        double *col = (double *)malloc(sizeof(double) * (size_t)m);
+        if (!col) {
+#pragma omp critical
+            rc = ZO_NO_MEM;
+        } else {
+#pragma omp for schedule(static)
+            for (int64_t j = 0; j < d; ++j) {
+                for (int i = 0; i < m; ++i) {
+                    double v = zo_load((const char *)V + (size_t)i * (size_t)ldv * esz, j, dtype);
+                    col[i] = v != v ? INFINITY : v;
+                }
+                qsort(col, (size_t)m, sizeof(double), zo_cmp_double);
+                out[j] = (m & 1) ? col[m / 2] : (col[m / 2 - 1] + col[m / 2]) / 2.0;
+            }
+            free(col);
+        }
+    }
+    return rc;
+}
+
+/* Krum_b: for every candidate i the sum of the squared Euclidean distances to its
+ * m - b - 2 nearest neighbours among the other candidates; the candidate with the
+ * smallest sum is returned (*k_out; ties: the lowest index).  sums[m] receives the
+ * per-candidate sums, dist[m*m] (may be NULL) the squared distances.
+ * The definition needs at least one neighbour: m - b - 2 >= 1.  (The paper notes that
+ * Krum's guarantee needs 2b + 2 < m; its own toy example uses m = 6, b = 2, so that
+ * bound is not enforced here.) */
+int zo_krum(int dtype, const void *V, int64_t ldv, int64_t d, int m, int b,
+            int32_t *k_out, double *sums, double *dist)
+{
+    if (m < 1 || b < 0 || m - b - 2 < 1 || d < 1 || ldv < d) return ZO_BAD_ARG;
+    const size_t esz = dtype == ZO_BF16 ? 2 : 4;
+    double *D = dist ? dist : (double *)malloc(sizeof(double) * (size_t)m * (size_t)m);
+    double *row = (double *)malloc(sizeof(double) * (size_t)m);
+    if (!D || !row) return ZO_NO_MEM;
+#pragma omp parallel for schedule(dynamic)
+    for (int i = 0; i < m; ++i) {
+        const char *vi = (const char *)V + (size_t)i * (size_t)ldv * esz;
+        for (int j = 0; j < m; ++j) {
+            const char *vj = (const char *)V + (size_t)j * (size_t)ldv * esz;
+            double s = 0.0;
+            for (int64_t t = 0; t < d; ++t) {
+                double df = zo_load(vi, t, dtype) - zo_load(vj, t, dtype);
+                s += df * df;
+            }
+            D[(size_t)i * m + j] = s;
+        }
+    }
+    const int nn = m - b - 2;
+    int best = 0;
+    for (int i = 0; i < m; ++i) {
+        int c = 0;
+        for (int j = 0; j < m; ++j)
+            if (j != i) {
+                double v = D[(size_t)i * m + j];
+                row[c++] = v != v ? INFINITY : v;          /* a NaN distance is no neighbour */
+            }
+        qsort(row, (size_t)c, sizeof(double), zo_cmp_double);
+        double s = 0.0;
+        for (int t = 0; t < nn; ++t) s += row[t];
+        sums[i] = s;
+        if (s < sums[best]) best = i;
+    }
+    *k_out = best;
+    free(row);
+    if (!dist) free(D);
+    return ZO_OK;
+}

@@ -65,6 +65,10 @@ def _load():
         lib.zo_step.restype = i32
         lib.zo_step.argtypes = [i32, i32, i32, vp, i32, vp, vp, i64, i32, vp, vp, i32,
                                 dbl, dbl, i32, vp, vp, vp]
+        lib.zo_median.restype = i32
+        lib.zo_median.argtypes = [i32, vp, i64, i64, i32, vp]
+        lib.zo_krum.restype = i32
+        lib.zo_krum.argtypes = [i32, vp, i64, i64, i32, i32, vp, vp, vp]
         lib.zo_eval_count.restype = ctypes.c_longlong
         lib.zo_reset_eval_count.restype = None
         lib.zo_num_threads.restype = i32
@@ -186,6 +190,25 @@ def aggregate(dtype, V, ldv, d, m, idx):
     _check(_load().zo_aggregate(dtype, _ptr(V), int(ldv), int(d), int(m), _ptr(idx),
                                 idx.shape[0], _ptr(out)), "zo_aggregate")
     return out
+
+
+def median(dtype, V, ldv, d, m):
+    """Marginal median of the m candidates (the paper's Median baseline): float64 [d]."""
+    V = _params(V, dtype)
+    out = np.empty(d, dtype=np.float64)
+    _check(_load().zo_median(dtype, _ptr(V), int(ldv), int(d), int(m), _ptr(out)), "zo_median")
+    return out
+
+
+def krum(dtype, V, ldv, d, m, b):
+    """Krum_b (the paper's Krum baseline): returns (k, sums[m], dist[m, m])."""
+    V = _params(V, dtype)
+    k = np.zeros(1, dtype=np.int32)
+    sums = np.empty(m, dtype=np.float64)
+    dist = np.empty((m, m), dtype=np.float64)
+    _check(_load().zo_krum(dtype, _ptr(V), int(ldv), int(d), int(m), int(b), _ptr(k), _ptr(sums),
+                           _ptr(dist)), "zo_krum")
+    return int(k[0]), sums, dist
 
 
 def update(dtype, x, vbar, gamma):

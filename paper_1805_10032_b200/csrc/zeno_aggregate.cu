@@ -89,8 +89,8 @@ __global__ void __launch_bounds__(256) aggregate_vec_kernel(const T *V, int64_t 
                                                              float gamma) {
     constexpr int E = Group<T>::kElems;
     __shared__ int64_t rows_s[ZENO_MAX_CANDIDATES];
-    pdl_launch_dependents();
     pdl_wait();
+    pdl_launch_dependents();
     stage_rows(idx, k, m, ldv, rows_s);
     const int64_t groups = d / E;            // whole groups; the d % E tail columns follow below
     for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < groups;
@@ -149,8 +149,8 @@ __global__ void __launch_bounds__(256) aggregate_scalar_kernel(const T *V, int64
                                                                 int m, const int32_t *idx, int k,
                                                                 float *out, T *xu, float gamma) {
     __shared__ int64_t rows_s[ZENO_MAX_CANDIDATES];
-    pdl_launch_dependents();
     pdl_wait();
+    pdl_launch_dependents();
     stage_rows(idx, k, m, ldv, rows_s);
     for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < d;
          j += (int64_t)gridDim.x * blockDim.x) {

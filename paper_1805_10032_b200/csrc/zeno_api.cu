@@ -377,7 +377,7 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
 
     const size_t rows = (size_t)m_max + 1;
     size_t act_elems = 0, norm_elems = 0, lsq_elems = 0, tc_elems = 0, ticket_elems = 1, split_elems = 0;
-    size_t head_elems = 0;
+    size_t head_elems = 0, splitp_elems = 0, splitt_elems = 0;
     if (desc->kind == ZENO_LOSS_SOFTMAX_MLP) {
         int64_t off = 0, widest = 0;
         int slots = 0;
@@ -406,6 +406,11 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
             if (zeno::layer_tc_usable((zeno_dtype)desc->param_dtype, (int)in, (int)o, n_r_max < 128 ? n_r_max : 128) &&
                 c->use_tc) {
                 if (zeno::layer_tc_norm_slots((int)o) > layer_slots) layer_slots = zeno::layer_tc_norm_slots((int)o);
+                // scratch of the tiles that blocks share: two pieces per block, a ticket per tile
+                const size_t sp = (size_t)c->sm_count * 2 * 128 * (size_t)zeno::layer_tc_n_pad(n_r_max < 128 ? n_r_max : 128);
+                if (sp > splitp_elems) splitp_elems = sp;
+                const size_t tk = rows * (size_t)((o + 127) / 128);
+                if (tk > splitt_elems) splitt_elems = tk;
                 const size_t need = (l == 0 ? 1 : rows) * 2 * (size_t)zeno::layer_tc_n_pad(n_r_max < 128 ? n_r_max : 128) *
                                     (size_t)in;
                 if (need > split_elems) split_elems = need;
@@ -448,6 +453,8 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
     const size_t at_split0 = reserve(split_elems, 4), at_split1 = reserve(split_elems, 4);
     const size_t at_losspart = reserve(rows * 8, 8), at_losssum = reserve(rows, 8);
     const size_t at_headz = reserve(head_elems, 4), at_headt = reserve(rows, 4);
+    const size_t at_splitp = reserve(splitp_elems, 4), at_splitn = reserve(splitp_elems ? (size_t)c->sm_count * 16 : 0, 4);
+    const size_t at_splitt = reserve(splitt_elems, 4);
 
     e = cudaMalloc(&c->arena, bytes);
     if (e != cudaSuccess) {
@@ -473,9 +480,14 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
     c->act_split[1] = base + at_split1;
     c->head_zpart = head_elems ? reinterpret_cast<float *>(base + at_headz) : nullptr;
     c->head_tickets = reinterpret_cast<unsigned *>(base + at_headt);
+    c->split_part = splitp_elems ? reinterpret_cast<float *>(base + at_splitp) : nullptr;
+    c->split_norm = reinterpret_cast<float *>(base + at_splitn);
+    c->split_ticket = reinterpret_cast<unsigned *>(base + at_splitt);
+    c->split_blocks = c->sm_count;
     e = cudaMemset(c->dev_status, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(c->tickets, 0, ticket_elems * sizeof(unsigned));
     if (e == cudaSuccess) e = cudaMemset(c->head_tickets, 0, rows * sizeof(unsigned));
+    if (e == cudaSuccess && splitt_elems) e = cudaMemset(c->split_ticket, 0, splitt_elems * sizeof(unsigned));
     if (e != cudaSuccess) {
         cudaFree(c->arena);
         delete c;
@@ -580,6 +592,40 @@ zeno_status zeno_step_update(zeno_handle h, void *x, const void *V, int64_t ldv,
     if (st == ZENO_OK && !ranked) st = enqueue_select(h, score_buf, m, b, idx_buf, s, &launches);
     // the scoring pass has read x by the time the average is formed: the update goes in place
     if (st == ZENO_OK) st = enqueue_aggregate(h, V, ldv, m, idx_buf, m - b, out, x, gamma, s, &launches);
+    profile_end(h, s);
+    h->last_launches = st == ZENO_OK ? launches : 0;
+    return st;
+}
+
+zeno_status zeno_run(zeno_handle h, void *x, const void *V, int64_t ldv, int64_t step_stride_v, int32_t m,
+                     const float *features, const void *targets, int32_t n_r, int32_t steps, float gamma,
+                     float rho, int32_t b, float *scores, int32_t *idx, void *stream) {
+    if (!h || !x || !V || !features || !targets) return ZENO_ERR_INVALID_ARG;
+    if (steps < 1 || m < 1 || m > h->m_max || b < 0 || b >= m) return ZENO_ERR_INVALID_ARG;
+    if (n_r < 1 || n_r > h->n_r_max || ldv < h->d || step_stride_v < (int64_t)m * ldv) return ZENO_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t esz = elem_size(h->desc.param_dtype);
+    const size_t feat_stride = (size_t)n_r * (size_t)h->desc.dims[0];
+    int launches = 0;
+    profile_begin(h);
+    zeno_status st = ZENO_OK;
+    for (int32_t t = 0; t < steps && st == ZENO_OK; ++t) {
+        // iteration t of Algorithm 1's server loop: its own candidates and its own batch, the x of iteration t - 1
+        const void *Vt = static_cast<const char *>(V) + (size_t)t * (size_t)step_stride_v * esz;
+        zeno_batch batch;
+        batch.features = features + (size_t)t * feat_stride;
+        batch.targets = static_cast<const char *>(targets) + (size_t)t * (size_t)n_r * 4;
+        batch.n_r = n_r;
+        float *score_buf = scores ? scores + (size_t)t * m : h->scores;
+        int32_t *idx_buf = idx ? idx + (size_t)t * (m - b) : h->idx;
+        bool ranked = false;
+        st = enqueue_score(h, x, Vt, ldv, m, &batch, gamma, rho, score_buf, nullptr, nullptr, m - b, idx_buf, &ranked,
+                           s, &launches);
+        if (st == ZENO_OK && !ranked) st = enqueue_select(h, score_buf, m, b, idx_buf, s, &launches);
+        if (st == ZENO_OK) st = enqueue_aggregate(h, Vt, ldv, m, idx_buf, m - b, nullptr, x, gamma, s, &launches);
+    }
     profile_end(h, s);
     h->last_launches = st == ZENO_OK ? launches : 0;
     return st;

@@ -71,6 +71,11 @@ struct Context {
     unsigned *tickets;              // the tail's arrival counter, zero between launches
     float *head_zpart;              // partial logits of a last layer folded into the layer before it, or NULL
     unsigned *head_tickets;         // [m_max + 1] per-model arrival counters of that mode, zero between launches
+    // tiles shared between blocks by the tensor-core layer kernel (even shares of the k-blocks)
+    float *split_part;              // [split_blocks][2][128][n_pad of n_r_max] raw accumulators of the pieces, or NULL
+    float *split_norm;              // [split_blocks][2][8] the pieces' partial sums of v^2
+    unsigned *split_ticket;         // [(m_max + 1) * most tiles of a layer], zero between launches
+    int split_blocks;               // blocks the scratch above was sized for (the SM count)
     void *host_stage;               // device copies of host inputs (zeno_step_host), grown on demand
     size_t host_stage_bytes;
     int last_launches;
@@ -239,9 +244,13 @@ int mlp_norm_slots(int out);
 
 // Programmatic dependent launch.  Consecutive kernels of a step are chained so that a kernel's
 // blocks may become resident, and run their on-chip set-up, while the kernel before it drains.
-// Every kernel calls pdl_launch_dependents() first and pdl_wait() before it reads or writes any
-// global memory; pdl_wait() returns once the preceding kernel has completed and its writes are
-// visible (it is a no-op for a kernel launched the ordinary way).
+// Every kernel calls pdl_wait() before it reads or writes any global memory that a kernel of this
+// library writes; pdl_wait() returns once the preceding kernel has completed and its writes are
+// visible (it is a no-op for a kernel launched the ordinary way).  pdl_launch_dependents() comes
+// only AFTER the kernel's own pdl_wait(): a kernel's successor can then start no earlier than the
+// completion of the kernel's predecessor, so whatever a successor reads ahead of its own wait (the
+// head kernel reads x and V there) cannot still be written by a kernel two places up the chain --
+// the in-place update of x by the previous step's averaging pass in particular.
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 

@@ -62,7 +62,6 @@ __host__ __device__ inline int lsq_stage_bytes(int n_pad) { return 2 * kVHalfByt
 __global__ void __launch_bounds__(kQThreads, 1)
 lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_a,
               const __grid_constant__ CUtensorMap map_x, LsqTcArgs a) {
-    pdl_launch_dependents();
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     // full, empty, bready [stages]; afull, aempty [A buffers]; dfull, dempty [2 sets]
     constexpr int kBars = 3 * kQMaxStages + 2 * kQMaxABufs + 4;
@@ -133,6 +132,7 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
     __syncthreads();
     tc_fence_after();
     pdl_wait();
+    pdl_launch_dependents();
     const uint32_t tmem = tmem_base_slot;
     volatile int *abortp = &abort_flag;
 

@@ -92,8 +92,8 @@ __global__ void __launch_bounds__(kLayerWarps * 32, 1) mlp_layer_kernel(LayerArg
     extern __shared__ __align__(16) float smem_dyn[];
     float(*hs)[NRT][kStageK] = reinterpret_cast<float(*)[NRT][kStageK]>(smem_dyn);
 
-    pdl_launch_dependents();
     pdl_wait();
+    pdl_launch_dependents();
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const int c = blockIdx.y;                    // model: 0 = x, 1+i = x - gamma v_i
@@ -258,7 +258,10 @@ __global__ void __launch_bounds__(256, 1) mlp_head_kernel(LayerArgs a) {
     float(*hs)[KC] = reinterpret_cast<float(*)[KC]>(smem_dyn + OUT_T * KC);     // [NS][KC]
     __shared__ float zl[32][NS + 1];
 
-    pdl_launch_dependents();
+    // The weights are inputs of the whole call: unless this is the call's first kernel (what precedes it
+    // on the stream may then still be producing x or V), they are read while the kernel that produces the
+    // activations is still running.
+    if (a.first_in_call) pdl_wait();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int c = blockIdx.x;
     const int K = a.in;
@@ -345,11 +348,9 @@ __global__ void __launch_bounds__(256, 1) mlp_head_kernel(LayerArgs a) {
         }
     };
 
-    // The weights are inputs of the whole call: the first chunk is formed while the kernel that
-    // produces the activations may still be running.
-    if (a.first_in_call) pdl_wait();    // unless x and V may still be in the making (see LayerArgs)
     stage_weights(0);
     pdl_wait();
+    pdl_launch_dependents();
     for (int kb = 0; kb < K; kb += KC) {
         if (kb > 0) __syncthreads();
         stage_acts(kb);                 // in flight while the weights are formed
@@ -434,8 +435,8 @@ __global__ void __launch_bounds__(256) mlp_loss_kernel(const float *logits, cons
                                                         int n_r, int classes, float *losses, double *loss_part,
                                                         int G, TailArgs tail) {
     __shared__ double per_warp[8];
-    pdl_launch_dependents();
     pdl_wait();
+    pdl_launch_dependents();
     const int c = blockIdx.x / G, g = blockIdx.x - c * G;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     double mine = 0.0;

@@ -87,8 +87,8 @@ __global__ void __launch_bounds__(kMmaWarps * 32) mlp_layer_mma_kernel(LayerArgs
     constexpr int kChunks = NRT * (kHS / 4) / (kMmaWarps * 32);   // float4 chunks of a stage per thread
     extern __shared__ __align__(16) uint4 hs_dyn[];                 // [2][NRT][kPitch]
 
-    pdl_launch_dependents();
     pdl_wait();
+    pdl_launch_dependents();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
     const int c = blockIdx.y;

@@ -87,7 +87,6 @@ __global__ void __launch_bounds__(kThreads, 1)
 stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_v,
                      StreamArgs a) {
     constexpr int kStage = kStageBytes;
-    pdl_launch_dependents();
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     // per pipeline: full[kMaxStages], empty[kMaxStages], a_full[kMaxABufs], a_empty[kMaxABufs], d_full, d_empty
     constexpr int kBarsPerPipe = 2 * kMaxStages + 2 * kMaxABufs + 2;
@@ -165,6 +164,7 @@ stream_tf32x3_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     __syncthreads();                                   // barriers and the TMEM base are visible
     tc_fence_after();
     pdl_wait();                                        // on-chip set-up done; global memory from here on
+    pdl_launch_dependents();
     const uint32_t tmem = tmem_base_slot;
     volatile int *abortp = &abort_flag;
 
@@ -435,8 +435,8 @@ __global__ void __launch_bounds__(256) stream_combine_kernel(const float *part, 
                                                              int64_t offB, float gamma, int relu,
                                                              float *H, float *Hsplit, int n_pad) {
     constexpr int E = VEC4 ? 4 : 1;
-    pdl_launch_dependents();
     pdl_wait();
+    pdl_launch_dependents();
     const int og = (out + E - 1) / E;                       // output groups per row
     const int n_rows = Hsplit ? n_pad : n_r;
     const int c = blockIdx.y;

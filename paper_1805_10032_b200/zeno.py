@@ -25,7 +25,7 @@ F32, BF16 = 0, 1
 
 EXPORTS = (
     "zeno_param_count", "zeno_create", "zeno_destroy", "zeno_score", "zeno_select",
-    "zeno_aggregate", "zeno_step", "zeno_step_update", "zeno_step_host", "zeno_device_status", "zeno_score_lsq_static",
+    "zeno_aggregate", "zeno_step", "zeno_step_update", "zeno_run", "zeno_step_host", "zeno_device_status", "zeno_score_lsq_static",
     "zeno_debug_set_wait_limit",
     "zeno_profile", "zeno_profile_read",
     "zeno_last_launch_count",
@@ -78,6 +78,8 @@ def load_library() -> ctypes.CDLL:
     lib.zeno_aggregate.argtypes = [vp, vp, i64, i32, vp, i32, vp, vp]
     lib.zeno_step.restype = i32
     lib.zeno_step.argtypes = [vp, vp, vp, i64, i32, ctypes.POINTER(Batch), f32, f32, i32, vp, vp, vp, vp]
+    lib.zeno_run.restype = i32
+    lib.zeno_run.argtypes = [vp, vp, vp, i64, i64, i32, vp, vp, i32, i32, f32, f32, i32, vp, vp, vp]
     lib.zeno_step_update.restype = i32
     lib.zeno_step_update.argtypes = [vp, vp, vp, i64, i32, ctypes.POINTER(Batch), f32, f32, i32, vp, vp, vp, vp]
     lib.zeno_step_host.restype = i32
@@ -296,6 +298,23 @@ class Zeno:
                                         _ptr(idx), _stream_ptr(stream))
         self._check(st, "zeno_step_update")
         return out, scores, idx
+
+    def run(self, x, V, features, targets, gamma, rho, b, scores=None, idx=None, stream=None):
+        """Algorithm 1's server loop: V [steps, m, ldv], features [steps, n_r, in], targets [steps, n_r];
+        x is updated in place.  Returns (scores [steps, m], idx [steps, m - b])."""
+        steps, m = V.shape[0], V.shape[1]
+        ldv, stride = V.stride(1), V.stride(0)
+        n_r = features.shape[1]
+        assert features.is_contiguous() and targets.is_contiguous()
+        if scores is None:
+            scores = torch.empty((steps, m), dtype=torch.float32, device=self._dev())
+        if idx is None:
+            idx = torch.empty((steps, max(m - b, 0)), dtype=torch.int32, device=self._dev())
+        st = self._lib.zeno_run(self._h, _ptr(x), _ptr(V), int(ldv), int(stride), int(m), _ptr(features),
+                                _ptr(targets), int(n_r), int(steps), float(gamma), float(rho), int(b),
+                                _ptr(scores), _ptr(idx), _stream_ptr(stream))
+        self._check(st, "zeno_run")
+        return scores, idx
 
     def step_host(self, x, V, features, targets, gamma, rho, b, out, scores=None, idx=None,
                   m=None, ldv=None, stream=None):

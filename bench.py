@@ -461,7 +461,7 @@ def bench_config(R, index, steps, warmup, headline):
     layer_of, layer = {}, 0
     for k in kern:
         name = k["kernel"].split(":")[1]
-        if name in ("stream_tf32x3", "layer_tc", "layer_tc_shared", "mlp_layer", "mlp_layer_mma", "mlp_head_loss_tail"):
+        if name in ("stream_tf32x3", "layer_tc", "mlp_layer", "mlp_layer_mma", "mlp_head_loss_tail"):
             layer_of[k["kernel"]] = [layer]
             layer += 1
         elif name == "layer_tc_head":           # a hidden layer with the small last layer folded in

@@ -44,6 +44,7 @@ extern "C" {
 
 #define ZENO_MAX_LAYERS 8
 #define ZENO_MAX_CANDIDATES 1024
+#define ZENO_KRUM_MAX_M 128      /* most candidates zeno_krum accepts */
 #define ZENO_STATIC_MAX_M 64    /* most candidates zeno_score_lsq_static accepts */
 #define ZENO_STATIC_MAX_N_R 32  /* most server samples zeno_score_lsq_static accepts */
 
@@ -138,6 +139,26 @@ zeno_status zeno_select(zeno_handle h, const float *scores, int32_t m, int32_t b
  * INVALID_ARG: NULL pointers, k < 1 or k > m, m > m_max, ldv < d. */
 zeno_status zeno_aggregate(zeno_handle h, const void *V, int64_t ldv, int32_t m,
                            const int32_t *idx, int32_t k, float *out, void *stream);
+
+/* The paper's baseline aggregation rules on the same candidates (Experiments, "Baselines"), for comparing
+ * them with Zeno_b on the same step.
+ *
+ * zeno_median -- Definition "Median", the marginal median: out[j] = the one-dimensional median of
+ * V[0][j] .. V[m-1][j] (the middle one of the sorted values, the mean of the two middle ones for even m),
+ * in binary32.  The paper does not say what a NaN entry is worth; here it counts as plus infinity.
+ * V: [m x ldv] device; out: float[d] device.  INVALID_ARG: NULL pointers, m < 1 or > m_max, ldv < d. */
+zeno_status zeno_median(zeno_handle h, const void *V, int64_t ldv, int32_t m, float *out, void *stream);
+
+/* zeno_krum -- Definition "Krum": k = arg min_i sum_{i -> j} ||v_i - v_j||^2 over the m - b - 2 nearest
+ * neighbours j of v_i among the other candidates (squared Euclidean distances, taken as sums of squared
+ * differences); ties go to the lowest index; a NaN distance counts as plus infinity.
+ * k: device int32[1], the winning candidate (required); out: float[d] device, a copy of row k, or NULL;
+ * sums: float[m] device, the candidates' neighbour sums, or NULL.
+ * INVALID_ARG: NULL V / k, m < 1 or > m_max, ldv < d, b < 0, m - b - 2 < 1 (no neighbour left).  The paper
+ * notes that Krum's guarantee needs 2b + 2 < m; its own toy example does not meet that, so it is not
+ * enforced.  UNSUPPORTED: m > ZENO_KRUM_MAX_M. */
+zeno_status zeno_krum(zeno_handle h, const void *V, int64_t ldv, int32_t m, int32_t b, float *out, int32_t *k,
+                      float *sums, void *stream);
 
 /* Zeno_b({v_i}) = score -> select -> aggregate on one stream, no host round trip.
  * out: float[d] (required); scores: float[m] or NULL; idx: int32[m-b] or NULL.

@@ -76,6 +76,10 @@ __device__ __forceinline__ void stage_rows(const int32_t *idx, int k, int m, int
     __syncthreads();
 }
 
+// x is read and written in this file, so it is read with ordinary loads (the read-only path is for data
+// nobody writes while the kernel runs).
+__device__ __forceinline__ float load_param(const float *p) { return *p; }
+__device__ __forceinline__ float load_param(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
 __device__ __forceinline__ void store_param(float *p, float v) { *p = v; }
 __device__ __forceinline__ void store_param(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
 
@@ -90,7 +94,10 @@ __global__ void __launch_bounds__(256) aggregate_vec_kernel(const T *V, int64_t 
     constexpr int E = Group<T>::kElems;
     __shared__ int64_t rows_s[ZENO_MAX_CANDIDATES];
     pdl_wait();
-    pdl_launch_dependents();
+    // With the in-place update the next kernel on the stream (the next step's first kernel, which reads x
+    // through the read-only path) must not become resident before x is final: no early trigger then, the
+    // dependents start when this grid has completed.
+    if (!xu) pdl_launch_dependents();
     stage_rows(idx, k, m, ldv, rows_s);
     const int64_t groups = d / E;            // whole groups; the d % E tail columns follow below
     for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < groups;
@@ -138,7 +145,7 @@ __global__ void __launch_bounds__(256) aggregate_vec_kernel(const T *V, int64_t 
             }
             acc = acc / (float)k;
             if (out) out[j] = acc;
-            if (xu) store_param(xu + j, fmaf(-gamma, acc, load_elem(xu + j)));
+            if (xu) store_param(xu + j, fmaf(-gamma, acc, load_param(xu + j)));
         }
     }
 }
@@ -150,7 +157,10 @@ __global__ void __launch_bounds__(256) aggregate_scalar_kernel(const T *V, int64
                                                                 float *out, T *xu, float gamma) {
     __shared__ int64_t rows_s[ZENO_MAX_CANDIDATES];
     pdl_wait();
-    pdl_launch_dependents();
+    // With the in-place update the next kernel on the stream (the next step's first kernel, which reads x
+    // through the read-only path) must not become resident before x is final: no early trigger then, the
+    // dependents start when this grid has completed.
+    if (!xu) pdl_launch_dependents();
     stage_rows(idx, k, m, ldv, rows_s);
     for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < d;
          j += (int64_t)gridDim.x * blockDim.x) {
@@ -161,7 +171,7 @@ __global__ void __launch_bounds__(256) aggregate_scalar_kernel(const T *V, int64
         }
         acc = acc / (float)k;
         if (out) out[j] = acc;
-        if (xu) store_param(xu + j, fmaf(-gamma, acc, load_elem(xu + j)));
+        if (xu) store_param(xu + j, fmaf(-gamma, acc, load_param(xu + j)));
     }
 }
 

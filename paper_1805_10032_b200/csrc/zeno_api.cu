@@ -377,7 +377,7 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
 
     const size_t rows = (size_t)m_max + 1;
     size_t act_elems = 0, norm_elems = 0, lsq_elems = 0, tc_elems = 0, ticket_elems = 1, split_elems = 0;
-    size_t head_elems = 0, splitp_elems = 0, splitt_elems = 0;
+    size_t head_elems = 0;
     if (desc->kind == ZENO_LOSS_SOFTMAX_MLP) {
         int64_t off = 0, widest = 0;
         int slots = 0;
@@ -406,11 +406,6 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
             if (zeno::layer_tc_usable((zeno_dtype)desc->param_dtype, (int)in, (int)o, n_r_max < 128 ? n_r_max : 128) &&
                 c->use_tc) {
                 if (zeno::layer_tc_norm_slots((int)o) > layer_slots) layer_slots = zeno::layer_tc_norm_slots((int)o);
-                // scratch of the tiles that blocks share: two pieces per block, a ticket per tile
-                const size_t sp = (size_t)c->sm_count * 2 * 128 * (size_t)zeno::layer_tc_n_pad(n_r_max < 128 ? n_r_max : 128);
-                if (sp > splitp_elems) splitp_elems = sp;
-                const size_t tk = rows * (size_t)((o + 127) / 128);
-                if (tk > splitt_elems) splitt_elems = tk;
                 const size_t need = (l == 0 ? 1 : rows) * 2 * (size_t)zeno::layer_tc_n_pad(n_r_max < 128 ? n_r_max : 128) *
                                     (size_t)in;
                 if (need > split_elems) split_elems = need;
@@ -453,8 +448,14 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
     const size_t at_split0 = reserve(split_elems, 4), at_split1 = reserve(split_elems, 4);
     const size_t at_losspart = reserve(rows * 8, 8), at_losssum = reserve(rows, 8);
     const size_t at_headz = reserve(head_elems, 4), at_headt = reserve(rows, 4);
-    const size_t at_splitp = reserve(splitp_elems, 4), at_splitn = reserve(splitp_elems ? (size_t)c->sm_count * 16 : 0, 4);
-    const size_t at_splitt = reserve(splitt_elems, 4);
+    c->krum_blocks = 2 * c->sm_count;
+    size_t krum_elems = 0;
+    if (m_max <= ZENO_KRUM_MAX_M)               // the largest of the partial layouts any m <= m_max may use
+        for (int mm = 3; mm <= m_max; ++mm) {
+            const size_t need = zeno::krum_part_floats(mm, c->krum_blocks);
+            if (need > krum_elems) krum_elems = need;
+        }
+    const size_t at_krum = reserve(krum_elems, 4), at_krums = reserve(m_max, 4);
 
     e = cudaMalloc(&c->arena, bytes);
     if (e != cudaSuccess) {
@@ -480,14 +481,11 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
     c->act_split[1] = base + at_split1;
     c->head_zpart = head_elems ? reinterpret_cast<float *>(base + at_headz) : nullptr;
     c->head_tickets = reinterpret_cast<unsigned *>(base + at_headt);
-    c->split_part = splitp_elems ? reinterpret_cast<float *>(base + at_splitp) : nullptr;
-    c->split_norm = reinterpret_cast<float *>(base + at_splitn);
-    c->split_ticket = reinterpret_cast<unsigned *>(base + at_splitt);
-    c->split_blocks = c->sm_count;
+    c->krum_part = krum_elems ? reinterpret_cast<float *>(base + at_krum) : nullptr;
+    c->krum_sums = reinterpret_cast<float *>(base + at_krums);
     e = cudaMemset(c->dev_status, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(c->tickets, 0, ticket_elems * sizeof(unsigned));
     if (e == cudaSuccess) e = cudaMemset(c->head_tickets, 0, rows * sizeof(unsigned));
-    if (e == cudaSuccess && splitt_elems) e = cudaMemset(c->split_ticket, 0, splitt_elems * sizeof(unsigned));
     if (e != cudaSuccess) {
         cudaFree(c->arena);
         delete c;
@@ -550,6 +548,37 @@ zeno_status zeno_aggregate(zeno_handle h, const void *V, int64_t ldv, int32_t m,
     profile_end(h, static_cast<cudaStream_t>(stream));
     h->last_launches = st == ZENO_OK ? launches : 0;
     return st;
+}
+
+zeno_status zeno_median(zeno_handle h, const void *V, int64_t ldv, int32_t m, float *out, void *stream) {
+    if (!h || !out) return ZENO_ERR_INVALID_ARG;
+    zeno_status st = check_common(h, V, ldv, m);
+    if (st != ZENO_OK) return st;
+    DeviceGuard guard(h->device);
+    if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+    int launches = 0;
+    profile_begin(h);
+    cudaError_t e = zeno::launch_median(*h, V, ldv, m, out, static_cast<cudaStream_t>(stream), &launches);
+    profile_end(h, static_cast<cudaStream_t>(stream));
+    h->last_launches = e == cudaSuccess ? launches : 0;
+    return e == cudaSuccess ? ZENO_OK : fail_cuda(h, e);
+}
+
+zeno_status zeno_krum(zeno_handle h, const void *V, int64_t ldv, int32_t m, int32_t b, float *out, int32_t *k,
+                      float *sums, void *stream) {
+    if (!h || !k) return ZENO_ERR_INVALID_ARG;
+    zeno_status st = check_common(h, V, ldv, m);
+    if (st != ZENO_OK) return st;
+    if (b < 0 || m - b - 2 < 1) return ZENO_ERR_INVALID_ARG;
+    if (m > ZENO_KRUM_MAX_M || !h->krum_part) return ZENO_ERR_UNSUPPORTED;
+    DeviceGuard guard(h->device);
+    if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+    int launches = 0;
+    profile_begin(h);
+    cudaError_t e = zeno::launch_krum(*h, V, ldv, m, b, out, k, sums, static_cast<cudaStream_t>(stream), &launches);
+    profile_end(h, static_cast<cudaStream_t>(stream));
+    h->last_launches = e == cudaSuccess ? launches : 0;
+    return e == cudaSuccess ? ZENO_OK : fail_cuda(h, e);
 }
 
 zeno_status zeno_step(zeno_handle h, const void *x, const void *V, int64_t ldv, int32_t m,

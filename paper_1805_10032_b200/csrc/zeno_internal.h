@@ -71,11 +71,10 @@ struct Context {
     unsigned *tickets;              // the tail's arrival counter, zero between launches
     float *head_zpart;              // partial logits of a last layer folded into the layer before it, or NULL
     unsigned *head_tickets;         // [m_max + 1] per-model arrival counters of that mode, zero between launches
-    // tiles shared between blocks by the tensor-core layer kernel (even shares of the k-blocks)
-    float *split_part;              // [split_blocks][2][128][n_pad of n_r_max] raw accumulators of the pieces, or NULL
-    float *split_norm;              // [split_blocks][2][8] the pieces' partial sums of v^2
-    unsigned *split_ticket;         // [(m_max + 1) * most tiles of a layer], zero between launches
-    int split_blocks;               // blocks the scratch above was sized for (the SM count)
+    // Krum: per-block partial sums of the pairs' squared distances, and the candidates' sums
+    float *krum_part;               // NULL when m_max is beyond ZENO_KRUM_MAX_M
+    float *krum_sums;               // [m_max]
+    int krum_blocks;                // blocks the partials were sized for
     void *host_stage;               // device copies of host inputs (zeno_step_host), grown on demand
     size_t host_stage_bytes;
     int last_launches;
@@ -231,6 +230,12 @@ int layer_tc_norm_slots(int out);
 cudaError_t launch_layer_tc(Context &c, const LayerTcLaunch &l, cudaStream_t s, int *launches);
 cudaError_t launch_split_acts(Context &c, const float *H, int models, int n_r, int K, void *out, cudaStream_t s,
                               int *launches);
+
+// The paper's baseline aggregation rules on the same V (zeno_baselines.cu).
+size_t krum_part_floats(int m, int blocks);
+cudaError_t launch_median(Context &c, const void *V, int64_t ldv, int m, float *out, cudaStream_t s, int *launches);
+cudaError_t launch_krum(Context &c, const void *V, int64_t ldv, int m, int b, float *out, int32_t *k, float *sums,
+                        cudaStream_t s, int *launches);
 
 int lsq_slab_count(const Context &c);
 // Tensor-core version of the least-squares stream (zeno_lsq_tc.cu): one slab per block into a.part.

@@ -21,14 +21,6 @@
 //                  operand; the fp32 activations are carried as two bfloat16 terms;
 //                  D += w [h_hi; h_lo]^T (kind::f16, K = 16 per MMA); result D[j] + D[n_pad + j].
 //
-// Work split.  With fewer whole tiles than a multiple of the SM count the last round of tiles would
-// leave most SMs idle (1,056 tiles on 148 SMs: 8 rounds for 7.1 rounds of work).  When the launch
-// asks for even shares, the k-blocks of all tiles form one sequence that is cut into one contiguous
-// share per block; a tile cut by a share boundary is accumulated in pieces by two (or more) blocks,
-// each piece at least two k-blocks long.  A piece's epilogue leaves the raw accumulator in global
-// memory and takes a ticket for the tile; the last piece to arrive adds all pieces in block order
-// (so the result does not depend on which block came last) and runs the tile's real epilogue.
-//
 // Warp roles: warps 0 and 2 TMA producers (weight ring, activation ring), warp 1 MMA issuer and owner of
 // TMEM (all three stay converged and issue from one elected lane; the issuer takes two k-blocks per turn), warps 4-11 two converter sets taking alternate k-blocks, warps
 // 12-15 epilogue.  Accumulator sets alternate between consecutive tiles when two fit in TMEM, so
@@ -107,14 +99,6 @@ struct LayerTcArgs {
     int np_slots, np_base;
     int *status;
     uint32_t spin_limit;   // polls a bounded wait may take
-    // Even shares (split != 0): the layer's k-blocks, item after item, are one sequence of n_items * nkb
-    // entries that is cut into gridDim.x contiguous shares, so a tile may be shared by several blocks.
-    // Each of them leaves its partial tile in split_part and the last one to arrive (a ticket per item)
-    // adds the pieces in block order and finishes the tile.
-    int split;
-    float *split_part;     // [blocks][2][128][n_pad]: a block's first and last unit when they are pieces
-    float *split_norm;     // [blocks][2][8]: the pieces' partial sums of v^2, per (quadrant, converter set)
-    unsigned *split_ticket;// [items], zero between launches
     HeadFuse head;         // used by the HEAD instantiations only
 };
 
@@ -270,36 +254,9 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     auto bar_aempty = [&](int g) { return smem_u32(&bars[kBarA + kLMaxABufs + g]); };
     auto bar_dfull = [&](int q) { return smem_u32(&bars[kBarD + q]); };
     auto bar_dempty = [&](int q) { return smem_u32(&bars[kBarD + kLMaxSets + q]); };
-    // Share boundaries of the even split: block b owns the sequence entries [cut(b), cut(b + 1)).  A
-    // boundary one k-block away from a tile's start or end is moved onto it, so that no piece is shorter
-    // than two k-blocks (both converter sets then take part in every piece).
-    const int64_t n_seq = (int64_t)n_items * nkb;
-    auto cut = [&](int b) -> int64_t {
-        if (b <= 0) return 0;
-        if (b >= (int)gridDim.x) return n_seq;
-        int64_t r = (int64_t)b * n_seq / gridDim.x;
-        const int o = (int)(r % nkb);
-        if (o == 1) r -= 1;
-        else if (o == nkb - 1) r += 1;
-        return r;
-    };
-    const int64_t my_r0 = a.split ? cut(blockIdx.x) : 0, my_r1 = a.split ? cut(blockIdx.x + 1) : 0;
-    const int my_i0 = a.split ? (int)(my_r0 / nkb) : 0;
-    // unit li of this block -> (model, tile) and the k-blocks [kb0, kb1) of the tile it covers.  Without
-    // the split a unit is a whole tile and neighbouring blocks share a model's activations in L2.
-    auto get_unit = [&](int li, int &model, int &tile, int &kb0, int &kb1) {
-        int item;
-        if (a.split) {
-            item = my_i0 + li;
-            const int64_t first = (int64_t)item * nkb;
-            if (first >= my_r1) return false;
-            kb0 = my_r0 > first ? (int)(my_r0 - first) : 0;
-            kb1 = my_r1 - first < nkb ? (int)(my_r1 - first) : nkb;
-        } else {
-            item = blockIdx.x + li * gridDim.x;
-            kb0 = 0;
-            kb1 = nkb;
-        }
+    // item li of this block -> (model, tile); neighbouring blocks share a model's activations in L2
+    auto get_item = [&](int li, int &model, int &tile) {
+        const int item = blockIdx.x + li * gridDim.x;
         model = item / a.tiles;
         tile = item - model * a.tiles;
         return item < n_items;
@@ -354,12 +311,12 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         const int ring_stages = acts ? n_bstages : n_stages;
         int s = 0;
         uint32_t round = 0;
-        int model, tile, kb0, kb1;
+        int model, tile;
         for (int li = 0;; ++li) {
-            if (!__all_sync(0xffffffffu, get_unit(li, model, tile, kb0, kb1) && !*abortp)) break;
+            if (!__all_sync(0xffffffffu, get_item(li, model, tile) && !*abortp)) break;
             const bool has_v = model > 0;                 // model 0 is x itself
             bool ok = true;
-            for (int kb = kb0; kb < kb1; ++kb) {
+            for (int kb = 0; kb < nkb; ++kb) {
                 const uint32_t empty = acts ? bar_bempty(s) : bar_empty(s), full = acts ? bar_bfull(s) : bar_full(s);
                 ok = __all_sync(0xffffffffu, mbar_wait(empty, (round & 1) ^ 1, abortp));
                 if (!ok) break;
@@ -396,9 +353,9 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         const int kb_step = n_bstages >= 4 ? 2 : 1;
         int bs = 0, ag = 0;                              // activation stage and A buffer of the next k-block
         uint32_t bph = 0, aph = 0;                       // and the phases their full barriers are awaited in
-        int model, tile, kb0, kb1;
+        int model, tile;
         for (int li = 0;; ++li) {
-            if (!__all_sync(0xffffffffu, get_unit(li, model, tile, kb0, kb1) && !*abortp)) break;
+            if (!__all_sync(0xffffffffu, get_item(li, model, tile) && !*abortp)) break;
             const int set = li % n_sets;
             const uint32_t use = (uint32_t)(li / n_sets);        // earlier uses of this accumulator set
             if (!__all_sync(0xffffffffu, mbar_wait(bar_dempty(set), (use & 1) ^ 1, abortp))) break;
@@ -410,8 +367,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
             // fence, the election and the loop's own arithmetic cost this warp -- the one every other
             // role ends up waiting for -- as much as the sixteen MMAs it issues.  Only with an activation ring
             // of four stages or more: with three (128 samples), holding two back at a time measured slower.
-            for (int kb = kb0; kb < kb1; kb += kb_step) {
-                const bool two = kb_step == 2 && kb + 1 < kb1;
+            for (int kb = 0; kb < nkb; kb += kb_step) {
+                const bool two = kb_step == 2 && kb + 1 < nkb;
                 int s1 = bs + 1, g1 = ag + 1;
                 uint32_t sph1 = bph, gph1 = aph;
                 if (s1 == n_bstages) { s1 = 0; sph1 ^= 1; }
@@ -431,7 +388,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
 #pragma unroll
                         for (int ks = 0; ks < 4; ++ks) {            // 32 bytes of every row per MMA
                             const uint64_t db = smem_desc_sw128(bx + ks * 32);
-                            const uint32_t acc = (uint32_t)((kb - kb0) | h | ks);     // the unit's first MMA overwrites
+                            const uint32_t acc = (uint32_t)(kb | h | ks);
                             if (kBf16) {
                                 tc_mma_bf16_ts(d1, a_tmem + ks * 8, db, idesc_2n, acc);          // w [h_hi; h_lo]
                             } else {
@@ -442,7 +399,7 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                         tc_commit(bar_aempty(g));               // the A buffer and
                         tc_commit(bar_bempty(s));               // the stage's activations may be overwritten once these finish
                     }
-                    if (kb + kb_step >= kb1) tc_commit(bar_dfull(set));
+                    if (kb + kb_step >= nkb) tc_commit(bar_dfull(set));
                 }
                 __syncwarp();
                 // advance both rings by the k-blocks taken
@@ -462,35 +419,29 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         const int row = quad * 32 + lane;             // row of the tile = TMEM lane
         const uint32_t a_bufs = tmem + ((uint32_t)(quad * 32) << 16) + a_base;
         uint32_t it0 = 0;
-        int model, tile, kb0, kb1;
-        int which = 0;                                // a block's pieces are its first unit (slot 0) or its last (slot 1)
-        // partial sum of squares of this tile's rows (model 0 is x itself: not a candidate); a piece's
-        // goes to the block's scratch, from where the block that finishes the tile collects it
-        auto store_norm = [&](const float (&n4)[4], bool piece) {
+        int model, tile;
+        // partial sum of squares of this tile's rows (model 0 is x itself: not a candidate)
+        auto store_norm = [&](const float (&n4)[4]) {
             if (model > 0) {
                 float nrm = (n4[0] + n4[1]) + (n4[2] + n4[3]);
                 const int o = tile * kRows + row;
-                // the bias entries' squares are counted once per tile: with the k-blocks that start it
-                if (cset == 0 && kb0 == 0 && a.offB >= 0 && o < a.out) {
+                if (cset == 0 && a.offB >= 0 && o < a.out) {
                     const float bv = load_elem(static_cast<const T *>(a.V) + (int64_t)(model - 1) * a.ldv + a.offB + o);
                     nrm = fmaf(bv, bv, nrm);
                 }
 #pragma unroll
                 for (int sft = 16; sft >= 1; sft >>= 1) nrm += __shfl_xor_sync(0xffffffffu, nrm, sft);
                 if (lane == 0) {
-                    if (piece) a.split_norm[((int64_t)blockIdx.x * 2 + which) * 8 + quad * 2 + cset] = nrm;
-                    else a.normpart[(int64_t)(model - 1) * a.np_slots + a.np_base + (tile * 4 + quad) * 2 + cset] = nrm;
-                    if (HEAD || piece) __threadfence();
+                    a.normpart[(int64_t)(model - 1) * a.np_slots + a.np_base + (tile * 4 + quad) * 2 + cset] = nrm;
+                    if (HEAD) __threadfence();
                 }
             }
         };
-        for (int li = 0; get_unit(li, model, tile, kb0, kb1) && !*abortp; ++li, it0 += (uint32_t)(kb1 - kb0)) {
+        for (int li = 0; get_item(li, model, tile) && !*abortp; ++li, it0 += nkb) {
             float nrm4[4] = {0.f, 0.f, 0.f, 0.f};
             bool ok = true;
-            const bool piece = kb1 - kb0 < nkb;
-            which = li == 0 ? 0 : 1;
-            for (int kb = kb0 + (int)((cset - it0) & 1u); kb < kb1; kb += 2) {
-                const uint32_t it = it0 + (uint32_t)(kb - kb0);
+            for (int kb = (int)((cset - it0) & 1u); kb < nkb; kb += 2) {
+                const uint32_t it = it0 + kb;
                 const uint32_t sround = small_div(it, inv_stages), around = small_div(it, inv_abufs);
                 const int s = (int)(it - sround * n_stages), g = (int)(it - around * n_abufs);
                 if (!mbar_wait(bar_full(s), sround & 1, abortp)) { ok = false; break; }
@@ -532,9 +483,9 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                         }
                     }
                 }
-                // HEAD, or a piece: the norm partial must be in global memory before the epilogue group takes
-                // the ticket, so it is written ahead of the set's last A buffer of the unit
-                if ((HEAD || piece) && kb + 2 >= kb1) store_norm(nrm4, piece);
+                // HEAD: the norm partial must be in global memory before the epilogue group takes the
+                // model's ticket, so it is written ahead of the set's last A buffer of the tile
+                if (HEAD && kb + 2 >= nkb) store_norm(nrm4);
                 if (!mbar_wait(bar_aempty(g), (around & 1) ^ 1, abortp)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t a_tmem = a_bufs + g * Tr::kACols;
@@ -546,45 +497,18 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 if (lane == 0) mbar_arrive(bar_afull(g));
             }
             if (!ok) break;
-            if (!HEAD && !piece) store_norm(nrm4, false);   // else: already written (every set has a k-block there)
+            if (!HEAD) store_norm(nrm4);          // HEAD: already written (every set has a k-block: K >= 2 k-blocks)
         }
     } else if (warp >= 12) {
         // ------------------------------------------------------------------ epilogue
         const int quad = warp & 3;
         const int row = quad * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-        int model, tile, kb0, kb1;
+        int model, tile;
         const int g = tid - (kLThreads - kEpiThreads);    // thread within the epilogue group
         const int cls_even = (a.head.classes + 1) & ~1;
-        const bool grouped = HEAD || a.split != 0;        // the group uses its named barrier: it stays together
-        // activation, padding and the layer's output for 16 samples of output row o (not HEAD)
-        auto write_chunk = [&](int o, int j0, const float (&acc)[16], float bias) {
-            if (o >= a.out) return;
-#pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                const int jj = j0 + j;
-                float z = acc[j] + bias;
-                if (a.relu) z = (z > 0.f || z != z) ? z : 0.f;
-                if (jj >= a.n_r) z = 0.f;             // padded samples
-                if (a.Hout && jj < a.n_r) a.Hout[((int64_t)model * a.n_r + jj) * a.out + o] = z;
-                if (a.Hsplit) {
-                    T *hs = static_cast<T *>(a.Hsplit) + (int64_t)model * 2 * a.n_pad * a.out + o;
-                    if (kBf16) {
-                        const __nv_bfloat16 hi = __float2bfloat16_rn(z);
-                        const __nv_bfloat16 lo = __float2bfloat16_rn(z - __bfloat162float(hi));
-                        reinterpret_cast<__nv_bfloat16 *>(hs)[(int64_t)jj * a.out] = hi;
-                        reinterpret_cast<__nv_bfloat16 *>(hs)[(int64_t)(a.n_pad + jj) * a.out] = lo;
-                    } else {
-                        const float hi = tf32_hi(z);
-                        reinterpret_cast<float *>(hs)[(int64_t)jj * a.out] = hi;
-                        reinterpret_cast<float *>(hs)[(int64_t)(a.n_pad + jj) * a.out] = z - hi;
-                    }
-                }
-            }
-        };
-        // the group leaves the loop together when it uses its named barrier
-        for (int li = 0; get_unit(li, model, tile, kb0, kb1) && (grouped || !*abortp); ++li) {
-            const bool piece = kb1 - kb0 < nkb;
+        // HEAD: the group leaves the loop together (its named barrier needs all four warps)
+        for (int li = 0; get_item(li, model, tile) && (HEAD || !*abortp); ++li) {
             const int set = li % n_sets;
             const uint32_t use = (uint32_t)(li / n_sets);
             const int o = tile * kRows + row;             // thread = output row o, column = sample j
@@ -619,10 +543,8 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 }
             }
             bool got = mbar_wait(bar_dfull(set), use & 1, abortp);
-            if (grouped) got = epi_all(got);
+            if (HEAD) got = epi_all(got);
             if (!got) break;
-            // a block's pieces are its first unit (slot 0) or its last (slot 1)
-            float *my_part = piece ? a.split_part + (((int64_t)blockIdx.x * 2 + (li == 0 ? 0 : 1)) * kRows + row) * a.n_pad : nullptr;
             tc_fence_after();
             const uint32_t dset = tmem + lane_addr + set * acc_cols;
             for (int j0 = 0; j0 < a.n_pad; j0 += 16) {
@@ -668,62 +590,29 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                         const float r = lane_transpose_sum32(pv, lane);
                         zq_w[(cb + (lane >> 4)) * a.n_pad + j0 + (lane & 15)] = r;
                     }
-                } else if (piece) {
-                    // the raw accumulator of this piece: 64 contiguous bytes per thread and chunk
+                } else if (o < a.out) {
 #pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        reinterpret_cast<float4 *>(my_part + j0)[q] = make_float4(acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
-                } else {
-                    write_chunk(o, j0, acc, bias);
-                }
-            }
-            if (!HEAD && piece) {
-                // Which blocks hold pieces of this tile: those whose shares meet its k-blocks.  The last of
-                // them to arrive adds the pieces in block order and finishes the tile.
-                const int item = model * a.tiles + tile;
-                const int64_t seq0 = (int64_t)item * nkb, seq1 = seq0 + nkb;
-                int b_lo = (int)(seq0 * gridDim.x / n_seq), b_hi = (int)((seq1 - 1) * gridDim.x / n_seq);
-                while (b_lo > 0 && cut(b_lo) > seq0) --b_lo;
-                while (cut(b_lo + 1) <= seq0) ++b_lo;
-                while (b_hi + 1 < (int)gridDim.x && cut(b_hi + 1) < seq1) ++b_hi;
-                while (cut(b_hi) >= seq1) --b_hi;
-                __threadfence();
-                epi_sync();
-                if (g == 0) {
-                    const unsigned tk = atomicAdd(a.split_ticket + item, 1u);
-                    head_last = tk == (unsigned)(b_hi - b_lo);
-                    if (head_last) a.split_ticket[item] = 0;             // ready for the next launch
-                }
-                epi_sync();
-                if (head_last) {                       // uniform in the group; rewritten only after the barrier below
-                    __threadfence();
-                    for (int j0 = 0; j0 < a.n_pad; j0 += 16) {
-                        float acc[16];
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) acc[j] = 0.f;
-                        for (int q = b_lo; q <= b_hi; ++q) {
-                            // block q's piece of this tile is its first unit if its share starts inside the tile
-                            const int which = (int)(cut(q) / nkb) == item ? 0 : 1;
-                            const float4 *src = reinterpret_cast<const float4 *>(
-                                a.split_part + (((int64_t)q * 2 + which) * kRows + row) * a.n_pad + j0);
-#pragma unroll
-                            for (int u = 0; u < 4; ++u) {
-                                const float4 t = __ldcg(src + u);
-                                acc[4 * u] += t.x; acc[4 * u + 1] += t.y; acc[4 * u + 2] += t.z; acc[4 * u + 3] += t.w;
+                    for (int j = 0; j < 16; ++j) {
+                        const int jj = j0 + j;
+                        float z = acc[j] + bias;
+                        if (a.relu) z = (z > 0.f || z != z) ? z : 0.f;
+                        if (jj >= a.n_r) z = 0.f;             // padded samples
+                        if (a.Hout && jj < a.n_r) a.Hout[((int64_t)model * a.n_r + jj) * a.out + o] = z;
+                        if (a.Hsplit) {
+                            T *hs = static_cast<T *>(a.Hsplit) + (int64_t)model * 2 * a.n_pad * a.out + o;
+                            if (kBf16) {
+                                const __nv_bfloat16 hi = __float2bfloat16_rn(z);
+                                const __nv_bfloat16 lo = __float2bfloat16_rn(z - __bfloat162float(hi));
+                                reinterpret_cast<__nv_bfloat16 *>(hs)[(int64_t)jj * a.out] = hi;
+                                reinterpret_cast<__nv_bfloat16 *>(hs)[(int64_t)(a.n_pad + jj) * a.out] = lo;
+                            } else {
+                                const float hi = tf32_hi(z);
+                                reinterpret_cast<float *>(hs)[(int64_t)jj * a.out] = hi;
+                                reinterpret_cast<float *>(hs)[(int64_t)(a.n_pad + jj) * a.out] = z - hi;
                             }
                         }
-                        write_chunk(o, j0, acc, bias);
-                    }
-                    if (g < 8 && model > 0) {              // the pieces' sums of squares, per (quadrant, converter set)
-                        float nrm = 0.f;
-                        for (int q = b_lo; q <= b_hi; ++q) {
-                            const int which = (int)(cut(q) / nkb) == item ? 0 : 1;
-                            nrm += __ldcg(a.split_norm + ((int64_t)q * 2 + which) * 8 + g);
-                        }
-                        a.normpart[(int64_t)(model - 1) * a.np_slots + a.np_base + tile * 8 + g] = nrm;
                     }
                 }
-                epi_sync();                            // head_last may be reused
             }
             if (HEAD) {
                 // the four warps' partial logits added in warp order: one set per tile in global memory
@@ -847,20 +736,6 @@ cudaError_t encode_maps(const LayerTcLaunch &l, CUtensorMap *map_x, CUtensorMap 
     return cudaSuccess;
 }
 
-// Even shares instead of whole tiles when the tiles do not fill the last round of blocks: at least a
-// tile's worth of k-blocks per share (so a tile meets at most one share boundary) and tiles long
-// enough for pieces of two k-blocks and more; only where whole tiles would leave more than a twentieth
-// of the SM rounds idle.  Not with the last layer folded in (its finish counts whole tiles).
-bool shares_tiles(const Context &c, const LayerTcLaunch &l, bool head) {
-    const int block_k = c.desc.param_dtype == ZENO_BF16 ? TcTraits<__nv_bfloat16>::kBlockK : TcTraits<float>::kBlockK;
-    const int items = (l.m + 1) * ((l.out + kRows - 1) / kRows);
-    const int sms = c.sm_count > 0 ? c.sm_count : 148;
-    const int nkb = (l.K + block_k - 1) / block_k;
-    const int whole_rounds = (items + sms - 1) / sms;
-    return !head && c.split_part != nullptr && items >= sms && nkb >= 6 && sms <= c.split_blocks &&
-           (double)items < 0.95 * (double)whole_rounds * sms;
-}
-
 template <typename T, bool LINEAR, bool HEAD>
 cudaError_t launch_typed(Context &c, const LayerTcLaunch &l, cudaStream_t s) {
     using Tr = TcTraits<T>;
@@ -903,21 +778,17 @@ cudaError_t launch_typed(Context &c, const LayerTcLaunch &l, cudaStream_t s) {
     a.status = c.dev_status;
     a.spin_limit = c.spin_limit;
     if (HEAD) a.head = *l.head; else a.head = HeadFuse{};
-    const int items = (l.m + 1) * a.tiles;
-    const int sms = c.sm_count > 0 ? c.sm_count : 148;
-    a.split = shares_tiles(c, l, HEAD);
-    a.split_part = c.split_part;
-    a.split_norm = c.split_norm;
-    a.split_ticket = c.split_ticket;
     static PerDeviceOnce attr_set;      // per instantiation and device
     if (attr_set.need(c.device)) {
         e = cudaFuncSetAttribute(layer_tc_kernel<T, LINEAR, HEAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, budget);
         if (e != cudaSuccess) return e;
         attr_set.mark(c.device);
     }
-    // whole tiles: the fewest blocks that give the same number of rounds as one block per SM
+    const int items = (l.m + 1) * a.tiles;
+    const int sms = c.sm_count > 0 ? c.sm_count : 148;
+    // equal shares: the fewest blocks that give the same number of rounds as one block per SM
     const int rounds = (items + sms - 1) / sms;
-    const int blocks = a.split ? sms : (items + rounds - 1) / rounds;
+    const int blocks = (items + rounds - 1) / rounds;
     return launch_chained(layer_tc_kernel<T, LINEAR, HEAD>, dim3(blocks), dim3(kLThreads), (size_t)a.stages * stage_bytes + (size_t)a.b_stages * b_bytes + 1024 + zq_bytes, s,
                           chain_launches(c), map_x, map_v, map_h, a);
 }
@@ -948,7 +819,7 @@ int layer_tc_head_slots(int out) { return (out + kRows - 1) / kRows * 4; }
 cudaError_t launch_layer_tc(Context &c, const LayerTcLaunch &l, cudaStream_t s, int *launches) {
     ++*launches;
     const bool head = l.head != nullptr && l.head->classes > 0 && !l.linear;
-    profile_mark(c, head ? "layer_tc_head" : shares_tiles(c, l, head) ? "layer_tc_shared" : "layer_tc", s);
+    profile_mark(c, head ? "layer_tc_head" : "layer_tc", s);
     if (c.desc.param_dtype == ZENO_BF16)
         return head ? launch_typed<__nv_bfloat16, false, true>(c, l, s) : launch_typed<__nv_bfloat16, false, false>(c, l, s);
     if (l.linear) return launch_typed<float, true, false>(c, l, s);

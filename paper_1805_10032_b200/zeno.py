@@ -25,7 +25,7 @@ F32, BF16 = 0, 1
 
 EXPORTS = (
     "zeno_param_count", "zeno_create", "zeno_destroy", "zeno_score", "zeno_select",
-    "zeno_aggregate", "zeno_step", "zeno_step_update", "zeno_run", "zeno_step_host", "zeno_device_status", "zeno_score_lsq_static",
+    "zeno_aggregate", "zeno_median", "zeno_krum", "zeno_step", "zeno_step_update", "zeno_run", "zeno_step_host", "zeno_device_status", "zeno_score_lsq_static",
     "zeno_debug_set_wait_limit",
     "zeno_profile", "zeno_profile_read",
     "zeno_last_launch_count",
@@ -76,6 +76,10 @@ def load_library() -> ctypes.CDLL:
     lib.zeno_select.argtypes = [vp, vp, i32, i32, vp, vp]
     lib.zeno_aggregate.restype = i32
     lib.zeno_aggregate.argtypes = [vp, vp, i64, i32, vp, i32, vp, vp]
+    lib.zeno_median.restype = i32
+    lib.zeno_median.argtypes = [vp, vp, i64, i32, vp, vp]
+    lib.zeno_krum.restype = i32
+    lib.zeno_krum.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, vp]
     lib.zeno_step.restype = i32
     lib.zeno_step.argtypes = [vp, vp, vp, i64, i32, ctypes.POINTER(Batch), f32, f32, i32, vp, vp, vp, vp]
     lib.zeno_run.restype = i32
@@ -261,6 +265,27 @@ class Zeno:
                                       _ptr(out), _stream_ptr(stream))
         self._check(st, "zeno_aggregate")
         return out
+
+    def median(self, V, m=None, ldv=None, out=None, stream=None):
+        """The marginal median of the candidates (the paper's Median baseline): out[d] float32."""
+        m = V.shape[0] if m is None else m
+        ldv = V.stride(0) if ldv is None else ldv
+        if out is None:
+            out = torch.empty(self.d, dtype=torch.float32, device=self._dev())
+        self._check(self._lib.zeno_median(self._h, _ptr(V), int(ldv), int(m), _ptr(out), _stream_ptr(stream)),
+                    "zeno_median")
+        return out
+
+    def krum(self, V, b, m=None, ldv=None, want_out=True, stream=None):
+        """Krum_b (the paper's Krum baseline): returns (out[d] or None, k int32[1], sums[m])."""
+        m = V.shape[0] if m is None else m
+        ldv = V.stride(0) if ldv is None else ldv
+        out = torch.empty(self.d, dtype=torch.float32, device=self._dev()) if want_out else None
+        k = torch.empty(1, dtype=torch.int32, device=self._dev())
+        sums = torch.empty(m, dtype=torch.float32, device=self._dev())
+        self._check(self._lib.zeno_krum(self._h, _ptr(V), int(ldv), int(m), int(b), _ptr(out), _ptr(k), _ptr(sums),
+                                        _stream_ptr(stream)), "zeno_krum")
+        return out, k, sums
 
     def step(self, x, V, features, targets, gamma, rho, b, m=None, ldv=None, out=None,
              scores=None, idx=None, want_scores=True, want_idx=True, stream=None):

@@ -46,13 +46,14 @@ SHRUNK = {
     # several tiles per model, an odd number of classes)
     "cfg4_ten_classes": (4, dict(dims=(264, 136, 200, 10), m=9, b=3, n_r=19, faults=[(3, "signflip")])),
     "cfg2_seven_classes": (2, dict(dims=(520, 200, 300, 7), n_r=30, m=12, b=5, faults=[(5, "noise200")])),
-    # tiles shared between blocks (more tiles than SMs, not a multiple of the SM count): the linear fp32 first
-    # layer, a later fp32 layer, and a bfloat16 model -- ragged row tiles and a ragged last k-block in each
-    "cfg3_shared_tiles_first_layer": (3, dict(dims=(200, 384, 10), m=100, b=40, n_r=5,
+    # more tiles than SMs, not a multiple of the SM count (several rounds of tiles per block, the last one
+    # partly empty): the linear fp32 first layer, a later fp32 layer, and a bfloat16 model -- ragged row
+    # tiles and a ragged last k-block in each
+    "cfg3_ragged_rounds_first_layer": (3, dict(dims=(200, 384, 10), m=100, b=40, n_r=5,
                                               faults=[(20, "signflip"), (20, "omniscient")])),
-    "cfg3_shared_tiles_later_layer": (3, dict(dims=(136, 264, 330, 10), m=100, b=40, n_r=9,
+    "cfg3_ragged_rounds_later_layer": (3, dict(dims=(136, 264, 330, 10), m=100, b=40, n_r=9,
                                               faults=[(20, "signflip"), (20, "omniscient")])),
-    "cfg4_shared_tiles": (4, dict(dims=(392, 264, 50), m=100, b=30, n_r=7, faults=[(30, "signflip")])),
+    "cfg4_ragged_rounds": (4, dict(dims=(392, 264, 50), m=100, b=30, n_r=7, faults=[(30, "signflip")])),
     "cfg5_small": (5, dict(d=70000, m=13, b=5, n_r=16, n_noise=5)),
     "cfg5_nr5": (5, dict(d=33333 * 4, m=70, b=30, n_r=5, n_noise=30)),
     # d a multiple of 32: the tensor-core stream fetches both k-blocks of a pair with one copy per operand
@@ -91,8 +92,8 @@ def kernels_of_a_step(w):
     ("cfg3_many_tiles", ["split_acts", "layer_tc", "stream_combine", "mlp_head_loss_tail", "aggregate"]),
     ("cfg4_128_samples", ["split_acts", "layer_tc", "layer_tc", "layer_tc", "mlp_loss_tail", "aggregate"]),
     ("cfg4_small", ["split_acts", "layer_tc", "layer_tc", "layer_tc", "mlp_loss_tail", "aggregate"]),
-    ("cfg3_shared_tiles_first_layer", ["split_acts", "layer_tc_shared", "stream_combine", "mlp_head_loss_tail", "aggregate"]),
-    ("cfg4_shared_tiles", ["split_acts", "layer_tc_shared", "layer_tc", "mlp_loss_tail", "aggregate"]),
+    ("cfg3_ragged_rounds_first_layer", ["split_acts", "layer_tc", "stream_combine", "mlp_head_loss_tail", "aggregate"]),
+    ("cfg4_ragged_rounds", ["split_acts", "layer_tc", "layer_tc", "mlp_loss_tail", "aggregate"]),
     ("cfg5_nr24_m64", ["lsq_tc", "lsq_finish", "select", "aggregate"]),
     ("cfg5_small", ["lsq_tc", "lsq_finish", "select", "aggregate"]),
 ])

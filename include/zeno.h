@@ -140,6 +140,26 @@ zeno_status zeno_select(zeno_handle h, const float *scores, int32_t m, int32_t b
 zeno_status zeno_aggregate(zeno_handle h, const void *V, int64_t ldv, int32_t m,
                            const int32_t *idx, int32_t k, float *out, void *stream);
 
+/* The score pass for a parameter vector that is sharded over several GPUs by column slice (the paper's
+ * model is m-way data parallel; Definition 2's score is what has to be put together across the slices).
+ * For the least-squares loss the residual A (x - gamma v) - y is linear in the parameters, so each GPU can
+ * take the products of its own columns and one sum over the GPUs gives the whole:
+ *
+ *   zeno_score_partial   on a handle made for the slice (dims[0] = the slice's length): x, V, features are
+ *                        the slice's columns (x [d_s], V [m x ldv], features A[:, slice] as [n_r x d_s]);
+ *                        writes sums[(m+1) x (n_r+1)] doubles on the device: row 0 = A_s x_s, row 1 + c =
+ *                        A_s v_c, last column of row 1 + c = the slice's share of ||v_c||^2 (0 in row 0).
+ *   (the caller adds the sums of all slices: an all-reduce of (m+1)(n_r+1) doubles)
+ *   zeno_score_from_sums from the total: losses[0] = ||A x - y||^2 / (2 n_r), losses[1 + c] the same at
+ *                        x - gamma v_c, norms, scores = Definition 2.  targets = y[n_r] (device).
+ *
+ * Every GPU then ranks the same scores (zeno_select) and averages its own slice (zeno_aggregate): no further
+ * exchange.  UNSUPPORTED: a handle that is not least squares.  Otherwise as zeno_score. */
+zeno_status zeno_score_partial(zeno_handle h, const void *x, const void *V, int64_t ldv, int32_t m,
+                               const float *features, int32_t n_r, double *sums, void *stream);
+zeno_status zeno_score_from_sums(zeno_handle h, const double *sums, const float *targets, int32_t m, int32_t n_r,
+                                 float gamma, float rho, float *scores, float *losses, float *norms, void *stream);
+
 /* The paper's baseline aggregation rules on the same candidates (Experiments, "Baselines"), for comparing
  * them with Zeno_b on the same step.
  *

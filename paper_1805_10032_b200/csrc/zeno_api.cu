@@ -550,6 +550,51 @@ zeno_status zeno_aggregate(zeno_handle h, const void *V, int64_t ldv, int32_t m,
     return st;
 }
 
+zeno_status zeno_score_partial(zeno_handle h, const void *x, const void *V, int64_t ldv, int32_t m,
+                               const float *features, int32_t n_r, double *sums, void *stream) {
+    if (!h || !sums) return ZENO_ERR_INVALID_ARG;
+    zeno_status st = check_common(h, V, ldv, m);
+    if (st != ZENO_OK) return st;
+    if (!x || !features || n_r < 1 || n_r > h->n_r_max) return ZENO_ERR_INVALID_ARG;
+    if (h->desc.kind != ZENO_LOSS_LEAST_SQUARES) return ZENO_ERR_UNSUPPORTED;
+    DeviceGuard guard(h->device);
+    if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+    zeno::LsqArgs a;
+    a.x = static_cast<const float *>(x);
+    a.V = static_cast<const float *>(V);
+    a.ldv = ldv;
+    a.d = h->d;
+    a.A = features;
+    a.n_r = n_r;
+    a.m = m;
+    a.part = h->lsq_part;
+    a.slabs = h->lsq_slabs;
+    int launches = 0;
+    profile_begin(h);
+    cudaError_t e = zeno::launch_lsq_partial(*h, a, score_rows_aligned(*h, x, V, ldv, features), sums,
+                                             static_cast<cudaStream_t>(stream), &launches);
+    profile_end(h, static_cast<cudaStream_t>(stream));
+    h->last_launches = e == cudaSuccess ? launches : 0;
+    return e == cudaSuccess ? ZENO_OK : fail_cuda(h, e);
+}
+
+zeno_status zeno_score_from_sums(zeno_handle h, const double *sums, const float *targets, int32_t m, int32_t n_r,
+                                 float gamma, float rho, float *scores, float *losses, float *norms, void *stream) {
+    if (!h || !sums || !targets || !scores) return ZENO_ERR_INVALID_ARG;
+    if (m < 1 || m > h->m_max || n_r < 1 || n_r > h->n_r_max) return ZENO_ERR_INVALID_ARG;
+    if (!isfinite(gamma) || !isfinite(rho) || rho < 0.f) return ZENO_ERR_INVALID_ARG;
+    if (h->desc.kind != ZENO_LOSS_LEAST_SQUARES) return ZENO_ERR_UNSUPPORTED;
+    DeviceGuard guard(h->device);
+    if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+    int launches = 0;
+    profile_begin(h);
+    cudaError_t e = zeno::launch_lsq_from_sums(*h, sums, m, n_r, targets, gamma, rho, losses, norms, scores,
+                                               static_cast<cudaStream_t>(stream), &launches);
+    profile_end(h, static_cast<cudaStream_t>(stream));
+    h->last_launches = e == cudaSuccess ? launches : 0;
+    return e == cudaSuccess ? ZENO_OK : fail_cuda(h, e);
+}
+
 zeno_status zeno_median(zeno_handle h, const void *V, int64_t ldv, int32_t m, float *out, void *stream) {
     if (!h || !out) return ZENO_ERR_INVALID_ARG;
     zeno_status st = check_common(h, V, ldv, m);

@@ -163,6 +163,11 @@ cudaError_t launch_mlp_layer(Context &c, const LayerArgs &a, bool aligned, cudaS
 cudaError_t launch_mlp_loss(Context &c, const float *logits, const int32_t *labels, int n_r,
                             int m, int classes, float *losses, const TailArgs &tail, cudaStream_t s,
                             int *launches);
+cudaError_t launch_lsq_partial(Context &c, const LsqArgs &a, bool aligned, double *sums, cudaStream_t s,
+                               int *launches);
+cudaError_t launch_lsq_from_sums(Context &c, const double *sums, int m, int n_r, const float *y, float gamma,
+                                 float rho, float *losses, float *norms, float *scores, cudaStream_t s,
+                                 int *launches);
 bool mlp_can_fuse_loss(int out, int n_r);
 // Warp-MMA version of the layer kernel (16-byte aligned rows, in % 8 == 0).
 cudaError_t launch_mlp_layer_mma(Context &c, const LayerArgs &a, cudaStream_t s, int *launches);

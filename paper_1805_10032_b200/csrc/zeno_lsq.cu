@@ -231,6 +231,41 @@ __global__ void __launch_bounds__(1024) lsq_finish_kernel(const float *part, int
     }
 }
 
+// The two halves of the finish for a parameter vector that is sharded over several GPUs by column slice:
+// the sums are additive over slices (the residual is linear in the parameters), so every GPU adds up its
+// own slab partials (in double, slab order), the sums of all GPUs are added by a collective in between,
+// and the losses and scores follow from the total.
+__global__ void __launch_bounds__(256) lsq_reduce_kernel(const float *part, int slabs, int n, double *sums) {
+    for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < n; t += gridDim.x * blockDim.x) {
+        double acc = 0.0;
+        for (int s = 0; s < slabs; ++s) acc += (double)part[(int64_t)s * n + t];
+        sums[t] = acc;
+    }
+}
+
+__global__ void __launch_bounds__(1024) lsq_from_sums_kernel(const double *sums /*[m+1][n_r+1]*/, int m, int n_r,
+                                                              const float *y, float gamma, float rho, float *losses,
+                                                              float *norms, float *scores) {
+    const int rows = m + 1, stride = n_r + 1;
+    __shared__ double f_s[ZENO_MAX_CANDIDATES + 1];
+    for (int r = threadIdx.x; r < rows; r += blockDim.x) {
+        double f = 0.0;
+        for (int j = 0; j < n_r; ++j) {
+            double res = sums[j] - (double)y[j];
+            if (r > 0) res -= (double)gamma * sums[r * stride + j];
+            f += res * res;
+        }
+        f_s[r] = f / (2.0 * n_r);
+        if (losses) losses[r] = (float)f_s[r];
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < m; i += blockDim.x) {
+        const double nv = sums[(i + 1) * stride + n_r];
+        if (norms) norms[i] = (float)nv;
+        scores[i] = (float)(f_s[0] - f_s[1 + i] - (double)rho * nv);
+    }
+}
+
 template <int NRT, int RB, bool VEC>
 cudaError_t launch_stream(const LsqArgs &a, cudaStream_t s) {
     const size_t smem = sizeof(float) * 2 * kStageFloats;
@@ -253,11 +288,10 @@ int lsq_slab_count(const Context &c) {
     return s < kMaxSlabs ? s : kMaxSlabs;
 }
 
-cudaError_t launch_lsq_score(Context &c, const LsqArgs &a_in, const float *y, float gamma,
-                             float rho, bool aligned, float *losses, float *norms, float *scores,
-                             cudaStream_t s, int *launches) {
+// The streaming pass over this handle's parameters: slab partials into a.part; *slabs_out slabs written.
+static cudaError_t launch_lsq_pass(Context &c, const LsqArgs &a_in, bool aligned, int *slabs_out, cudaStream_t s,
+                                   int *launches) {
     LsqArgs a = a_in;
-    const int rows = a.m + 1;
     const int nrt = a.n_r <= 8 ? 8 : (a.n_r <= 16 ? 16 : 32);
     // small problems: no more slabs than there are stages of A
     const int64_t stages = (a.d + (kStageFloats / nrt) - 1) / (kStageFloats / nrt);
@@ -279,13 +313,45 @@ cudaError_t launch_lsq_score(Context &c, const LsqArgs &a_in, const float *y, fl
         else
             e = aligned ? launch_stream<32, 4, true>(a, s) : launch_stream<32, 4, false>(a, s);
     }
+    *slabs_out = slabs;
+    return e;
+}
+
+cudaError_t launch_lsq_score(Context &c, const LsqArgs &a, const float *y, float gamma,
+                             float rho, bool aligned, float *losses, float *norms, float *scores,
+                             cudaStream_t s, int *launches) {
+    int slabs = 0;
+    cudaError_t e = launch_lsq_pass(c, a, aligned, &slabs, s, launches);
     if (e != cudaSuccess) return e;
     ++*launches;
     profile_mark(c, "lsq_finish", s);
     // the combined sums live behind the slab partials in the same workspace region
+    const int rows = a.m + 1;
     float *sums = a.part + (int64_t)slabs * rows * (a.n_r + 1);
     lsq_finish_kernel<<<1, 1024, 0, s>>>(a.part, slabs, a.m, a.n_r, y, gamma, rho, losses, norms,
                                          scores, sums);
+    return cudaGetLastError();
+}
+
+// This handle's slice of the sums: [m+1][n_r+1] doubles (row 0: A x, row 1 + c: A v_c; last column: ||v_c||^2).
+cudaError_t launch_lsq_partial(Context &c, const LsqArgs &a, bool aligned, double *sums, cudaStream_t s,
+                               int *launches) {
+    int slabs = 0;
+    cudaError_t e = launch_lsq_pass(c, a, aligned, &slabs, s, launches);
+    if (e != cudaSuccess) return e;
+    ++*launches;
+    profile_mark(c, "lsq_reduce", s);
+    const int n = (a.m + 1) * (a.n_r + 1);
+    lsq_reduce_kernel<<<(n + 255) / 256, 256, 0, s>>>(a.part, slabs, n, sums);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_lsq_from_sums(Context &c, const double *sums, int m, int n_r, const float *y, float gamma,
+                                 float rho, float *losses, float *norms, float *scores, cudaStream_t s,
+                                 int *launches) {
+    ++*launches;
+    profile_mark(c, "lsq_from_sums", s);
+    lsq_from_sums_kernel<<<1, 1024, 0, s>>>(sums, m, n_r, y, gamma, rho, losses, norms, scores);
     return cudaGetLastError();
 }
 

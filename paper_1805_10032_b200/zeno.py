@@ -25,7 +25,7 @@ F32, BF16 = 0, 1
 
 EXPORTS = (
     "zeno_param_count", "zeno_create", "zeno_destroy", "zeno_score", "zeno_select",
-    "zeno_aggregate", "zeno_median", "zeno_krum", "zeno_step", "zeno_step_update", "zeno_run", "zeno_step_host", "zeno_device_status", "zeno_score_lsq_static",
+    "zeno_aggregate", "zeno_score_partial", "zeno_score_from_sums", "zeno_median", "zeno_krum", "zeno_step", "zeno_step_update", "zeno_run", "zeno_step_host", "zeno_device_status", "zeno_score_lsq_static",
     "zeno_debug_set_wait_limit",
     "zeno_profile", "zeno_profile_read",
     "zeno_last_launch_count",
@@ -76,6 +76,10 @@ def load_library() -> ctypes.CDLL:
     lib.zeno_select.argtypes = [vp, vp, i32, i32, vp, vp]
     lib.zeno_aggregate.restype = i32
     lib.zeno_aggregate.argtypes = [vp, vp, i64, i32, vp, i32, vp, vp]
+    lib.zeno_score_partial.restype = i32
+    lib.zeno_score_partial.argtypes = [vp, vp, vp, i64, i32, vp, i32, vp, vp]
+    lib.zeno_score_from_sums.restype = i32
+    lib.zeno_score_from_sums.argtypes = [vp, vp, vp, i32, i32, f32, f32, vp, vp, vp, vp]
     lib.zeno_median.restype = i32
     lib.zeno_median.argtypes = [vp, vp, i64, i32, vp, vp]
     lib.zeno_krum.restype = i32
@@ -265,6 +269,29 @@ class Zeno:
                                       _ptr(out), _stream_ptr(stream))
         self._check(st, "zeno_aggregate")
         return out
+
+    def score_partial(self, x, V, features, m=None, ldv=None, sums=None, stream=None):
+        """This handle's column slice of the least-squares score sums: float64 [(m+1), (n_r+1)]."""
+        m = V.shape[0] if m is None else m
+        ldv = V.stride(0) if ldv is None else ldv
+        n_r = features.shape[0]
+        if sums is None:
+            sums = torch.empty((m + 1, n_r + 1), dtype=torch.float64, device=self._dev())
+        st = self._lib.zeno_score_partial(self._h, _ptr(x), _ptr(V), int(ldv), int(m), _ptr(features), int(n_r),
+                                          _ptr(sums), _stream_ptr(stream))
+        self._check(st, "zeno_score_partial")
+        return sums
+
+    def score_from_sums(self, sums, targets, gamma, rho, stream=None):
+        """Definition 2's scores from the sums of all slices: returns (scores[m], losses[m+1], norms[m])."""
+        m, n_r = sums.shape[0] - 1, sums.shape[1] - 1
+        scores = torch.empty(m, dtype=torch.float32, device=self._dev())
+        losses = torch.empty(m + 1, dtype=torch.float32, device=self._dev())
+        norms = torch.empty(m, dtype=torch.float32, device=self._dev())
+        st = self._lib.zeno_score_from_sums(self._h, _ptr(sums), _ptr(targets), int(m), int(n_r), float(gamma),
+                                            float(rho), _ptr(scores), _ptr(losses), _ptr(norms), _stream_ptr(stream))
+        self._check(st, "zeno_score_from_sums")
+        return scores, losses, norms
 
     def median(self, V, m=None, ldv=None, out=None, stream=None):
         """The marginal median of the candidates (the paper's Median baseline): out[d] float32."""

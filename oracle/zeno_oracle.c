@@ -440,3 +440,81 @@ int zo_krum(int dtype, const void *V, int64_t ldv, int64_t d, int m, int b,
     if (!dist) free(D);
     return ZO_OK;
 }
+
+/* ---- the workers' side of Algorithm 1, and the experiments' failures -------
+ *
+ * Algorithm 1, worker i: v_i = grad F_i(x) on the worker's own samples.  Written out for the two
+ * losses whose gradient has a closed form that needs no back-propagation through hidden layers:
+ * softmax regression (a one-layer model of the softmax family) and least squares.
+ *   softmax regression:  d/dW[c][k] = (1/n) sum_j (p_j[c] - [c = label_j]) a_j[k],
+ *                        d/db[c]    = (1/n) sum_j (p_j[c] - [c = label_j]),  p_j = softmax(W a_j + b);
+ *   least squares:       grad = A^T (A x - y) / n.
+ * flip != 0 is the experiments' label-flipping failure: every label is replaced by (classes - 1 - label)
+ * before the gradient is taken (the paper's "9 - label" for ten classes). */
+int zo_worker_gradient(int kind, int n_layers, const int64_t *dims, int has_bias, const void *x, int dtype,
+                       const float *features, const void *targets, int n, int flip, double *grad)
+{
+    if (n < 1) return ZO_BAD_ARG;
+    if (kind == ZO_LOSS_LEAST_SQUARES) {
+        const int64_t d = dims[0];
+        const float *y = (const float *)targets;
+        for (int64_t k = 0; k < d; ++k) grad[k] = 0.0;
+        for (int j = 0; j < n; ++j) {
+            double r = -(double)y[j];
+            for (int64_t k = 0; k < d; ++k) r += (double)features[(size_t)j * d + k] * zo_load(x, k, dtype);
+            for (int64_t k = 0; k < d; ++k) grad[k] += (double)features[(size_t)j * d + k] * r / (double)n;
+        }
+        return ZO_OK;
+    }
+    if (kind != ZO_LOSS_SOFTMAX_MLP || n_layers != 1) return ZO_BAD_ARG;
+    const int64_t in = dims[0], classes = dims[1];
+    const int32_t *labels = (const int32_t *)targets;
+    const int64_t d = classes * in + (has_bias ? classes : 0);
+    double *z = (double *)malloc(sizeof(double) * (size_t)classes);
+    if (!z) return ZO_NO_MEM;
+    for (int64_t k = 0; k < d; ++k) grad[k] = 0.0;
+    for (int j = 0; j < n; ++j) {
+        const float *a = features + (size_t)j * in;
+        double zmax = -INFINITY;
+        for (int64_t c = 0; c < classes; ++c) {
+            double s = has_bias ? zo_load(x, classes * in + c, dtype) : 0.0;
+            for (int64_t k = 0; k < in; ++k) s += zo_load(x, c * in + k, dtype) * (double)a[k];
+            z[c] = s;
+            if (s > zmax) zmax = s;
+        }
+        double se = 0.0;
+        for (int64_t c = 0; c < classes; ++c) se += exp(z[c] - zmax);
+        int64_t label = labels[j];
+        if (flip) label = classes - 1 - label;
+        for (int64_t c = 0; c < classes; ++c) {
+            const double delta = (exp(z[c] - zmax) / se - (c == label ? 1.0 : 0.0)) / (double)n;
+            for (int64_t k = 0; k < in; ++k) grad[c * in + k] += delta * (double)a[k];
+            if (has_bias) grad[classes * in + c] += delta;
+        }
+    }
+    free(z);
+    return ZO_OK;
+}
+
+/* The experiments' failures applied to the candidate matrix (float64 rows, [m][d]):
+ *   mode 0, bit-flipping: a faulty worker pushes the negative of its gradient, and the first faulty
+ *           row's (negated) gradient is copied over all other faulty rows;
+ *   mode 1, scaling: a faulty row becomes eps times its gradient (the failure model's toy example,
+ *           eps a large negative constant). */
+int zo_inject_faults(double *V, int64_t d, int m, const int32_t *faulty, int n_faulty, int mode, double eps)
+{
+    if (n_faulty < 0 || (mode != 0 && mode != 1)) return ZO_BAD_ARG;
+    for (int f = 0; f < n_faulty; ++f)
+        if (faulty[f] < 0 || faulty[f] >= m) return ZO_BAD_ARG;
+    if (n_faulty == 0) return ZO_OK;
+    if (mode == 0) {
+        double *first = V + (size_t)faulty[0] * d;
+        for (int64_t k = 0; k < d; ++k) first[k] = -first[k];
+        for (int f = 1; f < n_faulty; ++f)
+            memcpy(V + (size_t)faulty[f] * d, first, sizeof(double) * (size_t)d);
+    } else {
+        for (int f = 0; f < n_faulty; ++f)
+            for (int64_t k = 0; k < d; ++k) V[(size_t)faulty[f] * d + k] *= eps;
+    }
+    return ZO_OK;
+}

@@ -65,6 +65,10 @@ def _load():
         lib.zo_step.restype = i32
         lib.zo_step.argtypes = [i32, i32, i32, vp, i32, vp, vp, i64, i32, vp, vp, i32,
                                 dbl, dbl, i32, vp, vp, vp]
+        lib.zo_worker_gradient.restype = i32
+        lib.zo_worker_gradient.argtypes = [i32, i32, vp, i32, vp, i32, vp, vp, i32, i32, vp]
+        lib.zo_inject_faults.restype = i32
+        lib.zo_inject_faults.argtypes = [vp, i64, i32, vp, i32, i32, dbl]
         lib.zo_median.restype = i32
         lib.zo_median.argtypes = [i32, vp, i64, i64, i32, vp]
         lib.zo_krum.restype = i32
@@ -190,6 +194,31 @@ def aggregate(dtype, V, ldv, d, m, idx):
     _check(_load().zo_aggregate(dtype, _ptr(V), int(ldv), int(d), int(m), _ptr(idx),
                                 idx.shape[0], _ptr(out)), "zo_aggregate")
     return out
+
+
+def worker_gradient(kind, dtype, dims, has_bias, x, features, targets, flip=False):
+    """Algorithm 1, a worker's line: the gradient of the mean loss over its own samples at x (float64 [d]);
+    softmax regression (a one-layer model) and least squares.  flip: the label-flipping failure."""
+    dm = _dims(dims)
+    x = _params(x, dtype)
+    features = _features(features)
+    targets = _targets(kind, targets)
+    d = param_count(kind, dims, has_bias)
+    g = np.empty(d, dtype=np.float64)
+    _check(_load().zo_worker_gradient(kind, len(dm) - 1, _ptr(dm), int(has_bias), _ptr(x), dtype, _ptr(features),
+                                      _ptr(targets), targets.shape[0], int(bool(flip)), _ptr(g)),
+           "zo_worker_gradient")
+    return g
+
+
+def inject_faults(V, faulty, mode, eps=0.0):
+    """The experiments' failures on a float64 candidate matrix [m, d] (returns a modified copy):
+    mode 0 bit-flipping with copy-overwrite, mode 1 scaling by eps."""
+    V = np.array(V, dtype=np.float64, order="C", copy=True)
+    faulty = np.ascontiguousarray(faulty, dtype=np.int32)
+    _check(_load().zo_inject_faults(_ptr(V), V.shape[1], V.shape[0], _ptr(faulty), faulty.shape[0], int(mode),
+                                    float(eps)), "zo_inject_faults")
+    return V
 
 
 def median(dtype, V, ldv, d, m):

@@ -133,3 +133,63 @@ def test_krum_needs_a_neighbour(oracle):
         oracle.krum(F32, V, 3, 3, 5, 3)                        # m - b - 2 = 0
     k, _, _ = oracle.krum(F32, V, 3, 3, 5, 2)                  # one neighbour: fine, ties go to the lowest index
     assert k == 0
+
+
+# ---------------------------------------------------------------- the workers' side: gradients and failures
+# (Algorithm 1, worker lines; Experiments: label-flipping and bit-flipping failures; the failure model's
+# scaled gradient)
+
+MLP, LSQ = 0, 1
+
+
+def _fd_gradient(oracle, kind, dims, x, feats, tgts, h=1e-6):
+    """Central differences of the (already pinned) loss f_r, coordinate by coordinate, in float64."""
+    g = np.empty(x.shape[0])
+    for k in range(x.shape[0]):
+        e = np.zeros_like(x)
+        e[k] = h
+        g[k] = (oracle.loss(kind, dims, True, x + e, feats, tgts) - oracle.loss(kind, dims, True, x - e, feats, tgts)) / (2 * h)
+    return g
+
+
+def test_worker_gradient_softmax_regression_matches_finite_differences_of_the_loss(oracle):
+    r = _rng(21)
+    dims = (6, 4)
+    d = 6 * 4 + 4
+    x = r.standard_normal(d).astype(np.float32)
+    feats = r.standard_normal((5, 6)).astype(np.float32)
+    labels = r.integers(0, 4, 5).astype(np.int32)
+    g = oracle.worker_gradient(MLP, F32, dims, True, x, feats, labels)
+    fd = _fd_gradient(oracle, MLP, dims, x.astype(np.float64), feats, labels)
+    assert np.allclose(g, fd, rtol=1e-6, atol=1e-8)
+    # the label-flipping failure is the gradient on the labels classes - 1 - label
+    gf = oracle.worker_gradient(MLP, F32, dims, True, x, feats, labels, flip=True)
+    assert np.allclose(gf, oracle.worker_gradient(MLP, F32, dims, True, x, feats, (3 - labels).astype(np.int32)))
+    assert not np.allclose(gf, g)
+    # a gradient of a softmax model: the bias entries sum to zero (probabilities and one-hot both sum to one)
+    assert abs(g[24:].sum()) < 1e-12
+
+
+def test_worker_gradient_least_squares_is_the_normal_equations_residual(oracle):
+    r = _rng(22)
+    d, n = 9, 4
+    x = r.standard_normal(d).astype(np.float32)
+    A = r.standard_normal((n, d)).astype(np.float32)
+    y = r.standard_normal(n).astype(np.float32)
+    g = oracle.worker_gradient(LSQ, F32, (d, 1), False, x, A, y)
+    Ad = A.astype(np.float64)
+    assert np.allclose(g, Ad.T @ (Ad @ x.astype(np.float64) - y) / n, rtol=1e-12)
+    fd = _fd_gradient(oracle, LSQ, (d, 1), x.astype(np.float64), A, y)
+    assert np.allclose(g, fd, rtol=1e-6, atol=1e-8)
+
+
+def test_inject_faults_bit_flip_copies_one_negated_gradient_and_scaling_multiplies(oracle):
+    V = np.arange(20, dtype=np.float64).reshape(5, 4) + 1
+    out = oracle.inject_faults(V, [3, 1, 4], 0)
+    assert np.array_equal(out[3], -V[3]) and np.array_equal(out[1], -V[3]) and np.array_equal(out[4], -V[3])
+    assert np.array_equal(out[[0, 2]], V[[0, 2]])
+    out = oracle.inject_faults(V, [0, 2], 1, eps=-4.0)
+    assert np.array_equal(out[[0, 2]], -4.0 * V[[0, 2]]) and np.array_equal(out[[1, 3, 4]], V[[1, 3, 4]])
+    assert np.array_equal(oracle.inject_faults(V, [], 0), V)
+    with pytest.raises(Exception):
+        oracle.inject_faults(V, [5], 0)

@@ -160,6 +160,31 @@ zeno_status zeno_score_partial(zeno_handle h, const void *x, const void *V, int6
 zeno_status zeno_score_from_sums(zeno_handle h, const double *sums, const float *targets, int32_t m, int32_t n_r,
                                  float gamma, float rho, float *scores, float *losses, float *norms, void *stream);
 
+/* The workers' side of Algorithm 1 and the experiments' failures, on the device, so that a whole synchronous
+ * iteration (workers' gradients -> failures -> Zeno_b -> update) can be chained on one stream.  These calls
+ * build the step's input V; they are no part of the scoring path.
+ *
+ * zeno_worker_gradients -- Algorithm 1, worker i: v_i = grad F_i(x), the gradient of the mean loss over the
+ * worker's own n samples, written to row i of V (in V's storage type).  features: [m][n x dims[0]] binary32,
+ * targets: [m][n] int32 labels or binary32 y, one batch per worker; label_flip: int32[m] on the device or
+ * NULL -- where non-zero, that worker's labels are replaced by (classes - 1 - label) first (Experiments,
+ * label-flipping failure: "9 - label" for ten classes).  UNSUPPORTED: losses whose gradient needs
+ * back-propagation through hidden layers (only one-layer softmax models with at most 32 classes, and least
+ * squares in binary32, are served), or n beyond what a block's shared memory holds.
+ *
+ * zeno_inject_faults -- rows faulty[0..n_faulty) (device int32, entries outside [0, m) are skipped) of V
+ * are overwritten in place:
+ *   ZENO_FAULT_BIT_FLIP  Experiments, bit-flipping failure: the negative of row faulty[0]'s gradient, copied
+ *                        over every faulty row (all faulty gradients have the same value);
+ *   ZENO_FAULT_SCALE     the failure model's example: eps times the row's own gradient (eps a large
+ *                        negative constant). */
+#define ZENO_FAULT_BIT_FLIP 0
+#define ZENO_FAULT_SCALE 1
+zeno_status zeno_worker_gradients(zeno_handle h, const void *x, const float *features, const void *targets, int32_t n,
+                                  int32_t m, const int32_t *label_flip, void *V, int64_t ldv, void *stream);
+zeno_status zeno_inject_faults(zeno_handle h, void *V, int64_t ldv, int32_t m, const int32_t *faulty, int32_t n_faulty,
+                               int32_t mode, float eps, void *stream);
+
 /* The paper's baseline aggregation rules on the same candidates (Experiments, "Baselines"), for comparing
  * them with Zeno_b on the same step.
  *

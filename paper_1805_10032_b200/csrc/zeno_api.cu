@@ -5,6 +5,8 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "zeno_internal.h"
 
 using zeno::Context;
@@ -30,6 +32,12 @@ bool desc_ok(const zeno_model_desc *d) {
 }
 
 bool is_aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// A named range around an entry point, visible on a profiler's timeline (a no-op without one attached).
+struct Range {
+    explicit Range(const char *name) { nvtxRangePushA(name); }
+    ~Range() { nvtxRangePop(); }
+};
 
 // Switches to the handle's device for the duration of a call and back afterwards.
 struct DeviceGuard {
@@ -157,8 +165,9 @@ zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv,
         if (in_l < 128 || out_l < 128) return false;
         if (l > 0) return true;
         // first layer: the stream that shares the batch reads V once and nothing else, but it needs
-        // split-K partials to fill the SMs; with enough whole tiles for every SM this kernel wins
-        return (m + 1) * ((out_l + 127) / 128) >= 2 * c->sm_count;
+        // split-K partials to fill the SMs; with enough whole tiles for every SM this kernel wins, and
+        // beyond the stream's 64 samples it is the only tensor-core kernel there is
+        return (m + 1) * ((out_l + 127) / 128) >= 2 * c->sm_count || n_r > 64;
     };
     // the layer before a small last layer takes that layer, the loss and the tail along
     auto head_folds_into = [&](int l) {
@@ -341,6 +350,7 @@ int64_t zeno_param_count(const zeno_model_desc *desc) {
 
 zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m_max,
                         int32_t n_r_max, int32_t device) {
+    Range range("zeno_create");
     if (!out) return ZENO_ERR_INVALID_ARG;
     *out = nullptr;
     if (!desc) return ZENO_ERR_INVALID_ARG;
@@ -496,6 +506,7 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
 }
 
 zeno_status zeno_destroy(zeno_handle h) {
+    Range range("zeno_destroy");
     if (!h) return ZENO_ERR_INVALID_ARG;
     DeviceGuard guard(h->device);
     cudaError_t e = cudaFree(h->arena);
@@ -510,6 +521,7 @@ zeno_status zeno_destroy(zeno_handle h) {
 zeno_status zeno_score(zeno_handle h, const void *x, const void *V, int64_t ldv, int32_t m,
                        const zeno_batch *batch, float gamma, float rho, float *scores,
                        float *losses, float *norms, void *stream) {
+    Range range("zeno_score");
     if (!h) return ZENO_ERR_INVALID_ARG;
     DeviceGuard guard(h->device);
     if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
@@ -525,6 +537,7 @@ zeno_status zeno_score(zeno_handle h, const void *x, const void *V, int64_t ldv,
 
 zeno_status zeno_select(zeno_handle h, const float *scores, int32_t m, int32_t b, int32_t *idx,
                         void *stream) {
+    Range range("zeno_select");
     if (!h) return ZENO_ERR_INVALID_ARG;
     DeviceGuard guard(h->device);
     if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
@@ -538,6 +551,7 @@ zeno_status zeno_select(zeno_handle h, const float *scores, int32_t m, int32_t b
 
 zeno_status zeno_aggregate(zeno_handle h, const void *V, int64_t ldv, int32_t m, const int32_t *idx,
                            int32_t k, float *out, void *stream) {
+    Range range("zeno_aggregate");
     if (!h) return ZENO_ERR_INVALID_ARG;
     DeviceGuard guard(h->device);
     if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
@@ -552,6 +566,7 @@ zeno_status zeno_aggregate(zeno_handle h, const void *V, int64_t ldv, int32_t m,
 
 zeno_status zeno_score_partial(zeno_handle h, const void *x, const void *V, int64_t ldv, int32_t m,
                                const float *features, int32_t n_r, double *sums, void *stream) {
+    Range range("zeno_score_partial");
     if (!h || !sums) return ZENO_ERR_INVALID_ARG;
     zeno_status st = check_common(h, V, ldv, m);
     if (st != ZENO_OK) return st;
@@ -580,6 +595,7 @@ zeno_status zeno_score_partial(zeno_handle h, const void *x, const void *V, int6
 
 zeno_status zeno_score_from_sums(zeno_handle h, const double *sums, const float *targets, int32_t m, int32_t n_r,
                                  float gamma, float rho, float *scores, float *losses, float *norms, void *stream) {
+    Range range("zeno_score_from_sums");
     if (!h || !sums || !targets || !scores) return ZENO_ERR_INVALID_ARG;
     if (m < 1 || m > h->m_max || n_r < 1 || n_r > h->n_r_max) return ZENO_ERR_INVALID_ARG;
     if (!isfinite(gamma) || !isfinite(rho) || rho < 0.f) return ZENO_ERR_INVALID_ARG;
@@ -595,7 +611,51 @@ zeno_status zeno_score_from_sums(zeno_handle h, const double *sums, const float 
     return e == cudaSuccess ? ZENO_OK : fail_cuda(h, e);
 }
 
+zeno_status zeno_worker_gradients(zeno_handle h, const void *x, const float *features, const void *targets, int32_t n,
+                                  int32_t m, const int32_t *label_flip, void *V, int64_t ldv, void *stream) {
+    Range range("zeno_worker_gradients");
+    if (!h || !x || !features || !targets) return ZENO_ERR_INVALID_ARG;
+    zeno_status st = check_common(h, V, ldv, m);
+    if (st != ZENO_OK) return st;
+    if (n < 1) return ZENO_ERR_INVALID_ARG;
+    if (!zeno::worker_gradients_supported(*h, n)) return ZENO_ERR_UNSUPPORTED;
+    DeviceGuard guard(h->device);
+    if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+    int launches = 0;
+    profile_begin(h);
+    cudaError_t e = zeno::launch_worker_gradients(*h, x, features, targets, n, m, label_flip, V, ldv,
+                                                  static_cast<cudaStream_t>(stream), &launches);
+    profile_end(h, static_cast<cudaStream_t>(stream));
+    h->last_launches = e == cudaSuccess ? launches : 0;
+    return e == cudaSuccess ? ZENO_OK : fail_cuda(h, e);
+}
+
+zeno_status zeno_inject_faults(zeno_handle h, void *V, int64_t ldv, int32_t m, const int32_t *faulty, int32_t n_faulty,
+                               int32_t mode, float eps, void *stream) {
+    Range range("zeno_inject_faults");
+    if (!h) return ZENO_ERR_INVALID_ARG;
+    zeno_status st = check_common(h, V, ldv, m);
+    if (st != ZENO_OK) return st;
+    if (n_faulty < 0 || n_faulty > m || (n_faulty > 0 && !faulty)) return ZENO_ERR_INVALID_ARG;
+    if (mode != ZENO_FAULT_BIT_FLIP && mode != ZENO_FAULT_SCALE) return ZENO_ERR_INVALID_ARG;
+    if (mode == ZENO_FAULT_SCALE && !isfinite(eps)) return ZENO_ERR_INVALID_ARG;
+    if (n_faulty == 0) {
+        h->last_launches = 0;
+        return ZENO_OK;
+    }
+    DeviceGuard guard(h->device);
+    if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
+    int launches = 0;
+    profile_begin(h);
+    cudaError_t e = zeno::launch_inject_faults(*h, V, ldv, m, faulty, n_faulty, mode, eps, static_cast<cudaStream_t>(stream),
+                                               &launches);
+    profile_end(h, static_cast<cudaStream_t>(stream));
+    h->last_launches = e == cudaSuccess ? launches : 0;
+    return e == cudaSuccess ? ZENO_OK : fail_cuda(h, e);
+}
+
 zeno_status zeno_median(zeno_handle h, const void *V, int64_t ldv, int32_t m, float *out, void *stream) {
+    Range range("zeno_median");
     if (!h || !out) return ZENO_ERR_INVALID_ARG;
     zeno_status st = check_common(h, V, ldv, m);
     if (st != ZENO_OK) return st;
@@ -611,6 +671,7 @@ zeno_status zeno_median(zeno_handle h, const void *V, int64_t ldv, int32_t m, fl
 
 zeno_status zeno_krum(zeno_handle h, const void *V, int64_t ldv, int32_t m, int32_t b, float *out, int32_t *k,
                       float *sums, void *stream) {
+    Range range("zeno_krum");
     if (!h || !k) return ZENO_ERR_INVALID_ARG;
     zeno_status st = check_common(h, V, ldv, m);
     if (st != ZENO_OK) return st;
@@ -629,6 +690,7 @@ zeno_status zeno_krum(zeno_handle h, const void *V, int64_t ldv, int32_t m, int3
 zeno_status zeno_step(zeno_handle h, const void *x, const void *V, int64_t ldv, int32_t m,
                       const zeno_batch *batch, float gamma, float rho, int32_t b, float *out,
                       float *scores, int32_t *idx, void *stream) {
+    Range range("zeno_step");
     if (!h || !out) return ZENO_ERR_INVALID_ARG;
     if (m < 1 || m > h->m_max || b < 0 || b >= m) return ZENO_ERR_INVALID_ARG;
     DeviceGuard guard(h->device);
@@ -651,6 +713,7 @@ zeno_status zeno_step(zeno_handle h, const void *x, const void *V, int64_t ldv, 
 zeno_status zeno_step_update(zeno_handle h, void *x, const void *V, int64_t ldv, int32_t m,
                              const zeno_batch *batch, float gamma, float rho, int32_t b, float *out,
                              float *scores, int32_t *idx, void *stream) {
+    Range range("zeno_step_update");
     if (!h || !x) return ZENO_ERR_INVALID_ARG;
     if (m < 1 || m > h->m_max || b < 0 || b >= m) return ZENO_ERR_INVALID_ARG;
     DeviceGuard guard(h->device);
@@ -674,6 +737,7 @@ zeno_status zeno_step_update(zeno_handle h, void *x, const void *V, int64_t ldv,
 zeno_status zeno_run(zeno_handle h, void *x, const void *V, int64_t ldv, int64_t step_stride_v, int32_t m,
                      const float *features, const void *targets, int32_t n_r, int32_t steps, float gamma,
                      float rho, int32_t b, float *scores, int32_t *idx, void *stream) {
+    Range range("zeno_run");
     if (!h || !x || !V || !features || !targets) return ZENO_ERR_INVALID_ARG;
     if (steps < 1 || m < 1 || m > h->m_max || b < 0 || b >= m) return ZENO_ERR_INVALID_ARG;
     if (n_r < 1 || n_r > h->n_r_max || ldv < h->d || step_stride_v < (int64_t)m * ldv) return ZENO_ERR_INVALID_ARG;
@@ -709,6 +773,7 @@ zeno_status zeno_step_host(zeno_handle h, const void *x, const void *V, int64_t 
                            const float *features, const void *targets, int32_t n_r, float gamma,
                            float rho, int32_t b, float *out, float *scores, int32_t *idx,
                            void *stream) {
+    Range range("zeno_step_host");
     if (!h || !x || !V || !features || !targets || !out) return ZENO_ERR_INVALID_ARG;
     if (m < 1 || m > h->m_max || b < 0 || b >= m || ldv < h->d) return ZENO_ERR_INVALID_ARG;
     if (n_r < 1 || n_r > h->n_r_max) return ZENO_ERR_INVALID_ARG;

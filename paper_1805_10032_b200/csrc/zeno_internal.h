@@ -242,6 +242,13 @@ cudaError_t launch_median(Context &c, const void *V, int64_t ldv, int m, float *
 cudaError_t launch_krum(Context &c, const void *V, int64_t ldv, int m, int b, float *out, int32_t *k, float *sums,
                         cudaStream_t s, int *launches);
 
+// The workers' side of Algorithm 1 and the experiments' failures (zeno_workers.cu): builders of the step's input.
+bool worker_gradients_supported(const Context &c, int n);
+cudaError_t launch_worker_gradients(Context &c, const void *x, const float *features, const void *targets, int n, int m,
+                                    const int32_t *flip, void *V, int64_t ldv, cudaStream_t s, int *launches);
+cudaError_t launch_inject_faults(Context &c, void *V, int64_t ldv, int m, const int32_t *faulty, int n_faulty, int mode,
+                                 float eps, cudaStream_t s, int *launches);
+
 int lsq_slab_count(const Context &c);
 // Tensor-core version of the least-squares stream (zeno_lsq_tc.cu): one slab per block into a.part.
 bool lsq_tc_usable(const LsqArgs &a, bool aligned);

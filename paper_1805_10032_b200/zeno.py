@@ -21,11 +21,12 @@ MAX_CANDIDATES = 1024
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
 LOSS_SOFTMAX_MLP, LOSS_LEAST_SQUARES = 0, 1
+FAULT_BIT_FLIP, FAULT_SCALE = 0, 1
 F32, BF16 = 0, 1
 
 EXPORTS = (
     "zeno_param_count", "zeno_create", "zeno_destroy", "zeno_score", "zeno_select",
-    "zeno_aggregate", "zeno_score_partial", "zeno_score_from_sums", "zeno_median", "zeno_krum", "zeno_step", "zeno_step_update", "zeno_run", "zeno_step_host", "zeno_device_status", "zeno_score_lsq_static",
+    "zeno_aggregate", "zeno_worker_gradients", "zeno_inject_faults", "zeno_score_partial", "zeno_score_from_sums", "zeno_median", "zeno_krum", "zeno_step", "zeno_step_update", "zeno_run", "zeno_step_host", "zeno_device_status", "zeno_score_lsq_static",
     "zeno_debug_set_wait_limit",
     "zeno_profile", "zeno_profile_read",
     "zeno_last_launch_count",
@@ -76,6 +77,10 @@ def load_library() -> ctypes.CDLL:
     lib.zeno_select.argtypes = [vp, vp, i32, i32, vp, vp]
     lib.zeno_aggregate.restype = i32
     lib.zeno_aggregate.argtypes = [vp, vp, i64, i32, vp, i32, vp, vp]
+    lib.zeno_worker_gradients.restype = i32
+    lib.zeno_worker_gradients.argtypes = [vp, vp, vp, vp, i32, i32, vp, vp, i64, vp]
+    lib.zeno_inject_faults.restype = i32
+    lib.zeno_inject_faults.argtypes = [vp, vp, i64, i32, vp, i32, i32, f32, vp]
     lib.zeno_score_partial.restype = i32
     lib.zeno_score_partial.argtypes = [vp, vp, vp, i64, i32, vp, i32, vp, vp]
     lib.zeno_score_from_sums.restype = i32
@@ -269,6 +274,22 @@ class Zeno:
                                       _ptr(out), _stream_ptr(stream))
         self._check(st, "zeno_aggregate")
         return out
+
+    def worker_gradients(self, x, features, targets, V, label_flip=None, stream=None):
+        """Algorithm 1's worker lines: row i of V <- the gradient at x of worker i's mean loss over its own batch
+        (features [m, n, in], targets [m, n]); label_flip: int32 [m] device tensor or None."""
+        m, n = features.shape[0], features.shape[1]
+        st = self._lib.zeno_worker_gradients(self._h, _ptr(x), _ptr(features), _ptr(targets), int(n), int(m),
+                                             _ptr(label_flip), _ptr(V), int(V.stride(0)), _stream_ptr(stream))
+        self._check(st, "zeno_worker_gradients")
+        return V
+
+    def inject_faults(self, V, faulty, mode, eps=0.0, stream=None):
+        """The experiments' failures on the rows `faulty` (int32 device tensor) of V, in place."""
+        st = self._lib.zeno_inject_faults(self._h, _ptr(V), int(V.stride(0)), int(V.shape[0]), _ptr(faulty),
+                                          int(faulty.shape[0]), int(mode), float(eps), _stream_ptr(stream))
+        self._check(st, "zeno_inject_faults")
+        return V
 
     def score_partial(self, x, V, features, m=None, ldv=None, sums=None, stream=None):
         """This handle's column slice of the least-squares score sums: float64 [(m+1), (n_r+1)]."""

@@ -458,13 +458,8 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
     const size_t at_split0 = reserve(split_elems, 4), at_split1 = reserve(split_elems, 4);
     const size_t at_losspart = reserve(rows * 8, 8), at_losssum = reserve(rows, 8);
     const size_t at_headz = reserve(head_elems, 4), at_headt = reserve(rows, 4);
-    c->krum_blocks = 2 * c->sm_count;
-    size_t krum_elems = 0;
-    if (m_max <= ZENO_KRUM_MAX_M)               // the largest of the partial layouts any m <= m_max may use
-        for (int mm = 3; mm <= m_max; ++mm) {
-            const size_t need = zeno::krum_part_floats(mm, c->krum_blocks);
-            if (need > krum_elems) krum_elems = need;
-        }
+    c->krum_blocks = 8 * c->sm_count;
+    const size_t krum_elems = m_max <= ZENO_KRUM_MAX_M ? zeno::krum_part_floats(m_max, c->krum_blocks) : 0;
     const size_t at_krum = reserve(krum_elems, 4), at_krums = reserve(m_max, 4);
 
     e = cudaMalloc(&c->arena, bytes);

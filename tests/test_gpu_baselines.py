@@ -21,13 +21,44 @@ def _library():
 
 
 CASES = {
-    "cfg1": (1, dict()),                                                       # m = 20: registers, 32 slots
+    "cfg1": (1, dict()),                                                       # m = 20: one lane a column
     "cfg2_small_odd_m": (2, dict(dims=(300, 72, 40, 10), n_r=9, m=7, b=2, faults=[(2, "noise200")])),
-    "cfg3_m37": (3, dict(dims=(260, 44, 36, 10), m=37, b=15, n_r=7, faults=[(7, "signflip"), (8, "omniscient")])),  # 64 slots
-    "cfg3_m100": (3, dict(dims=(132, 40, 10), m=100, b=40, n_r=5, faults=[(20, "signflip"), (20, "omniscient")])),  # shared memory
+    "cfg3_m37": (3, dict(dims=(260, 44, 36, 10), m=37, b=15, n_r=7, faults=[(7, "signflip"), (8, "omniscient")])),  # two lanes a column
+    "cfg3_m100": (3, dict(dims=(132, 40, 10), m=100, b=40, n_r=5, faults=[(20, "signflip"), (20, "omniscient")])),  # four lanes a column
     "cfg4_bf16": (4, dict(dims=(264, 136, 72, 50), m=9, b=3, n_r=19, faults=[(3, "signflip")])),
     "cfg5_small": (5, dict(d=70001, m=13, b=5, n_r=16, n_noise=5, ldv=70003)),   # unaligned rows
 }
+
+
+# every compiled variant of the sorting network (columns of 8 .. 32 slots in one lane, then 2 .. 32 lanes a
+# column) at, below and above its limits, in both storage types; d leaves a ragged last group of columns
+MEDIAN_M = [1, 2, 3, 4, 7, 8, 9, 12, 13, 16, 17, 20, 21, 24, 25, 28, 29, 31, 32, 33, 63, 64, 65, 127, 128, 129, 255,
+            256, 257, 500, 512, 513, 1000, 1024]
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_median_every_network(oracle, dtype):
+    for m in MEDIAN_M:
+        if dtype == "fp32":
+            w = syn.make_config(5, d=301, m=m, b=0, n_r=4, n_noise=0, ldv=307, seed=1000 + m)
+            dt = 0
+        else:
+            w = syn.make_config(4, dims=(10, 13, 10), m=m, b=0, n_r=4, faults=[], seed=1000 + m)
+            dt = 1
+        if m >= 5:                                  # ties and special values in some columns
+            w.V[1, 0] = w.V[0, 0]
+            w.V[m - 1, 1] = float("inf")
+            w.V[m // 2, 2] = float("-inf")
+            w.V[2, 3] = float("nan")
+        want = oracle.median(dt, syn.to_numpy_params(w.V), w.ldv, w.d, w.m)
+        with zeno.from_workload(w) as z:
+            got = z.median(w.V.cuda()).cpu().numpy().astype(np.float64)
+        fin = np.isfinite(want)
+        assert np.array_equal(got[~fin], want[~fin]), m
+        if m % 2 == 1:
+            assert np.array_equal(got, want), (m, np.flatnonzero(got != want)[:5])     # a selection, exactly
+        else:                                       # the mean of two stored values formed in binary32: one rounding
+            assert np.all(np.abs(got[fin] - want[fin]) <= 1.2e-7 * np.maximum(np.abs(want[fin]), 1e-30) + 1e-45), m
 
 
 @pytest.mark.parametrize("name", sorted(CASES))
@@ -107,4 +138,4 @@ def test_krum_argument_errors_and_limits():
         with pytest.raises(zeno.ZenoError) as e:
             z.krum(w2.V.cuda(), 8)
         assert e.value.status == zeno.ERR_UNSUPPORTED
-        assert torch.isfinite(z.median(w2.V.cuda())).all()      # the median has no such limit (m = 130: 256 slots)
+        assert torch.isfinite(z.median(w2.V.cuda())).all()      # the median has no such limit

@@ -20,13 +20,23 @@
 // into fp32 registers every kFlush k-blocks (two sets alternate: one is drained while the other adds).
 //
 // Warp roles (every producer / issuer warp stays converged and issues from one elected lane):
-//   warp 0       TMA producer: per stage two 64-row boxes of V, two boxes of A, two 128-byte pieces of x
+//   warps 0, 16  TMA producers (warp 0 the even stages, warp 16 the odd ones: issuing a stage's copies takes one
+//                lane about 800 cycles, more than a stage may take): per stage two 64-row boxes of V, two boxes
+//                of A, two 128-byte pieces of x, or one copy of each when the rows allow
 //   warp 1       MMA issuer, owner of TMEM
-//   warps 2, 3   split the stage's rows of A (warp 2 the even k-block's, warp 3 the odd one's) into hi and lo
-//                terms (the MMA's B operand, 128-byte swizzled) and take A x from the same registers
+//   warps 2, 3, 18, 19   split the stage's rows of A (the first of a pair of warps the even k-block's, the
+//                second the odd one's; warps 2, 3 on even stages, 18, 19 on odd ones) into hi and lo terms
+//                (the MMA's B operand, 128-byte swizzled, in a ring of its own) and take A x from the same
+//                registers
 //   warps 4-11   two converter sets on alternate k-blocks: thread = TMEM lane; reads its 128 bytes of V,
 //                accumulates v^2, stores v_hi / v_lo to TMEM as the A operand
 //   warps 12-15  drain the accumulator sets into registers; at the end write the slab
+// A stage of the load ring is free again as soon as the converters and the splitters have read it into
+// registers; only the operand slots wait for the MMAs.  An operand slot is a TMEM buffer (A: the
+// candidates' entries) and a shared-memory buffer (B: the split rows of A) with ONE pair of barriers:
+// the issuing warp is the slowest link of the chain (cycle stamps: every barrier probe costs it 100 to
+// 500 cycles of shared-memory latency even when the phase has long completed), so it waits for one barrier
+// a k-block pair, probes the two pairs of a turn back to back, and commits once a pair.
 // Every mbarrier wait is bounded; a wait that gives up raises a status word and the block leaves through
 // the common teardown.
 #include "zeno_internal.h"
@@ -39,9 +49,9 @@ namespace {
 constexpr int kHalfRows = 64;               // candidates per half tile
 constexpr int kQBlockK = 32;                // floats per k-block = one 128-byte swizzle row
 constexpr int kVHalfBytes = kHalfRows * 128;
-constexpr int kQThreads = 32 * 16;
+constexpr int kQThreads = 32 * 20;
 constexpr int kQMaxStages = 8;
-constexpr int kQMaxABufs = 5;
+constexpr int kQMaxABufs = 5;               // operand slots
 constexpr int kQSmem = 217 * 1024;          // dynamic: the ring, reused for the result exchange at the end
 constexpr int kQTmemCols = 512;
 constexpr int kFlush = 32;                  // k-blocks accumulated in TMEM before a drain
@@ -49,22 +59,24 @@ constexpr int kFlush = 32;                  // k-blocks accumulated in TMEM befo
 struct LsqTcArgs {
     int m, n_r, n_pad;                      // n_pad: 16 or 32
     int nkb;                                // pairs of k-blocks in a block's k-range
-    int stages, n_abufs;
+    int stages, n_abufs;                    // stages of the load ring, operand slots
     int wide;                               // the tensor maps fetch both k-blocks of a pair in one copy (d % 32 == 0)
     float *part;                            // [blocks][m+1][n_r+1]
     int *status;
     uint32_t spin_limit;                    // polls a bounded wait may take
 };
 
-// bytes of a stage: V halves | [a_hi; a_lo] halves | raw A halves | x pieces (padded to 1 KB)
-__host__ __device__ inline int lsq_stage_bytes(int n_pad) { return 2 * kVHalfBytes + 2 * (2 * n_pad * 128) + 2 * (n_pad * 128) + 1024; }
+// bytes of a stage of the load ring: V halves | raw A halves | x pieces (padded to 1 KB)
+__host__ __device__ inline int lsq_stage_bytes(int n_pad) { return 2 * kVHalfBytes + 2 * (n_pad * 128) + 1024; }
+// bytes of a B operand: [a_hi; a_lo] of both halves
+__host__ __device__ inline int lsq_b_bytes(int n_pad) { return 2 * (2 * n_pad * 128); }
 
 __global__ void __launch_bounds__(kQThreads, 1)
 lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_a,
               const __grid_constant__ CUtensorMap map_x, LsqTcArgs a) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    // full, empty, bready [stages]; afull, aempty [A buffers]; dfull, dempty [2 sets]
-    constexpr int kBars = 3 * kQMaxStages + 2 * kQMaxABufs + 4;
+    // full, empty [stages]; ready, free [operand slots]; dfull, dempty [2 sets]
+    constexpr int kBars = 2 * kQMaxStages + 2 * kQMaxABufs + 4;
     __shared__ __align__(8) uint64_t bars[kBars];
     __shared__ __align__(8) uint64_t drain_bar;   // teardown after an abort: the issuer's last commit
     __shared__ __align__(8) uint64_t never_bar;   // nothing arrives here (test hook, see wait_for_nothing)
@@ -73,7 +85,7 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
     int &abort_flag = abort_state[0];
     __shared__ int issued[kQMaxStages];
     __shared__ float nrm_s[2][128];         // sums of squares per lane and converter set
-    __shared__ float z0_s[2][32];           // A x, per splitter warp
+    __shared__ float z0_s[4][32];           // A x, per splitter warp
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
@@ -81,39 +93,38 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
     if (tid == 64) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
 
     const int n_pad = a.n_pad, nkb = a.nkb, n_stages = a.stages, n_abufs = a.n_abufs;
-    const int b_bytes = 2 * n_pad * 128;                   // [a_hi; a_lo] of one half
     const int raw_bytes = n_pad * 128;
-    const int stage_bytes = lsq_stage_bytes(n_pad);
-    const int off_b = 2 * kVHalfBytes, off_raw = off_b + 2 * b_bytes, off_x = off_raw + 2 * raw_bytes;
+    const int stage_bytes = lsq_stage_bytes(n_pad), b_bytes = lsq_b_bytes(n_pad);
+    const int off_raw = 2 * kVHalfBytes, off_x = off_raw + 2 * raw_bytes;
     const int set_cols = 6 * n_pad;                        // D1 (4 n_pad) and D2 (2 n_pad), both halves side by side
     const int a_base = 2 * set_cols;
     const int n_flush = (nkb + kFlush - 1) / kFlush;
     const float inv_stages = 1.0f / (float)n_stages, inv_abufs = 1.0f / (float)n_abufs;
     uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t *bring = ring + (size_t)n_stages * stage_bytes;             // the B operands, 1 KB aligned like the stages
     // drained products per TMEM lane; written once the last accumulator set has been drained, when every
     // stage of the ring has been consumed
     float(*res)[33] = reinterpret_cast<float(*)[33]>(ring);
 
     auto bar_full = [&](int s) { return smem_u32(&bars[s]); };
     auto bar_empty = [&](int s) { return smem_u32(&bars[kQMaxStages + s]); };
-    auto bar_bready = [&](int s) { return smem_u32(&bars[2 * kQMaxStages + s]); };
-    auto bar_afull = [&](int g) { return smem_u32(&bars[3 * kQMaxStages + g]); };
-    auto bar_aempty = [&](int g) { return smem_u32(&bars[3 * kQMaxStages + kQMaxABufs + g]); };
-    auto bar_dfull = [&](int q) { return smem_u32(&bars[3 * kQMaxStages + 2 * kQMaxABufs + q]); };
-    auto bar_dempty = [&](int q) { return smem_u32(&bars[3 * kQMaxStages + 2 * kQMaxABufs + 2 + q]); };
+    constexpr int kBarA = 2 * kQMaxStages, kBarD = kBarA + 2 * kQMaxABufs;
+    auto bar_ready = [&](int g) { return smem_u32(&bars[kBarA + g]); };
+    auto bar_free = [&](int g) { return smem_u32(&bars[kBarA + kQMaxABufs + g]); };
+    auto bar_dfull = [&](int q) { return smem_u32(&bars[kBarD + q]); };
+    auto bar_dempty = [&](int q) { return smem_u32(&bars[kBarD + 2 + q]); };
 
     if (tid == 0) {
         abort_flag = 0;
         abort_state[1] = (int)a.spin_limit;
         for (int s = 0; s < kQMaxStages; ++s) {
             mbar_init(bar_full(s), 1);
-            mbar_init(bar_empty(s), 5);        // the four warps of a converter set and the MMAs' commit
-            mbar_init(bar_bready(s), 2);        // the two warps that split the rows of A
+            mbar_init(bar_empty(s), 6);        // the four warps of a converter set and the two that split the rows of A
             issued[s] = 0;
         }
         for (int g = 0; g < kQMaxABufs; ++g) {
-            mbar_init(bar_afull(g), 4);
-            mbar_init(bar_aempty(g), 1);
+            mbar_init(bar_ready(g), 6);        // a converter set's four warps and the two that split the rows of A
+            mbar_init(bar_free(g), 1);         // the MMAs' commit
         }
         for (int q = 0; q < 2; ++q) {
             mbar_init(bar_dfull(q), 1);
@@ -136,12 +147,12 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
     const uint32_t tmem = tmem_base_slot;
     volatile int *abortp = &abort_flag;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
-        wait_for_nothing(smem_u32(&never_bar), abortp);
-        int s = 0;
-        uint32_t round = 0;
-        for (int kb = 0; kb < nkb; ++kb) {
+    if (warp == 0 || warp == 16) {
+        // ------------------------------------------------------------------ TMA producers
+        if (warp == 0) wait_for_nothing(smem_u32(&never_bar), abortp);
+        for (int kb = warp == 0 ? 0 : 1; kb < nkb; kb += 2) {
+            const uint32_t round = small_div((uint32_t)kb, inv_stages);
+            const int s = kb - (int)round * n_stages;
             if (!__all_sync(0xffffffffu, mbar_wait(bar_empty(s), (round & 1) ^ 1, abortp))) break;
             if (elect_one()) {
                 const uint32_t dst = smem_u32(ring + (size_t)s * stage_bytes);
@@ -155,7 +166,9 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
                 // was what the ring waited for (cycle stamps: stages re-armed 1,400-2,200 cycles after they were
                 // free).  When d and ldv are multiples of 32 the maps see V and A as [row][k-block][32] and one box
                 // takes both k-blocks of the pair (a row's two 128-byte pieces then lie side by side in the stage),
-                // x comes as one 256-byte piece: three copies per stage.
+                // x comes as one 256-byte piece: three copies per stage.  (A map ordered [k-block][row][32] gives
+                // the stage layout of two separate boxes with one copy, but it fetches every row in two 128-byte
+                // visits and the kernel ran 7 % slower.)
                 const int n_loads = a.wide ? 3 : 6;
 #pragma unroll 1
                 for (int w = 0; w < n_loads; ++w) {    // V, A, x (of the two halves): ONE issue site
@@ -168,21 +181,17 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
                 }
             }
             __syncwarp();
-            if (++s == n_stages) {
-                s = 0;
-                ++round;
-            }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         const uint32_t idesc_base = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(128 >> 4) << 24);
         const uint32_t idesc_2n = idesc_base | ((uint32_t)((2 * n_pad) >> 3) << 17);
         const uint32_t idesc_4n = idesc_base | ((uint32_t)((4 * n_pad) >> 3) << 17);
-        int rs = 0, ag = 0;                              // ring stage and A buffer of the next k-block pair
-        uint32_t rph = 0, aph = 0;                       // and the phases their barriers are awaited in
-        // Two stages per turn of the loop (the operands are in place well ahead of this warp, and its
+        int ag = 0;                                      // operand slot of the next k-block pair
+        uint32_t aph = 0;                                // and the phase its barrier is awaited in
+        // Two k-block pairs per turn of the loop (the operands are in place well ahead of this warp, and its
         // waits, vote, fence and election cost as much as the MMAs it issues).  kFlush is even, so the two
-        // stages of a turn always add into the same accumulator set.
+        // pairs of a turn always add into the same accumulator set.
         for (int kb = 0; kb < nkb; kb += 2) {
             const bool two = kb + 1 < nkb;
             const int fl = kb / kFlush, in_fl = kb - fl * kFlush;
@@ -191,14 +200,15 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
                 if (!__all_sync(0xffffffffu, mbar_wait(bar_dempty(set), (((uint32_t)fl >> 1) & 1) ^ 1, abortp))) break;
                 tc_fence_after();
             }
-            int s1 = rs + 1, g1 = ag + 1;
-            uint32_t rph1 = rph, aph1 = aph;
-            if (s1 == n_stages) { s1 = 0; rph1 ^= 1; }
+            int g1 = ag + 1;
+            uint32_t aph1 = aph;
             if (g1 == n_abufs) { g1 = 0; aph1 ^= 1; }
-            if (!__all_sync(0xffffffffu, mbar_wait(bar_bready(rs), rph, abortp) && mbar_wait(bar_afull(ag), aph, abortp) &&
-                                             (!two || (mbar_wait(bar_bready(s1), rph1, abortp) &&
-                                                       mbar_wait(bar_afull(g1), aph1, abortp)))))
-                break;
+            // both probes are issued before either result is looked at
+            bool r0 = mbar_try_wait(bar_ready(ag), aph);
+            bool r1 = !two || mbar_try_wait(bar_ready(g1), aph1);
+            if (!r0) r0 = mbar_wait_poll(bar_ready(ag), aph, abortp);
+            if (!r1) r1 = mbar_wait_poll(bar_ready(g1), aph1, abortp);
+            if (!__all_sync(0xffffffffu, r0 && r1)) break;
             tc_fence_after();
             if (elect_one()) {
                 // D1 = v_hi [a_hi(even); a_hi(odd); a_lo(even); a_lo(odd)]^T, D2 = v_lo [a_hi(even); a_hi(odd)]^T:
@@ -207,9 +217,9 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
 #pragma unroll
                 for (int q = 0; q < 2; ++q) {
                     if (q == 1 && !two) break;
-                    const int s = q ? s1 : rs, g = q ? g1 : ag;
+                    const int g = q ? g1 : ag;
                     const uint32_t a_tmem = tmem + a_base + g * 64;
-                    const uint32_t bx = smem_u32(ring + (size_t)s * stage_bytes + off_b);
+                    const uint32_t bx = smem_u32(bring + (size_t)g * b_bytes);
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {
                         const uint64_t db = smem_desc_sw128(bx + ks * 32);
@@ -217,34 +227,32 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
                         tc_mma_tf32_ts(d1, a_tmem + ks * 8, db, idesc_4n, acc);
                         tc_mma_tf32_ts(d2, a_tmem + 32 + ks * 8, db, idesc_2n, acc);
                     }
-                    tc_commit(bar_aempty(g));
-                    tc_commit(bar_empty(s));
+                    tc_commit(bar_free(g));
                 }
                 const int last = two ? kb + 1 : kb;
                 if (last - fl * kFlush == kFlush - 1 || last + 1 == nkb) tc_commit(bar_dfull(set));
             }
             __syncwarp();
-            rs = two ? s1 + 1 : s1;
-            rph = rph1;
-            if (two && rs == n_stages) { rs = 0; rph ^= 1; }
             ag = two ? g1 + 1 : g1;
             aph = aph1;
             if (two && ag == n_abufs) { ag = 0; aph ^= 1; }
         }
-    } else if (warp == 2 || warp == 3) {
+    } else if (warp == 2 || warp == 3 || warp == 18 || warp == 19) {
         // ------------------------------------------------------------------ rows of A: split for the MMA, and A x
         // Warp 2 takes the even k-block's rows of every stage, warp 3 the odd one's.  All of a lane's rows
-        // are loaded before the first store: the stores go to the same shared array, so loads placed after
-        // them would wait for them, and the stage would reach the MMAs ~1,000 cycles later (cycle stamps).
-        const int h = warp - 2;
+        // are loaded before the first store (loads placed after stores to the same shared array would wait
+        // for them), and the stage is released as soon as they are in registers.
+        const int sset = warp >= 18 ? 1 : 0;          // set 0 takes the even stages, set 1 the odd
+        const int h = warp & 1;
         float accx[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};    // rows 4 u + lane / 8 (u < n_pad / 4)
         bool ok = true;
-        for (int kb = 0; kb < nkb && ok; ++kb) {
-            const uint32_t sround = small_div((uint32_t)kb, inv_stages);
-            const int s = kb - (int)sround * n_stages;
+        for (int kb = sset; kb < nkb && ok; kb += 2) {
+            const uint32_t sround = small_div((uint32_t)kb, inv_stages), bround = small_div((uint32_t)kb, inv_abufs);
+            const int s = kb - (int)sround * n_stages, gb = kb - (int)bround * n_abufs;
             ok = mbar_wait(bar_full(s), sround & 1, abortp);
             if (!ok) break;
-            uint8_t *st = ring + (size_t)s * stage_bytes;
+            const uint8_t *st = ring + (size_t)s * stage_bytes;
+            uint8_t *bop = bring + (size_t)gb * b_bytes;
             const float4 x4 = *reinterpret_cast<const float4 *>(st + off_x + h * 128 + (lane & 7) * 16);
             float4 v[8];
 #pragma unroll
@@ -254,6 +262,11 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
                 const int piece = a.wide ? 2 * j + h : h * n_pad + j;        // where row j of this warp's k-block landed
                 if (4 * u < n_pad) v[u] = *reinterpret_cast<const float4 *>(st + off_raw + piece * 128 + ((c ^ (piece & 7)) << 4));
             }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_empty(s));
+            ok = mbar_wait(bar_free(gb), (bround & 1) ^ 1, abortp);        // the MMAs that read this operand last are done
+            if (!ok) break;
+            tc_fence_after();
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
                 if (4 * u >= n_pad) break;
@@ -263,13 +276,13 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
                 const float4 hi = make_float4(tf32_hi(v[u].x), tf32_hi(v[u].y), tf32_hi(v[u].z), tf32_hi(v[u].w));
                 // B operand rows: a_hi of the even k-block, a_hi of the odd one, then the two a_lo blocks
                 // (n_pad % 8 == 0: every block starts in the same swizzle phase)
-                *reinterpret_cast<float4 *>(st + off_b + h * n_pad * 128 + sw) = hi;
-                *reinterpret_cast<float4 *>(st + off_b + (2 + h) * n_pad * 128 + sw) =
+                *reinterpret_cast<float4 *>(bop + h * n_pad * 128 + sw) = hi;
+                *reinterpret_cast<float4 *>(bop + (2 + h) * n_pad * 128 + sw) =
                     make_float4(v[u].x - hi.x, v[u].y - hi.y, v[u].z - hi.z, v[u].w - hi.w);
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> tensor-core reads
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_bready(s));
+            if (lane == 0) mbar_arrive(bar_ready(gb));
         }
         // A x: the eight lanes of a row add up
 #pragma unroll
@@ -278,7 +291,7 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
             t += __shfl_xor_sync(0xffffffffu, t, 1);
             t += __shfl_xor_sync(0xffffffffu, t, 2);
             t += __shfl_xor_sync(0xffffffffu, t, 4);
-            if ((lane & 7) == 0 && 4 * u + (lane >> 3) < 32) z0_s[warp - 2][4 * u + (lane >> 3)] = t;
+            if ((lane & 7) == 0 && 4 * u + (lane >> 3) < 32) z0_s[2 * sset + h][4 * u + (lane >> 3)] = t;
         }
     } else if (warp >= 4 && warp < 12) {
         // ------------------------------------------------------------------ converters
@@ -292,15 +305,28 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
             const uint32_t sround = small_div(it, inv_stages), around = small_div(it, inv_abufs);
             const int s = (int)(it - sround * n_stages), g = (int)(it - around * n_abufs);
             if (!mbar_wait(bar_full(s), sround & 1, abortp)) break;
-            // this lane's 128 bytes: box h, row r (two boxes one after the other), or row r, piece h (one box)
+            // this lane's 128 bytes: box h, row r (two boxes one after the other), or row r, piece h (one box).
+            // In the second layout the pieces of a quarter warp's eight lanes are two apart and their swizzle
+            // phases take only four values: every other group of four lanes reads its 16-byte chunks in the
+            // order 1, 0, 3, 2, .. (and swaps them back in registers), so that the eight lanes of a
+            // shared-memory access fall into eight different bank groups.
             const int piece = a.wide ? (((row & 63) << 1) | (row >> 6)) : row;
+            const int flip = a.wide ? ((row >> 2) & 1) : 0;
             const uint8_t *src = ring + (size_t)s * stage_bytes + piece * 128;
             float4 v[8];
             uint32_t hi[32], lo[32];
 #pragma unroll
-            for (int c = 0; c < 8; ++c) v[c] = *reinterpret_cast<const float4 *>(src + ((c ^ (piece & 7)) << 4));
+            for (int c = 0; c < 8; ++c) v[c] = *reinterpret_cast<const float4 *>(src + ((c ^ flip ^ (piece & 7)) << 4));
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_empty(s));
+            if (flip) {
+#pragma unroll
+                for (int c = 0; c < 8; c += 2) {
+                    const float4 t = v[c];
+                    v[c] = v[c + 1];
+                    v[c + 1] = t;
+                }
+            }
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
                 const float e[4] = {v[c].x, v[c].y, v[c].z, v[c].w};
@@ -312,17 +338,17 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
                     lo[4 * c + u] = __float_as_uint(e[u] - h);
                 }
             }
-            if (!mbar_wait(bar_aempty(g), (around & 1) ^ 1, abortp)) break;
+            if (!mbar_wait(bar_free(g), (around & 1) ^ 1, abortp)) break;
             tc_fence_after();
             tc_st32(a_bufs + g * 64, hi);
             tc_st32(a_bufs + g * 64 + 32, lo);
             tc_wait_st();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_afull(g));
+            if (lane == 0) mbar_arrive(bar_ready(g));
         }
         nrm_s[cset][row] = (nrm4[0] + nrm4[1]) + (nrm4[2] + nrm4[3]);
-    } else if (warp >= 12) {
+    } else if (warp >= 12 && warp < 16) {
         // ------------------------------------------------------------------ drains
         const int quad = warp & 3;
         const int row = quad * 32 + lane;
@@ -378,7 +404,7 @@ lsq_tc_kernel(const __grid_constant__ CUtensorMap map_v, const __grid_constant__
         const int r = t / stride, j = t - r * stride;
         float v;
         if (r == 0) {
-            v = j < a.n_r ? z0_s[0][j] + z0_s[1][j] : 0.f;
+            v = j < a.n_r ? (z0_s[0][j] + z0_s[1][j]) + (z0_s[2][j] + z0_s[3][j]) : 0.f;
         } else {
             const int c = r - 1;
             v = j < a.n_r ? res[c][j] + res[c + kHalfRows][j]
@@ -479,11 +505,11 @@ cudaError_t launch_lsq_tc(Context &c, const LsqArgs &a, int max_slabs, int *slab
     t.n_pad = n_pad;
     t.wide = wide ? 1 : 0;
     t.nkb = (int)((n_kblocks + 2 * (int64_t)blocks - 1) / (2 * (int64_t)blocks));
-    const int stage_bytes = lsq_stage_bytes(n_pad);
-    t.stages = (kQSmem - 1024) / stage_bytes;
-    if (t.stages > kQMaxStages) t.stages = kQMaxStages;
+    const int stage_bytes = lsq_stage_bytes(n_pad), b_bytes = lsq_b_bytes(n_pad);
     t.n_abufs = (kQTmemCols - 2 * 6 * n_pad) / 64;
     if (t.n_abufs > kQMaxABufs) t.n_abufs = kQMaxABufs;
+    t.stages = (kQSmem - 1024 - t.n_abufs * b_bytes) / stage_bytes;
+    if (t.stages > kQMaxStages) t.stages = kQMaxStages;
     t.part = a.part;
     t.status = c.dev_status;
     t.spin_limit = c.spin_limit;
@@ -494,7 +520,7 @@ cudaError_t launch_lsq_tc(Context &c, const LsqArgs &a, int max_slabs, int *slab
         attr_set.mark(c.device);
     }
     *slabs = blocks;
-    return launch_chained(lsq_tc_kernel, dim3(blocks), dim3(kQThreads), (size_t)t.stages * stage_bytes + 1024, s,
+    return launch_chained(lsq_tc_kernel, dim3(blocks), dim3(kQThreads), (size_t)t.stages * stage_bytes + (size_t)t.n_abufs * b_bytes + 1024, s,
                           chain_launches(c), map_v, map_a, map_x, t);
 }
 

@@ -28,6 +28,19 @@
  * Parameter-vector layout (the one both sides agree on): x and every row of
  * V are the flat concatenation, layer by layer, of W_l stored [out_l x in_l]
  * row-major followed by b_l[out_l] (if has_bias).  Least squares: just x[d].
+ *
+ * Convolutional network (kind 2; the paper's experiments train "a CNN with 4 convolutional layers
+ * followed by 1 fully connected layer" whose exact shape it does not print, so this one is this
+ * project's own and is stated here in full):
+ *   dims = {S, C_0, C_1, .., C_Lc, classes}, n_layers = Lc + 1 (Lc convolutional layers, Lc even, and the
+ *   dense layer); the input is C_0 planes of S x S values, [C_0][S][S] row-major.
+ *   Convolutional layer l (1-based): 3 x 3 windows, stride 1, zero padding 1, as a cross-correlation
+ *     out[co][y][x] = b[co] + sum_ci sum_dy sum_dx W[co][ci][dy][dx] in[ci][y + dy - 1][x + dx - 1],
+ *   followed by ReLU; after every second convolutional layer a 2 x 2 max pooling with stride 2 (a NaN in
+ *   the window gives NaN).  The dense layer takes the last planes flattened [C][y][x] to `classes`
+ *   logits; the loss is the softmax cross-entropy, as for kind 0.
+ *   Parameters: per convolutional layer W[C_l][C_{l-1}][3][3] then b[C_l]; then the dense layer's
+ *   W[classes][C_Lc (S / 2^(Lc/2))^2] and b[classes].
  */
 #include <math.h>
 #include <stdint.h>
@@ -37,7 +50,7 @@
 #include <omp.h>
 #endif
 
-enum { ZO_LOSS_SOFTMAX_MLP = 0, ZO_LOSS_LEAST_SQUARES = 1 };
+enum { ZO_LOSS_SOFTMAX_MLP = 0, ZO_LOSS_LEAST_SQUARES = 1, ZO_LOSS_SOFTMAX_CNN = 2 };
 enum { ZO_F32 = 0, ZO_BF16 = 1 };
 enum { ZO_OK = 0, ZO_BAD_ARG = 1, ZO_NO_MEM = 2 };
 
@@ -118,10 +131,37 @@ void zo_candidate_params(const void *x, const void *v, int64_t d, int dtype,
     }
 }
 
+/* side of the planes after all pooling steps, or 0 if the description is not a valid network */
+static int64_t zo_cnn_final_side(int n_layers, const int64_t *dims)
+{
+    int lc = n_layers - 1;
+    if (lc < 2 || (lc & 1))
+        return 0;
+    int64_t side = dims[0];
+    for (int l = 2; l <= lc; l += 2) {
+        if (side < 2 || (side & 1))
+            return 0;
+        side /= 2;
+    }
+    return side;
+}
+
 int64_t zo_param_count(int kind, int n_layers, const int64_t *dims, int has_bias)
 {
     if (kind == ZO_LOSS_LEAST_SQUARES)
         return dims[0];
+    if (kind == ZO_LOSS_SOFTMAX_CNN) {
+        int lc = n_layers - 1;
+        int64_t side = zo_cnn_final_side(n_layers, dims);
+        if (side == 0)
+            return 0;
+        int64_t d = 0;
+        for (int l = 1; l <= lc; ++l)
+            d += dims[l + 1] * dims[l] * 9 + (has_bias ? dims[l + 1] : 0);
+        int64_t classes = dims[lc + 2];
+        d += classes * dims[lc + 1] * side * side + (has_bias ? classes : 0);
+        return d;
+    }
     int64_t d = 0;
     for (int l = 0; l < n_layers; ++l)
         d += dims[l + 1] * dims[l] + (has_bias ? dims[l + 1] : 0);
@@ -168,8 +208,116 @@ static double zo_mlp_sample_loss(const double *w, int n_layers, const int64_t *d
     return zmax + log(se) - h[label];
 }
 
+/* the larger of two values; a NaN wins */
+static double zo_max_nan(double a, double b)
+{
+    if (a != a) return a;
+    if (b != b) return b;
+    return a > b ? a : b;
+}
+
+/* Softmax cross-entropy of the convolutional network described at the top of this file, one sample.
+ * feat: [C_0][S][S].  buf0, buf1: two buffers of the largest number of values any layer holds.
+ * logits_out (optional): the dense layer's outputs. */
+static double zo_cnn_sample_loss(const double *w, int n_layers, const int64_t *dims, int has_bias,
+                                 const float *feat, int32_t label, double *buf0, double *buf1,
+                                 double *logits_out)
+{
+    int lc = n_layers - 1;
+    int64_t side = dims[0];
+    double *h = buf0, *z = buf1;
+    for (int64_t k = 0; k < dims[1] * side * side; ++k)
+        h[k] = (double)feat[k];
+    const double *p = w;
+    for (int l = 1; l <= lc; ++l) {
+        int64_t cin = dims[l], cout = dims[l + 1];
+        const double *W = p;
+        const double *bias = has_bias ? p + cout * cin * 9 : NULL;
+        for (int64_t co = 0; co < cout; ++co)
+            for (int64_t y = 0; y < side; ++y)
+                for (int64_t x = 0; x < side; ++x) {
+                    double acc = bias ? bias[co] : 0.0;
+                    for (int64_t ci = 0; ci < cin; ++ci)
+                        for (int dy = 0; dy < 3; ++dy)
+                            for (int dx = 0; dx < 3; ++dx) {
+                                int64_t yy = y + dy - 1, xx = x + dx - 1;
+                                if (yy < 0 || yy >= side || xx < 0 || xx >= side)
+                                    continue; /* zero padding */
+                                acc += W[((co * cin + ci) * 3 + dy) * 3 + dx] * h[(ci * side + yy) * side + xx];
+                            }
+                    if (!(acc > 0.0))
+                        acc = (acc == acc) ? 0.0 : acc; /* ReLU; a NaN stays a NaN */
+                    z[(co * side + y) * side + x] = acc;
+                }
+        p += cout * cin * 9 + (has_bias ? cout : 0);
+        double *t = h; h = z; z = t;
+        if ((l & 1) == 0) { /* 2 x 2 max pooling, stride 2 */
+            int64_t half = side / 2;
+            for (int64_t c = 0; c < cout; ++c)
+                for (int64_t y = 0; y < half; ++y)
+                    for (int64_t x = 0; x < half; ++x) {
+                        const double *q = h + (c * side + 2 * y) * side + 2 * x;
+                        z[(c * half + y) * half + x] =
+                            zo_max_nan(zo_max_nan(q[0], q[1]), zo_max_nan(q[side], q[side + 1]));
+                    }
+            side = half;
+            t = h; h = z; z = t;
+        }
+    }
+    int64_t flat = dims[lc + 1] * side * side, C = dims[lc + 2];
+    const double *W = p;
+    const double *bias = has_bias ? p + C * flat : NULL;
+    for (int64_t c = 0; c < C; ++c) {
+        double acc = 0.0;
+        for (int64_t k = 0; k < flat; ++k)
+            acc += W[c * flat + k] * h[k];
+        if (bias)
+            acc += bias[c];
+        z[c] = acc;
+        if (logits_out)
+            logits_out[c] = acc;
+    }
+    double zmax = z[0];
+    for (int64_t c = 1; c < C; ++c)
+        if (z[c] > zmax) zmax = z[c];
+    double se = 0.0;
+    for (int64_t c = 0; c < C; ++c)
+        se += exp(z[c] - zmax);
+    return zmax + log(se) - z[label];
+}
+
+/* largest number of values a layer of the network holds (the input, any layer's planes, the logits) */
+static int64_t zo_cnn_widest(int n_layers, const int64_t *dims)
+{
+    int lc = n_layers - 1;
+    int64_t side = dims[0], widest = dims[1] * side * side;
+    for (int l = 1; l <= lc; ++l) {
+        if (dims[l + 1] * side * side > widest) widest = dims[l + 1] * side * side;
+        if ((l & 1) == 0) side /= 2;
+    }
+    if (dims[lc + 2] > widest) widest = dims[lc + 2];
+    return widest;
+}
+
+/* The network's logits for one sample (for the pins: the layers' arithmetic seen without the loss). */
+int zo_cnn_logits(int n_layers, const int64_t *dims, int has_bias, const double *w, const float *feat,
+                  double *logits)
+{
+    if (zo_cnn_final_side(n_layers, dims) == 0)
+        return ZO_BAD_ARG;
+    int64_t widest = zo_cnn_widest(n_layers, dims);
+    double *buf0 = (double *)malloc(sizeof(double) * (size_t)widest);
+    double *buf1 = (double *)malloc(sizeof(double) * (size_t)widest);
+    if (!buf0 || !buf1) { free(buf0); free(buf1); return ZO_NO_MEM; }
+    (void)zo_cnn_sample_loss(w, n_layers, dims, has_bias, feat, 0, buf0, buf1, logits);
+    free(buf0);
+    free(buf1);
+    return ZO_OK;
+}
+
 /* f_r(w) = (1/n_r) sum_j f(w; z_j)   (Definition 2).
  * kind 0: targets = int32 labels[n_r]; features [n_r x dims[0]] float32.
+ * kind 2: targets = int32 labels[n_r]; features [n_r x C_0 x S x S] float32 (see the top of the file).
  * kind 1: f(w; (a_j, y_j)) = (a_j . w - y_j)^2 / 2, features = A [n_r x d],
  *         targets = float32 y[n_r], so that f_r = ||A w - y||^2 / (2 n_r). */
 double zo_loss(int kind, int n_layers, const int64_t *dims, int has_bias,
@@ -186,6 +334,20 @@ double zo_loss(int kind, int n_layers, const int64_t *dims, int has_bias,
             double r = acc - (double)y[j];
             total += 0.5 * r * r;
         }
+    } else if (kind == ZO_LOSS_SOFTMAX_CNN) {
+        if (zo_cnn_final_side(n_layers, dims) == 0)
+            return NAN;
+        int64_t widest = zo_cnn_widest(n_layers, dims);
+        int64_t in_elems = dims[1] * dims[0] * dims[0];
+        double *buf0 = (double *)malloc(sizeof(double) * (size_t)widest);
+        double *buf1 = (double *)malloc(sizeof(double) * (size_t)widest);
+        if (!buf0 || !buf1) { free(buf0); free(buf1); return NAN; }
+        const int32_t *labels = (const int32_t *)targets;
+        for (int j = 0; j < n_r; ++j)
+            total += zo_cnn_sample_loss(w, n_layers, dims, has_bias, features + (int64_t)j * in_elems,
+                                        labels[j], buf0, buf1, NULL);
+        free(buf0);
+        free(buf1);
     } else {
         int64_t widest = 0;
         for (int l = 0; l <= n_layers; ++l)
@@ -454,6 +616,8 @@ int zo_krum(int dtype, const void *V, int64_t ldv, int64_t d, int m, int b,
 int zo_worker_gradient(int kind, int n_layers, const int64_t *dims, int has_bias, const void *x, int dtype,
                        const float *features, const void *targets, int n, int flip, double *grad)
 {
+    if (kind == ZO_LOSS_SOFTMAX_CNN)
+        return ZO_BAD_ARG; /* the workers' side is stated for the dense models and least squares only */
     if (n < 1) return ZO_BAD_ARG;
     if (kind == ZO_LOSS_LEAST_SQUARES) {
         const int64_t d = dims[0];

@@ -23,6 +23,7 @@ _LIB = os.path.join(_HERE, "libzeno_oracle.so")
 
 LOSS_SOFTMAX_MLP = 0
 LOSS_LEAST_SQUARES = 1
+LOSS_SOFTMAX_CNN = 2      # dims = [S, C_0, C_1, .., C_Lc, classes]: Lc convolutional layers and a dense one
 F32 = 0
 BF16 = 1
 
@@ -73,6 +74,8 @@ def _load():
         lib.zo_median.argtypes = [i32, vp, i64, i64, i32, vp]
         lib.zo_krum.restype = i32
         lib.zo_krum.argtypes = [i32, vp, i64, i64, i32, i32, vp, vp, vp]
+        lib.zo_cnn_logits.restype = i32
+        lib.zo_cnn_logits.argtypes = [i32, vp, i32, vp, vp, vp]
         lib.zo_eval_count.restype = ctypes.c_longlong
         lib.zo_reset_eval_count.restype = None
         lib.zo_num_threads.restype = i32
@@ -86,6 +89,12 @@ def _ptr(a):
 
 def _dims(dims):
     return np.ascontiguousarray(np.asarray(dims, dtype=np.int64))
+
+
+def _n_layers(kind, dm):
+    """Layers a dims list describes: its widths minus one, or (convolutional network) minus two,
+    since that list starts with the image side."""
+    return len(dm) - 2 if kind == LOSS_SOFTMAX_CNN else len(dm) - 1
 
 
 def _params(a, dtype):
@@ -130,7 +139,7 @@ def reset_eval_count() -> None:
 
 def param_count(kind, dims, has_bias=True) -> int:
     dm = _dims(dims)
-    return int(_load().zo_param_count(kind, len(dm) - 1, _ptr(dm), int(has_bias)))
+    return int(_load().zo_param_count(kind, _n_layers(kind, dm), _ptr(dm), int(has_bias)))
 
 
 def round_to_bf16(f: float) -> float:
@@ -155,8 +164,19 @@ def loss(kind, dims, has_bias, w, features, targets):
     features = _features(features)
     targets = _targets(kind, targets)
     n_r = targets.shape[0]
-    return float(_load().zo_loss(kind, len(dm) - 1, _ptr(dm), int(has_bias), _ptr(w),
+    return float(_load().zo_loss(kind, _n_layers(kind, dm), _ptr(dm), int(has_bias), _ptr(w),
                                  _ptr(features), _ptr(targets), n_r))
+
+
+def cnn_logits(dims, has_bias, w, feat):
+    """The convolutional network's logits for one sample (float64 [classes])."""
+    dm = _dims(dims)
+    w = np.ascontiguousarray(w, dtype=np.float64)
+    feat = _features(feat)
+    out = np.empty(int(dm[-1]), dtype=np.float64)
+    _check(_load().zo_cnn_logits(len(dm) - 2, _ptr(dm), int(has_bias), _ptr(w), _ptr(feat), _ptr(out)),
+           "zo_cnn_logits")
+    return out
 
 
 def score(kind, dtype, dims, has_bias, x, V, ldv, m, features, targets, gamma, rho):
@@ -170,7 +190,7 @@ def score(kind, dtype, dims, has_bias, x, V, ldv, m, features, targets, gamma, r
     s = np.empty(m, dtype=np.float64)
     f = np.empty(m + 1, dtype=np.float64)
     n = np.empty(m, dtype=np.float64)
-    rc = _load().zo_score(kind, dtype, len(dm) - 1, _ptr(dm), int(has_bias), _ptr(x), _ptr(V),
+    rc = _load().zo_score(kind, dtype, _n_layers(kind, dm), _ptr(dm), int(has_bias), _ptr(x), _ptr(V),
                           int(ldv), int(m), _ptr(features), _ptr(targets), n_r,
                           float(gamma), float(rho), _ptr(s), _ptr(f), _ptr(n))
     _check(rc, "zo_score")
@@ -262,7 +282,7 @@ def step(kind, dtype, dims, has_bias, x, V, ldv, m, features, targets, gamma, rh
     out = np.empty(d, dtype=np.float64)
     s = np.empty(m, dtype=np.float64)
     idx = np.empty(m - b, dtype=np.int32)
-    rc = _load().zo_step(kind, dtype, len(dm) - 1, _ptr(dm), int(has_bias), _ptr(x), _ptr(V),
+    rc = _load().zo_step(kind, dtype, _n_layers(kind, dm), _ptr(dm), int(has_bias), _ptr(x), _ptr(V),
                          int(ldv), int(m), _ptr(features), _ptr(targets), n_r,
                          float(gamma), float(rho), int(b), _ptr(out), _ptr(s), _ptr(idx))
     _check(rc, "zo_step")

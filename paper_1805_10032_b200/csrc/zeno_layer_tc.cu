@@ -373,9 +373,15 @@ layer_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
                 uint32_t sph1 = bph, gph1 = aph;
                 if (s1 == n_bstages) { s1 = 0; sph1 ^= 1; }
                 if (g1 == n_abufs) { g1 = 0; gph1 ^= 1; }
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_bfull(bs), bph, abortp) && mbar_wait(bar_afull(ag), aph, abortp) &&
-                                                 (!two || (mbar_wait(bar_bfull(s1), sph1, abortp) &&
-                                                           mbar_wait(bar_afull(g1), gph1, abortp))));
+                // all probes are issued before any result is looked at: each costs this warp a round trip to
+                // shared memory, and one after the other they took longer than issuing the MMAs
+                bool r0 = mbar_try_wait(bar_bfull(bs), bph), r1 = mbar_try_wait(bar_afull(ag), aph);
+                bool r2 = !two || mbar_try_wait(bar_bfull(s1), sph1), r3 = !two || mbar_try_wait(bar_afull(g1), gph1);
+                if (!r0) r0 = mbar_wait_poll(bar_bfull(bs), bph, abortp);
+                if (!r1) r1 = mbar_wait_poll(bar_afull(ag), aph, abortp);
+                if (!r2) r2 = mbar_wait_poll(bar_bfull(s1), sph1, abortp);
+                if (!r3) r3 = mbar_wait_poll(bar_afull(g1), gph1, abortp);
+                ok = __all_sync(0xffffffffu, r0 && r1 && r2 && r3);
                 if (!ok) break;
                 tc_fence_after();
                 if (elect_one()) {

@@ -205,9 +205,9 @@ def test_score_uses_the_cnn_loss_per_candidate(oracle):
     f0 = oracle.loss(CNN, dims, True, x.astype(np.float64), feats, labels)
     assert f[0] == f0
     for i in range(m):
-        wi = x.astype(np.float64) - np.float64(np.float32(gamma)) * V[i, :d].astype(np.float64)
+        wi = x.astype(np.float64) - gamma * V[i, :d].astype(np.float64)
         fi = oracle.loss(CNN, dims, True, wi, feats, labels)
         ni = float(np.sum(V[i, :d].astype(np.float64) ** 2))
         assert f[1 + i] == pytest.approx(fi, rel=1e-14)
         assert n[i] == pytest.approx(ni, rel=1e-14)
-        assert s[i] == pytest.approx(f0 - fi - np.float64(np.float32(rho)) * ni, rel=1e-12, abs=1e-15)
+        assert s[i] == pytest.approx(f0 - fi - rho * ni, rel=1e-12, abs=1e-15)

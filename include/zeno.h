@@ -63,7 +63,17 @@ typedef enum {
      * trains and reports (Experiments, evaluation metrics). */
     ZENO_LOSS_SOFTMAX_MLP = 0,
     /* f(x; (a, y)) = (a.x - y)^2 / 2, so that f_r(x) = ||A x - y||^2 / (2 n_r). */
-    ZENO_LOSS_LEAST_SQUARES = 1
+    ZENO_LOSS_LEAST_SQUARES = 1,
+    /* f(x; (a, y)) = -log softmax(CNN_x(a))[y] for a small convolutional network.  The paper's experiments
+     * train "a CNN with 4 convolutional layers followed by 1 fully connected layer" (Experiments, datasets and
+     * evaluation metrics) and do not print its shape; the network here is this library's own:
+     *   Lc convolutional layers (Lc even): 3 x 3 windows, stride 1, zero padding 1, as a cross-correlation
+     *     out[co][y][x] = b[co] + sum_ci sum_dy sum_dx W[co][ci][dy][dx] in[ci][y + dy - 1][x + dx - 1],
+     *   each followed by ReLU, every second one also by a 2 x 2 max pooling with stride 2 (a NaN in the window
+     *   gives NaN); then one dense layer from the last planes, flattened [C][y][x], to the classes' logits.
+     * Parameter vector: per convolutional layer W[C_l][C_{l-1}][3][3] then b[C_l]; then the dense layer's
+     * W[classes][C_Lc * side * side] and b[classes] (side = S / 2^(Lc/2)). */
+    ZENO_LOSS_SOFTMAX_CNN = 2
 } zeno_loss_kind;
 
 typedef enum {
@@ -76,15 +86,19 @@ typedef enum {
 typedef struct {
     int32_t kind;        /* zeno_loss_kind */
     int32_t param_dtype; /* zeno_dtype */
-    int32_t n_layers;    /* L; least squares: 1 */
-    int32_t has_bias;    /* MLP only */
-    int64_t dims[ZENO_MAX_LAYERS + 1]; /* MLP: widths, e.g. {3072,512,512,10}; least squares: {d, 1} */
+    int32_t n_layers;    /* L; least squares: 1; convolutional network: Lc + 1 (its dense layer counts) */
+    int32_t has_bias;    /* MLP and convolutional network */
+    int64_t dims[ZENO_MAX_LAYERS + 1]; /* MLP: widths, e.g. {3072,512,512,10}; least squares: {d, 1};
+                                          convolutional network: {S, C_0, C_1, .., C_Lc, classes}, e.g.
+                                          {32,3,32,32,64,64,10}: S x S images of C_0 planes (S even, at most 32,
+                                          and still even before each pooling), n_layers + 2 entries */
 } zeno_model_desc;
 
 /* The server's batch z_1..z_{n_r} (Definition 2), drawn by the caller after the
  * candidates arrive (Algorithm 1). */
 typedef struct {
-    const float *features; /* device, [n_r x dims[0]] row-major binary32 (least squares: A [n_r x d]) */
+    const float *features; /* device, [n_r x dims[0]] row-major binary32 (least squares: A [n_r x d];
+                              convolutional network: [n_r][C_0][S][S]) */
     const void *targets;   /* device, int32 labels[n_r] in [0, dims[L]) (MLP) or float y[n_r] (least squares) */
     int32_t n_r;
 } zeno_batch;

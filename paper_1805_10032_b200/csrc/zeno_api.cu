@@ -21,14 +21,36 @@ size_t round_up(size_t n, size_t q) { return (n + q - 1) / q * q; }
 
 size_t elem_size(int dtype) { return dtype == ZENO_BF16 ? 2 : 4; }
 
+// Convolutional network: dims = {S, C_0, C_1, .., C_Lc, classes}, n_layers = Lc + 1.  The side of the planes
+// the dense layer sees, or 0 if the description is not a network the kernels take.
+int64_t cnn_final_side(const zeno_model_desc *d) {
+    const int lc = d->n_layers - 1;
+    if (lc < 2 || (lc & 1) || d->n_layers + 1 > ZENO_MAX_LAYERS) return 0;
+    for (int l = 0; l <= d->n_layers + 1; ++l)
+        if (d->dims[l] < 1 || d->dims[l] > (int64_t)1 << 20) return 0;
+    int64_t side = d->dims[0];
+    for (int l = 1; l <= lc; ++l) {
+        if (!zeno::cnn_side_ok((int)side)) return 0;
+        if ((l & 1) == 0) side /= 2;
+    }
+    return side;
+}
+
 bool desc_ok(const zeno_model_desc *d) {
     if (!d) return false;
     if (d->kind == ZENO_LOSS_LEAST_SQUARES) return d->dims[0] >= 1;
+    if (d->kind == ZENO_LOSS_SOFTMAX_CNN) return cnn_final_side(d) > 0;
     if (d->kind != ZENO_LOSS_SOFTMAX_MLP) return false;
     if (d->n_layers < 1 || d->n_layers > ZENO_MAX_LAYERS) return false;
     for (int l = 0; l <= d->n_layers; ++l)
         if (d->dims[l] < 1 || d->dims[l] > (int64_t)1 << 30) return false;
     return true;
+}
+
+// values of one sample's features
+size_t feature_count(const zeno_model_desc &d) {
+    if (d.kind == ZENO_LOSS_SOFTMAX_CNN) return (size_t)(d.dims[1] * d.dims[0] * d.dims[0]);
+    return (size_t)d.dims[0];
 }
 
 bool is_aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
@@ -80,6 +102,8 @@ bool score_rows_aligned(const Context &c, const void *x, const void *V, int64_t 
     if (!is_aligned(x, vec_bytes) || !is_aligned(V, vec_bytes) || !is_aligned(features, 16)) return false;
     if (ldv % 4 != 0) return false;
     if (c.desc.kind == ZENO_LOSS_LEAST_SQUARES) return c.d % 4 == 0;
+    if (c.desc.kind == ZENO_LOSS_SOFTMAX_CNN)      // only the dense layer takes vector loads
+        return c.offW[c.desc.n_layers - 1] % 4 == 0 && c.cnn_flat % 4 == 0;
     for (int l = 0; l < c.desc.n_layers; ++l)
         if (c.offW[l] % 4 != 0 || c.desc.dims[l] % 4 != 0) return false;
     return true;
@@ -94,6 +118,92 @@ zeno_status check_common(const Context *c, const void *V, int64_t ldv, int32_t m
     if (!c || !V) return ZENO_ERR_INVALID_ARG;
     if (m < 1 || m > c->m_max) return ZENO_ERR_INVALID_ARG;
     if (ldv < c->d) return ZENO_ERR_INVALID_ARG;
+    return ZENO_OK;
+}
+
+// The convolutional network: its convolutional layers one launch each, then the dense layer with the
+// cross-entropy and the scoring tail as for the dense models.
+zeno_status enqueue_score_cnn(Context *c, const void *x, const void *V, int64_t ldv, int32_t m, const zeno_batch *batch,
+                              float gamma, float rho, float *scores, float *loss_buf, float *norms, int keep,
+                              int32_t *idx, bool *ranked, bool aligned, cudaStream_t s, int *launches) {
+    const int n_r = batch->n_r, L = c->desc.n_layers, lc = L - 1;
+    const int classes = (int)c->desc.dims[lc + 2];
+    zeno::TailArgs tail;
+    tail.normpart = c->normpart;
+    tail.np_slots = c->np_slots;
+    tail.used.layers = L;
+    tail.m = m;
+    tail.rho = rho;
+    tail.scores = scores;
+    tail.norms_out = norms;
+    tail.norm_tot = c->norms;
+    tail.loss_sum = c->loss_sum;
+    tail.n_r = n_r;
+    tail.idx = idx;
+    tail.keep = keep;
+    tail.ticket = c->tickets;
+    int side = (int)c->desc.dims[0];
+    cudaError_t e = cudaSuccess;
+    for (int l = 0; l < lc; ++l) {
+        zeno::CnnLayerArgs a;
+        a.x = x;
+        a.V = V;
+        a.ldv = ldv;
+        a.offW = c->offW[l];
+        a.offB = c->offB[l];
+        a.cin = (int)c->desc.dims[l + 1];
+        a.cout = (int)c->desc.dims[l + 2];
+        a.side = side;
+        a.pool = (l & 1) == 1;
+        a.Hin = l == 0 ? batch->features : c->act[(l - 1) & 1];
+        a.hin_cand_stride = l == 0 ? 0 : (int64_t)n_r * a.cin * side * side;
+        a.Hout = c->act[l & 1];
+        a.n_r = n_r;
+        a.m = m;
+        a.gamma = gamma;
+        a.normpart = c->normpart;
+        a.np_slots = c->np_slots;
+        a.np_base = c->np_base[l];
+        tail.used.base[l] = c->np_base[l];
+        tail.used.count[l] = zeno::cnn_norm_slots(a.cout);
+        e = zeno::launch_cnn_conv(*c, a, s, launches);
+        if (e != cudaSuccess) return fail_cuda(c, e);
+        if (a.pool) side /= 2;
+    }
+    const bool fuse_loss = zeno::mlp_can_fuse_loss(classes, n_r);
+    zeno::LayerArgs a;
+    a.x = x;
+    a.V = V;
+    a.ldv = ldv;
+    a.offW = c->offW[lc];
+    a.offB = c->offB[lc];
+    a.in = (int)c->cnn_flat;
+    a.out = classes;
+    a.Hin = c->act[(lc - 1) & 1];
+    a.hin_cand_stride = (int64_t)n_r * a.in;
+    a.Hout = c->act[lc & 1];
+    a.n_r = n_r;
+    a.m = m;
+    a.gamma = gamma;
+    a.relu = 0;
+    a.normpart = c->normpart;
+    a.np_slots = c->np_slots;
+    a.np_base = c->np_base[lc];
+    a.fuse_loss = fuse_loss;
+    a.first_in_call = 0;
+    tail.used.base[lc] = c->np_base[lc];
+    tail.used.count[lc] = zeno::mlp_norm_slots(a.out);
+    a.labels = static_cast<const int32_t *>(batch->targets);
+    a.losses = loss_buf;
+    a.tail = tail;
+    e = zeno::launch_mlp_layer(*c, a, aligned, s, launches);
+    if (e != cudaSuccess) return fail_cuda(c, e);
+    if (!fuse_loss) {
+        e = zeno::launch_mlp_loss(*c, c->act[lc & 1], static_cast<const int32_t *>(batch->targets), n_r, m, classes,
+                                  loss_buf, tail, s, launches);
+        if (e != cudaSuccess) return fail_cuda(c, e);
+    }
+    *ranked = keep > 0;
     return ZENO_OK;
 }
 
@@ -130,6 +240,9 @@ zeno_status enqueue_score(Context *c, const void *x, const void *V, int64_t ldv,
                                    aligned, loss_buf, norms, scores, s, launches);
         return e == cudaSuccess ? ZENO_OK : fail_cuda(c, e);
     }
+
+    if (c->desc.kind == ZENO_LOSS_SOFTMAX_CNN)
+        return enqueue_score_cnn(c, x, V, ldv, m, batch, gamma, rho, scores, loss_buf, norms, keep, idx, ranked, aligned, s, launches);
 
     const int L = c->desc.n_layers;
     zeno::TailArgs tail;
@@ -342,6 +455,13 @@ extern "C" {
 int64_t zeno_param_count(const zeno_model_desc *desc) {
     if (!desc_ok(desc)) return 0;
     if (desc->kind == ZENO_LOSS_LEAST_SQUARES) return desc->dims[0];
+    if (desc->kind == ZENO_LOSS_SOFTMAX_CNN) {
+        const int lc = desc->n_layers - 1;
+        const int64_t side = cnn_final_side(desc), classes = desc->dims[lc + 2];
+        int64_t d = 0;
+        for (int l = 1; l <= lc; ++l) d += desc->dims[l + 1] * desc->dims[l] * 9 + (desc->has_bias ? desc->dims[l + 1] : 0);
+        return d + classes * desc->dims[lc + 1] * side * side + (desc->has_bias ? classes : 0);
+    }
     int64_t d = 0;
     for (int l = 0; l < desc->n_layers; ++l)
         d += desc->dims[l + 1] * desc->dims[l] + (desc->has_bias ? desc->dims[l + 1] : 0);
@@ -354,7 +474,8 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
     if (!out) return ZENO_ERR_INVALID_ARG;
     *out = nullptr;
     if (!desc) return ZENO_ERR_INVALID_ARG;
-    if (desc->kind != ZENO_LOSS_SOFTMAX_MLP && desc->kind != ZENO_LOSS_LEAST_SQUARES)
+    if (desc->kind != ZENO_LOSS_SOFTMAX_MLP && desc->kind != ZENO_LOSS_LEAST_SQUARES &&
+        desc->kind != ZENO_LOSS_SOFTMAX_CNN)
         return ZENO_ERR_UNSUPPORTED;
     if (desc->param_dtype != ZENO_F32 && desc->param_dtype != ZENO_BF16) return ZENO_ERR_UNSUPPORTED;
     if (desc->kind == ZENO_LOSS_LEAST_SQUARES && desc->param_dtype != ZENO_F32)
@@ -435,6 +556,33 @@ zeno_status zeno_create(zeno_handle *out, const zeno_model_desc *desc, int32_t m
             slots += layer_slots;
             if (o > widest) widest = o;
         }
+        c->np_slots = slots;
+        act_elems = rows * (size_t)n_r_max * (size_t)widest;
+        norm_elems = (size_t)m_max * (size_t)slots;
+    } else if (desc->kind == ZENO_LOSS_SOFTMAX_CNN) {
+        // layers 0 .. Lc - 1: the convolutional ones; layer Lc: the dense one (served by the dense kernels)
+        const int lc = desc->n_layers - 1;
+        int64_t off = 0, side = desc->dims[0], widest = 0;
+        int slots = 0;
+        for (int l = 0; l < lc; ++l) {
+            const int64_t cin = desc->dims[l + 1], cout = desc->dims[l + 2];
+            c->offW[l] = off;
+            off += cout * cin * 9;
+            c->offB[l] = desc->has_bias ? off : -1;
+            if (desc->has_bias) off += cout;
+            c->np_base[l] = slots;
+            slots += zeno::cnn_norm_slots((int)cout);
+            if ((l & 1) == 1) side /= 2;                 // the pooling is folded into every second layer
+            if (cout * side * side > widest) widest = cout * side * side;
+        }
+        const int64_t classes = desc->dims[lc + 2];
+        c->cnn_flat = desc->dims[lc + 1] * side * side;
+        c->offW[lc] = off;
+        off += classes * c->cnn_flat;
+        c->offB[lc] = desc->has_bias ? off : -1;
+        c->np_base[lc] = slots;
+        slots += zeno::mlp_norm_slots((int)classes);
+        if (classes > widest) widest = classes;
         c->np_slots = slots;
         act_elems = rows * (size_t)n_r_max * (size_t)widest;
         norm_elems = (size_t)m_max * (size_t)slots;
@@ -740,7 +888,7 @@ zeno_status zeno_run(zeno_handle h, void *x, const void *V, int64_t ldv, int64_t
     if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t esz = elem_size(h->desc.param_dtype);
-    const size_t feat_stride = (size_t)n_r * (size_t)h->desc.dims[0];
+    const size_t feat_stride = (size_t)n_r * feature_count(h->desc);
     int launches = 0;
     profile_begin(h);
     zeno_status st = ZENO_OK;
@@ -776,7 +924,7 @@ zeno_status zeno_step_host(zeno_handle h, const void *x, const void *V, int64_t 
     if (guard.err != cudaSuccess) return fail_cuda(h, guard.err);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t esz = elem_size(h->desc.param_dtype);
-    const size_t in0 = (size_t)h->desc.dims[0];
+    const size_t in0 = feature_count(h->desc);
     const size_t x_bytes = round_up((size_t)h->d * esz, kAlign);
     const size_t v_bytes = round_up((size_t)m * (size_t)ldv * esz, kAlign);
     const size_t f_bytes = round_up((size_t)n_r * in0 * 4, kAlign);

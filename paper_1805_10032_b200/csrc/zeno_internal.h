@@ -51,6 +51,7 @@ struct Context {
     int64_t offB[ZENO_MAX_LAYERS];  // element offset of b_l, -1 without bias
     int np_base[ZENO_MAX_LAYERS];   // first norm-partial slot of layer l
     int np_slots;                   // norm-partial slots per candidate
+    int64_t cnn_flat;               // convolutional network: inputs of its dense layer
     void *arena;                    // the one device allocation everything below is carved from
     float *act[2];                  // activations [m_max+1][n_r_max][widest layer output]
     double *loss_part;              // [m_max + 1][8] per-block sums of the sample losses
@@ -182,6 +183,27 @@ cudaError_t launch_select(Context &c, const float *scores, int m, int b, int32_t
 cudaError_t launch_aggregate(Context &c, const void *V, int64_t ldv, int m,
                              const int32_t *idx, int k, float *out, void *xu, float gamma, bool aligned,
                              cudaStream_t s, int *launches);
+
+// One convolutional layer (3 x 3, stride 1, zero padding 1, ReLU, optionally followed by a 2 x 2 max
+// pooling) of all m + 1 models of a ZENO_LOSS_SOFTMAX_CNN handle.
+struct CnnLayerArgs {
+    const void *x;
+    const void *V;
+    int64_t ldv;
+    int64_t offW, offB;       // W[cout][cin][3][3], b[cout] (-1: none)
+    int cin, cout, side;      // input planes, output planes, the planes' side (before the pooling)
+    int pool;
+    const float *Hin;         // [m+1][n_r][cin][side][side] (the shared batch: stride 0)
+    int64_t hin_cand_stride;
+    float *Hout;              // [m+1][n_r][cout][side or side / 2]^2
+    int n_r, m;
+    float gamma;
+    float *normpart;
+    int np_slots, np_base;
+};
+bool cnn_side_ok(int side);
+int cnn_norm_slots(int cout);
+cudaError_t launch_cnn_conv(Context &c, const CnnLayerArgs &a, cudaStream_t s, int *launches);
 
 // Tensor-core stream for the first layer (fp32 storage).
 bool stream_tc_plan(int sms, int K, int out, int n_r, int m, StreamTcPlan *p);
@@ -324,6 +346,9 @@ __device__ __forceinline__ unsigned long long rank_key(float s, int index) {
     u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
     return ((unsigned long long)u << 32) | (unsigned)(0xffffffffu - (unsigned)index);
 }
+
+// ReLU that lets a NaN through
+__device__ __forceinline__ float relu_keep_nan(float z) { return (z > 0.f || z != z) ? z : 0.f; }
 
 template <typename T> struct is_bf16 { static constexpr bool value = false; };
 template <> struct is_bf16<__nv_bfloat16> { static constexpr bool value = true; };

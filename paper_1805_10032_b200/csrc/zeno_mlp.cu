@@ -64,7 +64,6 @@ __device__ __forceinline__ double warp_sum(double v) {
     return v;
 }
 
-__device__ __forceinline__ float relu_keep_nan(float z) { return (z > 0.f || z != z) ? z : 0.f; }
 
 // A lane's four k-indices inside a 128-wide block: vector path 4*lane + e (one 16-byte / 8-byte
 // load); scalar path 32*e + lane (coalesced).

@@ -157,6 +157,7 @@ __global__ void __launch_bounds__(256) inject_faults_kernel(T *V, int64_t ldv, i
 bool worker_gradients_supported(const Context &c, int n) {
     if (n < 1) return false;
     if (c.desc.kind == ZENO_LOSS_LEAST_SQUARES) return c.desc.param_dtype == ZENO_F32 && n <= 4096;
+    if (c.desc.kind != ZENO_LOSS_SOFTMAX_MLP) return false;
     return c.desc.n_layers == 1 && c.desc.dims[1] <= kWMaxClasses && (int64_t)n * c.desc.dims[1] * 4 <= 48 * 1024;
 }
 

@@ -28,9 +28,10 @@ BASE_SEED = 20260101
 @dataclass
 class Workload:
     name: str
-    kind: str                 # "mlp" (softmax cross-entropy ReLU MLP) or "lsq" (least squares)
+    kind: str                 # "mlp" (softmax cross-entropy ReLU MLP), "lsq" (least squares) or "cnn"
     dtype: str                # storage type of x and V: "f32" or "bf16"
-    dims: tuple               # mlp: layer widths (in, hidden..., classes); lsq: (d, 1)
+    dims: tuple               # mlp: layer widths (in, hidden..., classes); lsq: (d, 1);
+                              # cnn: (S, C_0, C_1, .., C_Lc, classes): image side, planes per layer, classes
     has_bias: bool
     m: int
     b: int
@@ -41,7 +42,7 @@ class Workload:
     ldv: int
     x: torch.Tensor           # [d]
     V: torch.Tensor           # [m, ldv]; columns >= d are padding (NaN for f32/bf16)
-    features: torch.Tensor    # [n_r, dims[0]] float32
+    features: torch.Tensor    # [n_r, dims[0]] float32 (cnn: [n_r, C_0, S, S])
     targets: torch.Tensor     # int32 labels [n_r] (mlp) or float32 y [n_r] (lsq)
     honest: torch.Tensor = field(default=None)  # bool [m], which rows are honest (metadata only)
     seed: int = 0
@@ -50,6 +51,12 @@ class Workload:
 def param_count(kind: str, dims: Sequence[int], has_bias: bool = True) -> int:
     if kind == "lsq":
         return int(dims[0])
+    if kind == "cnn":
+        side, chans, classes = dims[0], dims[1:-1], dims[-1]
+        lc = len(chans) - 1
+        conv = sum(chans[l] * chans[l - 1] * 9 + (chans[l] if has_bias else 0) for l in range(1, lc + 1))
+        side //= 2 ** (lc // 2)
+        return int(conv + classes * chans[-1] * side * side + (classes if has_bias else 0))
     return int(sum(dims[l + 1] * dims[l] + (dims[l + 1] if has_bias else 0)
                    for l in range(len(dims) - 1)))
 
@@ -182,6 +189,106 @@ def make_mlp_workload(name, seed, dims, dtype, m, b, n_r, gamma, rho, honest_std
                     targets=labels, honest=honest, seed=seed)
 
 
+def _cnn_split(flat, dims, has_bias):
+    """Views of the flat parameter vector: [(W[C_l, C_{l-1}, 3, 3], b or None)] and the dense (W, b)."""
+    side, chans, classes = dims[0], dims[1:-1], dims[-1]
+    lc = len(chans) - 1
+    off, conv = 0, []
+    for l in range(1, lc + 1):
+        n = chans[l] * chans[l - 1] * 9
+        W = flat[off:off + n].view(chans[l], chans[l - 1], 3, 3)
+        off += n
+        bvec = None
+        if has_bias:
+            bvec = flat[off:off + chans[l]]
+            off += chans[l]
+        conv.append((W, bvec))
+    side //= 2 ** (lc // 2)
+    n = classes * chans[-1] * side * side
+    W = flat[off:off + n].view(classes, chans[-1] * side * side)
+    off += n
+    bvec = flat[off:off + classes] if has_bias else None
+    return conv, (W, bvec)
+
+
+def cnn_he_init(dims, has_bias, gen, device) -> torch.Tensor:
+    """He-initialised weights N(0, 2/fan_in), zero biases, in the flat layout."""
+    side, chans, classes = dims[0], dims[1:-1], dims[-1]
+    lc = len(chans) - 1
+    parts = []
+    for l in range(1, lc + 1):
+        parts.append(_randn((chans[l] * chans[l - 1] * 9,), gen, device, (2.0 / (chans[l - 1] * 9)) ** 0.5))
+        if has_bias:
+            parts.append(torch.zeros(chans[l], device=device))
+    side //= 2 ** (lc // 2)
+    flat = chans[-1] * side * side
+    parts.append(_randn((classes * flat,), gen, device, (2.0 / flat) ** 0.5))
+    if has_bias:
+        parts.append(torch.zeros(classes, device=device))
+    return torch.cat(parts)
+
+
+def cnn_gradient(x_flat, dims, has_bias, feats, labels) -> torch.Tensor:
+    """A worker's gradient of the network's mean cross-entropy (torch autograd, float32): input data for the
+    candidates, like mlp_gradient."""
+    p = x_flat.detach().clone().float().requires_grad_(True)
+    conv, (W, bvec) = _cnn_split(p, dims, has_bias)
+    h = feats
+    for l, (Wc, bc) in enumerate(conv, start=1):
+        h = torch.relu(torch.nn.functional.conv2d(h, Wc, bc, padding=1))
+        if l % 2 == 0:
+            h = torch.nn.functional.max_pool2d(h, 2)
+    z = torch.nn.functional.linear(h.flatten(1), W, bvec)
+    loss = torch.nn.functional.cross_entropy(z, labels.long())
+    (g,) = torch.autograd.grad(loss, p)
+    return g.detach()
+
+
+def make_cnn_workload(name, seed, dims, dtype, m, b, n_r, gamma, rho, honest_std, faults, worker_batch=32,
+                      ldv: Optional[int] = None, device="cpu", has_bias=True) -> Workload:
+    """The convolutional model: images N(0, 1), uniform labels, He-initialised x, honest rows = a worker's
+    gradient + N(0, honest_std^2), faults as in make_mlp_workload."""
+    dims = tuple(int(v) for v in dims)
+    d = param_count("cnn", dims, has_bias)
+    ldv = round_up(d, 32) if ldv is None else int(ldv)
+    gen = _gen(seed, device)
+    gen_cpu = _gen(seed + 7919, "cpu")
+    side, c0, classes = dims[0], dims[1], dims[-1]
+    x = _store(cnn_he_init(dims, has_bias, gen, device), dtype)
+    feats = _randn((n_r, c0, side, side), gen, device)
+    labels = torch.randint(0, classes, (n_r,), generator=gen, device=device, dtype=torch.int32)
+    wfeats = _randn((worker_batch, c0, side, side), gen, device)
+    wlabels = torch.randint(0, classes, (worker_batch,), generator=gen, device=device, dtype=torch.int32)
+    g = cnn_gradient(x.float(), dims, has_bias, wfeats, wlabels)
+    n_faulty = sum(c for c, _ in faults)
+    n_honest = m - n_faulty
+    assert n_honest >= 1
+    perm = _shuffle_rows(m, gen_cpu)
+    V = _alloc_V(m, d, ldv, dtype, device)
+    honest = torch.zeros(m, dtype=torch.bool)
+    honest_sum = torch.zeros(d, device=device, dtype=torch.float32)
+    slot = 0
+    for _ in range(n_honest):
+        row = _store(g + _randn((d,), gen, device, honest_std), dtype)
+        V[perm[slot], :d] = row
+        honest[perm[slot]] = True
+        honest_sum += row.float()
+        slot += 1
+    for count, kind in faults:
+        if kind == "signflip":
+            row = _store(-4.0 * g, dtype)
+        elif kind == "omniscient":
+            row = _store(-1e3 * (honest_sum / n_honest), dtype)
+        for _ in range(count):
+            if kind == "noise200":
+                row = _store(_randn((d,), gen, device, 200.0), dtype)
+            V[perm[slot], :d] = row
+            slot += 1
+    return Workload(name=name, kind="cnn", dtype=dtype, dims=dims, has_bias=has_bias, m=m, b=b, n_r=n_r,
+                    gamma=gamma, rho=rho, d=d, ldv=ldv, x=x, V=V, features=feats, targets=labels,
+                    honest=honest, seed=seed)
+
+
 def make_lsq_workload(name, seed, d, m, b, n_r, gamma, rho, honest_std, n_noise, noise_std,
                       ldv: Optional[int] = None, device="cpu") -> Workload:
     """f(x) = ||A x - y||^2 / (2 n_r); A entries N(0, variance 1/d), y ~ N(0,1), x ~ N(0,1);
@@ -222,6 +329,10 @@ CONFIGS = {
             rho=5e-4, honest_std=0.05, faults=[(12, "signflip")]),
     5: dict(d=1 << 26, m=64, b=24, n_r=16, gamma=0.01, rho=1e-4, honest_std=0.01,
             n_noise=24, noise_std=100.0),
+    # the shape of the paper's own experiment: a CNN of four convolutional layers and a dense one on
+    # 32 x 32 x 3 images, 20 workers, 8 of them faulty, n_r = 4 (the network's widths are this project's)
+    6: dict(dims=(32, 3, 32, 32, 64, 64, 10), dtype="f32", m=20, b=8, n_r=4, gamma=0.1, rho=5e-4,
+            honest_std=0.02, faults=[(8, "signflip")]),
 }
 
 
@@ -231,6 +342,8 @@ def describe_config(index: int) -> dict:
     p = CONFIGS[index]
     if index == 5:
         kind, dims, dtype = "lsq", (p["d"], 1), "f32"
+    elif index == 6:
+        kind, dims, dtype = "cnn", tuple(p["dims"]), p["dtype"]
     else:
         kind, dims, dtype = "mlp", tuple(p["dims"]), p["dtype"]
     d = param_count(kind, dims)
@@ -243,11 +356,13 @@ def make_config(index: int, device="cpu", **ov) -> Workload:
     configuration for tests (e.g. dims=(96, 40, 24, 10), m=9, b=3, n_r=5)."""
     seed = ov.pop("seed", BASE_SEED + index)
     if index not in CONFIGS:
-        raise ValueError("config index must be 1..5")
+        raise ValueError("config index must be 1..6")
     p = dict(CONFIGS[index])
     p.update(ov)
     if index == 5:
         return make_lsq_workload("config5", seed, device=device, **p)
+    if index == 6:
+        return make_cnn_workload("config6", seed, device=device, **p)
     return make_mlp_workload(f"config{index}", seed, device=device, **p)
 
 

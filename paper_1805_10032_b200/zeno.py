@@ -20,7 +20,7 @@ MAX_LAYERS = 8
 MAX_CANDIDATES = 1024
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
-LOSS_SOFTMAX_MLP, LOSS_LEAST_SQUARES = 0, 1
+LOSS_SOFTMAX_MLP, LOSS_LEAST_SQUARES, LOSS_SOFTMAX_CNN = 0, 1, 2
 FAULT_BIT_FLIP, FAULT_SCALE = 0, 1
 F32, BF16 = 0, 1
 
@@ -129,7 +129,8 @@ def make_desc(kind: int, param_dtype: int, dims: Sequence[int], has_bias: bool =
     d = ModelDesc()
     d.kind = kind
     d.param_dtype = param_dtype
-    d.n_layers = len(dims) - 1
+    # a convolutional network's list starts with the image side: [S, C_0, C_1, .., C_Lc, classes]
+    d.n_layers = len(dims) - 2 if kind == LOSS_SOFTMAX_CNN else len(dims) - 1
     d.has_bias = int(has_bias)
     for i, v in enumerate(dims):
         d.dims[i] = int(v)
@@ -424,6 +425,6 @@ def score_lsq_static(x, V, A, y, gamma, rho, scores, losses=None, norms=None, m=
 
 def from_workload(w, m_max=None, n_r_max=None, device=0) -> "Zeno":
     """A handle shaped for a synthetic.Workload."""
-    kind = LOSS_LEAST_SQUARES if w.kind == "lsq" else LOSS_SOFTMAX_MLP
+    kind = {"lsq": LOSS_LEAST_SQUARES, "cnn": LOSS_SOFTMAX_CNN}.get(w.kind, LOSS_SOFTMAX_MLP)
     dt = BF16 if w.dtype == "bf16" else F32
     return Zeno(kind, dt, w.dims, w.has_bias, m_max or w.m, n_r_max or w.n_r, device)

@@ -19,7 +19,7 @@ SCORE_RTOL = 1e-4
 GAP_RTOL = 1e-3
 AGG_RTOL = 1e-5
 
-KIND = {"mlp": 0, "lsq": 1}
+KIND = {"mlp": 0, "lsq": 1, "cnn": 2}
 DTYPE = {"f32": 0, "bf16": 1}
 
 

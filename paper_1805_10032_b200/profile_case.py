@@ -18,7 +18,7 @@ from . import zeno
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--config", type=int, required=True, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--config", type=int, required=True, choices=[1, 2, 3, 4, 5, 6])
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--d", type=int, default=0, help="configuration 5 only: parameter count")
     ap.add_argument("--n-r", type=int, default=0)

@@ -78,7 +78,7 @@ def time_baselines(index, steps):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5, 6])
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--n-r", type=int, nargs="*", default=[])
     ap.add_argument("--b", type=int, nargs="*", default=[])

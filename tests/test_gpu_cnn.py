@@ -80,3 +80,17 @@ def test_nan_pixel_and_nan_candidate(oracle):
     assert 1 not in idx.cpu().tolist()
     ok = ~np.isnan(s_orc)
     assert np.allclose(s[ok], s_orc[ok], rtol=1e-3, atol=1e-6)
+
+
+def test_host_buffers(oracle):
+    """zeno_step_host with the convolutional model: the batch is [n_r][C_0][S][S] values per step."""
+    w = syn.make_config(6, dims=(8, 3, 8, 8, 10), m=5, b=2, n_r=3, faults=[(2, "signflip")])
+    out = torch.empty(w.d, dtype=torch.float32).pin_memory()
+    scores = torch.empty(w.m, dtype=torch.float32).pin_memory()
+    idx = torch.empty(w.m - w.b, dtype=torch.int32).pin_memory()
+    with zeno.from_workload(w) as z:
+        z.step_host(w.x.pin_memory(), w.V.pin_memory(), w.features.contiguous().pin_memory(), w.targets.pin_memory(),
+                    w.gamma, w.rho, w.b, out, scores=scores, idx=idx)
+        x, V, f, t = P.to_device(w)
+        out_d, scores_d, idx_d = z.step(x, V, f, t, w.gamma, w.rho, w.b)
+    assert torch.equal(out, out_d.cpu()) and torch.equal(scores, scores_d.cpu()) and torch.equal(idx, idx_d.cpu())

@@ -27,6 +27,7 @@ CASES = {
     "cfg2_mid_layers": (2, dict(dims=(520, 200, 136, 10), n_r=21, m=6, b=2, faults=[(2, "noise200")])),
     "cfg4_small": (4, dict(dims=(264, 136, 72, 50), m=9, b=3, n_r=19, faults=[(3, "signflip")])),
     "cfg5_small": (5, dict(d=70000, m=13, b=5, n_r=16, n_noise=5)),
+    "cfg6_cnn_small": (6, dict(dims=(8, 3, 8, 8, 12, 12, 10), m=7, b=2, n_r=5, faults=[(2, "signflip")])),
 }
 
 

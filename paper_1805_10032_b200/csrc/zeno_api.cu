@@ -654,6 +654,7 @@ zeno_status zeno_destroy(zeno_handle h) {
     DeviceGuard guard(h->device);
     cudaError_t e = cudaFree(h->arena);
     if (h->host_stage) cudaFree(h->host_stage);
+    free(h->tmap_cache);
     if (h->profile)
         for (int d = 0; d < zeno::kProfileDepth; ++d)
             for (int i = 0; i <= zeno::kMaxProfiled; ++i) cudaEventDestroy(h->events[d][i]);

@@ -77,6 +77,7 @@ struct Context {
     float *krum_sums;               // [m_max]
     int krum_blocks;                // blocks the partials were sized for
     void *host_stage;               // device copies of host inputs (zeno_step_host), grown on demand
+    void *tmap_cache;               // encoded tensor maps of the tensor-core kernels (host memory, malloc'ed), or NULL
     size_t host_stage_bytes;
     int last_launches;
     int last_cuda_error;

@@ -705,28 +705,24 @@ __global__ void __launch_bounds__(256) split_acts_kernel(const float *H, int mod
 }
 
 template <typename T>
-cudaError_t encode_maps(const LayerTcLaunch &l, CUtensorMap *map_x, CUtensorMap *map_v, CUtensorMap *map_h) {
+cudaError_t encode_maps(Context &c, const LayerTcLaunch &l, CUtensorMap *map_x, CUtensorMap *map_v, CUtensorMap *map_h) {
     using Tr = TcTraits<T>;
-    EncodeTiledFn enc = encode_tiled_fn();
-    if (!enc) return cudaErrorNotSupported;
+    if (!encode_tiled_fn()) return cudaErrorNotSupported;
     const cuuint64_t es = sizeof(T);
-    cuuint32_t ones[3] = {1, 1, 1};
     {
         cuuint64_t dims[3] = {(cuuint64_t)l.K, (cuuint64_t)l.out, 1};
         cuuint64_t strides[2] = {(cuuint64_t)l.K * es, (cuuint64_t)l.K * es * (cuuint64_t)l.out};
         cuuint32_t box[3] = {(cuuint32_t)Tr::kBlockK, kRows, 1};
-        if (enc(map_x, Tr::kMapType, 3, const_cast<T *>(static_cast<const T *>(l.x) + l.offW), dims, strides, box, ones,
-                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        if (encode_cached(c, map_x, Tr::kMapType, static_cast<const T *>(l.x) + l.offW, dims, strides, box,
+                          CU_TENSOR_MAP_SWIZZLE_128B) != CUDA_SUCCESS)
             return cudaErrorInvalidValue;
     }
     {
         cuuint64_t dims[3] = {(cuuint64_t)l.K, (cuuint64_t)l.out, (cuuint64_t)l.m};
         cuuint64_t strides[2] = {(cuuint64_t)l.K * es, (cuuint64_t)l.ldv * es};
         cuuint32_t box[3] = {(cuuint32_t)Tr::kBlockK, kRows, 1};
-        if (enc(map_v, Tr::kMapType, 3, const_cast<T *>(static_cast<const T *>(l.V) + l.offW), dims, strides, box, ones,
-                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        if (encode_cached(c, map_v, Tr::kMapType, static_cast<const T *>(l.V) + l.offW, dims, strides, box,
+                          CU_TENSOR_MAP_SWIZZLE_128B) != CUDA_SUCCESS)
             return cudaErrorInvalidValue;
     }
     {
@@ -734,9 +730,7 @@ cudaError_t encode_maps(const LayerTcLaunch &l, CUtensorMap *map_x, CUtensorMap 
         cuuint64_t dims[3] = {(cuuint64_t)l.K, rows, models};
         cuuint64_t strides[2] = {(cuuint64_t)l.K * es, (cuuint64_t)l.K * es * rows};
         cuuint32_t box[3] = {(cuuint32_t)Tr::kBlockK, (cuuint32_t)rows, 1};
-        if (enc(map_h, Tr::kMapType, 3, const_cast<void *>(l.Hsplit_in), dims, strides, box, ones,
-                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        if (encode_cached(c, map_h, Tr::kMapType, l.Hsplit_in, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B) != CUDA_SUCCESS)
             return cudaErrorInvalidValue;
     }
     return cudaSuccess;
@@ -746,7 +740,7 @@ template <typename T, bool LINEAR, bool HEAD>
 cudaError_t launch_typed(Context &c, const LayerTcLaunch &l, cudaStream_t s) {
     using Tr = TcTraits<T>;
     CUtensorMap map_x, map_v, map_h;
-    cudaError_t e = encode_maps<T>(l, &map_x, &map_v, &map_h);
+    cudaError_t e = encode_maps<T>(c, l, &map_x, &map_v, &map_h);
     if (e != cudaSuccess) return e;
     LayerTcArgs a;
     a.xparams = l.x;

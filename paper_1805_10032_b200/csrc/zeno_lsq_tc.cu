@@ -430,11 +430,9 @@ bool lsq_tc_usable(const LsqArgs &a, bool aligned) {
 
 // Fills a.part with one slab per block; *slabs = the number of slabs written.
 cudaError_t launch_lsq_tc(Context &c, const LsqArgs &a, int max_slabs, int *slabs, cudaStream_t s) {
-    EncodeTiledFn enc = encode_tiled_fn();
-    if (!enc) return cudaErrorNotSupported;
+    if (!encode_tiled_fn()) return cudaErrorNotSupported;
     const int n_pad = a.n_r <= 16 ? 16 : 32;
     CUtensorMap map_v, map_a, map_x;
-    cuuint32_t ones[3] = {1, 1, 1};
     const bool wide = a.d % kQBlockK == 0 && a.ldv % kQBlockK == 0;
     if (wide) {
         // [row][k-block][32]: the k-blocks of a row are 128 bytes apart, the rows ldv (or d) elements
@@ -443,27 +441,21 @@ cudaError_t launch_lsq_tc(Context &c, const LsqArgs &a, int max_slabs, int *slab
             cuuint64_t dims[3] = {kQBlockK, nkb_all, (cuuint64_t)a.m};
             cuuint64_t strides[2] = {128, (cuuint64_t)a.ldv * 4};
             cuuint32_t box[3] = {kQBlockK, 2, kHalfRows};
-            if (enc(&map_v, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(a.V), dims, strides, box, ones,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            if (encode_cached(c, &map_v, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, a.V, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B) != CUDA_SUCCESS)
                 return cudaErrorInvalidValue;
         }
         {
             cuuint64_t dims[3] = {kQBlockK, nkb_all, (cuuint64_t)a.n_r};
             cuuint64_t strides[2] = {128, (cuuint64_t)a.d * 4};
             cuuint32_t box[3] = {kQBlockK, 2, (cuuint32_t)n_pad};
-            if (enc(&map_a, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(a.A), dims, strides, box, ones,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            if (encode_cached(c, &map_a, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, a.A, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B) != CUDA_SUCCESS)
                 return cudaErrorInvalidValue;
         }
         {
             cuuint64_t dims[3] = {(cuuint64_t)a.d, 1, 1};
             cuuint64_t strides[2] = {(cuuint64_t)a.d * 4, (cuuint64_t)a.d * 4};
             cuuint32_t box[3] = {2 * kQBlockK, 1, 1};
-            if (enc(&map_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(a.x), dims, strides, box, ones,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            if (encode_cached(c, &map_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, a.x, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE) != CUDA_SUCCESS)
                 return cudaErrorInvalidValue;
         }
     } else {
@@ -471,27 +463,21 @@ cudaError_t launch_lsq_tc(Context &c, const LsqArgs &a, int max_slabs, int *slab
         cuuint64_t dims[3] = {(cuuint64_t)a.d, (cuuint64_t)a.m, 1};
         cuuint64_t strides[2] = {(cuuint64_t)a.ldv * 4, (cuuint64_t)a.ldv * 4 * (cuuint64_t)a.m};
         cuuint32_t box[3] = {kQBlockK, kHalfRows, 1};
-        if (enc(&map_v, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(a.V), dims, strides, box, ones,
-                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        if (encode_cached(c, &map_v, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, a.V, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B) != CUDA_SUCCESS)
             return cudaErrorInvalidValue;
     }
     {
         cuuint64_t dims[3] = {(cuuint64_t)a.d, (cuuint64_t)a.n_r, 1};
         cuuint64_t strides[2] = {(cuuint64_t)a.d * 4, (cuuint64_t)a.d * 4 * (cuuint64_t)a.n_r};
         cuuint32_t box[3] = {kQBlockK, (cuuint32_t)n_pad, 1};
-        if (enc(&map_a, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(a.A), dims, strides, box, ones,
-                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        if (encode_cached(c, &map_a, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, a.A, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B) != CUDA_SUCCESS)
             return cudaErrorInvalidValue;
     }
     {
         cuuint64_t dims[3] = {(cuuint64_t)a.d, 1, 1};
         cuuint64_t strides[2] = {(cuuint64_t)a.d * 4, (cuuint64_t)a.d * 4};
         cuuint32_t box[3] = {kQBlockK, 1, 1};
-        if (enc(&map_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(a.x), dims, strides, box, ones,
-                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        if (encode_cached(c, &map_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, a.x, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE) != CUDA_SUCCESS)
             return cudaErrorInvalidValue;
     }
     }

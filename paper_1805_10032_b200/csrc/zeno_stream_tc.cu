@@ -564,27 +564,20 @@ int stream_tc_norm_slots(const StreamTcPlan &p) { return p.R * p.tiles_per_model
 cudaError_t launch_stream_tc(Context &c, const StreamTcPlan &p, const float *x, const float *V, int64_t ldv,
                              int64_t offW, int64_t offB, int K, int out, const float *X, int n_r, int m,
                              float *part, int np_base, cudaStream_t s, int *launches) {
-    EncodeTiledFn enc = encode_tiled_fn();
-    if (!enc) return cudaErrorNotSupported;
+    if (!encode_tiled_fn()) return cudaErrorNotSupported;
     CUtensorMap map_x, map_v;
     {   // x as a one-model stack, so that both operands go through the same 3-D path
         cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)out, 1};
         cuuint64_t strides[2] = {(cuuint64_t)K * 4, (cuuint64_t)K * 4 * (cuuint64_t)out};
         cuuint32_t box[3] = {kBlockK, kTileRows, 1};
-        cuuint32_t es[3] = {1, 1, 1};
-        CUresult r = enc(&map_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(x + offW), dims, strides,
-                         box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        CUresult r = encode_cached(c, &map_x, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, x + offW, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
         if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
     }
     {
         cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)out, (cuuint64_t)m};
         cuuint64_t strides[2] = {(cuuint64_t)K * 4, (cuuint64_t)ldv * 4};
         cuuint32_t box[3] = {kBlockK, kTileRows, 1};
-        cuuint32_t es[3] = {1, 1, 1};
-        CUresult r = enc(&map_v, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(V + offW), dims, strides,
-                         box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        CUresult r = encode_cached(c, &map_v, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, V + offW, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
         if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
     }
     StreamArgs a;

@@ -3,6 +3,8 @@
 #pragma once
 
 #include <cuda.h>
+#include <stdlib.h>
+#include <string.h>
 
 #include "zeno_internal.h"
 
@@ -173,5 +175,61 @@ inline EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
+// Tensor maps are descriptions of (pointer, shape, box): a handle sees the same few over and over, one step
+// after the other, so the encoded maps are kept per handle and looked up by what they describe (a few
+// dozen entries, replaced round robin).  All maps of this library have rank 3, element strides of one,
+// no interleave, 256-byte L2 promotion and no out-of-bounds fill value.
+struct TensorMapKey {
+    const void *base;
+    cuuint64_t dims[3];
+    cuuint64_t strides[2];
+    cuuint32_t box[3];
+    int type, swizzle;
+};
+struct TensorMapCache {
+    static constexpr int kEntries = 32;
+    CUtensorMap map[kEntries];
+    TensorMapKey key[kEntries];
+    bool valid[kEntries];
+    int next;
+};
+
+inline CUresult encode_cached(Context &c, CUtensorMap *out, CUtensorMapDataType type, const void *base,
+                              const cuuint64_t (&dims)[3], const cuuint64_t (&strides)[2], const cuuint32_t (&box)[3],
+                              CUtensorMapSwizzle swizzle) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return CUDA_ERROR_NOT_SUPPORTED;
+    if (!c.tmap_cache) {
+        const size_t bytes = (sizeof(TensorMapCache) + 63) / 64 * 64;
+        c.tmap_cache = aligned_alloc(64, bytes);
+        if (c.tmap_cache) memset(c.tmap_cache, 0, bytes);
+    }
+    TensorMapKey k;
+    memset(&k, 0, sizeof(k));
+    k.base = base;
+    for (int i = 0; i < 3; ++i) { k.dims[i] = dims[i]; k.box[i] = box[i]; }
+    k.strides[0] = strides[0];
+    k.strides[1] = strides[1];
+    k.type = (int)type;
+    k.swizzle = (int)swizzle;
+    TensorMapCache *cache = static_cast<TensorMapCache *>(c.tmap_cache);
+    if (cache)
+        for (int i = 0; i < TensorMapCache::kEntries; ++i)
+            if (cache->valid[i] && memcmp(&cache->key[i], &k, sizeof(k)) == 0) {
+                *out = cache->map[i];
+                return CUDA_SUCCESS;
+            }
+    cuuint32_t ones[3] = {1, 1, 1};
+    const CUresult r = enc(out, type, 3, const_cast<void *>(base), dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r == CUDA_SUCCESS && cache) {
+        const int i = cache->next;
+        cache->next = (i + 1) % TensorMapCache::kEntries;
+        cache->map[i] = *out;
+        cache->key[i] = k;
+        cache->valid[i] = true;
+    }
+    return r;
+}
 
 }  // namespace zeno
